@@ -1,0 +1,165 @@
+/*
+ * libcpattn -- cache-aware causal prefill attention under zigzag context parallelism (CP),
+ * hand-written for NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * Notation (paper Sections 2.1-2.2): P = prefix_len, the cached tokens of a request;
+ * R = new_len, its uncached suffix (the only tokens that are queries); L = P + R; C = CP
+ * degree; Hq / Hkv query / KV heads, G = Hq / Hkv; D = head dimension.  New token r sits at
+ * absolute position P + r and attends to keys 0 .. P + r (diagonal included).
+ *
+ * Conventions
+ *   - Every call returns an int: CP_OK (0) or a negative CP_ERR_* code; cp_strerror() names the
+ *     code and cp_last_error() gives a per-thread message for the last failing call.
+ *   - All buffers are owned by the caller.  "device" pointers are CUDA device memory of the
+ *     context's device, "host" pointers ordinary host memory.  The library allocates device
+ *     memory only inside cp_ctx_create().
+ *   - GPU calls validate their arguments first (an invalid call launches nothing), then only
+ *     ENQUEUE work on the given stream (a cudaStream_t passed as void*, NULL = default stream)
+ *     and return.  Device-side failures (a bounded wait that ran out) are recorded in a status
+ *     word that cp_ctx_poll_status() reads after the caller has synchronised.
+ *   - bf16 tensors are passed as void*; element strides are in elements.
+ */
+#ifndef CPATTN_H
+#define CPATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    CP_OK = 0,
+    CP_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, inconsistent lengths              */
+    CP_ERR_UNSUPPORTED = -2, /* D != 128, page_size != 64, odd Hq/Hkv ratio, misaligned strides    */
+    CP_ERR_WORKSPACE = -3,   /* workspace missing, misaligned or smaller than cp_workspace_bytes() */
+    CP_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                                */
+    CP_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (reported by poll_status)       */
+    CP_ERR_BOUNDS = -6       /* a host-visible index (page id, range) is out of range              */
+};
+
+enum { CP_DTYPE_BF16 = 0, CP_DTYPE_F32 = 1 };
+
+const char* cp_strerror(int code);
+const char* cp_last_error(void);
+
+/* ---------------------------------------------------------------------------------------------
+ * Context: one per (host thread, device).  Holds the device status word, the pinned staging
+ * buffer for tile lists and the resolved driver entry point for tensor-map encoding.
+ * cp_ctx_create() makes `device` current and allocates; cp_ctx_destroy() frees.
+ * cp_ctx_poll_status() synchronises the device-to-host copy of the status word on the default
+ * stream (call it after synchronising the streams you used): returns CP_OK or CP_ERR_TIMEOUT and,
+ * when `detail` is non-NULL, writes 4 int32 words {code, barrier id, block, iteration}; the
+ * status word is cleared by the call.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct cp_ctx cp_ctx;
+int cp_ctx_create(cp_ctx** ctx, int device);
+int cp_ctx_destroy(cp_ctx* ctx);
+int cp_ctx_poll_status(cp_ctx* ctx, int32_t* detail /* host, 4 words or NULL */);
+
+/* ---------------------------------------------------------------------------------------------
+ * cp_plan -- zigzag shard plan (paper Section 2.1, applied to the uncached suffix of Section 2.2).
+ * The R new tokens are padded on the right to a multiple of 2C: chunk length cl = ceil(R / 2C);
+ * chunk j = [min(j*cl, R), min((j+1)*cl, R)) (trailing chunks may be short or empty); shard k owns
+ * chunks k and 2C-1-k.  A chunk ending at q_end needs keys [0, P + q_end).  `pairs` is the number
+ * of visible (query, key) pairs of the shard; over all shards it sums to W(R,P) = R*P + R(R+1)/2
+ * (Eq. 1).  Host only, integer only.  out: host array of C entries.
+ * Errors: CP_ERR_INVALID_ARG if new_len < 1, prefix_len < 0, C < 1 or out == NULL.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int64_t q_begin[2]; /* new-token index, half-open; [0] = chunk k, [1] = chunk 2C-1-k */
+    int64_t q_end[2];
+    int64_t kv_end[2];  /* absolute, exclusive: P + q_end (kv_begin is always 0)          */
+    uint64_t pairs;
+} cp_shard_plan;
+int cp_plan(int64_t new_len, int64_t prefix_len, int32_t C, cp_shard_plan* out);
+
+/* ---------------------------------------------------------------------------------------------
+ * Paged KV cache.  Logical token t of a request, KV head g, dim d lives at element
+ *   page_table[t / page_size] * stride_page + (t % page_size) * stride_tok + g * stride_head + d.
+ * The new tokens' K and V are already in the cache at logical positions [P, P+R) when attention is
+ * called (the ranks gather K/V before attending, Section 2.1).  Default layout
+ * [num_pages, 64, Hkv, 128] bf16.  Supported: page_size == 64, D == 128; the three strides must be
+ * multiples of 8 elements and k, v 16-byte aligned (tensor-map rules).  Slots that no logical
+ * token maps to (tail of a last page, unreferenced pages) are never read into a result, but they
+ * must hold finite bf16 values (they may pass through a multiply by an exactly zero weight).
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    const void* k;      /* device, bf16 */
+    const void* v;      /* device, bf16 */
+    int64_t num_pages;
+    int32_t page_size;  /* 64  */
+    int32_t Hkv;
+    int32_t D;          /* 128 */
+    int32_t reserved;
+    int64_t stride_page, stride_tok, stride_head; /* elements */
+} cp_kv_cache;
+
+/* Workspace (device, 256-byte aligned) needed by the attention calls for a batch of B requests:
+ * the tile list of the persistent scheduler.  new_len, C: host arrays of B entries.
+ * Returns 0 on invalid arguments. */
+size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C);
+
+/* ---------------------------------------------------------------------------------------------
+ * cp_prefill_attn -- all C shards of one request in one launch (Sections 2.1-2.2).
+ *   q          device [R, Hq, D] bf16, new tokens in original order
+ *   page_table device int32, ceil((P+R)/page_size) entries, each in [0, num_pages)
+ *   scale      softmax scale (1/sqrt(D) in the paper's definition)
+ *   out        device [R, Hq, D] bf16; row r = softmax(scale * q_r K^T + mask) V, written at its
+ *              original position (the "restore order" step is fused into the store)
+ *   lse        device [Hq, R] fp32: natural-log sum-exp of the scaled scores of each row
+ * Every shard's q-tiles are cut at chunk boundaries of cp_plan(R, P, C); the result does not
+ * depend on C.  Requires Hq % Hkv == 0 and Hq / Hkv even (two query heads of one KV group share
+ * each K/V tile).  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ * ------------------------------------------------------------------------------------------- */
+int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
+                    int64_t prefix_len, int64_t new_len, int32_t C, int32_t Hq, float scale,
+                    void* out, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+/* cp_prefill_attn_batch -- B requests in ONE launch (persistent varlen tile scheduler, longest
+ * tiles first).  Host arrays: cu_new [B+1] (prefix sums of new_len; q/out rows of request b are
+ * [cu_new[b], cu_new[b+1])), prefix_len [B], C [B], cu_pages [B+1] (request b's page table is
+ * page_table[cu_pages[b] .. cu_pages[b+1]), with at least ceil((P_b+R_b)/page_size) entries).
+ * q/out: device [cu_new[B], Hq, D] bf16; lse: device [Hq, cu_new[B]] fp32. */
+int cp_prefill_attn_batch(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
+                          int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
+                          const int64_t* cu_pages, int32_t Hq, float scale, void* out, float* lse,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* cp_prefill_attn_shard -- only the rows of shard `shard` (0 <= shard < C) of cp_plan(R, P, C):
+ * what one CP rank computes.  partial_out: device [R, Hq, D] fp32, partial_lse: device [Hq, R]
+ * fp32; rows the shard does not own are written 0 with lse = -inf, so that cp_merge over the C
+ * shard partials reproduces cp_prefill_attn exactly. */
+int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
+                          int64_t prefix_len, int64_t new_len, int32_t C, int32_t shard, int32_t Hq,
+                          float scale, float* partial_out, float* partial_lse, void* workspace,
+                          size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * cp_merge -- N-way log-sum-exp combination of partial attention results over the same rows
+ * (what joins per-shard or KV-split partials into full-sequence attention).
+ *   partials device [N, T, H, D] fp32;  lses device [N, H, T] fp32 (natural log; -inf = "this
+ *   partial holds nothing for the row": its values are ignored even if non-finite)
+ *   out      device [T, H, D], bf16 or fp32 (out_dtype = CP_DTYPE_*)
+ *   lse_out  device [H, T] fp32 or NULL
+ * Per row: m = max_n lse_n; m = -inf -> out = 0, lse = -inf; else w_n = exp(lse_n - m),
+ * out = sum w_n O_n / sum w_n, lse = m + ln sum w_n.  Supported: D == 128, 1 <= N <= 32.
+ * ------------------------------------------------------------------------------------------- */
+int cp_merge(cp_ctx* ctx, const float* partials, const float* lses, int32_t N, int64_t T, int32_t H,
+             int32_t D, void* out, int32_t out_dtype, float* lse_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Paged <-> contiguous copies of n logical tokens starting at t_begin (the prefix-KV gather path
+ * as a standalone op).  k_rows / v_rows: device [n, Hkv, D] bf16, contiguous.  page_table: device.
+ * Bit-exact copies.  Either of the k/v pairs may be NULL to copy only the other.
+ * ------------------------------------------------------------------------------------------- */
+int cp_kv_gather(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin,
+                 int64_t n, void* k_rows, void* v_rows, void* stream);
+int cp_kv_append(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin,
+                 int64_t n, const void* k_rows, const void* v_rows, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CPATTN_H */

@@ -1,0 +1,732 @@
+// Cache-aware causal prefill attention for sm_100a: tcgen05 tensor cores with TMEM accumulators,
+// TMA-staged Q/K/V tiles (K/V fetched page by page through the page table), online softmax.
+//
+// One persistent CTA per SM walks a list of work units.  A unit is one query tile (<= 128 new
+// tokens of one zigzag chunk) for TWO query heads of the same KV group, so each K/V tile that
+// lands in shared memory feeds two 128x128 score tiles (GQA head sharing).  Warp roles:
+//   warps 0-3  softmax warpgroup for head 0 of the pair: one thread per query row
+//   warps 4-7  softmax warpgroup for head 1
+//   warp  8    TMA producer (lane 0 issues; the warp prefetches page ids)
+//   warp  9    tcgen05.mma issuer (one elected thread)
+// TMEM (512 columns): S0 | S1 | O0 | O1, each 128 fp32 columns; P (bf16) overwrites the first 64
+// columns of its S tile and is consumed from TMEM as the A operand of P*V.
+// The tensor pipe executes the MMAs of the issuing thread in order:
+//   S0(j+1) is issued behind PV0(j), S1(j+1) behind PV1(j), so while one warpgroup runs softmax
+//   on its tile the pipe works for the other one.
+// Every wait is bounded; on expiry the CTA records where it gave up in the status word, all roles
+// drain and the kernel returns normally.
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cstring>
+#include <vector>
+
+#include "internal.h"
+
+using namespace cpattn;
+
+namespace {
+
+constexpr int kD = 128;
+constexpr int kBlockM = 128;
+constexpr int kBlockN = 128;
+constexpr int kKvStages = 4;                       // ring of 32 KB tiles, K and V alternate
+constexpr uint32_t kTileBytes = kBlockN * kD * 2;  // 32768
+constexpr uint32_t kHalfBytes = kTileBytes / 2;    // one 64-dim half: 128 rows x 128 B
+constexpr uint32_t kPageBoxBytes = 64 * 64 * 2;    // one TMA box: 64 tokens x 64 dims
+constexpr int kThreads = 320;
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr uint32_t kSmemQ = 0;                                  // 2 heads x 32 KB
+constexpr uint32_t kSmemKV = 2 * kTileBytes;                    // kKvStages x 32 KB
+constexpr uint32_t kSmemBar = kSmemKV + kKvStages * kTileBytes; // mbarriers
+constexpr uint32_t kSmemBytes = kSmemBar + 256;
+constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;              // slack for manual alignment
+
+// barrier indices (8 bytes each, from kSmemBar); also the ids reported on a timeout
+enum Bar : uint32_t {
+    kBarQFull = 0, kBarQEmpty = 1,
+    kBarKvFull = 2,                       // + stage
+    kBarKvEmpty = kBarKvFull + kKvStages, // + stage
+    kBarSReady = kBarKvEmpty + kKvStages, // + wg
+    kBarPReady = kBarSReady + 2,          // + wg
+    kBarODone = kBarPReady + 2,           // + wg
+    kBarOFree = kBarODone + 2,            // + wg
+    kNumBars = kBarOFree + 2
+};
+static_assert(kNumBars * 8 + 16 <= 256, "barrier area");
+constexpr uint32_t kSmemTmemPtr = kSmemBar + kNumBars * 8;      // uint32: TMEM base address
+constexpr uint32_t kSmemAbort = kSmemTmemPtr + 4;               // uint32: set when a wait expired
+
+// TMEM columns
+constexpr uint32_t kTmemS = 0;     // + wg * 128
+constexpr uint32_t kTmemO = 256;   // + wg * 128
+
+constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
+constexpr float kRescaleThreshold = 8.0f;              // log2 units: keep a stale row max up to 2^8
+
+struct AttnParams {
+    const TileItem* items;
+    int32_t n_items;
+    int32_t pairs_per_tile;   // Hq / 2
+    int32_t group;            // Hq / Hkv
+    int32_t Hq;
+    const int32_t* page_table;
+    int32_t oob_page;         // a page coordinate outside the tensor map: TMA fills zeros
+    float scale_log2;         // scale * log2(e)
+    void* out;
+    int32_t out_f32;          // 0: bf16 [rows, Hq, D]; 1: fp32
+    float* lse;
+    int64_t lse_stride;       // total rows
+    int32_t* status;
+};
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+
+#define CP_R8(a, o) "=f"(a[o + 0]), "=f"(a[o + 1]), "=f"(a[o + 2]), "=f"(a[o + 3]), "=f"(a[o + 4]), "=f"(a[o + 5]), "=f"(a[o + 6]), "=f"(a[o + 7])
+#define CP_W8F(a, o) "f"(a[o + 0]), "f"(a[o + 1]), "f"(a[o + 2]), "f"(a[o + 3]), "f"(a[o + 4]), "f"(a[o + 5]), "f"(a[o + 6]), "f"(a[o + 7])
+#define CP_W8R(a, o) "r"(a[o + 0]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]), "r"(a[o + 5]), "r"(a[o + 6]), "r"(a[o + 7])
+
+// 32 consecutive fp32 columns of this thread's TMEM lane -> registers v[o .. o+31]
+#define TMEM_LD32(taddr, v, o)                                                                            \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                \
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                  \
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"                 \
+                 : CP_R8(v, o), CP_R8(v, o + 8), CP_R8(v, o + 16), CP_R8(v, o + 24) : "r"(taddr) : "memory")
+#define TMEM_ST32F(taddr, v, o)                                                                           \
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "                                         \
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                  \
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"                        \
+                 ::CP_W8F(v, o), CP_W8F(v, o + 8), CP_W8F(v, o + 16), CP_W8F(v, o + 24), "r"(taddr) : "memory")
+#define TMEM_ST32R(taddr, v, o)                                                                           \
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "                                         \
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                  \
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"                        \
+                 ::CP_W8R(v, o), CP_W8R(v, o + 8), CP_W8R(v, o + 16), CP_W8R(v, o + 24), "r"(taddr) : "memory")
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&b);
+}
+
+// tcgen05 shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+// K-major operand (Q, K): rows of 128 B, 8-row groups 1024 B apart (SBO); LBO unused.
+// MN-major operand (V): 64 dims contiguous per key row (128 B), 8-key groups 1024 B apart (SBO),
+// the next 64 dims one half-tile (16 KB) further (LBO).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(lbo_bytes >> 4) << 16;
+    d |= (uint64_t)(sbo_bytes >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = 128; bit 16 = B is MN-major
+constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((kBlockN >> 3) << 17) | ((kBlockM >> 4) << 24);
+constexpr uint32_t kIdescPV = kIdescS | (1u << 16);
+
+// Bounded wait on an mbarrier phase.  Returns false when the wait expired or another role already
+// gave up; the first to expire records {code, barrier id, block, iteration} in the status word.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar_base, uint32_t bar_id, uint32_t parity, volatile uint32_t* abort_flag,
+                                          int32_t* status, int iter) {
+    const uint32_t bar = bar_base + bar_id * 8;
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitLimitCycles) {
+            *abort_flag = 1;
+            if (atomicCAS(status, 0, CP_ERR_TIMEOUT) == 0) {
+                status[1] = (int32_t)bar_id;
+                status[2] = (int32_t)blockIdx.x;
+                status[3] = iter;
+            }
+            return false;
+        }
+    }
+}
+
+struct UnitInfo {
+    TileItem it;
+    int head0;
+    int kv_head;
+};
+
+// Serpentine static schedule over the longest-first unit list: in even rounds CTA c takes unit
+// round*grid + c, in odd rounds round*grid + (grid-1-c), which evens out the sorted lengths.
+__device__ __forceinline__ int64_t unit_index(int round) {
+    const int g = gridDim.x;
+    const int c = (round & 1) ? (g - 1 - (int)blockIdx.x) : (int)blockIdx.x;
+    return (int64_t)round * g + c;
+}
+__device__ __forceinline__ bool fetch_unit(const AttnParams& p, int round, UnitInfo& u) {
+    const int64_t idx = unit_index(round);
+    const int64_t total = (int64_t)p.n_items * p.pairs_per_tile;
+    if (idx >= total) return false;
+    const int item = (int)(idx / p.pairs_per_tile);
+    const int pair = (int)(idx - (int64_t)item * p.pairs_per_tile);
+    u.it = p.items[item];
+    u.head0 = 2 * pair;
+    u.kv_head = u.head0 / p.group;
+    return true;
+}
+
+// ------------------------------------------------------------------------------------------
+// Roles
+// ------------------------------------------------------------------------------------------
+__device__ void producer_role(const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV, const AttnParams& p,
+                              uint32_t smem_base, volatile uint32_t* abort_flag) {
+    const int lane = threadIdx.x & 31;
+    const uint32_t bars = smem_base + kSmemBar;
+    uint32_t kv_it = 0;   // ring slots filled so far
+    for (int round = 0;; ++round) {
+        UnitInfo u;
+        if (!fetch_unit(p, round, u)) break;
+        int ok = 1;
+        if (lane == 0) {
+            ok = mbar_wait(bars, kBarQEmpty, (round & 1) ^ 1, abort_flag, p.status, round);
+            if (ok) {
+                const uint32_t qbar = bars + kBarQFull * 8;
+                mbar_expect_tx(qbar, 2 * kTileBytes);
+                for (int h = 0; h < 2; ++h)
+                    for (int half = 0; half < 2; ++half)
+                        tma_load_3d(smem_base + kSmemQ + h * kTileBytes + half * kHalfBytes, tmQ, qbar, half * 64,
+                                    u.head0 + h, u.it.q_row0);
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) return;
+        const int n_tiles = u.it.n_kv_tiles;
+        for (int j0 = 0; j0 < n_tiles; j0 += 16) {
+            // the warp fetches the page ids of 16 KV tiles (32 pages) at once
+            const int pg = 2 * j0 + lane;
+            const int my_page = (pg < u.it.n_pages) ? __ldg(p.page_table + u.it.pt_base + pg) : p.oob_page;
+            const int jn = min(16, n_tiles - j0);
+            for (int jj = 0; jj < jn; ++jj) {
+                const int page_a = __shfl_sync(0xffffffffu, my_page, 2 * jj);
+                const int page_b = __shfl_sync(0xffffffffu, my_page, 2 * jj + 1);
+                for (int kv = 0; kv < 2; ++kv) {
+                    if (lane == 0) {
+                        const uint32_t slot = kv_it % kKvStages;
+                        ok = mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j0 + jj);
+                        if (ok) {
+                            const uint32_t fbar = bars + (kBarKvFull + slot) * 8;
+                            const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
+                            const CUtensorMap* map = kv ? tmV : tmK;
+                            mbar_expect_tx(fbar, kTileBytes);
+                            for (int half = 0; half < 2; ++half) {
+                                tma_load_4d(dst + half * kHalfBytes, map, fbar, half * 64, u.kv_head, 0, page_a);
+                                tma_load_4d(dst + half * kHalfBytes + kPageBoxBytes, map, fbar, half * 64, u.kv_head, 0, page_b);
+                            }
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) return;
+                    ++kv_it;
+                }
+            }
+        }
+    }
+}
+
+__device__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base, volatile uint32_t* abort_flag) {
+    const uint32_t bars = smem_base + kSmemBar;
+    uint32_t kv_it = 0;        // ring slots consumed so far
+    uint32_t tile_cnt = 0;     // KV tiles processed so far (phase of s_ready / p_ready)
+    const uint32_t q_addr = smem_base + kSmemQ;
+
+    auto issue_s = [&](int wg, uint32_t k_addr) {
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks) {
+            const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+            mma_ss(tmem_base + kTmemS + wg * 128, make_desc(q_addr + wg * kTileBytes + off, 16, 1024),
+                   make_desc(k_addr + off, 16, 1024), kIdescS, ks > 0);
+        }
+    };
+    auto issue_pv = [&](int wg, uint32_t v_addr, bool accumulate) {
+#pragma unroll
+        for (int ks = 0; ks < kBlockN / 16; ++ks)
+            mma_ts(tmem_base + kTmemO + wg * 128, tmem_base + kTmemS + wg * 128 + ks * 8,
+                   make_desc(v_addr + ks * 2048, kHalfBytes, 1024), kIdescPV, accumulate || ks > 0);
+    };
+#define MMA_WAIT(id, parity, it) if (!mbar_wait(bars, (id), (parity), abort_flag, p.status, (it))) return
+
+    for (int round = 0;; ++round) {
+        UnitInfo u;
+        if (!fetch_unit(p, round, u)) break;
+        const int n = u.it.n_kv_tiles;
+        MMA_WAIT(kBarQFull, round & 1, round);
+        // S(0) for both heads
+        uint32_t slot = kv_it % kKvStages;
+        MMA_WAIT(kBarKvFull + slot, (kv_it / kKvStages) & 1, 0);
+        tc_fence_after();
+        uint32_t k_addr = smem_base + kSmemKV + slot * kTileBytes;
+        issue_s(0, k_addr);
+        tc_commit(bars + (kBarSReady + 0) * 8);
+        issue_s(1, k_addr);
+        tc_commit(bars + (kBarSReady + 1) * 8);
+        tc_commit(bars + (kBarKvEmpty + slot) * 8);
+        if (n == 1) tc_commit(bars + kBarQEmpty * 8);
+        ++kv_it;
+        for (int j = 0; j < n; ++j) {
+            const uint32_t v_slot = kv_it % kKvStages;
+            const uint32_t v_par = (kv_it / kKvStages) & 1;
+            ++kv_it;
+            const uint32_t v_addr = smem_base + kSmemKV + v_slot * kTileBytes;
+            const bool more = (j + 1 < n);
+            uint32_t k_slot = 0;
+            if (more) {
+                k_slot = kv_it % kKvStages;
+                k_addr = smem_base + kSmemKV + k_slot * kTileBytes;
+            }
+            // head 0: O0 (+)= P0 V(j); then S0(j+1)
+            MMA_WAIT(kBarPReady + 0, tile_cnt & 1, j);
+            if (j == 0 && round > 0) MMA_WAIT(kBarOFree + 0, (round - 1) & 1, j);
+            MMA_WAIT(kBarKvFull + v_slot, v_par, j);
+            tc_fence_after();
+            issue_pv(0, v_addr, j > 0);
+            if (!more) tc_commit(bars + (kBarODone + 0) * 8);
+            if (more) {
+                MMA_WAIT(kBarKvFull + k_slot, (kv_it / kKvStages) & 1, j);
+                tc_fence_after();
+                issue_s(0, k_addr);
+                tc_commit(bars + (kBarSReady + 0) * 8);
+            }
+            // head 1
+            MMA_WAIT(kBarPReady + 1, tile_cnt & 1, j);
+            if (j == 0 && round > 0) MMA_WAIT(kBarOFree + 1, (round - 1) & 1, j);
+            tc_fence_after();
+            issue_pv(1, v_addr, j > 0);
+            if (!more) tc_commit(bars + (kBarODone + 1) * 8);
+            tc_commit(bars + (kBarKvEmpty + v_slot) * 8);
+            if (more) {
+                issue_s(1, k_addr);
+                tc_commit(bars + (kBarSReady + 1) * 8);
+                tc_commit(bars + (kBarKvEmpty + k_slot) * 8);
+                if (j + 2 == n) tc_commit(bars + kBarQEmpty * 8);
+                ++kv_it;
+            }
+            ++tile_cnt;
+        }
+    }
+#undef MMA_WAIT
+}
+
+__device__ void softmax_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base, volatile uint32_t* abort_flag,
+                             int wg) {
+    const uint32_t bars = smem_base + kSmemBar;
+    const int lane = threadIdx.x & 31;
+    const int warp_in_wg = (threadIdx.x >> 5) & 3;
+    const int row = warp_in_wg * 32 + lane;                        // query row of the tile == TMEM lane
+    const uint32_t lane_addr = (uint32_t)(warp_in_wg * 32) << 16;   // TMEM lane field of this warp
+    const uint32_t s_tmem = tmem_base + lane_addr + kTmemS + wg * 128;
+    const uint32_t o_tmem = tmem_base + lane_addr + kTmemO + wg * 128;
+    const float c = p.scale_log2;
+    uint32_t tile_cnt = 0;
+
+#define SM_WAIT(id, parity, it)                                                                  \
+    {                                                                                            \
+        int ok_ = mbar_wait(bars, (id), (parity), abort_flag, p.status, (it));                   \
+        if (!__all_sync(0xffffffffu, ok_)) return;                                               \
+    }
+
+    for (int round = 0;; ++round) {
+        UnitInfo u;
+        if (!fetch_unit(p, round, u)) break;
+        const int n = u.it.n_kv_tiles;
+        const int head = u.head0 + wg;
+        float m = -INFINITY;   // running row max in log2 units (possibly stale by < threshold)
+        float l = 0.f;         // running row sum of 2^(s - m)
+        for (int j = 0; j < n; ++j) {
+            SM_WAIT(kBarSReady + wg, tile_cnt & 1, j);
+            ++tile_cnt;
+            tc_fence_after();
+            float s[128];
+            TMEM_LD32(s_tmem + 0, s, 0);
+            TMEM_LD32(s_tmem + 32, s, 32);
+            TMEM_LD32(s_tmem + 64, s, 64);
+            TMEM_LD32(s_tmem + 96, s, 96);
+            tc_wait_ld();
+            // causal mask: row sees keys < kv_len0 + row; only tiles that reach past kv_len0 need it
+            if ((j + 1) * kBlockN > u.it.kv_len0) {
+                const int lim = u.it.kv_len0 + row - j * kBlockN;
+#pragma unroll
+                for (int i = 0; i < 128; ++i)
+                    if (i >= lim) s[i] = -INFINITY;
+            }
+            float mx = s[0];
+#pragma unroll
+            for (int i = 1; i < 128; ++i) mx = fmaxf(mx, s[i]);
+            const float m_new = fmaxf(m, mx * c);
+            if (j == 0) {
+                m = m_new;     // O is overwritten by the first P*V: nothing to rescale
+            } else {
+                const bool grow = (m_new - m) > kRescaleThreshold;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float m_upd = grow ? m_new : m;
+                    const float alpha = ex2(m - m_upd);
+                    l *= alpha;
+                    m = m_upd;
+                    // P*V(j-1) finished before S(j) was signalled (the pipe runs in issue order)
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        float o[32];
+                        TMEM_LD32(o_tmem + cc * 32, o, 0);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] *= alpha;
+                        TMEM_ST32F(o_tmem + cc * 32, o, 0);
+                    }
+                }
+            }
+            const float neg_m = -m;
+            uint32_t pk[64];
+            float sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < 64; ++i) {
+                const float p0 = ex2(fmaf(s[2 * i], c, neg_m));
+                const float p1 = ex2(fmaf(s[2 * i + 1], c, neg_m));
+                sum += p0 + p1;
+                pk[i] = pack_bf16(p0, p1);
+            }
+            l += sum;
+            TMEM_ST32R(s_tmem + 0, pk, 0);
+            TMEM_ST32R(s_tmem + 32, pk, 32);
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(bars + (kBarPReady + wg) * 8);
+        }
+        // epilogue: O / l -> global at the row's original position; LSE in natural log
+        SM_WAIT(kBarODone + wg, round & 1, n);
+        tc_fence_after();
+        const float inv_l = 1.f / l;
+        const bool valid = row < u.it.n_rows;
+        const int64_t grow_idx = (int64_t)u.it.q_row0 + row;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+            float o[32];
+            TMEM_LD32(o_tmem + cc * 32, o, 0);
+            tc_wait_ld();
+            if (valid) {
+                if (p.out_f32) {
+                    float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) +
+                                                            (grow_idx * p.Hq + head) * kD + cc * 32);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        dst[i] = make_float4(o[4 * i] * inv_l, o[4 * i + 1] * inv_l, o[4 * i + 2] * inv_l, o[4 * i + 3] * inv_l);
+                } else {
+                    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) +
+                                                          (grow_idx * p.Hq + head) * kD + cc * 32);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 v;
+                        v.x = pack_bf16(o[8 * i + 0] * inv_l, o[8 * i + 1] * inv_l);
+                        v.y = pack_bf16(o[8 * i + 2] * inv_l, o[8 * i + 3] * inv_l);
+                        v.z = pack_bf16(o[8 * i + 4] * inv_l, o[8 * i + 5] * inv_l);
+                        v.w = pack_bf16(o[8 * i + 6] * inv_l, o[8 * i + 7] * inv_l);
+                        dst[i] = v;
+                    }
+                }
+            }
+        }
+        if (valid) p.lse[(int64_t)head * p.lse_stride + grow_idx] = (m + lg2(l)) * 0.6931471805599453f;
+        tc_fence_before();
+        mbar_arrive(bars + (kBarOFree + wg) * 8);
+    }
+#undef SM_WAIT
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+               const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    volatile uint32_t* tmem_ptr = reinterpret_cast<volatile uint32_t*>(smem_gen + kSmemTmemPtr);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_gen + kSmemAbort);
+    const int warp = threadIdx.x >> 5;
+    const uint32_t bars = smem_base + kSmemBar;
+
+    if (threadIdx.x == 0) {
+        mbar_init(bars + kBarQFull * 8, 1);
+        mbar_init(bars + kBarQEmpty * 8, 1);
+        for (int s = 0; s < kKvStages; ++s) {
+            mbar_init(bars + (kBarKvFull + s) * 8, 1);
+            mbar_init(bars + (kBarKvEmpty + s) * 8, 1);
+        }
+        for (int w = 0; w < 2; ++w) {
+            mbar_init(bars + (kBarSReady + w) * 8, 1);
+            mbar_init(bars + (kBarPReady + w) * 8, 128);
+            mbar_init(bars + (kBarODone + w) * 8, 1);
+            mbar_init(bars + (kBarOFree + w) * 8, 128);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_base + kSmemTmemPtr), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_ptr;
+
+    if (warp < 4) {
+        softmax_role(p, smem_base, tmem_base, abort_flag, 0);
+    } else if (warp < 8) {
+        softmax_role(p, smem_base, tmem_base, abort_flag, 1);
+    } else if (warp == 8) {
+        producer_role(&tmQ, &tmK, &tmV, p, smem_base, abort_flag);
+    } else if (threadIdx.x == 9 * 32) {
+        mma_role(p, smem_base, tmem_base, abort_flag);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies that are still in flight time to land before shared memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+__global__ void fill_neg_inf_kernel(float* p, int64_t n) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        p[i] = -INFINITY;
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------
+int encode_maps(cp_ctx* ctx, const void* q, int64_t total_rows, int32_t Hq, const cp_kv_cache* c, CUtensorMap* tmQ,
+                CUtensorMap* tmK, CUtensorMap* tmV) {
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)Hq, (cuuint64_t)total_rows};
+        cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)Hq * kD * 2};
+        cuuint32_t box[3] = {64, 1, (cuuint32_t)kBlockM};
+        cuuint32_t es[3] = {1, 1, 1};
+        CUresult r = ctx->encode_tiled(tmQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box,
+                                       es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return set_error(CP_ERR_CUDA, "cuTensorMapEncodeTiled(q) failed with %d", (int)r);
+    }
+    for (int kv = 0; kv < 2; ++kv) {
+        cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)c->Hkv, (cuuint64_t)c->page_size, (cuuint64_t)c->num_pages};
+        cuuint64_t strides[3] = {(cuuint64_t)c->stride_head * 2, (cuuint64_t)c->stride_tok * 2,
+                                 (cuuint64_t)c->stride_page * 2};
+        cuuint32_t box[4] = {64, 1, 64, 1};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        CUresult r = ctx->encode_tiled(kv ? tmV : tmK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+                                       const_cast<void*>(kv ? c->v : c->k), dims, strides, box, es,
+                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return set_error(CP_ERR_CUDA, "cuTensorMapEncodeTiled(%s) failed with %d", kv ? "v" : "k", (int)r);
+    }
+    return CP_OK;
+}
+
+// Copies the tile list into the workspace through one of the context's two pinned staging buffers
+// (falls back to a pageable copy for lists that do not fit).
+int upload_tiles(cp_ctx* ctx, const std::vector<TileItem>& tiles, void* workspace, cudaStream_t s) {
+    const size_t bytes = tiles.size() * sizeof(TileItem);
+    uint8_t* dst = static_cast<uint8_t*>(workspace) + kWorkspaceHeader;
+    if (bytes > ctx->stage_bytes)
+        return check_cuda(cudaMemcpyAsync(dst, tiles.data(), bytes, cudaMemcpyHostToDevice, s), "tile list copy");
+    const int i = ctx->stage_next;
+    ctx->stage_next ^= 1;
+    if (ctx->stage_used[i])
+        if (int rc = check_cuda(cudaEventSynchronize(ctx->stage_event[i]), "cudaEventSynchronize(stage)")) return rc;
+    memcpy(ctx->h_stage[i], tiles.data(), bytes);
+    if (int rc = check_cuda(cudaMemcpyAsync(dst, ctx->h_stage[i], bytes, cudaMemcpyHostToDevice, s), "tile list copy"))
+        return rc;
+    ctx->stage_used[i] = true;
+    return check_cuda(cudaEventRecord(ctx->stage_event[i], s), "cudaEventRecord(stage)");
+}
+
+int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table, int32_t B,
+                const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C, const int64_t* cu_pages,
+                int32_t only_shard, int32_t Hq, float scale, void* out, int out_f32, float* lse, void* workspace,
+                size_t workspace_bytes, void* stream, const char* who) {
+    if (!ctx || !q || !page_table || !out || !lse || B < 1 || !cu_new || !prefix_len || !C || !cu_pages)
+        return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or B < 1", who);
+    if (int rc = validate_kv_cache(cache, who)) return rc;
+    if (Hq < 1 || Hq % cache->Hkv != 0)
+        return set_error(CP_ERR_INVALID_ARG, "%s: Hq=%d is not a multiple of Hkv=%d", who, Hq, cache->Hkv);
+    if ((Hq / cache->Hkv) % 2 != 0)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: Hq/Hkv=%d must be even (two query heads share each K/V tile)", who,
+                         Hq / cache->Hkv);
+    if (!(scale > 0.f)) return set_error(CP_ERR_INVALID_ARG, "%s: scale must be positive", who);
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return set_error(CP_ERR_INVALID_ARG, "%s: q and out must be 16-byte aligned", who);
+    if (cu_new[0] != 0 || cu_pages[0] != 0) return set_error(CP_ERR_INVALID_ARG, "%s: cu_new[0] and cu_pages[0] must be 0", who);
+    std::vector<int64_t> new_len(B);
+    for (int32_t b = 0; b < B; ++b) {
+        new_len[b] = cu_new[b + 1] - cu_new[b];
+        if (new_len[b] < 1 || prefix_len[b] < 0 || C[b] < 1)
+            return set_error(CP_ERR_INVALID_ARG, "%s: request %d has new_len=%lld prefix_len=%lld C=%d", who, b,
+                             (long long)new_len[b], (long long)prefix_len[b], C[b]);
+        const int64_t need = (prefix_len[b] + new_len[b] + cache->page_size - 1) / cache->page_size;
+        if (cu_pages[b + 1] - cu_pages[b] < need)
+            return set_error(CP_ERR_BOUNDS, "%s: request %d needs %lld page-table entries, has %lld", who, b,
+                             (long long)need, (long long)(cu_pages[b + 1] - cu_pages[b]));
+        if (prefix_len[b] + new_len[b] > 0x7fffff00ll)
+            return set_error(CP_ERR_UNSUPPORTED, "%s: request %d is longer than 2^31 tokens", who, b);
+    }
+    if (cu_new[B] > 0x7fffff00ll || cu_pages[B] > 0x7fffff00ll)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: more than 2^31 packed rows or pages", who);
+    const size_t need_ws = cp_workspace_bytes(B, new_len.data(), C);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need_ws)
+        return set_error(CP_ERR_WORKSPACE, "%s: workspace %p of %zu bytes; need %zu bytes, 256-byte aligned", who,
+                         workspace, workspace_bytes, need_ws);
+
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+    std::vector<TileItem> tiles;
+    build_tiles(B, cu_new, prefix_len, C, cu_pages, only_shard, tiles);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (tiles.empty()) return CP_OK;   // the shard owns no rows (only empty chunks)
+
+    CUtensorMap tmQ, tmK, tmV;
+    if (int rc = encode_maps(ctx, q, cu_new[B], Hq, cache, &tmQ, &tmK, &tmV)) return rc;
+    if (int rc = upload_tiles(ctx, tiles, workspace, s)) return rc;
+    if (!ctx->attn_attr_set) {
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
+        ctx->attn_attr_set = true;
+    }
+    AttnParams p;
+    p.items = reinterpret_cast<const TileItem*>(static_cast<uint8_t*>(workspace) + kWorkspaceHeader);
+    p.n_items = (int32_t)tiles.size();
+    p.pairs_per_tile = Hq / 2;
+    p.group = Hq / cache->Hkv;
+    p.Hq = Hq;
+    p.page_table = page_table;
+    p.oob_page = (int32_t)std::min<int64_t>(cache->num_pages, 0x7fffffff);
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.out = out;
+    p.out_f32 = out_f32;
+    p.lse = lse;
+    p.lse_stride = cu_new[B];
+    p.status = ctx->d_status;
+    const int64_t units = (int64_t)tiles.size() * p.pairs_per_tile;
+    const int grid = (int)std::min<int64_t>(units, ctx->num_sms);
+    cp_attn_kernel<<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
+    return check_cuda(cudaGetLastError(), who);
+}
+
+}  // namespace
+
+extern "C" int cp_prefill_attn_batch(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
+                                     int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
+                                     const int64_t* cu_pages, int32_t Hq, float scale, void* out, float* lse,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
+    return attn_common(ctx, q, cache, page_table, B, cu_new, prefix_len, C, cu_pages, -1, Hq, scale, out, 0, lse,
+                       workspace, workspace_bytes, stream, "cp_prefill_attn_batch");
+}
+
+extern "C" int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
+                               int64_t prefix_len, int64_t new_len, int32_t C, int32_t Hq, float scale, void* out,
+                               float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!cache || new_len < 1 || prefix_len < 0)
+        return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn: cache is NULL, new_len < 1 or prefix_len < 0");
+    const int64_t cu_new[2] = {0, new_len};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
+    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, Hq, scale, out, 0, lse,
+                       workspace, workspace_bytes, stream, "cp_prefill_attn");
+}
+
+extern "C" int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
+                                     int64_t prefix_len, int64_t new_len, int32_t C, int32_t shard, int32_t Hq,
+                                     float scale, float* partial_out, float* partial_lse, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+    if (!cache || new_len < 1 || prefix_len < 0 || C < 1 || shard < 0 || shard >= C || !partial_out || !partial_lse || Hq < 1)
+        return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_shard: bad sizes or shard %d not in [0, %d)", shard, C);
+    if (!ctx) return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_shard: ctx is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+    // rows the shard does not own: zeros with lse = -inf (the identity element of cp_merge)
+    if (int rc = check_cuda(cudaMemsetAsync(partial_out, 0, (size_t)new_len * Hq * kD * sizeof(float), s),
+                            "cudaMemsetAsync(partial_out)")) return rc;
+    const int64_t n_lse = new_len * Hq;
+    fill_neg_inf_kernel<<<(int)std::min<int64_t>((n_lse + 255) / 256, 4096), 256, 0, s>>>(partial_lse, n_lse);
+    if (int rc = check_cuda(cudaGetLastError(), "fill_neg_inf launch")) return rc;
+    const int64_t cu_new[2] = {0, new_len};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
+    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, Hq, scale, partial_out, 1,
+                       partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_shard");
+}

@@ -1,0 +1,62 @@
+// Internal declarations shared by the translation units of libcpattn (not part of the ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "cpattn.h"
+
+namespace cpattn {
+
+// One query tile of the persistent scheduler: up to 128 consecutive new tokens of one chunk of
+// one request.  Every tile is processed once per pair of query heads.
+struct TileItem {
+    int32_t q_row0;     // first row in the packed q / out tensors
+    int32_t n_rows;     // 1..128
+    int32_t kv_len0;    // keys visible to the first row: P + r0 + 1 (row i sees kv_len0 + i)
+    int32_t pt_base;    // offset of the request's page table in the packed page table
+    int32_t n_pages;    // entries of that page table
+    int32_t n_kv_tiles; // ceil((kv_len0 + n_rows - 1) / 128)
+    int32_t request;
+    int32_t shard;
+};
+static_assert(sizeof(TileItem) == 32, "TileItem layout");
+
+constexpr size_t kWorkspaceHeader = 256;
+constexpr int kTileRows = 128;
+constexpr int kStatusWords = 4;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+int set_error(int code, const char* fmt, ...);
+int check_cuda(cudaError_t e, const char* what);
+
+// Host planner pieces (plan.cpp)
+int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C);
+// Builds the tile list of a batch, cut at the chunk boundaries of every request's zigzag plan and
+// sorted longest first.  only_shard < 0 keeps all shards.
+int validate_kv_cache(const cp_kv_cache* c, const char* who);
+int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
+                const int64_t* cu_pages, int32_t only_shard, std::vector<TileItem>& out);
+
+}  // namespace cpattn
+
+struct cp_ctx {
+    int device;
+    int num_sms;
+    int32_t* d_status;                 // kStatusWords int32 on the device
+    int32_t* h_status;                 // pinned mirror
+    void* h_stage[2];                  // pinned staging buffers for tile lists
+    size_t stage_bytes;
+    cudaEvent_t stage_event[2];
+    bool stage_used[2];
+    int stage_next;
+    cpattn::EncodeTiledFn encode_tiled;
+    bool attn_attr_set;
+};

@@ -1,0 +1,85 @@
+// cp_kv_gather / cp_kv_append: bit-exact copies between a paged KV cache and contiguous rows,
+// addressed through the page table.  One 16-byte vector per thread; HBM-bound.
+#include <algorithm>
+
+#include "internal.h"
+
+using namespace cpattn;
+
+namespace {
+
+// kToPaged = false: paged -> rows (gather); true: rows -> paged (append).
+template <bool kToPaged>
+__global__ void __launch_bounds__(256)
+kv_copy_kernel(uint4* __restrict__ paged_k, uint4* __restrict__ paged_v, uint4* __restrict__ rows_k,
+               uint4* __restrict__ rows_v, const int32_t* __restrict__ page_table, int64_t t_begin, int64_t n,
+               int page_size, int Hkv, int vec_per_head, int64_t stride_page8, int64_t stride_tok8,
+               int64_t stride_head8) {
+    const int vec_per_tok = Hkv * vec_per_head;
+    const int64_t total = n * vec_per_tok;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t tok = i / vec_per_tok;
+        const int rem = (int)(i - tok * vec_per_tok);
+        const int g = rem / vec_per_head;
+        const int c = rem - g * vec_per_head;
+        const int64_t t = t_begin + tok;
+        const int64_t off = (int64_t)page_table[t / page_size] * stride_page8 + (t % page_size) * stride_tok8 +
+                            (int64_t)g * stride_head8 + c;
+        if (kToPaged) {
+            if (rows_k) paged_k[off] = rows_k[i];
+            if (rows_v) paged_v[off] = rows_v[i];
+        } else {
+            if (rows_k) rows_k[i] = paged_k[off];
+            if (rows_v) rows_v[i] = paged_v[off];
+        }
+    }
+}
+
+int validate_cache(const cp_kv_cache* c, const char* who) {
+    if (!c || !c->k || !c->v || c->num_pages < 1 || c->Hkv < 1)
+        return set_error(CP_ERR_INVALID_ARG, "%s: cache is NULL or has null / non-positive fields", who);
+    if (c->page_size != 64 || c->D != 128)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: page_size=%d D=%d, only 64 / 128 are supported", who, c->page_size,
+                         c->D);
+    if ((c->stride_page | c->stride_tok | c->stride_head) & 7 || c->stride_page < 1 || c->stride_tok < 1 ||
+        c->stride_head < 1)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: strides must be positive multiples of 8 elements", who);
+    if (((uintptr_t)c->k | (uintptr_t)c->v) & 15)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: k and v must be 16-byte aligned", who);
+    return CP_OK;
+}
+
+template <bool kToPaged>
+int kv_copy(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin, int64_t n,
+            const void* k_rows, const void* v_rows, void* stream, const char* who) {
+    if (!ctx || !page_table || t_begin < 0 || n < 0)
+        return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or negative range", who);
+    if (int rc = validate_cache(cache, who)) return rc;
+    if (!k_rows && !v_rows) return set_error(CP_ERR_INVALID_ARG, "%s: both row pointers are NULL", who);
+    if (((uintptr_t)k_rows | (uintptr_t)v_rows) & 15)
+        return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
+    if (n == 0) return CP_OK;
+    const int vec_per_head = cache->D / 8;
+    const int64_t total = n * cache->Hkv * vec_per_head;
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
+    kv_copy_kernel<kToPaged><<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        (uint4*)cache->k, (uint4*)cache->v, (uint4*)k_rows, (uint4*)v_rows, page_table, t_begin, n, cache->page_size,
+        cache->Hkv, vec_per_head, cache->stride_page / 8, cache->stride_tok / 8, cache->stride_head / 8);
+    return check_cuda(cudaGetLastError(), who);
+}
+
+}  // namespace
+
+namespace cpattn {
+int validate_kv_cache(const cp_kv_cache* c, const char* who) { return validate_cache(c, who); }
+}
+
+extern "C" int cp_kv_gather(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin,
+                            int64_t n, void* k_rows, void* v_rows, void* stream) {
+    return kv_copy<false>(ctx, cache, page_table, t_begin, n, k_rows, v_rows, stream, "cp_kv_gather");
+}
+
+extern "C" int cp_kv_append(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin,
+                            int64_t n, const void* k_rows, const void* v_rows, void* stream) {
+    return kv_copy<true>(ctx, cache, page_table, t_begin, n, k_rows, v_rows, stream, "cp_kv_append");
+}

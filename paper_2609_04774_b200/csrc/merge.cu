@@ -1,0 +1,120 @@
+// cp_merge: N-way log-sum-exp combination of partial attention results.  HBM-bound streaming
+// kernel: one warp per (token, head) row of 128 floats, each lane owning one float4 of the row.
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "internal.h"
+
+using namespace cpattn;
+
+namespace {
+
+constexpr int kMergeD = 128;
+constexpr int kTokPerCta = 8;    // tokens per CTA: 8 consecutive lse floats = one 32-byte sector
+constexpr int kHeadsPerWarp = 4; // consecutive heads (2 KB of every partial) handled by one warp
+constexpr int kMergeThreads = 32 * kTokPerCta;
+
+__device__ __forceinline__ float4 ld_stream(const float4* p) {
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+
+// Grid: x = ceil(H / kHeadsPerWarp), y = ceil(T / kTokPerCta).  Warp w of the CTA handles token
+// y*8 + w and heads x*4 .. x*4+3.  NMAX > 0: N <= NMAX, loop fully unrolled with the loads of all
+// partials in flight before the first use.
+template <int NMAX, bool kOutBf16>
+__global__ void __launch_bounds__(kMergeThreads)
+merge_kernel(const float* __restrict__ partials, const float* __restrict__ lses, int N, int64_t T, int H,
+             void* __restrict__ out, float* __restrict__ lse_out) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int64_t t = (int64_t)blockIdx.y * kTokPerCta + warp;
+    const int h0 = blockIdx.x * kHeadsPerWarp;
+    if (t >= T) return;
+    const int64_t row_stride4 = kMergeD / 4;                          // float4 per row
+    const int64_t part_stride4 = T * (int64_t)H * row_stride4;        // float4 per partial
+    const float4* src = reinterpret_cast<const float4*>(partials) + (t * H + h0) * row_stride4 + lane;
+
+#pragma unroll
+    for (int hh = 0; hh < kHeadsPerWarp; ++hh) {
+        const int h = h0 + hh;
+        if (h >= H) break;
+        // lane n < N holds lse of partial n; max / sum by warp shuffles
+        float my = -INFINITY;
+        if (lane < N) my = lses[((int64_t)lane * H + h) * T + t];
+        float4 x[NMAX];
+#pragma unroll
+        for (int n = 0; n < NMAX; ++n)
+            if (n < N) x[n] = ld_stream(src + n * part_stride4 + hh * row_stride4);
+        float m = my;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        const bool dead = (m == -INFINITY);
+        const float w = (dead || my == -INFINITY) ? 0.f : __expf(my - m);
+        float ws = w;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
+        const float inv = dead ? 0.f : 1.f / ws;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int n = 0; n < NMAX; ++n) {
+            if (n < N) {
+                const float wn = __shfl_sync(0xffffffffu, w, n) * inv;
+                if (wn > 0.f) {   // a zero weight hides whatever the partial holds
+                    acc.x = fmaf(wn, x[n].x, acc.x);
+                    acc.y = fmaf(wn, x[n].y, acc.y);
+                    acc.z = fmaf(wn, x[n].z, acc.z);
+                    acc.w = fmaf(wn, x[n].w, acc.w);
+                }
+            }
+        }
+        const int64_t orow = (t * H + h) * kMergeD + lane * 4;
+        if (kOutBf16) {
+            __nv_bfloat162 a = __floats2bfloat162_rn(acc.x, acc.y);
+            __nv_bfloat162 b = __floats2bfloat162_rn(acc.z, acc.w);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&a);
+            pk.y = *reinterpret_cast<uint32_t*>(&b);
+            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + orow) = pk;
+        } else {
+            *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + orow) = acc;
+        }
+        if (lse_out != nullptr && lane == 0) lse_out[(int64_t)h * T + t] = dead ? -INFINITY : m + __logf(ws);
+    }
+}
+
+template <int NMAX>
+void launch_merge(const float* partials, const float* lses, int N, int64_t T, int H, void* out, int out_dtype,
+                  float* lse_out, cudaStream_t s) {
+    dim3 grid((H + kHeadsPerWarp - 1) / kHeadsPerWarp, (unsigned)((T + kTokPerCta - 1) / kTokPerCta));
+    if (out_dtype == CP_DTYPE_BF16)
+        merge_kernel<NMAX, true><<<grid, kMergeThreads, 0, s>>>(partials, lses, N, T, H, out, lse_out);
+    else
+        merge_kernel<NMAX, false><<<grid, kMergeThreads, 0, s>>>(partials, lses, N, T, H, out, lse_out);
+}
+
+}  // namespace
+
+extern "C" int cp_merge(cp_ctx* ctx, const float* partials, const float* lses, int32_t N, int64_t T, int32_t H,
+                        int32_t D, void* out, int32_t out_dtype, float* lse_out, void* stream) {
+    if (!ctx || !partials || !lses || !out || N < 1 || T < 1 || H < 1)
+        return set_error(CP_ERR_INVALID_ARG, "cp_merge: null pointer or non-positive size (N=%d T=%lld H=%d)", N,
+                         (long long)T, H);
+    if (D != kMergeD) return set_error(CP_ERR_UNSUPPORTED, "cp_merge: D=%d, only 128 is supported", D);
+    if (N > 32) return set_error(CP_ERR_UNSUPPORTED, "cp_merge: N=%d, at most 32 partials", N);
+    if (out_dtype != CP_DTYPE_BF16 && out_dtype != CP_DTYPE_F32)
+        return set_error(CP_ERR_INVALID_ARG, "cp_merge: out_dtype=%d", out_dtype);
+    if ((T + kTokPerCta - 1) / kTokPerCta > 65535 * 1024ll)
+        return set_error(CP_ERR_UNSUPPORTED, "cp_merge: T=%lld too large", (long long)T);
+    if (((uintptr_t)partials | (uintptr_t)out) & 15)
+        return set_error(CP_ERR_INVALID_ARG, "cp_merge: partials and out must be 16-byte aligned");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (N <= 2) launch_merge<2>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
+    else if (N <= 4) launch_merge<4>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
+    else if (N <= 8) launch_merge<8>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
+    else if (N <= 16) launch_merge<16>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
+    else launch_merge<32>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
+    return check_cuda(cudaGetLastError(), "cp_merge launch");
+}

@@ -1,0 +1,66 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, and the integer planner matches the oracle bit for bit."""
+import ctypes
+import itertools
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import reference as orc
+from paper_2609_04774_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load()
+
+
+def test_library_exports_every_declared_symbol(lib):
+    header = open(os.path.join(ROOT, "include", "cpattn.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(cp_[a-z_0-9]+)\s*\(", header))
+    assert declared, "no declarations found"
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_struct_layouts_match_header():
+    assert ctypes.sizeof(binding.cp_shard_plan) == 56
+    assert ctypes.sizeof(binding.cp_kv_cache) == 64
+
+
+def test_cp_plan_bit_exact_against_oracle(lib):
+    cases = list(itertools.product(list(range(1, 70)) + [127, 128, 129, 1000, 4096], [0, 1, 64, 12288], [1, 2, 3, 4, 5, 8]))
+    cases += [(1024, 0, 2), (4096, 12288, 4), (131072, 0, 8), (32768, 32768, 8), (65536, 64, 7)]
+    for R, P, C in cases:
+        assert binding.cp_plan(R, P, C) == orc.plan(R, P, C), (R, P, C)
+
+
+def test_cp_plan_rejects_bad_arguments(lib):
+    for args in [(0, 0, 1), (-3, 0, 2), (5, -1, 1), (5, 0, 0)]:
+        with pytest.raises(binding.CpError) as e:
+            binding.cp_plan(*args)
+        assert e.value.code == binding.CP_ERR_INVALID_ARG
+    assert b"cp_plan" in lib.cp_last_error()
+    assert lib.cp_strerror(-5) == b"CP_ERR_TIMEOUT"
+
+
+def test_workspace_bytes(lib):
+    assert binding.cp_workspace_bytes([1024], [2]) == 256 + 32 * (8 + 4)
+    assert binding.cp_workspace_bytes([5, 300], [4, 1]) == 256 + 32 * ((1 + 8) + (3 + 2))
+    assert binding.cp_workspace_bytes([0], [1]) == 0
+
+
+def test_gpu_calls_fail_cleanly_without_a_device(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    with pytest.raises(binding.CpError) as e:
+        binding.Context(0)
+    assert e.value.code in (binding.CP_ERR_CUDA, binding.CP_ERR_INVALID_ARG)

@@ -1,0 +1,221 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded
+inputs.  Planner and page indexing bit-exact; attention within max-abs 2e-2 / mean-abs 2e-3 and LSE
+within 1e-3; merge within fp32 round-off."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import reference as orc
+from paper_2609_04774_b200 import binding
+from paper_2609_04774_b200 import workloads as wl
+from tests.gpu_util import DeviceWorkload, bf16_to_f64, bits_to_bf16, compare
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    c.close()
+
+
+def oracle_request(mat, b, rows=None):
+    w = mat.wl
+    r = w.requests[b]
+    q = mat.q[w.cu_new[b]:w.cu_new[b + 1]]
+    pt = mat.page_table[w.cu_pages[b]:w.cu_pages[b + 1]]
+    if rows is None:
+        return orc.attn_full(q, mat.k_pages, mat.v_pages, pt, r.prefix_len, w.Hkv, w.scale)
+    return orc.attn_rows(q, mat.k_pages, mat.v_pages, pt, r.prefix_len, w.Hkv, w.scale, rows)
+
+
+def check_batch(ctx, w, pair_budget=3e8, seed_rows=123):
+    """Run the whole batch in one launch; compare every request (all rows when cheap, otherwise the
+    rows around every tile / chunk boundary plus seeded random rows)."""
+    mat = wl.materialize(w)
+    dev = DeviceWorkload(mat)
+    out, lse = dev.run_batch(ctx)
+    stats = []
+    for b, r in enumerate(w.requests):
+        lo, hi = int(w.cu_new[b]), int(w.cu_new[b + 1])
+        if r.new_len * (r.prefix_len + r.new_len / 2) * w.Hq <= pair_budget:
+            rows = np.arange(r.new_len)
+        else:
+            n = max(16, int(pair_budget / (w.Hq * (r.prefix_len + r.new_len / 2))))
+            cl = -(-r.new_len // (2 * r.C))
+            edges = [x for j in range(2 * r.C + 1) for x in (j * cl - 1, j * cl, j * cl + 127, j * cl + 128)]
+            rnd = wl.sample_rows(seed_rows + b, 1, r.new_len, n)[0]
+            rows = np.unique(np.clip(np.concatenate([edges, rnd, [0, r.new_len - 1]]), 0, r.new_len - 1))
+        ref_o, ref_l = oracle_request(mat, b, rows)
+        stats.append(compare(out[lo:hi][rows], lse[:, lo:hi][:, rows], ref_o, ref_l, "%s req %d" % (w.name, b)))
+    return dev, out, lse, stats
+
+
+def test_plan_matches_oracle_on_device_box():
+    for R, P, C in [(1024, 0, 2), (4096, 12288, 4), (131072, 0, 8), (32768, 32768, 8), (333, 192, 3)]:
+        assert binding.cp_plan(R, P, C) == orc.plan(R, P, C)
+
+
+def test_merge_parity(ctx):
+    for (N, T, H, dt) in [(2, 100, 5, torch.float32), (4, 37, 64, torch.bfloat16), (8, 64, 7, torch.float32),
+                          (3, 9, 1, torch.bfloat16), (1, 20, 4, torch.float32), (16, 33, 3, torch.float32)]:
+        parts, lses = wl.merge_inputs(6, N, T, H, 128, neg_inf_frac=5)
+        if N > 2:
+            lses[:, H - 1, 3] = -np.inf        # a row that is dead in every partial
+            parts[2, 5, 0] = np.nan            # junk behind a -inf lse must be ignored
+            lses[2, 0, 5] = -np.inf
+        ref_o, ref_l = orc.merge(parts, lses)
+        out = torch.empty((T, H, 128), dtype=dt, device="cuda")
+        lse_out = torch.empty((H, T), dtype=torch.float32, device="cuda")
+        binding.cp_merge(ctx, torch.from_numpy(parts).cuda(), torch.from_numpy(lses).cuda(), out, lse_out)
+        torch.cuda.synchronize()
+        o = out.float().cpu().numpy().astype(np.float64)
+        tol = 1e-5 if dt == torch.float32 else 2.0 ** -8
+        assert np.abs(o - ref_o).max() <= tol * max(1.0, np.abs(ref_o).max()), (N, T, H)
+        l = lse_out.cpu().numpy().astype(np.float64)
+        assert np.array_equal(np.isneginf(l), np.isneginf(ref_l))
+        fin = np.isfinite(ref_l)
+        assert np.abs(l[fin] - ref_l[fin]).max() <= 1e-5 * np.abs(ref_l[fin]).max()
+
+
+def test_kv_gather_append_bit_exact(ctx):
+    w = wl.small_mixed()
+    mat = wl.materialize(w)
+    k = bits_to_bf16(mat.k_pages)
+    v = bits_to_bf16(mat.v_pages)
+    cache = binding.make_cache(k, v)
+    b = 0
+    r = w.requests[b]
+    pt_host = mat.page_table[w.cu_pages[b]:w.cu_pages[b + 1]]
+    pt = torch.from_numpy(pt_host.copy()).cuda()
+    t0, n = 37, r.total_len - 37
+    kr = torch.zeros((n, w.Hkv, w.D), dtype=torch.bfloat16, device="cuda")
+    vr = torch.zeros_like(kr)
+    binding.cp_kv_gather(ctx, cache, pt, t0, n, kr, vr)
+    torch.cuda.synchronize()
+    assert np.array_equal(kr.view(torch.int16).cpu().numpy().view(np.uint16), orc.kv_gather(mat.k_pages, pt_host, t0, t0 + n))
+    assert np.array_equal(vr.view(torch.int16).cpu().numpy().view(np.uint16), orc.kv_gather(mat.v_pages, pt_host, t0, t0 + n))
+    # append new rows and compare the whole pool with the oracle's append
+    newk = wl.normal_bf16(5, wl.TID_K, (n, w.Hkv, w.D))
+    newv = wl.normal_bf16(5, wl.TID_V, (n, w.Hkv, w.D))
+    binding.cp_kv_append(ctx, cache, pt, t0, n, bits_to_bf16(newk), bits_to_bf16(newv))
+    torch.cuda.synchronize()
+    kp, vp = mat.k_pages.copy(), mat.v_pages.copy()
+    orc.kv_append(kp, pt_host, t0, newk)
+    orc.kv_append(vp, pt_host, t0, newv)
+    assert np.array_equal(k.view(torch.int16).cpu().numpy().view(np.uint16), kp)
+    assert np.array_equal(v.view(torch.int16).cpu().numpy().view(np.uint16), vp)
+
+
+def test_attention_small_mixed_batch(ctx):
+    dev, out, lse, _ = check_batch(ctx, wl.small_mixed())
+    # run-to-run bitwise determinism
+    o1 = dev.out.clone()
+    l1 = dev.lse.clone()
+    dev.run_batch(ctx)
+    assert torch.equal(o1.view(torch.int16), dev.out.view(torch.int16)) and torch.equal(l1, dev.lse)
+
+
+def test_attention_config1(ctx):
+    check_batch(ctx, wl.config1())
+
+
+def test_single_request_entry_point_and_c_invariance(ctx):
+    w = wl.Workload("one", 21, 8, 2, [wl.Request(517, 320, 1)])
+    mat = wl.materialize(w)
+    dev = DeviceWorkload(mat)
+    ref_o, ref_l = oracle_request(mat, 0)
+    ws = torch.zeros(binding.cp_workspace_bytes([517], [8]), dtype=torch.uint8, device="cuda")
+    outs = []
+    for C in (1, 2, 3, 8):
+        dev.out.fill_(float("nan"))
+        binding.cp_prefill_attn(ctx, dev.q, dev.cache, dev.page_table, 320, 517, C, w.Hq, w.scale, dev.out, dev.lse, ws)
+        torch.cuda.synchronize()
+        ctx.poll_status()
+        compare(bf16_to_f64(dev.out), dev.lse.cpu().numpy().astype(np.float64), ref_o, ref_l, "C=%d" % C)
+        outs.append(dev.out.clone())
+
+
+def test_shard_partials_merge_to_full(ctx):
+    w = wl.Workload("shards", 22, 8, 2, [wl.Request(700, 192, 3)])
+    r = w.requests[0]
+    mat = wl.materialize(w)
+    dev = DeviceWorkload(mat)
+    out_full, lse_full = dev.run_batch(ctx)
+    C = r.C
+    parts = torch.full((C, r.new_len, w.Hq, w.D), float("nan"), dtype=torch.float32, device="cuda")
+    lses = torch.full((C, w.Hq, r.new_len), float("nan"), dtype=torch.float32, device="cuda")
+    plan = orc.plan(r.new_len, r.prefix_len, C)
+    for k in range(C):
+        binding.cp_prefill_attn_shard(ctx, dev.q, dev.cache, dev.page_table, r.prefix_len, r.new_len, C, k, w.Hq,
+                                      w.scale, parts[k], lses[k], dev.ws)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    for k in range(C):
+        own = np.zeros(r.new_len, dtype=bool)
+        own[orc.shard_rows(plan[k])] = True
+        lk = lses[k].cpu().numpy()
+        assert np.isfinite(lk[:, own]).all() and np.isneginf(lk[:, ~own]).all()
+        assert (parts[k].cpu().numpy()[~own] == 0).all()
+    merged = torch.empty((r.new_len, w.Hq, w.D), dtype=torch.bfloat16, device="cuda")
+    mlse = torch.empty((w.Hq, r.new_len), dtype=torch.float32, device="cuda")
+    binding.cp_merge(ctx, parts, lses, merged, mlse)
+    torch.cuda.synchronize()
+    ref_o, ref_l = oracle_request(mat, 0)
+    compare(bf16_to_f64(merged), mlse.cpu().numpy().astype(np.float64), ref_o, ref_l, "merged shards")
+    assert np.abs(bf16_to_f64(merged) - out_full).max() <= 2.0 ** -7 * max(1.0, np.abs(out_full).max())
+
+
+def test_argument_validation_launches_nothing(ctx):
+    w = wl.Workload("val", 23, 8, 2, [wl.Request(64, 0, 1)])
+    dev = DeviceWorkload(wl.materialize(w))
+    small = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.CpError) as e:
+        binding.cp_prefill_attn(ctx, dev.q, dev.cache, dev.page_table, 0, 64, 1, w.Hq, w.scale, dev.out, dev.lse, small)
+    assert e.value.code == binding.CP_ERR_WORKSPACE
+    with pytest.raises(binding.CpError) as e:
+        binding.cp_prefill_attn(ctx, dev.q, dev.cache, dev.page_table, 0, 64, 1, 6, w.scale, dev.out, dev.lse, dev.ws)
+    assert e.value.code == binding.CP_ERR_UNSUPPORTED      # Hq/Hkv = 3 is odd
+    with pytest.raises(binding.CpError) as e:
+        binding.cp_prefill_attn(ctx, dev.q, dev.cache, dev.page_table, 0, 0, 1, w.Hq, w.scale, dev.out, dev.lse, dev.ws)
+    assert e.value.code == binding.CP_ERR_INVALID_ARG
+    bad = binding.make_cache(dev.k, dev.v)
+    bad.page_size = 32
+    with pytest.raises(binding.CpError) as e:
+        binding.cp_prefill_attn(ctx, dev.q, bad, dev.page_table, 0, 64, 1, w.Hq, w.scale, dev.out, dev.lse, dev.ws)
+    assert e.value.code == binding.CP_ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    assert torch.isnan(dev.out.float()).all()               # nothing was written
+
+
+def test_attention_config2_full(ctx):
+    check_batch(ctx, wl.config2(), pair_budget=1e11)
+
+
+def test_attention_config4_varlen(ctx):
+    check_batch(ctx, wl.config4(), pair_budget=1.5e8)
+
+
+def test_attention_config5_sampled(ctx):
+    check_batch(ctx, wl.config5(), pair_budget=1.2e9)
+
+
+def test_attention_config3_sampled(ctx):
+    # 512 seeded random rows for every head, compared exactly, plus chunk-boundary rows for all heads.
+    w = wl.config3()
+    mat = wl.materialize(w)
+    dev = DeviceWorkload(mat)
+    out, lse = dev.run_batch(ctx)
+    r = w.requests[0]
+    rows = wl.sample_rows(w.seed, w.Hq, r.new_len, 512)                       # [Hq, 512]
+    heads = np.repeat(np.arange(w.Hq, dtype=np.int32), 512)
+    ro, rl = orc.attn_pairs(mat.q, mat.k_pages, mat.v_pages, mat.page_table, 0, w.Hkv, w.scale, rows.reshape(-1), heads)
+    got_o = out[rows.reshape(-1), heads]
+    got_l = lse[heads, rows.reshape(-1)]
+    compare(got_o, got_l, ro, rl, "cfg3 sampled")
+    cl = r.new_len // (2 * r.C)
+    edge = np.unique(np.clip([x for j in range(2 * r.C + 1) for x in (j * cl - 1, j * cl)], 0, r.new_len - 1))
+    eo, el = orc.attn_rows(mat.q, mat.k_pages, mat.v_pages, mat.page_table, 0, w.Hkv, w.scale, edge[::3])
+    compare(out[edge[::3]], lse[:, edge[::3]], eo, el, "cfg3 chunk edges")
+    assert np.isfinite(lse).all() and np.isfinite(out).all()
