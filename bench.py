@@ -1,0 +1,508 @@
+#!/usr/bin/env python
+"""Benchmark of libcpattn's hot path: cache-aware causal prefill attention under zigzag CP.
+
+Default mode prints ONE JSON line for the headline workload (BASELINE config 2: Llama-3-8B-shaped
+layer, 12288 cached + 4096 new tokens, C=4, paged KV).  A step is one pass of the hot path over the
+batch: cp_plan (host) -> tile schedule -> one persistent attention launch over all C shards reading
+K/V through the page table and storing rows at their original positions.  `value` is measured with
+inputs resident in HBM; `e2e` goes through the same C-ABI calls from pinned HOST buffers (q, the new
+tokens' K/V rows appended into the paged cache, page table up; out and lse down).
+
+Other modes (`--mode merge|table|configs`) write the cp_merge sweep, the measured prefill-time
+table over (new_len, prefix_len, C) and the per-config numbers as JSON lines to `--out`.
+
+`--impl reference` times the CPU fp64 oracle (host cores) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_04774_b200 import workloads as wl  # noqa: E402
+
+METRIC = "causal_effective_prefill_attention_tflops"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def get_workload(cfg: int) -> wl.Workload:
+    return wl.CONFIGS[cfg]()
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks sampling during the timed region
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    smax.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------------------------
+# device-side runner
+# ----------------------------------------------------------------------------------------------
+class Runner:
+    """Holds device copies of one workload and runs steps through the C ABI."""
+
+    def __init__(self, w: wl.Workload, device: int, need_host: bool = False):
+        import torch
+        from paper_2609_04774_b200 import binding, build
+        build.build()
+        self.torch, self.binding, self.w = torch, binding, w
+        torch.cuda.set_device(device)
+        self.ctx = binding.Context(device)
+        mat = wl.materialize(w)
+        self.mat = mat
+
+        def dev(bits):
+            return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+        self.q, self.k, self.v = dev(mat.q), dev(mat.k_pages), dev(mat.v_pages)
+        self.page_table = torch.from_numpy(mat.page_table).cuda()
+        self.cache = binding.make_cache(self.k, self.v)
+        self.out = torch.empty((w.total_new, w.Hq, w.D), dtype=torch.bfloat16, device="cuda")
+        self.lse = torch.empty((w.Hq, w.total_new), dtype=torch.float32, device="cuda")
+        self.new_len = [r.new_len for r in w.requests]
+        self.prefix = [r.prefix_len for r in w.requests]
+        self.Cs = [r.C for r in w.requests]
+        self.ws = torch.zeros(binding.cp_workspace_bytes(self.new_len, self.Cs), dtype=torch.uint8, device="cuda")
+        self.cu_new, self.cu_pages = w.cu_new, w.cu_pages
+        if need_host:
+            self._host_buffers()
+
+    def _host_buffers(self):
+        """Pinned host copies of one step's inputs: q, the new tokens' K/V rows, the page table."""
+        torch, w, mat = self.torch, self.w, self.mat
+        self.h_q = torch.from_numpy(mat.q.view(np.int16)).view(torch.bfloat16).pin_memory()
+        newk, newv = [], []
+        for b, r in enumerate(w.requests):
+            pt = mat.page_table[w.cu_pages[b]:w.cu_pages[b + 1]]
+            idx = np.arange(r.prefix_len, r.total_len)
+            newk.append(mat.k_pages[pt[idx // wl.PAGE], idx % wl.PAGE])
+            newv.append(mat.v_pages[pt[idx // wl.PAGE], idx % wl.PAGE])
+        self.h_newk = torch.from_numpy(np.concatenate(newk).view(np.int16)).view(torch.bfloat16).pin_memory()
+        self.h_newv = torch.from_numpy(np.concatenate(newv).view(np.int16)).view(torch.bfloat16).pin_memory()
+        self.h_pt = torch.from_numpy(mat.page_table).pin_memory()
+        self.d_newk = torch.empty_like(self.h_newk, device="cuda")
+        self.d_newv = torch.empty_like(self.h_newv, device="cuda")
+        self.h_out = torch.empty(self.out.shape, dtype=torch.bfloat16).pin_memory()
+        self.h_lse = torch.empty(self.lse.shape, dtype=torch.float32).pin_memory()
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in (self.h_q, self.h_newk, self.h_newv, self.h_pt))
+        self.d2h_bytes = sum(t.numel() * t.element_size() for t in (self.h_out, self.h_lse))
+
+    def step(self):
+        """One pass of the hot path with device-resident inputs: plan + schedule + attention launch."""
+        b, w = self.binding, self.w
+        for r in w.requests:
+            b.cp_plan(r.new_len, r.prefix_len, r.C)
+        b.cp_prefill_attn_batch(self.ctx, self.q, self.cache, self.page_table, self.cu_new, self.prefix, self.Cs,
+                                self.cu_pages, w.Hq, w.scale, self.out, self.lse, self.ws)
+
+    def step_e2e(self):
+        """The same pass from host buffers: copies in, KV append through the page table, attention, copies out."""
+        b, w = self.binding, self.w
+        self.q.copy_(self.h_q, non_blocking=True)
+        self.page_table.copy_(self.h_pt, non_blocking=True)
+        self.d_newk.copy_(self.h_newk, non_blocking=True)
+        self.d_newv.copy_(self.h_newv, non_blocking=True)
+        row0 = 0
+        for i, r in enumerate(w.requests):
+            b.cp_plan(r.new_len, r.prefix_len, r.C)
+            pt = self.page_table[int(self.cu_pages[i]):int(self.cu_pages[i + 1])]
+            b.cp_kv_append(self.ctx, self.cache, pt, r.prefix_len, r.new_len, self.d_newk[row0:row0 + r.new_len],
+                           self.d_newv[row0:row0 + r.new_len])
+            row0 += r.new_len
+        b.cp_prefill_attn_batch(self.ctx, self.q, self.cache, self.page_table, self.cu_new, self.prefix, self.Cs,
+                                self.cu_pages, w.Hq, w.scale, self.out, self.lse, self.ws)
+        self.h_out.copy_(self.out, non_blocking=True)
+        self.h_lse.copy_(self.lse, non_blocking=True)
+
+    def launches_per_step(self, e2e=False):
+        return 1 + (len(self.w.requests) if e2e else 0)
+
+
+def timed_loop(torch, fn, steps, warmup, dist=None):
+    """W warm-up steps, then exactly `steps` steps between CUDA events; returns total ms and per-step ms list."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+        torch.cuda.synchronize()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    evs[0].record()
+    for i in range(steps):
+        fn()
+        evs[i + 1].record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+        torch.cuda.synchronize()
+    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+    return evs[0].elapsed_time(evs[steps]), per
+
+
+def kernel_only_ms(torch, runner, steps):
+    """Average duration of the attention launch alone: events recorded directly around each launch on the
+    launching stream, after the loop above has warmed everything up."""
+    w, b = runner.w, runner.binding
+    ds = []
+    for _ in range(steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        b.cp_prefill_attn_batch(runner.ctx, runner.q, runner.cache, runner.page_table, runner.cu_new, runner.prefix,
+                                runner.Cs, runner.cu_pages, w.Hq, w.scale, runner.out, runner.lse, runner.ws)
+        e1.record()
+        ds.append((e0, e1))
+    torch.cuda.synchronize()
+    return statistics.mean(a.elapsed_time(c) for a, c in ds)
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ----------------------------------------------------------------------------------------------
+def oracle_sample(w: wl.Workload, mat, rows_per_request: int, seed: int, threads=None):
+    """Time the oracle on `rows_per_request` seeded rows (all heads) of every request; returns
+    (seconds, visible pairs evaluated per query head summed over heads, threads used)."""
+    from oracle import reference as orc
+    threads = threads or orc.host_threads()
+    pairs = 0
+    t0 = time.perf_counter()
+    for b, r in enumerate(w.requests):
+        n = min(rows_per_request, r.new_len)
+        rows = np.unique(wl.sample_rows(seed + b, 1, r.new_len, n)[0])
+        q = mat.q[w.cu_new[b]:w.cu_new[b + 1]]
+        pt = mat.page_table[w.cu_pages[b]:w.cu_pages[b + 1]]
+        orc.attn_rows(q, mat.k_pages, mat.v_pages, pt, r.prefix_len, w.Hkv, w.scale, rows, n_threads=threads)
+        pairs += int((r.prefix_len + rows + 1).sum()) * w.Hq
+    return time.perf_counter() - t0, pairs, threads
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU oracle as it stands, one bounded sample of the workload per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import reference as orc
+    orc.build()
+    w = get_workload(args.config)
+    mat = wl.materialize(w)
+    rows = args.ref_rows
+    for i in range(args.warmup):
+        oracle_sample(w, mat, rows, 1000 + i)
+    tot_t, tot_pairs, threads = 0.0, 0, orc.host_threads()
+    for i in range(args.steps):
+        t, p, threads = oracle_sample(w, mat, rows, 2000 + i)
+        tot_t += t
+        tot_pairs += p
+    value = 4 * w.D * tot_pairs / tot_t / 1e12
+    sample = "%d seeded rows x %d heads per request per step (%d steps)" % (rows, w.Hq, args.steps)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / max(args.steps, 1), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "Hq": w.Hq, "Hkv": w.Hkv, "D": w.D, "seed": w.seed},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------
+# main (ours)
+# ----------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+    peaks = load_peaks()
+    w = get_workload(args.config)
+    runner = Runner(w, local, need_host=True)
+    flops = w.flops()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    total_ms, per = timed_loop(torch, runner.step, args.steps, args.warmup, dist)
+    e2e_ms, _ = timed_loop(torch, runner.step_e2e, max(3, args.steps // 4), 3, dist)
+    e2e_steps = max(3, args.steps // 4)
+    kern_ms = kernel_only_ms(torch, runner, min(args.steps, 50))
+    clocks = sampler.stop() if rank == 0 else None
+    runner.ctx.poll_status()
+
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = total_ms / args.steps
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    e2e_value = world * flops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    achieved = flops / (kern_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "requests": len(w.requests), "new_tokens": w.total_new, "Hq": w.Hq,
+                   "Hkv": w.Hkv, "D": w.D, "page_size": wl.PAGE, "seed": w.seed, "pairs": w.pairs(),
+                   "l2": "inputs (q+kv+out = %.0f MB) exceed the 126 MB L2; no flush between steps" %
+                         ((2 * w.total_new * w.Hq * w.D * 2 + 2 * sum(r.total_len for r in w.requests) * w.Hkv * w.D * 2) / 1e6),
+                   "multi_gpu": "independent replicas of the workload per rank, no collective"},
+        "tokens_per_s": world * w.total_new / (ms_per_step * 1e-3),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": runner.h2d_bytes,
+                "d2h_bytes_per_step": runner.d2h_bytes, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": args.steps * runner.launches_per_step(),
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak, "traffic": None, "kernel": "cp_attn_kernel",
+                     "kernel_ms": kern_ms, "peak_source": "%s burst bf16 (of %s)" % (peaks["_source"], peaks["_source"]),
+                     "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                     "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS},
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        from oracle import reference as orc
+        orc.build()
+        t, pairs, threads = oracle_sample(w, runner.mat, args.cpu_rows, 4242)
+        line["cpu_baseline"] = {"value": 4 * w.D * pairs / t / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": "%d seeded rows x %d heads per request (%.1f s)" % (args.cpu_rows, w.Hq, t)}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------------------------
+# extra modes: per-config numbers, merge sweep, prefill-time table
+# ----------------------------------------------------------------------------------------------
+def run_configs(args, out):
+    import torch
+    peaks = load_peaks()
+    for cfg in args.configs:
+        w = get_workload(cfg)
+        runner = Runner(w, 0)
+        steps = max(3, min(args.steps, int(2000 / max(1.0, w.flops() / 1e12))))
+        total_ms, per = timed_loop(torch, runner.step, steps, 3)
+        runner.ctx.poll_status()
+        ms = total_ms / steps
+        tf = w.flops() / (ms * 1e-3) / 1e12
+        out.write(json.dumps({"mode": "config", "config": cfg, "workload": w.name, "ms": ms, "ms_best": min(per),
+                              "tflops": tf, "tokens_per_s": w.total_new / (ms * 1e-3),
+                              "frac_nominal_2250": tf / NOMINAL_BF16_TFLOPS, "frac_measured_burst": tf / peaks["bf16_tflops"],
+                              "frac_measured_sustained": tf / peaks["bf16_tflops_sustained"], "steps": steps}) + "\n")
+        out.flush()
+        del runner
+        torch.cuda.empty_cache()
+
+
+def run_merge_sweep(args, out):
+    import torch
+    from paper_2609_04774_b200 import binding, build
+    build.build()
+    peaks = load_peaks()
+    ctx = binding.Context(0)
+    H, D = 64, 128
+    for T in args.merge_T:
+        for N in (2, 4, 8):
+            for dt in (torch.bfloat16, torch.float32):
+                in_bytes = N * T * H * (D * 4 + 4)
+                out_bytes = T * H * (D * dt.itemsize) + 4 * T * H
+                if in_bytes > 100e9:
+                    continue
+                parts = torch.randn((N, T, H, D), dtype=torch.float32, device="cuda")
+                lses = 8 + 2 * torch.randn((N, H, T), dtype=torch.float32, device="cuda")
+                lses[0].view(-1)[::16] = float("-inf")
+                o = torch.empty((T, H, D), dtype=dt, device="cuda")
+                lo = torch.empty((H, T), dtype=torch.float32, device="cuda")
+                flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if in_bytes < 512e6 else None
+
+                def fn():
+                    if flush is not None:
+                        flush.zero_()
+                    binding.cp_merge(ctx, parts, lses, o, lo)
+
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                ds = []
+                for _ in range(args.merge_reps):
+                    if flush is not None:
+                        flush.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    binding.cp_merge(ctx, parts, lses, o, lo)
+                    e1.record()
+                    ds.append((e0, e1))
+                torch.cuda.synchronize()
+                ms = [a.elapsed_time(b) for a, b in ds]
+                med = statistics.median(ms)
+                gbs = (in_bytes + out_bytes) / (med * 1e-3) / 1e9
+                out.write(json.dumps({"mode": "merge", "T": T, "N": N, "H": H, "out": str(dt).split(".")[-1],
+                                      "bytes": in_bytes + out_bytes, "ms_median": med, "ms_best": min(ms), "GBps": gbs,
+                                      "frac_nominal_8000": gbs / NOMINAL_HBM_GBS, "frac_measured_copy": gbs / peaks["hbm_gbs"],
+                                      "l2_flush": flush is not None}) + "\n")
+                out.flush()
+                del parts, lses, o, lo, flush
+                torch.cuda.empty_cache()
+
+
+def run_table(args, out):
+    """Measured prefill-time table over (new_len, prefix_len, C): all-shard time and the slowest /
+    fastest single shard (what one CP rank would compute), with W(R,P) of Eq. (1) -- the inputs of the
+    paper's cache-aware prefill-time model (Eq. 2)."""
+    import torch
+    from paper_2609_04774_b200 import binding, build
+    build.build()
+    ctx = binding.Context(0)
+    Hq, Hkv, D = 32, 8, 128
+    out.write("R,P,C,W,W_over_C,t_all_ms,t_shard_max_ms,t_shard_min_ms\n")
+    for R in args.table_R:
+        for hit in (0.0, 0.25, 0.5, 0.75, 0.9):
+            L = int(round(R / (1 - hit)))
+            P = (L - R) // wl.PAGE * wl.PAGE
+            w0 = wl.Workload("table", 7, Hq, Hkv, [wl.Request(R, P, 1)])
+            mat = wl.materialize(w0)
+            dev = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+            q, k, v = dev(mat.q), dev(mat.k_pages), dev(mat.v_pages)
+            pt = torch.from_numpy(mat.page_table).cuda()
+            cache = binding.make_cache(k, v)
+            o = torch.empty((R, Hq, D), dtype=torch.bfloat16, device="cuda")
+            lse = torch.empty((Hq, R), dtype=torch.float32, device="cuda")
+            po = torch.empty((R, Hq, D), dtype=torch.float32, device="cuda")
+            ws = torch.zeros(binding.cp_workspace_bytes([R], [8]), dtype=torch.uint8, device="cuda")
+
+            def timeit(fn, reps):
+                for _ in range(2):
+                    fn()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(reps):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / reps
+
+            W = R * P + R * (R + 1) // 2
+            reps = max(2, min(20, int(2e12 / (4 * D * Hq * W))))
+            for C in (1, 2, 4, 8):
+                t_all = timeit(lambda: binding.cp_prefill_attn(ctx, q, cache, pt, P, R, C, Hq, w0.scale, o, lse, ws), reps)
+                ts = [timeit(lambda: binding.cp_prefill_attn_shard(ctx, q, cache, pt, P, R, C, s, Hq, w0.scale, po, lse, ws), reps)
+                      for s in range(C)]
+                out.write("%d,%d,%d,%d,%.1f,%.4f,%.4f,%.4f\n" % (R, P, C, W, W / C, t_all, max(ts), min(ts)))
+                out.flush()
+            ctx.poll_status()
+            del q, k, v, o, po, lse
+            torch.cuda.empty_cache()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="BASELINE config number of the headline workload")
+    ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table"])
+    ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5])
+    ap.add_argument("--merge-T", type=int, nargs="*", default=[4096, 16384, 65536, 262144])
+    ap.add_argument("--merge-reps", type=int, default=20)
+    ap.add_argument("--table-R", type=int, nargs="*", default=[1024, 2048, 4096, 8192, 16384, 32768, 65536, 131072])
+    ap.add_argument("--out", default=None)
+    ap.add_argument("--cpu-rows", type=int, default=1024, help="rows per request of the cpu_baseline sample")
+    ap.add_argument("--ref-rows", type=int, default=96, help="rows per request per step of --impl reference")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.mode == "bench":
+        return run_ours(args)
+    out = open(args.out, "w") if args.out else sys.stdout
+    {"configs": run_configs, "merge": run_merge_sweep, "table": run_table}[args.mode](args, out)
+
+
+if __name__ == "__main__":
+    main()
