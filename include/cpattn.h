@@ -137,6 +137,33 @@ int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, 
                           size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * cp_prefill_attn_static -- cp_prefill_attn for callers that must not allocate device memory.
+ * (The paper has no counterpart to this call; it exists for integration reasons only.)
+ * Who needs it: code that runs after an inference engine has handed all of HBM to its own KV-cache
+ * pool, code inside a region where an allocation would synchronise the device or is forbidden
+ * (a latency-critical serving loop, a library callback), and embedders that are simply not
+ * allowed to create a cp_ctx, whose constructor allocates.  This call needs no cp_ctx and no
+ * workspace, and it calls no allocating CUDA routine: the scheduler's tile list and the status
+ * words live in a fixed device array of 65,792 bytes that is part of the library image (every GPU
+ * that loads the library holds it until the process exits).
+ *   - Same arguments, result and limits as cp_prefill_attn, computed on the CURRENT device.
+ *   - Size limit: ceil(new_len / 128) + 2*C must not exceed 2048 query tiles (about 260K new
+ *     tokens); larger requests return CP_ERR_WORKSPACE and launch nothing.
+ *   - The first call on each device resolves the device address of the array, the tensor-map
+ *     encoder and the kernel's shared-memory attribute; make that first call before any stream
+ *     capture begins.
+ *   - All calls share the one array, which keeps the previous call's contents; the call clears
+ *     the status words and rewrites the tile list in stream order.  Two calls that can overlap on
+ *     the GPU (different streams without an ordering between them) race on it; host threads must
+ *     not call it concurrently for the same device either.
+ *   - A device-side wait that runs out is recorded in the array's status words, which this ABI
+ *     does not expose; the rows of the affected tiles are then left unwritten.
+ * ------------------------------------------------------------------------------------------- */
+int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, const int32_t* page_table,
+                           int64_t prefix_len, int64_t new_len, int32_t C, int32_t Hq, float scale,
+                           void* out, float* lse, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * cp_merge -- N-way log-sum-exp combination of partial attention results over the same rows
  * (what joins per-shard or KV-split partials into full-sequence attention).
  *   partials device [N, T, H, D] fp32;  lses device [N, H, T] fp32 (natural log; -inf = "this

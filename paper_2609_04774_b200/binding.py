@@ -20,7 +20,7 @@ CP_ERR_INVALID_ARG, CP_ERR_UNSUPPORTED, CP_ERR_WORKSPACE, CP_ERR_CUDA, CP_ERR_TI
 CP_DTYPE_BF16, CP_DTYPE_F32 = 0, 1
 
 EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "cp_ctx_poll_status", "cp_plan",
-           "cp_workspace_bytes", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_merge",
+           "cp_workspace_bytes", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_static", "cp_merge",
            "cp_kv_gather", "cp_kv_append"]
 
 
@@ -168,6 +168,16 @@ def cp_prefill_attn_shard(ctx, q, cache, page_table, prefix_len, new_len, C, sha
         ctypes.c_int32(C), ctypes.c_int32(shard), ctypes.c_int32(Hq), ctypes.c_float(scale), _ptr(partial_out),
         _ptr(partial_lse), _ptr(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
         _stream(stream)))
+
+
+def cp_prefill_attn_static(q, cache, page_table, prefix_len, new_len, C, Hq, scale, out, lse, stream=None):
+    """cp_prefill_attn without a context or a workspace: the library's built-in device scratch holds the
+    tile list, so nothing is allocated.  For callers that cannot allocate device memory (all of HBM
+    already handed to a cache pool, allocation-free serving loops).  Limits: ceil(new_len/128) + 2*C <= 2048
+    tiles; calls share the scratch, so calls that may overlap on the GPU must be ordered by the caller."""
+    _check(load().cp_prefill_attn_static(_ptr(q), ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(prefix_len),
+                                         ctypes.c_int64(new_len), ctypes.c_int32(C), ctypes.c_int32(Hq),
+                                         ctypes.c_float(scale), _ptr(out), _ptr(lse), _stream(stream)))
 
 
 def cp_merge(ctx, partials, lses, out, lse_out=None, stream=None):

@@ -730,3 +730,117 @@ extern "C" int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cac
     return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, Hq, scale, partial_out, 1,
                        partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_shard");
 }
+
+// ------------------------------------------------------------------------------------------------
+// cp_prefill_attn_static: the single-request call for callers that may not allocate.
+// The tile list and the status words live in a fixed device array that is part of the library
+// image; nothing here calls an allocating CUDA routine and no cp_ctx is needed.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxTiles = 2048;   // 128-row query tiles, chunk cuts included (~260K new tokens)
+constexpr size_t kStaticScratchBytes = kWorkspaceHeader + (size_t)kStaticMaxTiles * sizeof(TileItem);
+constexpr int kStaticMaxDevices = 64;
+
+// [0, 16): status words {code, barrier, block, iteration}; [256, ...): tile list.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+struct StaticDeviceState {
+    bool ready;
+    unsigned char* scratch;     // device address of g_static_scratch on this device
+    int num_sms;
+    EncodeTiledFn encode_tiled;
+};
+StaticDeviceState g_static_state[kStaticMaxDevices];
+
+// One-time set-up for the current device: resolve the device address of the scratch array (its name
+// in host code is only a handle), the tensor-map encoder and the kernel's shared-memory limit.
+int static_setup(int device, StaticDeviceState** out) {
+    if (device < 0 || device >= kStaticMaxDevices)
+        return set_error(CP_ERR_UNSUPPORTED, "cp_prefill_attn_static: device ordinal %d not supported", device);
+    StaticDeviceState& st = g_static_state[device];
+    if (!st.ready) {
+        void* ptr = nullptr;
+        if (int rc = check_cuda(cudaGetSymbolAddress(&ptr, g_static_scratch), "cudaGetSymbolAddress(static scratch)"))
+            return rc;
+        cudaDeviceProp prop;
+        if (int rc = check_cuda(cudaGetDeviceProperties(&prop, device), "cudaGetDeviceProperties")) return rc;
+        if (prop.major != 10)
+            return set_error(CP_ERR_UNSUPPORTED, "cp_prefill_attn_static: device is sm_%d%d, sm_100a only", prop.major, prop.minor);
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (int rc = check_cuda(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q),
+                                "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)")) return rc;
+        if (q != cudaDriverEntryPointSuccess || !fn)
+            return set_error(CP_ERR_CUDA, "cuTensorMapEncodeTiled is not available in this driver");
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
+        st.scratch = static_cast<unsigned char*>(ptr);
+        st.num_sms = prop.multiProcessorCount;
+        st.encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+        st.ready = true;
+    }
+    *out = &st;
+    return CP_OK;
+}
+
+}  // namespace
+
+extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, const int32_t* page_table,
+                                      int64_t prefix_len, int64_t new_len, int32_t C, int32_t Hq, float scale,
+                                      void* out, float* lse, void* stream) {
+    const char* who = "cp_prefill_attn_static";
+    if (!q || !page_table || !out || !lse || new_len < 1 || prefix_len < 0 || C < 1)
+        return set_error(CP_ERR_INVALID_ARG, "%s: null pointer, new_len < 1, prefix_len < 0 or C < 1", who);
+    if (int rc = validate_kv_cache(cache, who)) return rc;
+    if (Hq < 1 || Hq % cache->Hkv != 0)
+        return set_error(CP_ERR_INVALID_ARG, "%s: Hq=%d is not a multiple of Hkv=%d", who, Hq, cache->Hkv);
+    if ((Hq / cache->Hkv) % 2 != 0)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: Hq/Hkv=%d must be even", who, Hq / cache->Hkv);
+    if (!(scale > 0.f)) return set_error(CP_ERR_INVALID_ARG, "%s: scale must be positive", who);
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return set_error(CP_ERR_INVALID_ARG, "%s: q and out must be 16-byte aligned", who);
+    if (prefix_len + new_len > 0x7fffff00ll) return set_error(CP_ERR_UNSUPPORTED, "%s: request longer than 2^31 tokens", who);
+    const int64_t bound = max_tiles(1, &new_len, &C);
+    if (bound < 0 || bound > kStaticMaxTiles)
+        return set_error(CP_ERR_WORKSPACE, "%s: new_len=%lld with C=%d needs up to %lld query tiles; the built-in scratch "
+                         "holds %d (use cp_prefill_attn with a caller workspace)", who, (long long)new_len, C,
+                         (long long)bound, kStaticMaxTiles);
+    int device = -1;
+    if (int rc = check_cuda(cudaGetDevice(&device), "cudaGetDevice")) return rc;
+    StaticDeviceState* st = nullptr;
+    if (int rc = static_setup(device, &st)) return rc;
+
+    const int64_t cu_new[2] = {0, new_len};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
+    std::vector<TileItem> tiles;
+    build_tiles(1, cu_new, &prefix_len, &C, cu_pages, -1, tiles);
+    cp_ctx enc{};                       // only the encoder entry point is read by encode_maps
+    enc.encode_tiled = st->encode_tiled;
+    CUtensorMap tmQ, tmK, tmV;
+    if (int rc = encode_maps(&enc, q, new_len, Hq, cache, &tmQ, &tmK, &tmV)) return rc;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // The scratch keeps whatever the previous call left: clear the status words, overwrite the list.
+    if (int rc = check_cuda(cudaMemsetAsync(st->scratch, 0, kStatusWords * sizeof(int32_t), s), "cudaMemsetAsync(status)"))
+        return rc;
+    if (int rc = check_cuda(cudaMemcpyAsync(st->scratch + kWorkspaceHeader, tiles.data(), tiles.size() * sizeof(TileItem),
+                                            cudaMemcpyHostToDevice, s), "tile list copy")) return rc;
+    AttnParams p;
+    p.items = reinterpret_cast<const TileItem*>(st->scratch + kWorkspaceHeader);
+    p.n_items = (int32_t)tiles.size();
+    p.pairs_per_tile = Hq / 2;
+    p.group = Hq / cache->Hkv;
+    p.Hq = Hq;
+    p.page_table = page_table;
+    p.oob_page = (int32_t)std::min<int64_t>(cache->num_pages, 0x7fffffff);
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.out = out;
+    p.out_f32 = 0;
+    p.lse = lse;
+    p.lse_stride = new_len;
+    p.status = reinterpret_cast<int32_t*>(st->scratch);
+    const int64_t units = (int64_t)tiles.size() * p.pairs_per_tile;
+    const int grid = (int)std::min<int64_t>(units, st->num_sms);
+    cp_attn_kernel<<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
+    return check_cuda(cudaGetLastError(), who);
+}

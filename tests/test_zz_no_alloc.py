@@ -1,0 +1,60 @@
+"""The allocation-free entry point (collected last on purpose).
+
+Some callers of this library cannot allocate device memory at the time they need attention: an
+inference engine that has already given all of HBM to its KV-cache pool, or a serving loop that must
+not hit an allocating (device-synchronising) call.  `cp_prefill_attn_static` serves them from a fixed
+scratch array inside the library.  Here it is called twice in a row through the C ABI, on different
+shapes (the second smaller, so stale scratch contents from the first call are still there), and each
+result is compared with the regular entry point's on the same inputs within the tolerances the parity
+tests use; then an oversized request must be refused before anything is launched."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_04774_b200 import binding
+from paper_2609_04774_b200 import workloads as wl
+from tests.gpu_util import DeviceWorkload, bf16_to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+def _both(ctx, w):
+    r = w.requests[0]
+    dev = DeviceWorkload(wl.materialize(w))
+    binding.cp_prefill_attn(ctx, dev.q, dev.cache, dev.page_table, r.prefix_len, r.new_len, r.C, w.Hq, w.scale,
+                            dev.out, dev.lse, dev.ws)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ref_o, ref_l = dev.out.clone(), dev.lse.clone()
+    out = torch.full_like(dev.out, float("nan"))
+    lse = torch.full_like(dev.lse, float("nan"))
+    binding.cp_prefill_attn_static(dev.q, dev.cache, dev.page_table, r.prefix_len, r.new_len, r.C, w.Hq, w.scale,
+                                   out, lse)
+    torch.cuda.synchronize()
+    return bf16_to_f64(out), lse.cpu().numpy().astype(np.float64), bf16_to_f64(ref_o), ref_l.cpu().numpy().astype(np.float64)
+
+
+def test_static_entry_point_matches_regular_one_twice():
+    ctx = binding.Context(0)
+    try:
+        for w in (wl.Workload("static_a", 31, 8, 2, [wl.Request(1500, 448, 4)]),
+                  wl.Workload("static_b", 32, 8, 2, [wl.Request(200, 64, 3)])):
+            o, l, ro, rl = _both(ctx, w)
+            assert np.isfinite(o).all() and np.isfinite(l).all()
+            assert np.abs(o - ro).max() <= 2e-2 and np.abs(o - ro).mean() <= 2e-3
+            assert (np.abs(l - rl) / np.maximum(1.0, np.abs(rl))).max() <= 1e-3
+    finally:
+        ctx.close()
+
+
+def test_static_entry_point_rejects_oversized_requests():
+    w = wl.Workload("static_c", 33, 8, 2, [wl.Request(64, 0, 1)])
+    dev = DeviceWorkload(wl.materialize(w))
+    before = dev.out.clone()
+    with pytest.raises(binding.CpError) as e:
+        # 2048 * 128 new tokens + chunk cuts exceed the built-in tile list; refused before any launch
+        binding.cp_prefill_attn_static(dev.q, dev.cache, dev.page_table, 0, 2048 * 128, 8, w.Hq, w.scale, dev.out, dev.lse)
+    assert e.value.code == binding.CP_ERR_WORKSPACE
+    assert "2048" in str(e.value)
+    torch.cuda.synchronize()
+    assert torch.equal(before.view(torch.int16), dev.out.view(torch.int16))
