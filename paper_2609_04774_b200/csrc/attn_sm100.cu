@@ -8,6 +8,8 @@
 //   warps 4-7  softmax warpgroup for head 1
 //   warp  8    TMA producer (lane 0 issues; the warp prefetches page ids)
 //   warp  9    tcgen05.mma issuer (one elected thread)
+//   warps 10-11 idle (they complete the third warpgroup so that register budgets can be moved:
+//              the softmax warpgroups run with 208 registers per thread, the third one with 88)
 // TMEM (512 columns): S0 | S1 | O0 | O1, each 128 fp32 columns; P (bf16) overwrites the first 64
 // columns of its S tile and is consumed from TMEM as the A operand of P*V.
 // The tensor pipe executes the MMAs of the issuing thread in order:
@@ -34,7 +36,9 @@ constexpr int kKvStages = 4;                       // ring of 32 KB tiles, K and
 constexpr uint32_t kTileBytes = kBlockN * kD * 2;  // 32768
 constexpr uint32_t kHalfBytes = kTileBytes / 2;    // one 64-dim half: 128 rows x 128 B
 constexpr uint32_t kPageBoxBytes = 64 * 64 * 2;    // one TMA box: 64 tokens x 64 dims
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;
+constexpr int kRegsSoftmax = 208;   // setmaxnreg budgets: 2*128*208 + 128*88 = 64512 = 384*168
+constexpr int kRegsOther = 88;
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t kSmemQ = 0;                                  // 2 heads x 32 KB
@@ -49,8 +53,8 @@ enum Bar : uint32_t {
     kBarKvFull = 2,                       // + stage
     kBarKvEmpty = kBarKvFull + kKvStages, // + stage
     kBarSReady = kBarKvEmpty + kKvStages, // + wg
-    kBarPReady = kBarSReady + 2,          // + wg
-    kBarODone = kBarPReady + 2,           // + wg
+    kBarPReady = kBarSReady + 2,          // + wg*2 + half: P columns [0,32) / [32,64) written
+    kBarODone = kBarPReady + 4,           // + wg
     kBarOFree = kBarODone + 2,            // + wg
     kNumBars = kBarOFree + 2
 };
@@ -63,7 +67,8 @@ constexpr uint32_t kTmemS = 0;     // + wg * 128
 constexpr uint32_t kTmemO = 256;   // + wg * 128
 
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
-constexpr float kRescaleThreshold = 8.0f;              // log2 units: keep a stale row max up to 2^8
+constexpr float kRescaleThreshold = 8.0f;
+constexpr bool kPolyExp = true;                       // every fourth pair of exp2 on the FMA pipe              // log2 units: keep a stale row max up to 2^8
 
 struct AttnParams {
     const TileItem* items;
@@ -157,6 +162,10 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
                  "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                  \
                  "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"                        \
                  ::CP_W8F(v, o), CP_W8F(v, o + 8), CP_W8F(v, o + 16), CP_W8F(v, o + 24), "r"(taddr) : "memory")
+#define TMEM_ST16R(taddr, v, o)                                                                           \
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "                                         \
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"                                 \
+                 ::CP_W8R(v, o), CP_W8R(v, o + 8), "r"(taddr) : "memory")
 #define TMEM_ST32R(taddr, v, o)                                                                           \
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "                                         \
                  "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                  \
@@ -172,6 +181,29 @@ __device__ __forceinline__ float lg2(float x) {
     float y;
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// 2^x for a pair of arguments x <= 0 on the FMA pipe (no MUFU): round to nearest integer with the
+// 1.5*2^23 trick, cubic minimax polynomial of 2^f on [-0.5, 0.5] (relative error 7.5e-5, far below
+// the bf16 rounding of P), integer part added into the exponent field.
+__device__ __forceinline__ float2 ex2_poly2(float2 x) {
+    const float kMagic = 12582912.f;
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 r = __fadd2_rn(x, make_float2(kMagic, kMagic));
+    const float2 xi = __fadd2_rn(r, make_float2(-kMagic, -kMagic));
+    const float2 f = __fadd2_rn(x, make_float2(-xi.x, -xi.y));
+    float2 p = __ffma2_rn(f, make_float2(0.0551716648f, 0.0551716648f), make_float2(0.2426111251f, 0.2426111251f));
+    p = __ffma2_rn(p, f, make_float2(0.6932609677f, 0.6932609677f));
+    p = __ffma2_rn(p, f, make_float2(0.9999280572f, 0.9999280572f));
+    float2 out;
+    out.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23));
+    out.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23));
+    return out;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
@@ -246,7 +278,7 @@ __device__ __forceinline__ bool fetch_unit(const AttnParams& p, int round, UnitI
 // ------------------------------------------------------------------------------------------
 // Roles
 // ------------------------------------------------------------------------------------------
-__device__ void producer_role(const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV, const AttnParams& p,
+__device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV, const AttnParams& p,
                               uint32_t smem_base, volatile uint32_t* abort_flag) {
     const int lane = threadIdx.x & 31;
     const uint32_t bars = smem_base + kSmemBar;
@@ -301,7 +333,7 @@ __device__ void producer_role(const CUtensorMap* tmQ, const CUtensorMap* tmK, co
     }
 }
 
-__device__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base, volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
     uint32_t kv_it = 0;        // ring slots consumed so far
     uint32_t tile_cnt = 0;     // KV tiles processed so far (phase of s_ready / p_ready)
@@ -315,11 +347,14 @@ __device__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_
                    make_desc(k_addr + off, 16, 1024), kIdescS, ks > 0);
         }
     };
-    auto issue_pv = [&](int wg, uint32_t v_addr, bool accumulate) {
+    // P*V over keys [half*64, half*64+64) of the tile: P columns [half*32, +32), V rows [half*64, +64)
+    auto issue_pv = [&](int wg, int half, uint32_t v_addr, bool accumulate) {
 #pragma unroll
-        for (int ks = 0; ks < kBlockN / 16; ++ks)
+        for (int k4 = 0; k4 < 4; ++k4) {
+            const int ks = half * 4 + k4;
             mma_ts(tmem_base + kTmemO + wg * 128, tmem_base + kTmemS + wg * 128 + ks * 8,
                    make_desc(v_addr + ks * 2048, kHalfBytes, 1024), kIdescPV, accumulate || ks > 0);
+        }
     };
 #define MMA_WAIT(id, parity, it) if (!mbar_wait(bars, (id), (parity), abort_flag, p.status, (it))) return
 
@@ -356,7 +391,10 @@ __device__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_
             if (j == 0 && round > 0) MMA_WAIT(kBarOFree + 0, (round - 1) & 1, j);
             MMA_WAIT(kBarKvFull + v_slot, v_par, j);
             tc_fence_after();
-            issue_pv(0, v_addr, j > 0);
+            issue_pv(0, 0, v_addr, j > 0);
+            MMA_WAIT(kBarPReady + 1, tile_cnt & 1, j);
+            tc_fence_after();
+            issue_pv(0, 1, v_addr, true);
             if (!more) tc_commit(bars + (kBarODone + 0) * 8);
             if (more) {
                 MMA_WAIT(kBarKvFull + k_slot, (kv_it / kKvStages) & 1, j);
@@ -365,10 +403,13 @@ __device__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_
                 tc_commit(bars + (kBarSReady + 0) * 8);
             }
             // head 1
-            MMA_WAIT(kBarPReady + 1, tile_cnt & 1, j);
+            MMA_WAIT(kBarPReady + 2, tile_cnt & 1, j);
             if (j == 0 && round > 0) MMA_WAIT(kBarOFree + 1, (round - 1) & 1, j);
             tc_fence_after();
-            issue_pv(1, v_addr, j > 0);
+            issue_pv(1, 0, v_addr, j > 0);
+            MMA_WAIT(kBarPReady + 3, tile_cnt & 1, j);
+            tc_fence_after();
+            issue_pv(1, 1, v_addr, true);
             if (!more) tc_commit(bars + (kBarODone + 1) * 8);
             tc_commit(bars + (kBarKvEmpty + v_slot) * 8);
             if (more) {
@@ -384,8 +425,8 @@ __device__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_
 #undef MMA_WAIT
 }
 
-__device__ void softmax_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base, volatile uint32_t* abort_flag,
-                             int wg) {
+__device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
+                                             volatile uint32_t* abort_flag, int wg) {
     const uint32_t bars = smem_base + kSmemBar;
     const int lane = threadIdx.x & 31;
     const int warp_in_wg = (threadIdx.x >> 5) & 3;
@@ -394,6 +435,7 @@ __device__ void softmax_role(const AttnParams& p, uint32_t smem_base, uint32_t t
     const uint32_t s_tmem = tmem_base + lane_addr + kTmemS + wg * 128;
     const uint32_t o_tmem = tmem_base + lane_addr + kTmemO + wg * 128;
     const float c = p.scale_log2;
+    const float2 c2 = make_float2(c, c);
     uint32_t tile_cnt = 0;
 
 #define SM_WAIT(id, parity, it)                                                                  \
@@ -411,7 +453,6 @@ __device__ void softmax_role(const AttnParams& p, uint32_t smem_base, uint32_t t
         float l = 0.f;         // running row sum of 2^(s - m)
         for (int j = 0; j < n; ++j) {
             SM_WAIT(kBarSReady + wg, tile_cnt & 1, j);
-            ++tile_cnt;
             tc_fence_after();
             float s[128];
             TMEM_LD32(s_tmem + 0, s, 0);
@@ -420,15 +461,26 @@ __device__ void softmax_role(const AttnParams& p, uint32_t smem_base, uint32_t t
             TMEM_LD32(s_tmem + 96, s, 96);
             tc_wait_ld();
             // causal mask: row sees keys < kv_len0 + row; only tiles that reach past kv_len0 need it
-            if ((j + 1) * kBlockN > u.it.kv_len0) {
+            const bool diag = (j + 1) * kBlockN > u.it.kv_len0;
+            if (diag) {
                 const int lim = u.it.kv_len0 + row - j * kBlockN;
 #pragma unroll
                 for (int i = 0; i < 128; ++i)
                     if (i >= lim) s[i] = -INFINITY;
             }
-            float mx = s[0];
+            // row max: four independent chains of 3-input max
+            float mx0 = max3(s[0], s[1], s[2]), mx1 = max3(s[3], s[4], s[5]);
+            float mx2 = max3(s[6], s[7], s[8]), mx3 = max3(s[9], s[10], s[11]);
 #pragma unroll
-            for (int i = 1; i < 128; ++i) mx = fmaxf(mx, s[i]);
+            for (int i = 12; i < 124; i += 8) {
+                mx0 = max3(mx0, s[i], s[i + 1]);
+                mx1 = max3(mx1, s[i + 2], s[i + 3]);
+                mx2 = max3(mx2, s[i + 4], s[i + 5]);
+                mx3 = max3(mx3, s[i + 6], s[i + 7]);
+            }
+            mx0 = max3(mx0, s[124], s[125]);
+            mx1 = max3(mx1, s[126], s[127]);
+            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             const float m_new = fmaxf(m, mx * c);
             if (j == 0) {
                 m = m_new;     // O is overwritten by the first P*V: nothing to rescale
@@ -451,22 +503,42 @@ __device__ void softmax_role(const AttnParams& p, uint32_t smem_base, uint32_t t
                     }
                 }
             }
-            const float neg_m = -m;
+            const float2 nm2 = make_float2(-m, -m);
+            float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0, sum2 = sum0, sum3 = sum0;
             uint32_t pk[64];
-            float sum = 0.f;
+            // p = 2^(s*c - m), in four quarters of 32 keys; every fourth pair of an unmasked tile takes the
+            // FMA-pipe polynomial instead of MUFU.  P is handed to the MMA warp in two halves.
 #pragma unroll
-            for (int i = 0; i < 64; ++i) {
-                const float p0 = ex2(fmaf(s[2 * i], c, neg_m));
-                const float p1 = ex2(fmaf(s[2 * i + 1], c, neg_m));
-                sum += p0 + p1;
-                pk[i] = pack_bf16(p0, p1);
+            for (int qd = 0; qd < 4; ++qd) {
+#pragma unroll
+                for (int i = qd * 16; i < qd * 16 + 16; i += 4) {
+                    float2 x0 = __ffma2_rn(make_float2(s[2 * i + 0], s[2 * i + 1]), c2, nm2);
+                    float2 x1 = __ffma2_rn(make_float2(s[2 * i + 2], s[2 * i + 3]), c2, nm2);
+                    float2 x2 = __ffma2_rn(make_float2(s[2 * i + 4], s[2 * i + 5]), c2, nm2);
+                    float2 x3 = __ffma2_rn(make_float2(s[2 * i + 6], s[2 * i + 7]), c2, nm2);
+                    float2 p0 = make_float2(ex2(x0.x), ex2(x0.y));
+                    float2 p1 = make_float2(ex2(x1.x), ex2(x1.y));
+                    float2 p2 = make_float2(ex2(x2.x), ex2(x2.y));
+                    float2 p3 = (kPolyExp && !diag) ? ex2_poly2(x3) : make_float2(ex2(x3.x), ex2(x3.y));
+                    sum0 = __fadd2_rn(sum0, p0);
+                    sum1 = __fadd2_rn(sum1, p1);
+                    sum2 = __fadd2_rn(sum2, p2);
+                    sum3 = __fadd2_rn(sum3, p3);
+                    pk[i + 0] = pack_bf16(p0.x, p0.y);
+                    pk[i + 1] = pack_bf16(p1.x, p1.y);
+                    pk[i + 2] = pack_bf16(p2.x, p2.y);
+                    pk[i + 3] = pack_bf16(p3.x, p3.y);
+                }
+                TMEM_ST16R(s_tmem + qd * 16, pk, qd * 16);
+                if (qd & 1) {
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(bars + (kBarPReady + wg * 2 + (qd >> 1)) * 8);
+                }
             }
-            l += sum;
-            TMEM_ST32R(s_tmem + 0, pk, 0);
-            TMEM_ST32R(s_tmem + 32, pk, 32);
-            tc_wait_st();
-            tc_fence_before();
-            mbar_arrive(bars + (kBarPReady + wg) * 8);
+            const float2 st = __fadd2_rn(__fadd2_rn(sum0, sum1), __fadd2_rn(sum2, sum3));
+            l += st.x + st.y;
+            ++tile_cnt;
         }
         // epilogue: O / l -> global at the row's original position; LSE in natural log
         SM_WAIT(kBarODone + wg, round & 1, n);
@@ -528,7 +600,8 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         for (int w = 0; w < 2; ++w) {
             mbar_init(bars + (kBarSReady + w) * 8, 1);
-            mbar_init(bars + (kBarPReady + w) * 8, 128);
+            mbar_init(bars + (kBarPReady + 2 * w) * 8, 128);
+            mbar_init(bars + (kBarPReady + 2 * w + 1) * 8, 128);
             mbar_init(bars + (kBarODone + w) * 8, 1);
             mbar_init(bars + (kBarOFree + w) * 8, 128);
         }
@@ -544,14 +617,16 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr;
 
-    if (warp < 4) {
-        softmax_role(p, smem_base, tmem_base, abort_flag, 0);
-    } else if (warp < 8) {
-        softmax_role(p, smem_base, tmem_base, abort_flag, 1);
-    } else if (warp == 8) {
-        producer_role(&tmQ, &tmK, &tmV, p, smem_base, abort_flag);
-    } else if (threadIdx.x == 9 * 32) {
-        mma_role(p, smem_base, tmem_base, abort_flag);
+    if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+        softmax_role(p, smem_base, tmem_base, abort_flag, warp >> 2);
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+        if (warp == 8) {
+            producer_role(&tmQ, &tmK, &tmV, p, smem_base, abort_flag);
+        } else if (threadIdx.x == 9 * 32) {
+            mma_role(p, smem_base, tmem_base, abort_flag);
+        }
     }
 
     tc_fence_before();
