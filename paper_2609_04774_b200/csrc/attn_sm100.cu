@@ -7,14 +7,15 @@
 //   warps 0-3  softmax warpgroup for head 0 of the pair: one thread per query row
 //   warps 4-7  softmax warpgroup for head 1
 //   warp  8    TMA producer (lane 0 issues; the warp prefetches page ids)
-//   warp  9    tcgen05.mma issuer (one elected thread)
+//   warp  9    tcgen05.mma issuer (warp-uniform loop, one elected lane issues)
 //   warps 10-11 idle (they complete the third warpgroup so that register budgets can be moved:
 //              the softmax warpgroups run with 208 registers per thread, the third one with 88)
 // TMEM (512 columns): S0 | S1 | O0 | O1, each 128 fp32 columns; P (bf16) overwrites the first 64
 // columns of its S tile and is consumed from TMEM as the A operand of P*V.
-// The tensor pipe executes the MMAs of the issuing thread in order:
-//   S0(j+1) is issued behind PV0(j), S1(j+1) behind PV1(j), so while one warpgroup runs softmax
-//   on its tile the pipe works for the other one.
+// The tensor pipe executes the MMAs of the issuing thread in order, PV0(j) S0(j+1) PV1(j) S1(j+1):
+// S(j+1) follows P*V(j) of the same head (P overwrites S), and while one warpgroup runs softmax on
+// its tile the pipe works for the other head.  P is handed over in four pieces of 32 keys, so P*V
+// starts while the rest of the row is still being exponentiated.
 // Every wait is bounded; on expiry the CTA records where it gave up in the status word, all roles
 // drain and the kernel returns normally.
 #include <cuda_bf16.h>
@@ -32,7 +33,7 @@ namespace {
 constexpr int kD = 128;
 constexpr int kBlockM = 128;
 constexpr int kBlockN = 128;
-constexpr int kKvStages = 4;                       // ring of 32 KB tiles, K and V alternate
+constexpr int kKvStages = 5;                       // ring of 32 KB tiles, K and V alternate
 constexpr uint32_t kTileBytes = kBlockN * kD * 2;  // 32768
 constexpr uint32_t kHalfBytes = kTileBytes / 2;    // one 64-dim half: 128 rows x 128 B
 constexpr uint32_t kPageBoxBytes = 64 * 64 * 2;    // one TMA box: 64 tokens x 64 dims
@@ -53,8 +54,8 @@ enum Bar : uint32_t {
     kBarKvFull = 2,                       // + stage
     kBarKvEmpty = kBarKvFull + kKvStages, // + stage
     kBarSReady = kBarKvEmpty + kKvStages, // + wg
-    kBarPReady = kBarSReady + 2,          // + wg*2 + half: P columns [0,32) / [32,64) written
-    kBarODone = kBarPReady + 4,           // + wg
+    kBarPReady = kBarSReady + 2,          // + wg*4 + quarter: P columns [16*quarter, +16) written
+    kBarODone = kBarPReady + 8,           // + wg
     kBarOFree = kBarODone + 2,            // + wg
     kNumBars = kBarOFree + 2
 };
@@ -66,9 +67,11 @@ constexpr uint32_t kSmemAbort = kSmemTmemPtr + 4;               // uint32: set w
 constexpr uint32_t kTmemS = 0;     // + wg * 128
 constexpr uint32_t kTmemO = 256;   // + wg * 128
 
+constexpr uint32_t kTryWaitHintNs = 200000;             // the thread may stay suspended this long per try
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
 constexpr float kRescaleThreshold = 8.0f;
-constexpr bool kPolyExp = true;                       // every fourth pair of exp2 on the FMA pipe              // log2 units: keep a stale row max up to 2^8
+constexpr int kPieces = 2;                            // P is handed to the MMA warp in this many pieces (1, 2 or 4)
+constexpr int kPolyOf4 = 1;                            // pairs out of every four whose exp2 runs on the FMA pipe              // log2 units: keep a stale row max up to 2^8
 
 struct AttnParams {
     const TileItem* items;
@@ -104,9 +107,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kTryWaitHintNs) : "memory");
     return ok != 0;
 }
 
@@ -122,6 +125,16 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 
+// True in exactly one lane of the (converged) warp.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -227,17 +240,21 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((kBlockN >> 3) << 17) | ((kBlockM >> 4) << 24);
 constexpr uint32_t kIdescPV = kIdescS | (1u << 16);
 
-// Bounded wait on an mbarrier phase.  Returns false when the wait expired or another role already
-// gave up; the first to expire records {code, barrier id, block, iteration} in the status word.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar_base, uint32_t bar_id, uint32_t parity, volatile uint32_t* abort_flag,
+// Bounded wait on an mbarrier phase.  The fast path is a single try; the slow path spins with a cycle
+// limit.  When the limit runs out the first thread to notice records {code, barrier id, block,
+// iteration} in the status word and raises the CTA's abort flag; from then on every wait of the CTA
+// gives up after one failed try, so all roles run off the end of their loops without blocking (the
+// results are garbage, the status word says so) and the kernel returns normally.
+__device__ __forceinline__ void mbar_wait(uint32_t bar_base, uint32_t bar_id, uint32_t parity, volatile uint32_t* abort_flag,
                                           int32_t* status, int iter) {
     const uint32_t bar = bar_base + bar_id * 8;
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
     while (true) {
+        if (*abort_flag) return;
+#pragma unroll 1
         for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
+            if (mbar_try_wait(bar, parity)) return;
         if (clock64() - t0 > kWaitLimitCycles) {
             *abort_flag = 1;
             if (atomicCAS(status, 0, CP_ERR_TIMEOUT) == 0) {
@@ -245,10 +262,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar_base, uint32_t bar_id, ui
                 status[2] = (int32_t)blockIdx.x;
                 status[3] = iter;
             }
-            return false;
+            return;
         }
     }
 }
+
+// Optional phase trace (build with -DCPATTN_TRACE): block 0 stamps clock64() at fixed points of the
+// first 64 KV tiles of its first unit into the area behind the status words.
+#ifndef CPATTN_TRACE_ROW
+#define CPATTN_TRACE_ROW 0
+#endif
+#ifdef CPATTN_TRACE
+#define CP_TRACE(who, j, e)                                                                              \
+    if (blockIdx.x == 0 && round == 0 && (j) < 64)                                                       \
+        reinterpret_cast<long long*>(p.status + 16)[(((who)*64 + (j)) * 8) + (e)] = clock64();
+#else
+#define CP_TRACE(who, j, e)
+#endif
 
 struct UnitInfo {
     TileItem it;
@@ -286,20 +316,16 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
     for (int round = 0;; ++round) {
         UnitInfo u;
         if (!fetch_unit(p, round, u)) break;
-        int ok = 1;
         if (lane == 0) {
-            ok = mbar_wait(bars, kBarQEmpty, (round & 1) ^ 1, abort_flag, p.status, round);
-            if (ok) {
-                const uint32_t qbar = bars + kBarQFull * 8;
-                mbar_expect_tx(qbar, 2 * kTileBytes);
-                for (int h = 0; h < 2; ++h)
-                    for (int half = 0; half < 2; ++half)
-                        tma_load_3d(smem_base + kSmemQ + h * kTileBytes + half * kHalfBytes, tmQ, qbar, half * 64,
-                                    u.head0 + h, u.it.q_row0);
-            }
+            mbar_wait(bars, kBarQEmpty, (round & 1) ^ 1, abort_flag, p.status, round);
+            const uint32_t qbar = bars + kBarQFull * 8;
+            mbar_expect_tx(qbar, 2 * kTileBytes);
+            for (int h = 0; h < 2; ++h)
+                for (int half = 0; half < 2; ++half)
+                    tma_load_3d(smem_base + kSmemQ + h * kTileBytes + half * kHalfBytes, tmQ, qbar, half * 64,
+                                u.head0 + h, u.it.q_row0);
         }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok) return;
+        __syncwarp();
         const int n_tiles = u.it.n_kv_tiles;
         for (int j0 = 0; j0 < n_tiles; j0 += 16) {
             // the warp fetches the page ids of 16 KV tiles (32 pages) at once
@@ -312,20 +338,17 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
                 for (int kv = 0; kv < 2; ++kv) {
                     if (lane == 0) {
                         const uint32_t slot = kv_it % kKvStages;
-                        ok = mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j0 + jj);
-                        if (ok) {
-                            const uint32_t fbar = bars + (kBarKvFull + slot) * 8;
-                            const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
-                            const CUtensorMap* map = kv ? tmV : tmK;
-                            mbar_expect_tx(fbar, kTileBytes);
-                            for (int half = 0; half < 2; ++half) {
-                                tma_load_4d(dst + half * kHalfBytes, map, fbar, half * 64, u.kv_head, 0, page_a);
-                                tma_load_4d(dst + half * kHalfBytes + kPageBoxBytes, map, fbar, half * 64, u.kv_head, 0, page_b);
-                            }
+                        mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j0 + jj);
+                        const uint32_t fbar = bars + (kBarKvFull + slot) * 8;
+                        const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
+                        const CUtensorMap* map = kv ? tmV : tmK;
+                        mbar_expect_tx(fbar, kTileBytes);
+                        for (int half = 0; half < 2; ++half) {
+                            tma_load_4d(dst + half * kHalfBytes, map, fbar, half * 64, u.kv_head, 0, page_a);
+                            tma_load_4d(dst + half * kHalfBytes + kPageBoxBytes, map, fbar, half * 64, u.kv_head, 0, page_b);
                         }
                     }
-                    ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (!ok) return;
+                    __syncwarp();
                     ++kv_it;
                 }
             }
@@ -333,96 +356,224 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
     }
 }
 
-__device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base, volatile uint32_t* abort_flag) {
+// The issuer warp alternates between the two heads in a fixed order, PV0(j) S0(j+1) PV1(j) S1(j+1):
+// the tensor pipe executes in issue order, which keeps the two softmax warpgroups half a period apart
+// (one exponentiates while the pipe works for the other).  P arrives in four pieces of 32 keys, so
+// P*V starts while the rest of the row is still being exponentiated.  The whole warp runs the loop
+// (waits included) so that addresses and descriptors stay warp-uniform; one elected lane issues.
+__device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
+                                         volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
     uint32_t kv_it = 0;        // ring slots consumed so far
-    uint32_t tile_cnt = 0;     // KV tiles processed so far (phase of s_ready / p_ready)
-    const uint32_t q_addr = smem_base + kSmemQ;
+    uint32_t tile_cnt = 0;     // KV tiles processed so far (phase of p_ready)
+    const uint64_t q_desc0 = make_desc(smem_base + kSmemQ, 16, 1024);
+    const uint64_t k_desc0 = make_desc(smem_base + kSmemKV, 16, 1024);           // K-major view of a ring slot
+    const uint64_t v_desc0 = make_desc(smem_base + kSmemKV, kHalfBytes, 1024);   // MN-major view of a ring slot
 
-    auto issue_s = [&](int wg, uint32_t k_addr) {
+    auto issue_s = [&](int wg, uint32_t slot) {
+        if (elect_one()) {
 #pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) {
-            const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-            mma_ss(tmem_base + kTmemS + wg * 128, make_desc(q_addr + wg * kTileBytes + off, 16, 1024),
-                   make_desc(k_addr + off, 16, 1024), kIdescS, ks > 0);
+            for (int ks = 0; ks < kD / 16; ++ks) {
+                const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+                mma_ss(tmem_base + kTmemS + wg * 128, q_desc0 + (wg * (kTileBytes >> 4)) + off,
+                       k_desc0 + slot * (kTileBytes >> 4) + off, kIdescS, ks > 0);
+            }
+            tc_commit(bars + (kBarSReady + wg) * 8);
         }
+        __syncwarp();
     };
-    // P*V over keys [half*64, half*64+64) of the tile: P columns [half*32, +32), V rows [half*64, +64)
-    auto issue_pv = [&](int wg, int half, uint32_t v_addr, bool accumulate) {
+    // P*V over one piece of the tile's keys: 128/kPieces keys = 8/kPieces MMAs of 16 keys
+    auto issue_pv = [&](int wg, int part, uint32_t slot, bool accumulate) {
+        if (elect_one()) {
 #pragma unroll
-        for (int k4 = 0; k4 < 4; ++k4) {
-            const int ks = half * 4 + k4;
-            mma_ts(tmem_base + kTmemO + wg * 128, tmem_base + kTmemS + wg * 128 + ks * 8,
-                   make_desc(v_addr + ks * 2048, kHalfBytes, 1024), kIdescPV, accumulate || ks > 0);
+            for (int k2 = 0; k2 < 8 / kPieces; ++k2) {
+                const int ks = part * (8 / kPieces) + k2;
+                mma_ts(tmem_base + kTmemO + wg * 128, tmem_base + kTmemS + wg * 128 + ks * 8,
+                       v_desc0 + slot * (kTileBytes >> 4) + ks * (2048 >> 4), kIdescPV, accumulate || ks > 0);
+            }
         }
+        __syncwarp();
     };
-#define MMA_WAIT(id, parity, it) if (!mbar_wait(bars, (id), (parity), abort_flag, p.status, (it))) return
+    auto commit = [&](uint32_t bar_id) {
+        if (elect_one()) tc_commit(bars + bar_id * 8);
+        __syncwarp();
+    };
+#define MMA_WAIT(id, parity, it) mbar_wait(bars, (id), (parity), abort_flag, p.status, (it))
 
     for (int round = 0;; ++round) {
         UnitInfo u;
         if (!fetch_unit(p, round, u)) break;
         const int n = u.it.n_kv_tiles;
         MMA_WAIT(kBarQFull, round & 1, round);
-        // S(0) for both heads
         uint32_t slot = kv_it % kKvStages;
         MMA_WAIT(kBarKvFull + slot, (kv_it / kKvStages) & 1, 0);
         tc_fence_after();
-        uint32_t k_addr = smem_base + kSmemKV + slot * kTileBytes;
-        issue_s(0, k_addr);
-        tc_commit(bars + (kBarSReady + 0) * 8);
-        issue_s(1, k_addr);
-        tc_commit(bars + (kBarSReady + 1) * 8);
-        tc_commit(bars + (kBarKvEmpty + slot) * 8);
-        if (n == 1) tc_commit(bars + kBarQEmpty * 8);
+        issue_s(0, slot);
+        issue_s(1, slot);
+        commit(kBarKvEmpty + slot);
+        if (n == 1) commit(kBarQEmpty);
         ++kv_it;
+#pragma unroll 1
         for (int j = 0; j < n; ++j) {
             const uint32_t v_slot = kv_it % kKvStages;
             const uint32_t v_par = (kv_it / kKvStages) & 1;
             ++kv_it;
-            const uint32_t v_addr = smem_base + kSmemKV + v_slot * kTileBytes;
             const bool more = (j + 1 < n);
-            uint32_t k_slot = 0;
-            if (more) {
-                k_slot = kv_it % kKvStages;
-                k_addr = smem_base + kSmemKV + k_slot * kTileBytes;
+            const uint32_t k_slot = kv_it % kKvStages;
+            const uint32_t k_par = (kv_it / kKvStages) & 1;
+#pragma unroll
+            for (int wg = 0; wg < 2; ++wg) {
+                if (j == 0 && round > 0) MMA_WAIT(kBarOFree + wg, (round - 1) & 1, j);
+                if (wg == 0) {
+                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2, j, 6); }
+                    MMA_WAIT(kBarKvFull + v_slot, v_par, j);
+                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2, j, 7); }
+                }
+#pragma unroll
+                for (int part = 0; part < kPieces; ++part) {
+                    MMA_WAIT(kBarPReady + wg * 4 + part, tile_cnt & 1, j);
+                    tc_fence_after();
+                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, part); }
+                    issue_pv(wg, part, v_slot, j > 0);
+                }
+                if (wg == 1) commit(kBarKvEmpty + v_slot);
+                if (more) {
+                    if (wg == 0) MMA_WAIT(kBarKvFull + k_slot, k_par, j);
+                    tc_fence_after();
+                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, 4); }
+                    issue_s(wg, k_slot);
+                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, 5); }
+                    if (wg == 1) {
+                        commit(kBarKvEmpty + k_slot);
+                        if (j + 2 == n) commit(kBarQEmpty);
+                    }
+                } else {
+                    commit(kBarODone + wg);
+                }
             }
-            // head 0: O0 (+)= P0 V(j); then S0(j+1)
-            MMA_WAIT(kBarPReady + 0, tile_cnt & 1, j);
-            if (j == 0 && round > 0) MMA_WAIT(kBarOFree + 0, (round - 1) & 1, j);
-            MMA_WAIT(kBarKvFull + v_slot, v_par, j);
-            tc_fence_after();
-            issue_pv(0, 0, v_addr, j > 0);
-            MMA_WAIT(kBarPReady + 1, tile_cnt & 1, j);
-            tc_fence_after();
-            issue_pv(0, 1, v_addr, true);
-            if (!more) tc_commit(bars + (kBarODone + 0) * 8);
-            if (more) {
-                MMA_WAIT(kBarKvFull + k_slot, (kv_it / kKvStages) & 1, j);
-                tc_fence_after();
-                issue_s(0, k_addr);
-                tc_commit(bars + (kBarSReady + 0) * 8);
-            }
-            // head 1
-            MMA_WAIT(kBarPReady + 2, tile_cnt & 1, j);
-            if (j == 0 && round > 0) MMA_WAIT(kBarOFree + 1, (round - 1) & 1, j);
-            tc_fence_after();
-            issue_pv(1, 0, v_addr, j > 0);
-            MMA_WAIT(kBarPReady + 3, tile_cnt & 1, j);
-            tc_fence_after();
-            issue_pv(1, 1, v_addr, true);
-            if (!more) tc_commit(bars + (kBarODone + 1) * 8);
-            tc_commit(bars + (kBarKvEmpty + v_slot) * 8);
-            if (more) {
-                issue_s(1, k_addr);
-                tc_commit(bars + (kBarSReady + 1) * 8);
-                tc_commit(bars + (kBarKvEmpty + k_slot) * 8);
-                if (j + 2 == n) tc_commit(bars + kBarQEmpty * 8);
-                ++kv_it;
-            }
+            if (more) ++kv_it;
             ++tile_cnt;
         }
     }
 #undef MMA_WAIT
+}
+
+// Row max of 32 raw scores into four independent chains.
+__device__ __forceinline__ void max32(const float (&s)[32], float& a0, float& a1, float& a2, float& a3) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 8) {
+        a0 = max3(a0, s[i], s[i + 1]);
+        a1 = max3(a1, s[i + 2], s[i + 3]);
+        a2 = max3(a2, s[i + 4], s[i + 5]);
+        a3 = max3(a3, s[i + 6], s[i + 7]);
+    }
+}
+// Columns at or beyond `lim` are above the causal diagonal for this row.
+__device__ __forceinline__ void mask32(float (&s)[32], int lim) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        if (i >= lim) s[i] = -INFINITY;
+}
+// p = 2^(s*c - m) for 32 keys -> 16 packed bf16 pairs; row sums into four accumulators.  In unmasked
+// tiles kPolyOf4 of every four pairs take the FMA-pipe polynomial instead of MUFU.
+template <bool kMasked>
+__device__ __forceinline__ void exp32(const float (&s)[32], uint32_t (&pk)[16], float2 c2, float2 nm2, float2& sum0,
+                                      float2& sum1, float2& sum2, float2& sum3) {
+#pragma unroll
+    for (int i = 0; i < 16; i += 4) {
+        const float2 x0 = __ffma2_rn(make_float2(s[2 * i + 0], s[2 * i + 1]), c2, nm2);
+        const float2 x1 = __ffma2_rn(make_float2(s[2 * i + 2], s[2 * i + 3]), c2, nm2);
+        const float2 x2 = __ffma2_rn(make_float2(s[2 * i + 4], s[2 * i + 5]), c2, nm2);
+        const float2 x3 = __ffma2_rn(make_float2(s[2 * i + 6], s[2 * i + 7]), c2, nm2);
+        const float2 p0 = make_float2(ex2(x0.x), ex2(x0.y));
+        const float2 p1 = make_float2(ex2(x1.x), ex2(x1.y));
+        const float2 p2 = (kPolyOf4 >= 2 && !kMasked) ? ex2_poly2(x2) : make_float2(ex2(x2.x), ex2(x2.y));
+        const float2 p3 = (kPolyOf4 >= 1 && !kMasked) ? ex2_poly2(x3) : make_float2(ex2(x3.x), ex2(x3.y));
+        sum0 = __fadd2_rn(sum0, p0);
+        sum1 = __fadd2_rn(sum1, p1);
+        sum2 = __fadd2_rn(sum2, p2);
+        sum3 = __fadd2_rn(sum3, p3);
+        pk[i + 0] = pack_bf16(p0.x, p0.y);
+        pk[i + 1] = pack_bf16(p1.x, p1.y);
+        pk[i + 2] = pack_bf16(p2.x, p2.y);
+        pk[i + 3] = pack_bf16(p3.x, p3.y);
+    }
+}
+
+// One 128x128 score tile of one head: two passes over the row in TMEM, 32 columns at a time with the
+// next piece's load in flight (row max; then exponentials, row sum, P back to TMEM in four pieces,
+// each signalled to the MMA warp).  Short code and few live registers on purpose: two warps per SM
+// sub-partition run it half a period apart and it has to stay resident in the instruction cache.
+// kMasked: the tile reaches past the causal diagonal of some rows; `lim` = visible columns of this row.
+template <bool kMasked>
+__device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, uint32_t p_bar0, float c, int lim,
+                                             bool first, float& m, float& l) {
+    float a[32], b[32];
+    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+    TMEM_LD32(s_tmem + 0, a, 0);
+    tc_wait_ld();
+    TMEM_LD32(s_tmem + 32, b, 0);
+    if (kMasked) mask32(a, lim);
+    max32(a, mx0, mx1, mx2, mx3);
+    tc_wait_ld();
+    TMEM_LD32(s_tmem + 64, a, 0);
+    if (kMasked) mask32(b, lim - 32);
+    max32(b, mx0, mx1, mx2, mx3);
+    tc_wait_ld();
+    TMEM_LD32(s_tmem + 96, b, 0);
+    if (kMasked) mask32(a, lim - 64);
+    max32(a, mx0, mx1, mx2, mx3);
+    tc_wait_ld();
+    TMEM_LD32(s_tmem + 0, a, 0);            // first piece of the second pass
+    if (kMasked) mask32(b, lim - 96);
+    max32(b, mx0, mx1, mx2, mx3);
+
+    const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+    const float m_new = fmaxf(m, mx * c);
+    if (first) {
+        m = m_new;     // O is overwritten by the first P*V: nothing to rescale
+    } else {
+        const bool grow = (m_new - m) > kRescaleThreshold;
+        if (__any_sync(0xffffffffu, grow)) {
+            const float m_upd = grow ? m_new : m;
+            const float alpha = ex2(m - m_upd);
+            l *= alpha;
+            m = m_upd;
+            // P*V of the previous tile finished before this S was signalled (the pipe runs in issue order)
+            tc_wait_ld();
+#pragma unroll 1
+            for (int cc = 0; cc < 4; ++cc) {
+                float o[32];
+                TMEM_LD32(o_tmem + cc * 32, o, 0);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] *= alpha;
+                TMEM_ST32F(o_tmem + cc * 32, o, 0);
+            }
+        }
+    }
+    const float2 c2 = make_float2(c, c);
+    const float2 nm2 = make_float2(-m, -m);
+    float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0, sum2 = sum0, sum3 = sum0;
+    uint32_t pk[16];
+#define CP_P_PIECE(cur, nxt, q)                                                         \
+    tc_wait_ld();                                                                       \
+    if ((q) < 3) TMEM_LD32(s_tmem + ((q) + 1) * 32, nxt, 0);                            \
+    if (kMasked) mask32(cur, lim - (q) * 32);                                           \
+    exp32<kMasked>(cur, pk, c2, nm2, sum0, sum1, sum2, sum3);                           \
+    TMEM_ST16R(s_tmem + (q) * 16, pk, 0);                                               \
+    if (((q) + 1) % (4 / kPieces) == 0) {                                               \
+        tc_wait_st();                                                                   \
+        tc_fence_before();                                                              \
+        mbar_arrive(p_bar0 + ((q) / (4 / kPieces)) * 8);                                \
+    }
+    CP_P_PIECE(a, b, 0)
+    CP_P_PIECE(b, a, 1)
+    CP_P_PIECE(a, b, 2)
+    CP_P_PIECE(b, a, 3)
+#undef CP_P_PIECE
+    const float2 st = __fadd2_rn(__fadd2_rn(sum0, sum1), __fadd2_rn(sum2, sum3));
+    l += st.x + st.y;
 }
 
 __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
@@ -434,15 +585,13 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
     const uint32_t lane_addr = (uint32_t)(warp_in_wg * 32) << 16;   // TMEM lane field of this warp
     const uint32_t s_tmem = tmem_base + lane_addr + kTmemS + wg * 128;
     const uint32_t o_tmem = tmem_base + lane_addr + kTmemO + wg * 128;
+    const uint32_t p_bar0 = bars + (kBarPReady + wg * 4) * 8;
     const float c = p.scale_log2;
-    const float2 c2 = make_float2(c, c);
     uint32_t tile_cnt = 0;
 
 #define SM_WAIT(id, parity, it)                                                                  \
-    {                                                                                            \
-        int ok_ = mbar_wait(bars, (id), (parity), abort_flag, p.status, (it));                   \
-        if (!__all_sync(0xffffffffu, ok_)) return;                                               \
-    }
+    mbar_wait(bars, (id), (parity), abort_flag, p.status, (it));                                 \
+    __syncwarp();
 
     for (int round = 0;; ++round) {
         UnitInfo u;
@@ -451,93 +600,18 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
         const int head = u.head0 + wg;
         float m = -INFINITY;   // running row max in log2 units (possibly stale by < threshold)
         float l = 0.f;         // running row sum of 2^(s - m)
+        // tiles below n_full lie entirely under the causal diagonal of every row of the q-tile
+        const int n_full = u.it.kv_len0 / kBlockN;
+#pragma unroll 1
         for (int j = 0; j < n; ++j) {
             SM_WAIT(kBarSReady + wg, tile_cnt & 1, j);
             tc_fence_after();
-            float s[128];
-            TMEM_LD32(s_tmem + 0, s, 0);
-            TMEM_LD32(s_tmem + 32, s, 32);
-            TMEM_LD32(s_tmem + 64, s, 64);
-            TMEM_LD32(s_tmem + 96, s, 96);
-            tc_wait_ld();
-            // causal mask: row sees keys < kv_len0 + row; only tiles that reach past kv_len0 need it
-            const bool diag = (j + 1) * kBlockN > u.it.kv_len0;
-            if (diag) {
-                const int lim = u.it.kv_len0 + row - j * kBlockN;
-#pragma unroll
-                for (int i = 0; i < 128; ++i)
-                    if (i >= lim) s[i] = -INFINITY;
-            }
-            // row max: four independent chains of 3-input max
-            float mx0 = max3(s[0], s[1], s[2]), mx1 = max3(s[3], s[4], s[5]);
-            float mx2 = max3(s[6], s[7], s[8]), mx3 = max3(s[9], s[10], s[11]);
-#pragma unroll
-            for (int i = 12; i < 124; i += 8) {
-                mx0 = max3(mx0, s[i], s[i + 1]);
-                mx1 = max3(mx1, s[i + 2], s[i + 3]);
-                mx2 = max3(mx2, s[i + 4], s[i + 5]);
-                mx3 = max3(mx3, s[i + 6], s[i + 7]);
-            }
-            mx0 = max3(mx0, s[124], s[125]);
-            mx1 = max3(mx1, s[126], s[127]);
-            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-            const float m_new = fmaxf(m, mx * c);
-            if (j == 0) {
-                m = m_new;     // O is overwritten by the first P*V: nothing to rescale
-            } else {
-                const bool grow = (m_new - m) > kRescaleThreshold;
-                if (__any_sync(0xffffffffu, grow)) {
-                    const float m_upd = grow ? m_new : m;
-                    const float alpha = ex2(m - m_upd);
-                    l *= alpha;
-                    m = m_upd;
-                    // P*V(j-1) finished before S(j) was signalled (the pipe runs in issue order)
-#pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        float o[32];
-                        TMEM_LD32(o_tmem + cc * 32, o, 0);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] *= alpha;
-                        TMEM_ST32F(o_tmem + cc * 32, o, 0);
-                    }
-                }
-            }
-            const float2 nm2 = make_float2(-m, -m);
-            float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0, sum2 = sum0, sum3 = sum0;
-            uint32_t pk[64];
-            // p = 2^(s*c - m), in four quarters of 32 keys; every fourth pair of an unmasked tile takes the
-            // FMA-pipe polynomial instead of MUFU.  P is handed to the MMA warp in two halves.
-#pragma unroll
-            for (int qd = 0; qd < 4; ++qd) {
-#pragma unroll
-                for (int i = qd * 16; i < qd * 16 + 16; i += 4) {
-                    float2 x0 = __ffma2_rn(make_float2(s[2 * i + 0], s[2 * i + 1]), c2, nm2);
-                    float2 x1 = __ffma2_rn(make_float2(s[2 * i + 2], s[2 * i + 3]), c2, nm2);
-                    float2 x2 = __ffma2_rn(make_float2(s[2 * i + 4], s[2 * i + 5]), c2, nm2);
-                    float2 x3 = __ffma2_rn(make_float2(s[2 * i + 6], s[2 * i + 7]), c2, nm2);
-                    float2 p0 = make_float2(ex2(x0.x), ex2(x0.y));
-                    float2 p1 = make_float2(ex2(x1.x), ex2(x1.y));
-                    float2 p2 = make_float2(ex2(x2.x), ex2(x2.y));
-                    float2 p3 = (kPolyExp && !diag) ? ex2_poly2(x3) : make_float2(ex2(x3.x), ex2(x3.y));
-                    sum0 = __fadd2_rn(sum0, p0);
-                    sum1 = __fadd2_rn(sum1, p1);
-                    sum2 = __fadd2_rn(sum2, p2);
-                    sum3 = __fadd2_rn(sum3, p3);
-                    pk[i + 0] = pack_bf16(p0.x, p0.y);
-                    pk[i + 1] = pack_bf16(p1.x, p1.y);
-                    pk[i + 2] = pack_bf16(p2.x, p2.y);
-                    pk[i + 3] = pack_bf16(p3.x, p3.y);
-                }
-                TMEM_ST16R(s_tmem + qd * 16, pk, qd * 16);
-                if (qd & 1) {
-                    tc_wait_st();
-                    tc_fence_before();
-                    mbar_arrive(bars + (kBarPReady + wg * 2 + (qd >> 1)) * 8);
-                }
-            }
-            const float2 st = __fadd2_rn(__fadd2_rn(sum0, sum1), __fadd2_rn(sum2, sum3));
-            l += st.x + st.y;
+            if (row == CPATTN_TRACE_ROW) { CP_TRACE(wg, j, 0); }
+            if (j < n_full)
+                softmax_tile<false>(s_tmem, o_tmem, p_bar0, c, 0, j == 0, m, l);
+            else
+                softmax_tile<true>(s_tmem, o_tmem, p_bar0, c, u.it.kv_len0 + row - j * kBlockN, j == 0, m, l);
+            if (row == CPATTN_TRACE_ROW) { CP_TRACE(wg, j, 6); }
             ++tile_cnt;
         }
         // epilogue: O / l -> global at the row's original position; LSE in natural log
@@ -546,7 +620,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
         const float inv_l = 1.f / l;
         const bool valid = row < u.it.n_rows;
         const int64_t grow_idx = (int64_t)u.it.q_row0 + row;
-#pragma unroll
+#pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
             float o[32];
             TMEM_LD32(o_tmem + cc * 32, o, 0);
@@ -600,8 +674,7 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         for (int w = 0; w < 2; ++w) {
             mbar_init(bars + (kBarSReady + w) * 8, 1);
-            mbar_init(bars + (kBarPReady + 2 * w) * 8, 128);
-            mbar_init(bars + (kBarPReady + 2 * w + 1) * 8, 128);
+            for (int q4 = 0; q4 < 4; ++q4) mbar_init(bars + (kBarPReady + 4 * w + q4) * 8, 128);
             mbar_init(bars + (kBarODone + w) * 8, 1);
             mbar_init(bars + (kBarOFree + w) * 8, 128);
         }
@@ -624,7 +697,7 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
         if (warp == 8) {
             producer_role(&tmQ, &tmK, &tmV, p, smem_base, abort_flag);
-        } else if (threadIdx.x == 9 * 32) {
+        } else if (warp == 9) {
             mma_role(p, smem_base, tmem_base, abort_flag);
         }
     }

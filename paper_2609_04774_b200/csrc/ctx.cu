@@ -58,8 +58,8 @@ extern "C" int cp_ctx_create(cp_ctx** out, int device) {
     c->device = device;
     c->num_sms = prop.multiProcessorCount;
     c->stage_bytes = 8u << 20;
-    int rc = check_cuda(cudaMalloc(&c->d_status, kStatusWords * sizeof(int32_t)), "cudaMalloc(status)");
-    if (!rc) rc = check_cuda(cudaMemset(c->d_status, 0, kStatusWords * sizeof(int32_t)), "cudaMemset(status)");
+    int rc = check_cuda(cudaMalloc(&c->d_status, kStatusBytes), "cudaMalloc(status)");
+    if (!rc) rc = check_cuda(cudaMemset(c->d_status, 0, kStatusBytes), "cudaMemset(status)");
     if (!rc) rc = check_cuda(cudaMallocHost(&c->h_status, kStatusWords * sizeof(int32_t)), "cudaMallocHost(status)");
     for (int i = 0; i < 2 && !rc; ++i) {
         rc = check_cuda(cudaMallocHost(&c->h_stage[i], c->stage_bytes), "cudaMallocHost(stage)");
@@ -95,6 +95,14 @@ extern "C" int cp_ctx_destroy(cp_ctx* c) {
     delete c;
     return CP_OK;
 }
+
+#ifdef CPATTN_TRACE
+// Trace builds only: copy the status buffer (status words + phase trace) to the host.
+extern "C" int cp_debug_read_status_buffer(cp_ctx* c, void* dst, size_t bytes) {
+    if (!c || !dst || bytes > kStatusBytes) return set_error(CP_ERR_INVALID_ARG, "cp_debug_read_status_buffer");
+    return check_cuda(cudaMemcpy(dst, c->d_status, bytes, cudaMemcpyDeviceToHost), "cudaMemcpy(trace)");
+}
+#endif
 
 extern "C" int cp_ctx_poll_status(cp_ctx* c, int32_t* detail) {
     if (!c) return set_error(CP_ERR_INVALID_ARG, "cp_ctx_poll_status: ctx is NULL");

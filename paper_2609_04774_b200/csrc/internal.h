@@ -29,6 +29,11 @@ static_assert(sizeof(TileItem) == 32, "TileItem layout");
 constexpr size_t kWorkspaceHeader = 256;
 constexpr int kTileRows = 128;
 constexpr int kStatusWords = 4;
+#ifdef CPATTN_TRACE
+constexpr size_t kStatusBytes = 64 + 4 * 64 * 8 * sizeof(long long);   // status words + phase trace
+#else
+constexpr size_t kStatusBytes = kStatusWords * sizeof(int32_t);
+#endif
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
