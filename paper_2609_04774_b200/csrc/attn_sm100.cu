@@ -370,33 +370,23 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
     const uint64_t k_desc0 = make_desc(smem_base + kSmemKV, 16, 1024);           // K-major view of a ring slot
     const uint64_t v_desc0 = make_desc(smem_base + kSmemKV, kHalfBytes, 1024);   // MN-major view of a ring slot
 
-    auto issue_s = [&](int wg, uint32_t slot) {
-        if (elect_one()) {
+    // S = Q K^T for one head: 8 MMAs of 16 dims (issued by the elected lane only)
+    auto mma_s = [&](int wg, uint32_t slot) {
 #pragma unroll
-            for (int ks = 0; ks < kD / 16; ++ks) {
-                const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
-                mma_ss(tmem_base + kTmemS + wg * 128, q_desc0 + (wg * (kTileBytes >> 4)) + off,
-                       k_desc0 + slot * (kTileBytes >> 4) + off, kIdescS, ks > 0);
-            }
-            tc_commit(bars + (kBarSReady + wg) * 8);
+        for (int ks = 0; ks < kD / 16; ++ks) {
+            const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+            mma_ss(tmem_base + kTmemS + wg * 128, q_desc0 + (wg * (kTileBytes >> 4)) + off,
+                   k_desc0 + slot * (kTileBytes >> 4) + off, kIdescS, ks > 0);
         }
-        __syncwarp();
     };
-    // P*V over one piece of the tile's keys: 128/kPieces keys = 8/kPieces MMAs of 16 keys
-    auto issue_pv = [&](int wg, int part, uint32_t slot, bool accumulate) {
-        if (elect_one()) {
+    // O += P V over one piece of the tile's keys: 128/kPieces keys = 8/kPieces MMAs of 16 keys
+    auto mma_pv = [&](int wg, int part, uint32_t slot, bool accumulate) {
 #pragma unroll
-            for (int k2 = 0; k2 < 8 / kPieces; ++k2) {
-                const int ks = part * (8 / kPieces) + k2;
-                mma_ts(tmem_base + kTmemO + wg * 128, tmem_base + kTmemS + wg * 128 + ks * 8,
-                       v_desc0 + slot * (kTileBytes >> 4) + ks * (2048 >> 4), kIdescPV, accumulate || ks > 0);
-            }
+        for (int k2 = 0; k2 < 8 / kPieces; ++k2) {
+            const int ks = part * (8 / kPieces) + k2;
+            mma_ts(tmem_base + kTmemO + wg * 128, tmem_base + kTmemS + wg * 128 + ks * 8,
+                   v_desc0 + slot * (kTileBytes >> 4) + ks * (2048 >> 4), kIdescPV, accumulate || ks > 0);
         }
-        __syncwarp();
-    };
-    auto commit = [&](uint32_t bar_id) {
-        if (elect_one()) tc_commit(bars + bar_id * 8);
-        __syncwarp();
     };
 #define MMA_WAIT(id, parity, it) mbar_wait(bars, (id), (parity), abort_flag, p.status, (it))
 
@@ -405,13 +395,18 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
         if (!fetch_unit(p, round, u)) break;
         const int n = u.it.n_kv_tiles;
         MMA_WAIT(kBarQFull, round & 1, round);
-        uint32_t slot = kv_it % kKvStages;
-        MMA_WAIT(kBarKvFull + slot, (kv_it / kKvStages) & 1, 0);
+        const uint32_t slot0 = kv_it % kKvStages;
+        MMA_WAIT(kBarKvFull + slot0, (kv_it / kKvStages) & 1, 0);
         tc_fence_after();
-        issue_s(0, slot);
-        issue_s(1, slot);
-        commit(kBarKvEmpty + slot);
-        if (n == 1) commit(kBarQEmpty);
+        if (elect_one()) {
+            mma_s(0, slot0);
+            tc_commit(bars + (kBarSReady + 0) * 8);
+            mma_s(1, slot0);
+            tc_commit(bars + (kBarSReady + 1) * 8);
+            tc_commit(bars + (kBarKvEmpty + slot0) * 8);
+            if (n == 1) tc_commit(bars + kBarQEmpty * 8);
+        }
+        __syncwarp();
         ++kv_it;
 #pragma unroll 1
         for (int j = 0; j < n; ++j) {
@@ -421,35 +416,36 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
             const bool more = (j + 1 < n);
             const uint32_t k_slot = kv_it % kKvStages;
             const uint32_t k_par = (kv_it / kKvStages) & 1;
+            // K(j+1) and V(j) were requested long ago; check them before the P hand-over
+            MMA_WAIT(kBarKvFull + v_slot, v_par, j);
+            if (more) MMA_WAIT(kBarKvFull + k_slot, k_par, j);
 #pragma unroll
             for (int wg = 0; wg < 2; ++wg) {
                 if (j == 0 && round > 0) MMA_WAIT(kBarOFree + wg, (round - 1) & 1, j);
-                if (wg == 0) {
-                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2, j, 6); }
-                    MMA_WAIT(kBarKvFull + v_slot, v_par, j);
-                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2, j, 7); }
-                }
 #pragma unroll
                 for (int part = 0; part < kPieces; ++part) {
                     MMA_WAIT(kBarPReady + wg * 4 + part, tile_cnt & 1, j);
                     tc_fence_after();
                     if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, part); }
-                    issue_pv(wg, part, v_slot, j > 0);
-                }
-                if (wg == 1) commit(kBarKvEmpty + v_slot);
-                if (more) {
-                    if (wg == 0) MMA_WAIT(kBarKvFull + k_slot, k_par, j);
-                    tc_fence_after();
-                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, 4); }
-                    issue_s(wg, k_slot);
-                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, 5); }
-                    if (wg == 1) {
-                        commit(kBarKvEmpty + k_slot);
-                        if (j + 2 == n) commit(kBarQEmpty);
+                    if (elect_one()) {
+                        mma_pv(wg, part, v_slot, j > 0);
+                        if (part == kPieces - 1) {
+                            if (more) {
+                                mma_s(wg, k_slot);
+                                tc_commit(bars + (kBarSReady + wg) * 8);
+                            } else {
+                                tc_commit(bars + (kBarODone + wg) * 8);
+                            }
+                            if (wg == 1) {
+                                tc_commit(bars + (kBarKvEmpty + v_slot) * 8);
+                                if (more) tc_commit(bars + (kBarKvEmpty + k_slot) * 8);
+                                if (j + 2 == n) tc_commit(bars + kBarQEmpty * 8);
+                            }
+                        }
                     }
-                } else {
-                    commit(kBarODone + wg);
+                    __syncwarp();
                 }
+                if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, 5); }
             }
             if (more) ++kv_it;
             ++tile_cnt;
@@ -500,34 +496,31 @@ __device__ __forceinline__ void exp32(const float (&s)[32], uint32_t (&pk)[16], 
     }
 }
 
-// One 128x128 score tile of one head: two passes over the row in TMEM, 32 columns at a time with the
-// next piece's load in flight (row max; then exponentials, row sum, P back to TMEM in four pieces,
-// each signalled to the MMA warp).  Short code and few live registers on purpose: two warps per SM
-// sub-partition run it half a period apart and it has to stay resident in the instruction cache.
+// One 128x128 score tile of one head: the row is read from TMEM once (four 32-column loads, one
+// wait), reduced to its max, exponentiated in four pieces of 32 keys, and P goes back to TMEM piece
+// by piece, each hand-over signalled to the MMA warp.  Straight-line code in both variants (no
+// per-element branches) so that the scheduler can overlap the MUFU, FMA and ALU pipes.
 // kMasked: the tile reaches past the causal diagonal of some rows; `lim` = visible columns of this row.
 template <bool kMasked>
 __device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, uint32_t p_bar0, float c, int lim,
                                              bool first, float& m, float& l) {
-    float a[32], b[32];
+    float s0[32], s1[32], s2[32], s3[32];
+    TMEM_LD32(s_tmem + 0, s0, 0);
+    TMEM_LD32(s_tmem + 32, s1, 0);
+    TMEM_LD32(s_tmem + 64, s2, 0);
+    TMEM_LD32(s_tmem + 96, s3, 0);
+    tc_wait_ld();
+    if (kMasked) {
+        mask32(s0, lim);
+        mask32(s1, lim - 32);
+        mask32(s2, lim - 64);
+        mask32(s3, lim - 96);
+    }
     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-    TMEM_LD32(s_tmem + 0, a, 0);
-    tc_wait_ld();
-    TMEM_LD32(s_tmem + 32, b, 0);
-    if (kMasked) mask32(a, lim);
-    max32(a, mx0, mx1, mx2, mx3);
-    tc_wait_ld();
-    TMEM_LD32(s_tmem + 64, a, 0);
-    if (kMasked) mask32(b, lim - 32);
-    max32(b, mx0, mx1, mx2, mx3);
-    tc_wait_ld();
-    TMEM_LD32(s_tmem + 96, b, 0);
-    if (kMasked) mask32(a, lim - 64);
-    max32(a, mx0, mx1, mx2, mx3);
-    tc_wait_ld();
-    TMEM_LD32(s_tmem + 0, a, 0);            // first piece of the second pass
-    if (kMasked) mask32(b, lim - 96);
-    max32(b, mx0, mx1, mx2, mx3);
-
+    max32(s0, mx0, mx1, mx2, mx3);
+    max32(s1, mx0, mx1, mx2, mx3);
+    max32(s2, mx0, mx1, mx2, mx3);
+    max32(s3, mx0, mx1, mx2, mx3);
     const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
     const float m_new = fmaxf(m, mx * c);
     if (first) {
@@ -540,7 +533,6 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, u
             l *= alpha;
             m = m_upd;
             // P*V of the previous tile finished before this S was signalled (the pipe runs in issue order)
-            tc_wait_ld();
 #pragma unroll 1
             for (int cc = 0; cc < 4; ++cc) {
                 float o[32];
@@ -556,10 +548,7 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, u
     const float2 nm2 = make_float2(-m, -m);
     float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0, sum2 = sum0, sum3 = sum0;
     uint32_t pk[16];
-#define CP_P_PIECE(cur, nxt, q)                                                         \
-    tc_wait_ld();                                                                       \
-    if ((q) < 3) TMEM_LD32(s_tmem + ((q) + 1) * 32, nxt, 0);                            \
-    if (kMasked) mask32(cur, lim - (q) * 32);                                           \
+#define CP_P_PIECE(cur, q)                                                              \
     exp32<kMasked>(cur, pk, c2, nm2, sum0, sum1, sum2, sum3);                           \
     TMEM_ST16R(s_tmem + (q) * 16, pk, 0);                                               \
     if (((q) + 1) % (4 / kPieces) == 0) {                                               \
@@ -567,10 +556,10 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, u
         tc_fence_before();                                                              \
         mbar_arrive(p_bar0 + ((q) / (4 / kPieces)) * 8);                                \
     }
-    CP_P_PIECE(a, b, 0)
-    CP_P_PIECE(b, a, 1)
-    CP_P_PIECE(a, b, 2)
-    CP_P_PIECE(b, a, 3)
+    CP_P_PIECE(s0, 0)
+    CP_P_PIECE(s1, 1)
+    CP_P_PIECE(s2, 2)
+    CP_P_PIECE(s3, 3)
 #undef CP_P_PIECE
     const float2 st = __fadd2_rn(__fadd2_rn(sum0, sum1), __fadd2_rn(sum2, sum3));
     l += st.x + st.y;
