@@ -135,7 +135,7 @@ class Runner:
         self.new_len = [r.new_len for r in w.requests]
         self.prefix = [r.prefix_len for r in w.requests]
         self.Cs = [r.C for r in w.requests]
-        self.ws = torch.zeros(binding.cp_workspace_bytes(self.new_len, self.Cs), dtype=torch.uint8, device="cuda")
+        self.ws = torch.zeros(binding.cp_workspace_bytes(self.new_len, self.Cs, w.Hq), dtype=torch.uint8, device="cuda")
         self.cu_new, self.cu_pages = w.cu_new, w.cu_pages
         if need_host:
             self._host_buffers()
@@ -451,7 +451,7 @@ def run_table(args, out):
             o = torch.empty((R, Hq, D), dtype=torch.bfloat16, device="cuda")
             lse = torch.empty((Hq, R), dtype=torch.float32, device="cuda")
             po = torch.empty((R, Hq, D), dtype=torch.float32, device="cuda")
-            ws = torch.zeros(binding.cp_workspace_bytes([R], [8]), dtype=torch.uint8, device="cuda")
+            ws = torch.zeros(binding.cp_workspace_bytes([R], [8], Hq), dtype=torch.uint8, device="cuda")
 
             def timeit(fn, reps):
                 for _ in range(2):

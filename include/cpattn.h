@@ -96,10 +96,25 @@ typedef struct {
     int64_t stride_page, stride_tok, stride_head; /* elements */
 } cp_kv_cache;
 
-/* Workspace (device, 256-byte aligned) needed by the attention calls for a batch of B requests:
- * the tile list of the persistent scheduler.  new_len, C: host arrays of B entries.
+/* Workspace (device, 256-byte aligned) needed by the attention calls for a batch of B requests with
+ * Hq query heads: the work lists of the persistent scheduler and the fp32 partial results of the
+ * (query tile, head pair) units whose KV range is split over several CTAs for load balance (about
+ * 55 MB of fixed partial space plus 16 bytes per unit).  new_len, C: host arrays of B entries.
  * Returns 0 on invalid arguments. */
-size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C);
+size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C, int32_t Hq);
+
+/* cp_schedule_inspect -- host only: the work distribution the attention calls would use for a batch
+ * on a device with num_sms SMs (the varlen tile schedule: query tiles of at most 128 rows cut at the
+ * chunk boundaries of every request's zigzag plan; one unit per tile and pair of query heads; whole
+ * units longest first onto the least loaded CTA, the remainder cut along KV so that every CTA gets
+ * the same number of KV tile steps).  summary (8 values): CTAs, query tiles, pieces, split units,
+ * partial slots, largest / smallest per-CTA load in KV tile steps, their total.  pieces (optional,
+ * 6 int32 per piece: cta, tile, head pair, first KV tile, end KV tile, partial slot or -1) and
+ * items (optional, 4 int32 per tile: first packed row, rows, keys visible to the first row, KV tiles)
+ * are filled when non-NULL and large enough (CP_ERR_WORKSPACE otherwise). */
+int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
+                        int32_t Hq, int32_t num_sms, int64_t* summary, int32_t* pieces, int64_t max_pieces,
+                        int32_t* items, int64_t max_items);
 
 /* ---------------------------------------------------------------------------------------------
  * cp_prefill_attn -- all C shards of one request in one launch (Sections 2.1-2.2).
@@ -110,7 +125,8 @@ size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C);
  *              original position (the "restore order" step is fused into the store)
  *   lse        device [Hq, R] fp32: natural-log sum-exp of the scaled scores of each row
  * Every shard's q-tiles are cut at chunk boundaries of cp_plan(R, P, C); the result does not
- * depend on C.  Requires Hq % Hkv == 0 and Hq / Hkv even (two query heads of one KV group share
+ * depend on C.  One persistent launch computes all tiles; the few units that were split along KV
+ * to balance the SMs are combined by a second small launch (an LSE merge of their partials).  Requires Hq % Hkv == 0 and Hq / Hkv even (two query heads of one KV group share
  * each K/V tile).  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
  * ------------------------------------------------------------------------------------------- */
 int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,

@@ -20,7 +20,7 @@ CP_ERR_INVALID_ARG, CP_ERR_UNSUPPORTED, CP_ERR_WORKSPACE, CP_ERR_CUDA, CP_ERR_TI
 CP_DTYPE_BF16, CP_DTYPE_F32 = 0, 1
 
 EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "cp_ctx_poll_status", "cp_plan",
-           "cp_workspace_bytes", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_static", "cp_merge",
+           "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_static", "cp_merge",
            "cp_kv_gather", "cp_kv_append"]
 
 
@@ -125,10 +125,30 @@ def cp_plan(new_len: int, prefix_len: int, C: int):
             for s in arr[:C]]
 
 
-def cp_workspace_bytes(new_len, C) -> int:
+def cp_workspace_bytes(new_len, C, Hq) -> int:
     nl, cs = _i64(new_len).reshape(-1), _i32(C).reshape(-1)
     return int(load().cp_workspace_bytes(ctypes.c_int32(nl.size), nl.ctypes.data_as(ctypes.c_void_p),
-                                         cs.ctypes.data_as(ctypes.c_void_p)))
+                                         cs.ctypes.data_as(ctypes.c_void_p), ctypes.c_int32(Hq)))
+
+
+def cp_schedule_inspect(cu_new, prefix_len, C, Hq, num_sms=148, want_lists=True):
+    """Host-only view of the varlen tile schedule: (summary dict, pieces [n,6] int32, items [n,4] int32)."""
+    cu_new, prefix_len, C = _i64(cu_new), _i64(prefix_len), _i32(C)
+    B = prefix_len.size
+    summary = np.zeros(8, dtype=np.int64)
+    args = [ctypes.c_int32(B), cu_new.ctypes.data_as(ctypes.c_void_p), prefix_len.ctypes.data_as(ctypes.c_void_p),
+            C.ctypes.data_as(ctypes.c_void_p), ctypes.c_int32(Hq), ctypes.c_int32(num_sms),
+            summary.ctypes.data_as(ctypes.c_void_p)]
+    _check(load().cp_schedule_inspect(*args, None, ctypes.c_int64(0), None, ctypes.c_int64(0)))
+    keys = ["grid", "tiles", "pieces", "split_units", "slots", "max_load", "min_load", "total"]
+    info = dict(zip(keys, (int(x) for x in summary)))
+    if not want_lists:
+        return info, None, None
+    pieces = np.zeros((info["pieces"], 6), dtype=np.int32)
+    items = np.zeros((info["tiles"], 4), dtype=np.int32)
+    _check(load().cp_schedule_inspect(*args, pieces.ctypes.data_as(ctypes.c_void_p), ctypes.c_int64(pieces.shape[0]),
+                                      items.ctypes.data_as(ctypes.c_void_p), ctypes.c_int64(items.shape[0])))
+    return info, pieces, items
 
 
 def make_cache(k_pages, v_pages) -> cp_kv_cache:

@@ -76,6 +76,10 @@ constexpr int kPolyOf4 = 1;                            // pairs out of every fou
 struct AttnParams {
     const TileItem* items;
     int32_t n_items;
+    const int32_t* cta_off;    // explicit schedule: pieces of CTA b are pieces[cta_off[b] .. cta_off[b+1]);
+    const PieceEntry* pieces;  // NULL: implicit serpentine schedule over whole units (no KV splits)
+    float* partial_o;          // [slots][2 heads][128 rows][128] fp32, normalised partial outputs
+    float* partial_lse;        // [slots][2 heads][128 rows]
     int32_t pairs_per_tile;   // Hq / 2
     int32_t group;            // Hq / Hkv
     int32_t Hq;
@@ -280,26 +284,44 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar_base, uint32_t bar_id, ui
 #define CP_TRACE(who, j, e)
 #endif
 
+// One piece of work of a CTA: KV tiles [t_begin, t_end) of one query tile for one pair of heads.
 struct UnitInfo {
     TileItem it;
     int head0;
     int kv_head;
+    int t_begin, t_end;   // KV tile range of this piece
+    int slot;             // < 0: whole unit, final rows; >= 0: partial slot
 };
 
-// Serpentine static schedule over the longest-first unit list: in even rounds CTA c takes unit
-// round*grid + c, in odd rounds round*grid + (grid-1-c), which evens out the sorted lengths.
-__device__ __forceinline__ int64_t unit_index(int round) {
-    const int g = gridDim.x;
-    const int c = (round & 1) ? (g - 1 - (int)blockIdx.x) : (int)blockIdx.x;
-    return (int64_t)round * g + c;
-}
+// Two schedules.  Explicit (p.pieces != NULL): the host lists, per CTA, whole units and the KV
+// ranges of units that were split to fill every CTA to the same number of KV tile steps.  Implicit:
+// serpentine over the longest-first unit list -- in even rounds CTA c takes unit round*grid + c, in
+// odd rounds round*grid + (grid-1-c), which evens out the sorted lengths; whole units only.
 __device__ __forceinline__ bool fetch_unit(const AttnParams& p, int round, UnitInfo& u) {
-    const int64_t idx = unit_index(round);
-    const int64_t total = (int64_t)p.n_items * p.pairs_per_tile;
-    if (idx >= total) return false;
-    const int item = (int)(idx / p.pairs_per_tile);
-    const int pair = (int)(idx - (int64_t)item * p.pairs_per_tile);
-    u.it = p.items[item];
+    int item, pair;
+    if (p.pieces != nullptr) {
+        const int idx = p.cta_off[blockIdx.x] + round;
+        if (idx >= p.cta_off[blockIdx.x + 1]) return false;
+        const PieceEntry e = p.pieces[idx];
+        item = e.item;
+        pair = e.pair;
+        u.t_begin = e.t_begin;
+        u.t_end = e.t_end;
+        u.slot = e.slot;
+        u.it = p.items[item];
+    } else {
+        const int g = gridDim.x;
+        const int c = (round & 1) ? (g - 1 - (int)blockIdx.x) : (int)blockIdx.x;
+        const int64_t idx = (int64_t)round * g + c;
+        const int64_t total = (int64_t)p.n_items * p.pairs_per_tile;
+        if (idx >= total) return false;
+        item = (int)(idx / p.pairs_per_tile);
+        pair = (int)(idx - (int64_t)item * p.pairs_per_tile);
+        u.it = p.items[item];
+        u.t_begin = 0;
+        u.t_end = u.it.n_kv_tiles;
+        u.slot = -1;
+    }
     u.head0 = 2 * pair;
     u.kv_head = u.head0 / p.group;
     return true;
@@ -326,8 +348,8 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
                                 u.head0 + h, u.it.q_row0);
         }
         __syncwarp();
-        const int n_tiles = u.it.n_kv_tiles;
-        for (int j0 = 0; j0 < n_tiles; j0 += 16) {
+        const int n_tiles = u.t_end;
+        for (int j0 = u.t_begin; j0 < n_tiles; j0 += 16) {
             // the warp fetches the page ids of 16 KV tiles (32 pages) at once
             const int pg = 2 * j0 + lane;
             const int my_page = (pg < u.it.n_pages) ? __ldg(p.page_table + u.it.pt_base + pg) : p.oob_page;
@@ -393,7 +415,7 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
     for (int round = 0;; ++round) {
         UnitInfo u;
         if (!fetch_unit(p, round, u)) break;
-        const int n = u.it.n_kv_tiles;
+        const int n = u.t_end;
         MMA_WAIT(kBarQFull, round & 1, round);
         const uint32_t slot0 = kv_it % kKvStages;
         MMA_WAIT(kBarKvFull + slot0, (kv_it / kKvStages) & 1, 0);
@@ -404,12 +426,12 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
             mma_s(1, slot0);
             tc_commit(bars + (kBarSReady + 1) * 8);
             tc_commit(bars + (kBarKvEmpty + slot0) * 8);
-            if (n == 1) tc_commit(bars + kBarQEmpty * 8);
+            if (u.t_begin + 1 == n) tc_commit(bars + kBarQEmpty * 8);
         }
         __syncwarp();
         ++kv_it;
 #pragma unroll 1
-        for (int j = 0; j < n; ++j) {
+        for (int j = u.t_begin; j < n; ++j) {
             const uint32_t v_slot = kv_it % kKvStages;
             const uint32_t v_par = (kv_it / kKvStages) & 1;
             ++kv_it;
@@ -421,14 +443,14 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
             if (more) MMA_WAIT(kBarKvFull + k_slot, k_par, j);
 #pragma unroll
             for (int wg = 0; wg < 2; ++wg) {
-                if (j == 0 && round > 0) MMA_WAIT(kBarOFree + wg, (round - 1) & 1, j);
+                if (j == u.t_begin && round > 0) MMA_WAIT(kBarOFree + wg, (round - 1) & 1, j);
 #pragma unroll
                 for (int part = 0; part < kPieces; ++part) {
                     MMA_WAIT(kBarPReady + wg * 4 + part, tile_cnt & 1, j);
                     tc_fence_after();
                     if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, part); }
                     if (elect_one()) {
-                        mma_pv(wg, part, v_slot, j > 0);
+                        mma_pv(wg, part, v_slot, j > u.t_begin);
                         if (part == kPieces - 1) {
                             if (more) {
                                 mma_s(wg, k_slot);
@@ -545,7 +567,10 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, u
         }
     }
     const float2 c2 = make_float2(c, c);
-    const float2 nm2 = make_float2(-m, -m);
+    // a row that has seen no key yet (only possible in masked tiles of a KV-split piece) keeps m = -inf;
+    // subtracting 0 instead keeps its weights at exactly 0 rather than NaN
+    const float m_sub = (kMasked && m == -INFINITY) ? 0.f : m;
+    const float2 nm2 = make_float2(-m_sub, -m_sub);
     float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0, sum2 = sum0, sum3 = sum0;
     uint32_t pk[16];
 #define CP_P_PIECE(cur, q)                                                              \
@@ -585,39 +610,43 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
     for (int round = 0;; ++round) {
         UnitInfo u;
         if (!fetch_unit(p, round, u)) break;
-        const int n = u.it.n_kv_tiles;
+        const int n = u.t_end;
         const int head = u.head0 + wg;
         float m = -INFINITY;   // running row max in log2 units (possibly stale by < threshold)
         float l = 0.f;         // running row sum of 2^(s - m)
         // tiles below n_full lie entirely under the causal diagonal of every row of the q-tile
         const int n_full = u.it.kv_len0 / kBlockN;
 #pragma unroll 1
-        for (int j = 0; j < n; ++j) {
+        for (int j = u.t_begin; j < n; ++j) {
             SM_WAIT(kBarSReady + wg, tile_cnt & 1, j);
             tc_fence_after();
             if (row == CPATTN_TRACE_ROW) { CP_TRACE(wg, j, 0); }
             if (j < n_full)
-                softmax_tile<false>(s_tmem, o_tmem, p_bar0, c, 0, j == 0, m, l);
+                softmax_tile<false>(s_tmem, o_tmem, p_bar0, c, 0, j == u.t_begin, m, l);
             else
-                softmax_tile<true>(s_tmem, o_tmem, p_bar0, c, u.it.kv_len0 + row - j * kBlockN, j == 0, m, l);
+                softmax_tile<true>(s_tmem, o_tmem, p_bar0, c, u.it.kv_len0 + row - j * kBlockN, j == u.t_begin, m, l);
             if (row == CPATTN_TRACE_ROW) { CP_TRACE(wg, j, 6); }
             ++tile_cnt;
         }
         // epilogue: O / l -> global at the row's original position; LSE in natural log
         SM_WAIT(kBarODone + wg, round & 1, n);
         tc_fence_after();
-        const float inv_l = 1.f / l;
+        // a row of a KV-split piece may see none of the piece's keys: l = 0, written as O = 0, lse = -inf
+        const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
+        const bool partial = u.slot >= 0;
         const bool valid = row < u.it.n_rows;
         const int64_t grow_idx = (int64_t)u.it.q_row0 + row;
+        float* part_row = p.partial_o + (((int64_t)max(u.slot, 0) * 2 + wg) * kBlockM + row) * kD;
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
             float o[32];
             TMEM_LD32(o_tmem + cc * 32, o, 0);
             tc_wait_ld();
             if (valid) {
-                if (p.out_f32) {
-                    float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) +
-                                                            (grow_idx * p.Hq + head) * kD + cc * 32);
+                if (partial || p.out_f32) {
+                    float4* dst = partial ? reinterpret_cast<float4*>(part_row + cc * 32)
+                                          : reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) +
+                                                                      (grow_idx * p.Hq + head) * kD + cc * 32);
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
                         dst[i] = make_float4(o[4 * i] * inv_l, o[4 * i + 1] * inv_l, o[4 * i + 2] * inv_l, o[4 * i + 3] * inv_l);
@@ -636,7 +665,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
                 }
             }
         }
-        if (valid) p.lse[(int64_t)head * p.lse_stride + grow_idx] = (m + lg2(l)) * 0.6931471805599453f;
+        if (valid) {
+            const float lse_val = (l > 0.f) ? (m + lg2(l)) * 0.6931471805599453f : -INFINITY;
+            if (partial) p.partial_lse[((int64_t)u.slot * 2 + wg) * kBlockM + row] = lse_val;
+            else p.lse[(int64_t)head * p.lse_stride + grow_idx] = lse_val;
+        }
         tc_fence_before();
         mbar_arrive(bars + (kBarOFree + wg) * 8);
     }
@@ -709,6 +742,90 @@ __global__ void fill_neg_inf_kernel(float* p, int64_t n) {
         p[i] = -INFINITY;
 }
 
+// LSE merge of the KV-split units: block b combines the partial slots of merges[b] into the final
+// rows.  One warp per (head, row), one float4 per lane; weights exp(lse_k - max) by fast exp.
+struct FixupParams {
+    const TileItem* items;
+    const MergeEntry* merges;
+    const int32_t* merge_slots;
+    const float* partial_o;
+    const float* partial_lse;
+    void* out;
+    int32_t out_f32;
+    int32_t Hq;
+    float* lse;
+    int64_t lse_stride;
+};
+
+constexpr int kFixupRowsPerBlock = 16;    // 8 warps x 2 (head, row) combinations
+
+// grid = (split units, 256 / kFixupRowsPerBlock): each warp combines two rows; the partial LSEs of a
+// row are loaded 32 slots at a time (lane k holds slot k), max and sum by warp shuffles.
+__global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p) {
+    const MergeEntry me = p.merges[blockIdx.x];
+    const TileItem it = p.items[me.item];
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int r2 = 0; r2 < 2; ++r2) {
+        const int hr = blockIdx.y * kFixupRowsPerBlock + warp * 2 + r2;
+        const int wg = hr / kBlockM;
+        const int row = hr - wg * kBlockM;
+        if (row >= it.n_rows) continue;
+        // pass 1: max of the partial LSEs (lane k of each group of 32 slots holds slot k)
+        float m = -INFINITY;
+        for (int base = 0; base < me.n_slots; base += 32) {
+            if (base + lane < me.n_slots) {
+                const int slot = p.merge_slots[me.slot_off + base + lane];
+                m = fmaxf(m, p.partial_lse[((int64_t)slot * 2 + wg) * kBlockM + row]);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        // pass 2: weights exp(lse_k - m) and the weighted sum of the partial rows
+        float wsum = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int base = 0; base < me.n_slots; base += 32) {
+            int my_slot = 0;
+            float w_mine = 0.f;
+            if (base + lane < me.n_slots) {
+                my_slot = p.merge_slots[me.slot_off + base + lane];
+                const float my_lse = p.partial_lse[((int64_t)my_slot * 2 + wg) * kBlockM + row];
+                w_mine = (my_lse == -INFINITY) ? 0.f : __expf(my_lse - m);
+            }
+            wsum += w_mine;
+            const int cnt = min(32, me.n_slots - base);
+            for (int k = 0; k < cnt; ++k) {
+                const float w = __shfl_sync(0xffffffffu, w_mine, k);
+                const int slot = __shfl_sync(0xffffffffu, my_slot, k);
+                if (w > 0.f) {     // a zero weight hides whatever the slot holds for this row
+                    const float4 x = reinterpret_cast<const float4*>(p.partial_o + (((int64_t)slot * 2 + wg) * kBlockM + row) * kD)[lane];
+                    acc.x = fmaf(w, x.x, acc.x);
+                    acc.y = fmaf(w, x.y, acc.y);
+                    acc.z = fmaf(w, x.z, acc.z);
+                    acc.w = fmaf(w, x.w, acc.w);
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+        const float inv = 1.f / wsum;     // every row of a unit sees at least key 0, so wsum > 0
+        const int head = 2 * me.pair + wg;
+        const int64_t grow = (int64_t)it.q_row0 + row;
+        const int64_t off = (grow * p.Hq + head) * kD + lane * 4;
+        if (p.out_f32) {
+            *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off) =
+                make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+        } else {
+            uint2 pk;
+            pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+            pk.y = pack_bf16(acc.z * inv, acc.w * inv);
+            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off) = pk;
+        }
+        if (lane == 0) p.lse[(int64_t)head * p.lse_stride + grow] = m + __logf(wsum);
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
@@ -739,19 +856,18 @@ int encode_maps(cp_ctx* ctx, const void* q, int64_t total_rows, int32_t Hq, cons
     return CP_OK;
 }
 
-// Copies the tile list into the workspace through one of the context's two pinned staging buffers
-// (falls back to a pageable copy for lists that do not fit).
-int upload_tiles(cp_ctx* ctx, const std::vector<TileItem>& tiles, void* workspace, cudaStream_t s) {
-    const size_t bytes = tiles.size() * sizeof(TileItem);
-    uint8_t* dst = static_cast<uint8_t*>(workspace) + kWorkspaceHeader;
+// Copies a host block into the workspace through one of the context's two pinned staging buffers
+// (falls back to a pageable copy for blocks that do not fit).
+int upload_block(cp_ctx* ctx, const std::vector<uint8_t>& block, void* dst, cudaStream_t s) {
+    const size_t bytes = block.size();
     if (bytes > ctx->stage_bytes)
-        return check_cuda(cudaMemcpyAsync(dst, tiles.data(), bytes, cudaMemcpyHostToDevice, s), "tile list copy");
+        return check_cuda(cudaMemcpyAsync(dst, block.data(), bytes, cudaMemcpyHostToDevice, s), "schedule copy");
     const int i = ctx->stage_next;
     ctx->stage_next ^= 1;
     if (ctx->stage_used[i])
         if (int rc = check_cuda(cudaEventSynchronize(ctx->stage_event[i]), "cudaEventSynchronize(stage)")) return rc;
-    memcpy(ctx->h_stage[i], tiles.data(), bytes);
-    if (int rc = check_cuda(cudaMemcpyAsync(dst, ctx->h_stage[i], bytes, cudaMemcpyHostToDevice, s), "tile list copy"))
+    memcpy(ctx->h_stage[i], block.data(), bytes);
+    if (int rc = check_cuda(cudaMemcpyAsync(dst, ctx->h_stage[i], bytes, cudaMemcpyHostToDevice, s), "schedule copy"))
         return rc;
     ctx->stage_used[i] = true;
     return check_cuda(cudaEventRecord(ctx->stage_event[i], s), "cudaEventRecord(stage)");
@@ -787,28 +903,47 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     }
     if (cu_new[B] > 0x7fffff00ll || cu_pages[B] > 0x7fffff00ll)
         return set_error(CP_ERR_UNSUPPORTED, "%s: more than 2^31 packed rows or pages", who);
-    const size_t need_ws = cp_workspace_bytes(B, new_len.data(), C);
+    const size_t need_ws = cp_workspace_bytes(B, new_len.data(), C, Hq);
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need_ws)
         return set_error(CP_ERR_WORKSPACE, "%s: workspace %p of %zu bytes; need %zu bytes, 256-byte aligned", who,
                          workspace, workspace_bytes, need_ws);
 
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    std::vector<TileItem> tiles;
-    build_tiles(B, cu_new, prefix_len, C, cu_pages, only_shard, tiles);
+    Schedule sch;
+    build_tiles(B, cu_new, prefix_len, C, cu_pages, only_shard, sch.items);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (tiles.empty()) return CP_OK;   // the shard owns no rows (only empty chunks)
+    if (sch.items.empty()) return CP_OK;   // the shard owns no rows (only empty chunks)
+    if (int rc = build_schedule(Hq / 2, ctx->num_sms, sch)) return rc;
+    const WorkspaceLayout lay = workspace_layout(sch.items.size(), sch.pieces.size(), sch.merges.size(),
+                                                 sch.merge_slots.size(), sch.grid, sch.n_slots);
+    if (lay.total > workspace_bytes)
+        return set_error(CP_ERR_WORKSPACE, "%s: schedule needs %zu workspace bytes, have %zu", who, lay.total, workspace_bytes);
 
     CUtensorMap tmQ, tmK, tmV;
     if (int rc = encode_maps(ctx, q, cu_new[B], Hq, cache, &tmQ, &tmK, &tmV)) return rc;
-    if (int rc = upload_tiles(ctx, tiles, workspace, s)) return rc;
+    // one contiguous block: items | cta_off | pieces | merges | merge_slots (offsets as in the layout)
+    std::vector<uint8_t> block(lay.partial_o - lay.items, 0);
+    memcpy(block.data() + (lay.items - lay.items), sch.items.data(), sch.items.size() * sizeof(TileItem));
+    memcpy(block.data() + (lay.cta_off - lay.items), sch.cta_off.data(), sch.cta_off.size() * sizeof(int32_t));
+    memcpy(block.data() + (lay.pieces - lay.items), sch.pieces.data(), sch.pieces.size() * sizeof(PieceEntry));
+    if (!sch.merges.empty()) {
+        memcpy(block.data() + (lay.merges - lay.items), sch.merges.data(), sch.merges.size() * sizeof(MergeEntry));
+        memcpy(block.data() + (lay.merge_slots - lay.items), sch.merge_slots.data(), sch.merge_slots.size() * sizeof(int32_t));
+    }
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (int rc = upload_block(ctx, block, ws + lay.items, s)) return rc;
     if (!ctx->attn_attr_set) {
         if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
         ctx->attn_attr_set = true;
     }
     AttnParams p;
-    p.items = reinterpret_cast<const TileItem*>(static_cast<uint8_t*>(workspace) + kWorkspaceHeader);
-    p.n_items = (int32_t)tiles.size();
+    p.items = reinterpret_cast<const TileItem*>(ws + lay.items);
+    p.n_items = (int32_t)sch.items.size();
+    p.cta_off = reinterpret_cast<const int32_t*>(ws + lay.cta_off);
+    p.pieces = reinterpret_cast<const PieceEntry*>(ws + lay.pieces);
+    p.partial_o = reinterpret_cast<float*>(ws + lay.partial_o);
+    p.partial_lse = reinterpret_cast<float*>(ws + lay.partial_lse);
     p.pairs_per_tile = Hq / 2;
     p.group = Hq / cache->Hkv;
     p.Hq = Hq;
@@ -820,10 +955,24 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.lse = lse;
     p.lse_stride = cu_new[B];
     p.status = ctx->d_status;
-    const int64_t units = (int64_t)tiles.size() * p.pairs_per_tile;
-    const int grid = (int)std::min<int64_t>(units, ctx->num_sms);
-    cp_attn_kernel<<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
-    return check_cuda(cudaGetLastError(), who);
+    cp_attn_kernel<<<sch.grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
+    if (int rc = check_cuda(cudaGetLastError(), who)) return rc;
+    if (!sch.merges.empty()) {
+        FixupParams f;
+        f.items = p.items;
+        f.merges = reinterpret_cast<const MergeEntry*>(ws + lay.merges);
+        f.merge_slots = reinterpret_cast<const int32_t*>(ws + lay.merge_slots);
+        f.partial_o = p.partial_o;
+        f.partial_lse = p.partial_lse;
+        f.out = out;
+        f.out_f32 = out_f32;
+        f.Hq = Hq;
+        f.lse = lse;
+        f.lse_stride = cu_new[B];
+        cp_attn_fixup_kernel<<<dim3((unsigned)sch.merges.size(), 2 * kBlockM / kFixupRowsPerBlock), 256, 0, s>>>(f);
+        if (int rc = check_cuda(cudaGetLastError(), "cp_attn_fixup launch")) return rc;
+    }
+    return CP_OK;
 }
 
 }  // namespace
@@ -965,6 +1114,10 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     AttnParams p;
     p.items = reinterpret_cast<const TileItem*>(st->scratch + kWorkspaceHeader);
     p.n_items = (int32_t)tiles.size();
+    p.cta_off = nullptr;       // implicit schedule over whole units: no piece lists, no partial results
+    p.pieces = nullptr;
+    p.partial_o = nullptr;
+    p.partial_lse = nullptr;
     p.pairs_per_tile = Hq / 2;
     p.group = Hq / cache->Hkv;
     p.Hq = Hq;

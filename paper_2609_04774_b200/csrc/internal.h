@@ -26,6 +26,49 @@ struct TileItem {
 };
 static_assert(sizeof(TileItem) == 32, "TileItem layout");
 
+// One entry of a CTA's work list: KV tiles [t_begin, t_end) of query tile `item` for head pair `pair`.
+// slot < 0: the piece covers the whole KV range of the unit and writes the final rows; otherwise it
+// writes a normalised fp32 partial (+ LSE) into partial slot `slot`, merged afterwards.
+struct PieceEntry {
+    int32_t item;
+    int16_t pair;
+    int16_t slot;
+    int32_t t_begin;
+    int32_t t_end;
+};
+static_assert(sizeof(PieceEntry) == 16, "PieceEntry layout");
+
+// A (query tile, head pair) unit whose KV range was split over several CTAs: its partial slots.
+struct MergeEntry {
+    int32_t item;
+    int32_t pair;
+    int32_t n_slots;
+    int32_t slot_off;   // into the flat slot list
+};
+
+// Host-side schedule of one launch.
+struct Schedule {
+    std::vector<TileItem> items;        // query tiles, longest first
+    std::vector<int32_t> cta_off;       // grid + 1 offsets into pieces
+    std::vector<PieceEntry> pieces;
+    std::vector<MergeEntry> merges;
+    std::vector<int32_t> merge_slots;
+    int32_t grid = 0;
+    int32_t n_slots = 0;
+};
+
+// Device layout of a schedule inside the workspace (byte offsets from the workspace base).
+struct WorkspaceLayout {
+    size_t items, cta_off, pieces, merges, merge_slots, partial_o, partial_lse, total;
+};
+
+constexpr int kMaxGrid = 192;                          // upper bound on CTAs (SMs) a schedule may use
+constexpr int kMaxSlots = 2 * kMaxGrid + 32;           // partial slots a schedule may use
+constexpr int kMinShareTiles = 8;                      // smallest per-CTA share worth spreading work for
+constexpr int kMinPieceTiles = 4;                      // never cut a unit into pieces shorter than this
+constexpr size_t kPartialRowFloats = 128;              // fp32 values of one partial row
+constexpr size_t kPartialSlotRows = 2 * 128;           // two heads x 128 query rows per slot
+
 constexpr size_t kWorkspaceHeader = 256;
 constexpr int kTileRows = 128;
 constexpr int kStatusWords = 4;
@@ -49,6 +92,12 @@ int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C);
 int validate_kv_cache(const cp_kv_cache* c, const char* who);
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
                 const int64_t* cu_pages, int32_t only_shard, std::vector<TileItem>& out);
+// Distributes the (tile, head pair) units of s.items over `grid_max` CTAs: whole units longest first
+// onto the least loaded CTA while they fit under the per-CTA share, the rest cut into KV ranges that
+// fill every CTA to the same number of KV tiles.  Fills cta_off / pieces / merges / merge_slots.
+int build_schedule(int32_t pairs_per_tile, int32_t grid_max, Schedule& s);
+WorkspaceLayout workspace_layout(size_t n_items, size_t n_pieces, size_t n_merges, size_t n_merge_slots, size_t grid,
+                                 size_t n_slots);
 
 }  // namespace cpattn
 

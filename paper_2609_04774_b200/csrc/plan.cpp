@@ -1,5 +1,7 @@
 // Host-side integer work: the zigzag shard plan and the q-tile list of the persistent scheduler.
 #include <algorithm>
+#include <climits>
+#include <cstdint>
 
 #include "internal.h"
 
@@ -60,6 +62,113 @@ int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, con
     return CP_OK;
 }
 
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+WorkspaceLayout workspace_layout(size_t n_items, size_t n_pieces, size_t n_merges, size_t n_merge_slots, size_t grid,
+                                 size_t n_slots) {
+    WorkspaceLayout w;
+    size_t off = kWorkspaceHeader;
+    w.items = off;        off = align_up(off + n_items * sizeof(TileItem), 256);
+    w.cta_off = off;      off = align_up(off + (grid + 1) * sizeof(int32_t), 256);
+    w.pieces = off;       off = align_up(off + n_pieces * sizeof(PieceEntry), 256);
+    w.merges = off;       off = align_up(off + n_merges * sizeof(MergeEntry), 256);
+    w.merge_slots = off;  off = align_up(off + n_merge_slots * sizeof(int32_t), 256);
+    w.partial_o = off;    off = align_up(off + n_slots * kPartialSlotRows * kPartialRowFloats * sizeof(float), 256);
+    w.partial_lse = off;  off = align_up(off + n_slots * kPartialSlotRows * sizeof(float), 256);
+    w.total = off;
+    return w;
+}
+
+int build_schedule(int32_t pairs_per_tile, int32_t grid_max, Schedule& s) {
+    const int64_t n_items = (int64_t)s.items.size();
+    const int64_t n_units = n_items * pairs_per_tile;
+    int64_t W = 0;
+    for (const TileItem& t : s.items) W += (int64_t)t.n_kv_tiles * pairs_per_tile;
+    if (W <= 0 || W > 0x7fffffffll) return set_error(CP_ERR_UNSUPPORTED, "schedule: %lld KV tile steps", (long long)W);
+    grid_max = std::min(grid_max, kMaxGrid);
+    // per-CTA share of KV tile steps; never below a short unit's length (cutting those only adds
+    // prologues and merges), which also shrinks the grid for tiny problems
+    int32_t longest = 0;
+    for (const TileItem& t : s.items) longest = std::max(longest, t.n_kv_tiles);
+    const int64_t T = std::max<int64_t>((W + grid_max - 1) / grid_max, std::min<int32_t>(longest, kMinShareTiles));
+    const int32_t G = (int32_t)std::max<int64_t>(1, std::min<int64_t>(grid_max, (W + T - 1) / T));
+    s.grid = G;
+
+    std::vector<int64_t> load(G, 0);
+    std::vector<std::vector<PieceEntry>> lists(G);
+    struct TailUnit { int32_t item; int32_t pair; int32_t n; };
+    std::vector<TailUnit> tail;
+
+    // 1. whole units, longest first, onto the least loaded CTA while they fit under the share
+    using Slot = std::pair<int64_t, int32_t>;             // (load, cta); smallest first
+    std::vector<Slot> heap;
+    heap.reserve(G);
+    for (int32_t c = 0; c < G; ++c) heap.push_back({0, c});
+    auto cmp = [](const Slot& a, const Slot& b) { return a > b; };
+    std::make_heap(heap.begin(), heap.end(), cmp);
+    for (int64_t i = 0; i < n_items; ++i) {
+        const int32_t n = s.items[i].n_kv_tiles;
+        for (int32_t pr = 0; pr < pairs_per_tile; ++pr) {
+            std::pop_heap(heap.begin(), heap.end(), cmp);
+            Slot& top = heap.back();
+            if (top.first + n <= T) {
+                lists[top.second].push_back({(int32_t)i, (int16_t)pr, (int16_t)-1, 0, n});
+                top.first += n;
+                load[top.second] = top.first;
+            } else {
+                tail.push_back({(int32_t)i, pr, n});
+            }
+            std::push_heap(heap.begin(), heap.end(), cmp);
+        }
+    }
+    (void)n_units;
+
+    // 2. the remaining units, cut into KV ranges that fill every CTA up to the share
+    const int64_t minp = std::min<int64_t>(kMinPieceTiles, std::max<int64_t>(1, T));   // shortest piece worth a cut
+    struct Cut { int32_t cta; int32_t t_begin; int32_t t_end; };
+    std::vector<std::vector<Cut>> cuts(tail.size());
+    int32_t c = 0;
+    for (size_t u = 0; u < tail.size(); ++u) {
+        int32_t t = 0;
+        const int32_t n = tail[u].n;
+        while (t < n) {
+            while (c < G - 1 && T - load[c] < std::min<int64_t>(minp, n - t)) ++c;   // CTA is full
+            int64_t len = std::min<int64_t>(n - t, std::max<int64_t>(T - load[c], 0));
+            if (c == G - 1 || len <= 0) len = n - t;                                        // last CTA takes what is left
+            if (n - t - len > 0 && n - t - len < minp) len = n - t;                           // no tiny remainder
+            cuts[u].push_back({c, t, (int32_t)(t + len)});
+            load[c] += len;
+            t += (int32_t)len;
+        }
+    }
+    s.merges.clear();
+    s.merge_slots.clear();
+    int32_t n_slots = 0;
+    for (size_t u = 0; u < tail.size(); ++u) {
+        const bool split = cuts[u].size() > 1;
+        if (split) s.merges.push_back({tail[u].item, tail[u].pair, (int32_t)cuts[u].size(), (int32_t)s.merge_slots.size()});
+        for (const Cut& k : cuts[u]) {
+            int16_t slot = -1;
+            if (split) {
+                slot = (int16_t)n_slots++;
+                s.merge_slots.push_back(slot);
+            }
+            lists[k.cta].push_back({tail[u].item, (int16_t)tail[u].pair, slot, k.t_begin, k.t_end});
+        }
+    }
+    if (n_slots > kMaxSlots) return set_error(CP_ERR_UNSUPPORTED, "schedule: %d partial slots", n_slots);
+    s.n_slots = n_slots;
+
+    s.cta_off.assign(G + 1, 0);
+    s.pieces.clear();
+    for (int32_t k = 0; k < G; ++k) {
+        s.cta_off[k] = (int32_t)s.pieces.size();
+        s.pieces.insert(s.pieces.end(), lists[k].begin(), lists[k].end());
+    }
+    s.cta_off[G] = (int32_t)s.pieces.size();
+    return CP_OK;
+}
+
 }  // namespace cpattn
 
 using namespace cpattn;
@@ -81,9 +190,60 @@ extern "C" int cp_plan(int64_t new_len, int64_t prefix_len, int32_t C, cp_shard_
     return CP_OK;
 }
 
-extern "C" size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C) {
-    if (B < 1 || !new_len || !C) return 0;
+extern "C" size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C, int32_t Hq) {
+    if (B < 1 || !new_len || !C || Hq < 2) return 0;
     const int64_t n = max_tiles(B, new_len, C);
     if (n < 0) return 0;
-    return kWorkspaceHeader + (size_t)n * sizeof(TileItem);
+    const size_t pairs = (size_t)Hq / 2;
+    // every unit is one piece, plus at most one extra piece per cut; the partial slots are bounded
+    return workspace_layout((size_t)n, (size_t)n * pairs + kMaxSlots, kMaxSlots, kMaxSlots, kMaxGrid, kMaxSlots).total;
+}
+
+extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
+                                   int32_t Hq, int32_t num_sms, int64_t* summary, int32_t* pieces, int64_t max_pieces,
+                                   int32_t* items, int64_t max_items) {
+    if (B < 1 || !cu_new || !prefix_len || !C || Hq < 2 || Hq % 2 != 0 || num_sms < 1 || !summary)
+        return set_error(CP_ERR_INVALID_ARG, "cp_schedule_inspect: bad arguments");
+    std::vector<int64_t> cu_pages(B + 1, 0);
+    for (int32_t b = 0; b < B; ++b) {
+        const int64_t R = cu_new[b + 1] - cu_new[b];
+        if (R < 1 || prefix_len[b] < 0 || C[b] < 1) return set_error(CP_ERR_INVALID_ARG, "cp_schedule_inspect: request %d", b);
+        cu_pages[b + 1] = cu_pages[b] + (prefix_len[b] + R + 63) / 64;
+    }
+    Schedule sch;
+    build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), -1, sch.items);
+    if (int rc = build_schedule(Hq / 2, num_sms, sch)) return rc;
+    int64_t max_load = 0, min_load = INT64_MAX, total = 0;
+    for (int32_t c = 0; c < sch.grid; ++c) {
+        int64_t load = 0;
+        for (int32_t k = sch.cta_off[c]; k < sch.cta_off[c + 1]; ++k) load += sch.pieces[k].t_end - sch.pieces[k].t_begin;
+        max_load = std::max(max_load, load);
+        min_load = std::min(min_load, load);
+        total += load;
+    }
+    summary[0] = sch.grid;
+    summary[1] = (int64_t)sch.items.size();
+    summary[2] = (int64_t)sch.pieces.size();
+    summary[3] = (int64_t)sch.merges.size();
+    summary[4] = sch.n_slots;
+    summary[5] = max_load;
+    summary[6] = min_load;
+    summary[7] = total;
+    if (pieces) {
+        if ((int64_t)sch.pieces.size() > max_pieces) return set_error(CP_ERR_WORKSPACE, "cp_schedule_inspect: %zu pieces", sch.pieces.size());
+        for (int32_t c = 0; c < sch.grid; ++c)
+            for (int32_t k = sch.cta_off[c]; k < sch.cta_off[c + 1]; ++k) {
+                const PieceEntry& e = sch.pieces[k];
+                int32_t* o = pieces + (int64_t)k * 6;
+                o[0] = c; o[1] = e.item; o[2] = e.pair; o[3] = e.t_begin; o[4] = e.t_end; o[5] = e.slot;
+            }
+    }
+    if (items) {
+        if ((int64_t)sch.items.size() > max_items) return set_error(CP_ERR_WORKSPACE, "cp_schedule_inspect: %zu items", sch.items.size());
+        for (size_t i = 0; i < sch.items.size(); ++i) {
+            int32_t* o = items + (int64_t)i * 4;
+            o[0] = sch.items[i].q_row0; o[1] = sch.items[i].n_rows; o[2] = sch.items[i].kv_len0; o[3] = sch.items[i].n_kv_tiles;
+        }
+    }
+    return CP_OK;
 }

@@ -28,7 +28,7 @@ class DeviceWorkload:
         self.lse = torch.full((wl.Hq, wl.total_new), float("nan"), dtype=torch.float32, device="cuda")
         nl = [r.new_len for r in wl.requests]
         cs = [r.C for r in wl.requests]
-        self.ws = torch.zeros(binding.cp_workspace_bytes(nl, cs), dtype=torch.uint8, device="cuda")
+        self.ws = torch.zeros(binding.cp_workspace_bytes(nl, cs, wl.Hq), dtype=torch.uint8, device="cuda")
 
     def run_batch(self, ctx):
         wl = self.wl

@@ -52,9 +52,13 @@ def test_cp_plan_rejects_bad_arguments(lib):
 
 
 def test_workspace_bytes(lib):
-    assert binding.cp_workspace_bytes([1024], [2]) == 256 + 32 * (8 + 4)
-    assert binding.cp_workspace_bytes([5, 300], [4, 1]) == 256 + 32 * ((1 + 8) + (3 + 2))
-    assert binding.cp_workspace_bytes([0], [1]) == 0
+    small = binding.cp_workspace_bytes([1024], [2], 8)
+    big = binding.cp_workspace_bytes([131072], [8], 32)
+    assert 50e6 < small < 60e6                       # dominated by the fixed partial-result space
+    assert big - small == pytest.approx((1040 - 12) * 32 + (1040 * 16 - 12 * 4) * 16, abs=1024)
+    assert small % 256 == 0 and big % 256 == 0
+    assert binding.cp_workspace_bytes([0], [1], 8) == 0
+    assert binding.cp_workspace_bytes([64], [1], 1) == 0
 
 
 def test_gpu_calls_fail_cleanly_without_a_device(lib):

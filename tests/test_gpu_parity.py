@@ -126,7 +126,7 @@ def test_single_request_entry_point_and_c_invariance(ctx):
     mat = wl.materialize(w)
     dev = DeviceWorkload(mat)
     ref_o, ref_l = oracle_request(mat, 0)
-    ws = torch.zeros(binding.cp_workspace_bytes([517], [8]), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(binding.cp_workspace_bytes([517], [8], w.Hq), dtype=torch.uint8, device="cuda")
     outs = []
     for C in (1, 2, 3, 8):
         dev.out.fill_(float("nan"))

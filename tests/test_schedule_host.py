@@ -1,0 +1,76 @@
+"""Host-side checks of the varlen tile schedule (no GPU): every (query tile, head pair, KV tile) step is
+covered exactly once, per-CTA loads are balanced, split units have consistent partial slots."""
+import numpy as np
+import pytest
+
+from paper_2609_04774_b200 import binding, build
+from paper_2609_04774_b200 import workloads as wl
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+
+
+def check(w, num_sms=148):
+    cu_new = w.cu_new
+    prefix = [r.prefix_len for r in w.requests]
+    Cs = [r.C for r in w.requests]
+    info, pieces, items = binding.cp_schedule_inspect(cu_new, prefix, Cs, w.Hq, num_sms)
+    HP = w.Hq // 2
+    # tiles: rows tile [0, total_new) exactly, never straddle a request or a chunk, at most 128 rows
+    rows = np.zeros(w.total_new, dtype=np.int32)
+    for q0, n, kv0, nt in items:
+        assert 1 <= n <= 128 and nt == -(-(kv0 + n - 1) // 128)
+        rows[q0:q0 + n] += 1
+        b = int(np.searchsorted(cu_new, q0, side="right") - 1)
+        r = w.requests[b]
+        r0 = q0 - cu_new[b]
+        assert r0 + n <= r.new_len and kv0 == r.prefix_len + r0 + 1
+        cl = -(-r.new_len // (2 * r.C))
+        assert r0 // cl == (r0 + n - 1) // cl                      # inside one zigzag chunk
+    assert (rows == 1).all()
+    # pieces: per unit the KV tile ranges tile [0, n_kv_tiles) exactly; slots only on split units
+    cover = {}
+    loads = np.zeros(info["grid"], dtype=np.int64)
+    slots = set()
+    for cta, item, pair, t0, t1, slot in pieces:
+        assert 0 <= cta < info["grid"] and 0 <= pair < HP and 0 <= t0 < t1 <= items[item][3]
+        cover.setdefault((item, pair), []).append((t0, t1, slot))
+        loads[cta] += t1 - t0
+        if slot >= 0:
+            assert slot not in slots
+            slots.add(slot)
+    assert len(cover) == len(items) * HP
+    n_split = 0
+    for (item, pair), segs in cover.items():
+        segs.sort()
+        assert segs[0][0] == 0 and segs[-1][1] == items[item][3]
+        for a, b2 in zip(segs, segs[1:]):
+            assert a[1] == b2[0]
+        if len(segs) == 1:
+            assert segs[0][2] == -1
+        else:
+            n_split += 1
+            assert all(s[2] >= 0 for s in segs)
+    assert n_split == info["split_units"] and len(slots) == info["slots"] <= 2 * 192 + 32
+    assert loads.sum() == info["total"] == sum(int(it[3]) for it in items) * HP
+    assert loads.max() == info["max_load"] and loads.min() == info["min_load"]
+    return info, loads
+
+
+def test_schedule_covers_and_balances_all_configs():
+    for cfg in (1, 2, 4, 5, 3):
+        w = wl.CONFIGS[cfg]()
+        info, loads = check(w)
+        share = -(-info["total"] // info["grid"])
+        assert info["max_load"] <= 1.01 * share + 4, (cfg, info)   # at most one short remainder above the share
+        assert loads.mean() >= 0.97 * info["max_load"] - 1, (cfg, info)   # the slowest CTA is within 3 % of the mean
+
+
+def test_schedule_small_and_odd_shapes():
+    for w in (wl.small_mixed(), wl.Workload("one_row", 1, 4, 2, [wl.Request(1, 0, 1)]),
+              wl.Workload("long_prefix", 2, 8, 2, [wl.Request(7, 100000, 2)]),
+              wl.Workload("many_small", 3, 8, 2, [wl.Request(3 + i, 64 * (i % 3), 1 + i % 4) for i in range(40)])):
+        for sms in (1, 7, 148):
+            check(w, sms)
