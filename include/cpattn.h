@@ -106,8 +106,8 @@ size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C, i
 /* cp_schedule_inspect -- host only: the work distribution the attention calls would use for a batch
  * on a device with num_sms SMs (the varlen tile schedule: query tiles of at most 128 rows cut at the
  * chunk boundaries of every request's zigzag plan; one unit per tile and pair of query heads; whole
- * units longest first onto the least loaded CTA, the remainder cut along KV so that every CTA gets
- * the same number of KV tile steps).  summary (8 values): CTAs, query tiles, pieces, split units,
+ * units longest first dealt to the CTAs in serpentine order, the remainder cut along KV so that every
+ * CTA gets the same number of KV tile steps).  summary (8 values): CTAs, query tiles, pieces, split units,
  * partial slots, largest / smallest per-CTA load in KV tile steps, their total.  pieces (optional,
  * 6 int32 per piece: cta, tile, head pair, first KV tile, end KV tile, partial slot or -1) and
  * items (optional, 4 int32 per tile: first packed row, rows, keys visible to the first row, KV tiles)

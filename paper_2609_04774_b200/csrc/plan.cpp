@@ -80,92 +80,99 @@ WorkspaceLayout workspace_layout(size_t n_items, size_t n_pieces, size_t n_merge
 }
 
 int build_schedule(int32_t pairs_per_tile, int32_t grid_max, Schedule& s) {
+    const int32_t HP = pairs_per_tile;
     const int64_t n_items = (int64_t)s.items.size();
-    const int64_t n_units = n_items * pairs_per_tile;
+    const int64_t n_units = n_items * HP;
     int64_t W = 0;
-    for (const TileItem& t : s.items) W += (int64_t)t.n_kv_tiles * pairs_per_tile;
-    if (W <= 0 || W > 0x7fffffffll) return set_error(CP_ERR_UNSUPPORTED, "schedule: %lld KV tile steps", (long long)W);
+    int32_t longest = 0;
+    for (const TileItem& t : s.items) {
+        W += (int64_t)t.n_kv_tiles * HP;
+        longest = std::max(longest, t.n_kv_tiles);
+    }
+    if (W <= 0 || W > 0x7fffffffll || n_units > 0x7fffffffll)
+        return set_error(CP_ERR_UNSUPPORTED, "schedule: %lld KV tile steps", (long long)W);
     grid_max = std::min(grid_max, kMaxGrid);
     // per-CTA share of KV tile steps; never below a short unit's length (cutting those only adds
     // prologues and merges), which also shrinks the grid for tiny problems
-    int32_t longest = 0;
-    for (const TileItem& t : s.items) longest = std::max(longest, t.n_kv_tiles);
     const int64_t T = std::max<int64_t>((W + grid_max - 1) / grid_max, std::min<int32_t>(longest, kMinShareTiles));
     const int32_t G = (int32_t)std::max<int64_t>(1, std::min<int64_t>(grid_max, (W + T - 1) / T));
     s.grid = G;
 
+    // 1. whole units, longest first, dealt to the CTAs in serpentine order (0..G-1, G-1..0, ...) while
+    //    they fit under the share; what does not fit goes to the tail
     std::vector<int64_t> load(G, 0);
-    std::vector<std::vector<PieceEntry>> lists(G);
+    std::vector<int32_t> count(G, 0);                  // pieces per CTA
+    std::vector<int16_t> cta_of((size_t)n_units);      // CTA of a whole unit, -1 = tail
     struct TailUnit { int32_t item; int32_t pair; int32_t n; };
     std::vector<TailUnit> tail;
-
-    // 1. whole units, longest first, onto the least loaded CTA while they fit under the share
-    using Slot = std::pair<int64_t, int32_t>;             // (load, cta); smallest first
-    std::vector<Slot> heap;
-    heap.reserve(G);
-    for (int32_t c = 0; c < G; ++c) heap.push_back({0, c});
-    auto cmp = [](const Slot& a, const Slot& b) { return a > b; };
-    std::make_heap(heap.begin(), heap.end(), cmp);
-    for (int64_t i = 0; i < n_items; ++i) {
-        const int32_t n = s.items[i].n_kv_tiles;
-        for (int32_t pr = 0; pr < pairs_per_tile; ++pr) {
-            std::pop_heap(heap.begin(), heap.end(), cmp);
-            Slot& top = heap.back();
-            if (top.first + n <= T) {
-                lists[top.second].push_back({(int32_t)i, (int16_t)pr, (int16_t)-1, 0, n});
-                top.first += n;
-                load[top.second] = top.first;
-            } else {
-                tail.push_back({(int32_t)i, pr, n});
+    {
+        int64_t k = 0;   // running index over the units that were dealt
+        for (int64_t i = 0; i < n_items; ++i) {
+            const int32_t n = s.items[i].n_kv_tiles;
+            for (int32_t pr = 0; pr < HP; ++pr) {
+                const int64_t r = k / G;
+                const int32_t pos = (int32_t)(k - r * G);
+                const int32_t c = (r & 1) ? G - 1 - pos : pos;
+                if (load[c] + n <= T) {
+                    load[c] += n;
+                    ++count[c];
+                    cta_of[(size_t)(i * HP + pr)] = (int16_t)c;
+                    ++k;
+                } else {
+                    cta_of[(size_t)(i * HP + pr)] = -1;
+                    tail.push_back({(int32_t)i, pr, n});
+                }
             }
-            std::push_heap(heap.begin(), heap.end(), cmp);
         }
     }
-    (void)n_units;
 
-    // 2. the remaining units, cut into KV ranges that fill every CTA up to the share
+    // 2. the tail, cut into KV ranges that fill every CTA up to the share
     const int64_t minp = std::min<int64_t>(kMinPieceTiles, std::max<int64_t>(1, T));   // shortest piece worth a cut
-    struct Cut { int32_t cta; int32_t t_begin; int32_t t_end; };
-    std::vector<std::vector<Cut>> cuts(tail.size());
+    struct Cut { int32_t unit; int32_t cta; int32_t t_begin; int32_t t_end; int32_t slot; };
+    std::vector<Cut> cuts;
+    s.merges.clear();
+    s.merge_slots.clear();
+    int32_t n_slots = 0;
     int32_t c = 0;
     for (size_t u = 0; u < tail.size(); ++u) {
         int32_t t = 0;
         const int32_t n = tail[u].n;
+        const size_t first = cuts.size();
         while (t < n) {
-            while (c < G - 1 && T - load[c] < std::min<int64_t>(minp, n - t)) ++c;   // CTA is full
+            while (c < G - 1 && T - load[c] < std::min<int64_t>(minp, n - t)) ++c;          // CTA is full
             int64_t len = std::min<int64_t>(n - t, std::max<int64_t>(T - load[c], 0));
             if (c == G - 1 || len <= 0) len = n - t;                                        // last CTA takes what is left
             if (n - t - len > 0 && n - t - len < minp) len = n - t;                           // no tiny remainder
-            cuts[u].push_back({c, t, (int32_t)(t + len)});
+            cuts.push_back({(int32_t)u, c, t, (int32_t)(t + len), -1});
             load[c] += len;
+            ++count[c];
             t += (int32_t)len;
         }
-    }
-    s.merges.clear();
-    s.merge_slots.clear();
-    int32_t n_slots = 0;
-    for (size_t u = 0; u < tail.size(); ++u) {
-        const bool split = cuts[u].size() > 1;
-        if (split) s.merges.push_back({tail[u].item, tail[u].pair, (int32_t)cuts[u].size(), (int32_t)s.merge_slots.size()});
-        for (const Cut& k : cuts[u]) {
-            int16_t slot = -1;
-            if (split) {
-                slot = (int16_t)n_slots++;
-                s.merge_slots.push_back(slot);
+        if (cuts.size() - first > 1) {
+            s.merges.push_back({tail[u].item, tail[u].pair, (int32_t)(cuts.size() - first), (int32_t)s.merge_slots.size()});
+            for (size_t k = first; k < cuts.size(); ++k) {
+                cuts[k].slot = n_slots++;
+                s.merge_slots.push_back(cuts[k].slot);
             }
-            lists[k.cta].push_back({tail[u].item, (int16_t)tail[u].pair, slot, k.t_begin, k.t_end});
         }
     }
     if (n_slots > kMaxSlots) return set_error(CP_ERR_UNSUPPORTED, "schedule: %d partial slots", n_slots);
     s.n_slots = n_slots;
 
+    // 3. per-CTA lists: whole units in dealing order, then the CTA's KV ranges
     s.cta_off.assign(G + 1, 0);
-    s.pieces.clear();
-    for (int32_t k = 0; k < G; ++k) {
-        s.cta_off[k] = (int32_t)s.pieces.size();
-        s.pieces.insert(s.pieces.end(), lists[k].begin(), lists[k].end());
+    for (int32_t k = 0; k < G; ++k) s.cta_off[k + 1] = s.cta_off[k] + count[k];
+    s.pieces.resize((size_t)s.cta_off[G]);
+    std::vector<int32_t> fill(s.cta_off.begin(), s.cta_off.end() - 1);
+    for (int64_t i = 0; i < n_items; ++i) {
+        const int32_t n = s.items[i].n_kv_tiles;
+        for (int32_t pr = 0; pr < HP; ++pr) {
+            const int16_t k = cta_of[(size_t)(i * HP + pr)];
+            if (k >= 0) s.pieces[(size_t)fill[k]++] = {(int32_t)i, (int16_t)pr, (int16_t)-1, 0, n};
+        }
     }
-    s.cta_off[G] = (int32_t)s.pieces.size();
+    for (const Cut& k : cuts)
+        s.pieces[(size_t)fill[k.cta]++] = {tail[k.unit].item, (int16_t)tail[k.unit].pair, (int16_t)k.slot, k.t_begin, k.t_end};
     return CP_OK;
 }
 
