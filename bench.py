@@ -3,13 +3,15 @@
 
 Default mode prints ONE JSON line for the headline workload (BASELINE config 2: Llama-3-8B-shaped
 layer, 12288 cached + 4096 new tokens, C=4, paged KV).  A step is one pass of the hot path over the
-batch: cp_plan (host) -> tile schedule -> one persistent attention launch over all C shards reading
-K/V through the page table and storing rows at their original positions.  `value` is measured with
-inputs resident in HBM; `e2e` goes through the same C-ABI calls from pinned HOST buffers (q, the new
-tokens' K/V rows appended into the paged cache, page table up; out and lse down).
+batch: cp_plan (host) -> varlen tile schedule (host, uploaded by a copy kernel) -> one persistent
+attention launch over all C shards reading K/V through the page table and storing rows at their
+original positions -> LSE merge of the units whose KV range was split across CTAs.  `value` is
+measured with inputs resident in HBM; `e2e` goes through the same C-ABI calls from pinned HOST
+buffers (q, the new tokens' K/V rows appended into the paged cache, page table up; out and lse down).
 
-Other modes (`--mode merge|table|configs`) write the cp_merge sweep, the measured prefill-time
-table over (new_len, prefix_len, C) and the per-config numbers as JSON lines to `--out`.
+Other modes (`--mode merge|table|configs|kvcopy`) write the cp_merge sweep, the measured prefill-time
+table over (new_len, prefix_len, C), the per-config numbers and the paged KV copy bandwidth as JSON
+lines to `--out`.
 
 `--impl reference` times the CPU fp64 oracle (host cores) on a bounded sample of the same workload.
 """
@@ -35,6 +37,9 @@ METRIC = "causal_effective_prefill_attention_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one cp_attn_kernel launch, from the ncu capture
+# summarised in profiles/ (per workload name)
+ATTN_TRAFFIC_BYTES = {"cfg2_R4096_P12288_C4": 244_072_704}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -188,7 +193,27 @@ class Runner:
         self.h_lse.copy_(self.lse, non_blocking=True)
 
     def launches_per_step(self, e2e=False):
-        return 1 + (len(self.w.requests) if e2e else 0)
+        """Kernels of this library per step: schedule copy + attention (+ LSE fix-up when units were split)."""
+        info, _, _ = self.binding.cp_schedule_inspect(self.cu_new, self.prefix, self.Cs, self.w.Hq,
+                                                      self.torch.cuda.get_device_properties(0).multi_processor_count,
+                                                      want_lists=False)
+        self.schedule = info
+        return 2 + (1 if info["split_units"] > 0 else 0) + (len(self.w.requests) if e2e else 0)
+
+
+def max_over_ranks(torch, dist, values, device):
+    """MAX all-reduce of a list of per-rank timings (no-op without a process group)."""
+    if dist is None:
+        return list(values)
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_value(world, flops_per_rank, ms_per_step):
+    """Aggregate over all ranks: every rank runs its own replica of the workload (weak scaling), the job
+    is as slow as its slowest rank."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
 
 
 def timed_loop(torch, fn, steps, warmup, dist=None):
@@ -309,18 +334,15 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     runner.ctx.poll_status()
 
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = max_over_ranks(torch, dist, [total_ms, e2e_ms], "cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
     ms_per_step = total_ms / args.steps
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
-    e2e_value = world * flops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    value = whole_job_value(world, flops, ms_per_step)
+    e2e_value = whole_job_value(world, flops, e2e_ms / e2e_steps)
     achieved = flops / (kern_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops"]
     line = {
@@ -336,9 +358,10 @@ def run_ours(args):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": runner.h2d_bytes,
                 "d2h_bytes_per_step": runner.d2h_bytes, "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": args.steps * runner.launches_per_step(),
+        "schedule": runner.schedule,
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved / peak, "traffic": None, "kernel": "cp_attn_kernel",
-                     "kernel_ms": kern_ms, "peak_source": "%s burst bf16 (of %s)" % (peaks["_source"], peaks["_source"]),
+                     "frac": achieved / peak, "traffic": ATTN_TRAFFIC_BYTES.get(w.name), "kernel": "cp_attn_kernel",
+                     "kernel_ms": kern_ms, "kernel_ms_covers": "schedule copy + cp_attn_kernel + LSE fix-up of one step", "peak_source": "%s burst bf16 (of %s)" % (peaks["_source"], peaks["_source"]),
                      "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
                      "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS},
         "clocks": clocks,
@@ -428,6 +451,47 @@ def run_merge_sweep(args, out):
                 torch.cuda.empty_cache()
 
 
+def run_kvcopy(args, out):
+    """cp_kv_gather / cp_kv_append bandwidth: n tokens x 8 KV heads x 128 dims, K and V, shuffled pages."""
+    import torch
+    from paper_2609_04774_b200 import binding, build
+    build.build()
+    peaks = load_peaks()
+    ctx = binding.Context(0)
+    Hkv, D = 8, 128
+    for n in (16384, 131072, 1048576):
+        pages = n // wl.PAGE
+        k = torch.randn((pages, wl.PAGE, Hkv, D), device="cuda").to(torch.bfloat16)
+        v = torch.randn((pages, wl.PAGE, Hkv, D), device="cuda").to(torch.bfloat16)
+        pt = torch.from_numpy(wl.permutation(9, wl.TID_PERM, pages)).cuda()
+        cache = binding.make_cache(k, v)
+        kr = torch.empty((n, Hkv, D), dtype=torch.bfloat16, device="cuda")
+        vr = torch.empty_like(kr)
+        moved = 2 * 2 * n * Hkv * D * 2 + 4 * pages          # K and V, read + written, plus the table
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if moved < 512e6 else None
+        for name, fn in (("gather", lambda: binding.cp_kv_gather(ctx, cache, pt, 0, n, kr, vr)),
+                         ("append", lambda: binding.cp_kv_append(ctx, cache, pt, 0, n, kr, vr))):
+            ds = []
+            for i in range(13):
+                if flush is not None:
+                    flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                if i >= 3:
+                    ds.append((e0, e1))
+            torch.cuda.synchronize()
+            ms = statistics.median(a.elapsed_time(b) for a, b in ds)
+            gbs = moved / (ms * 1e-3) / 1e9
+            out.write(json.dumps({"mode": "kvcopy", "op": name, "tokens": n, "bytes": moved, "ms_median": ms, "GBps": gbs,
+                                  "frac_nominal_8000": gbs / NOMINAL_HBM_GBS, "frac_measured_copy": gbs / peaks["hbm_gbs"],
+                                  "l2_flush": flush is not None}) + "\n")
+            out.flush()
+        del k, v, kr, vr, flush
+        torch.cuda.empty_cache()
+
+
 def run_table(args, out):
     """Measured prefill-time table over (new_len, prefix_len, C): all-shard time and the slowest /
     fastest single shard (what one CP rank would compute), with W(R,P) of Eq. (1) -- the inputs of the
@@ -485,7 +549,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="BASELINE config number of the headline workload")
-    ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table"])
+    ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table", "kvcopy"])
     ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5])
     ap.add_argument("--merge-T", type=int, nargs="*", default=[4096, 16384, 65536, 262144])
     ap.add_argument("--merge-reps", type=int, default=20)
@@ -501,7 +565,7 @@ def main():
     if args.mode == "bench":
         return run_ours(args)
     out = open(args.out, "w") if args.out else sys.stdout
-    {"configs": run_configs, "merge": run_merge_sweep, "table": run_table}[args.mode](args, out)
+    {"configs": run_configs, "merge": run_merge_sweep, "table": run_table, "kvcopy": run_kvcopy}[args.mode](args, out)
 
 
 if __name__ == "__main__":

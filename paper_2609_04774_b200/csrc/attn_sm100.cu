@@ -21,6 +21,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -114,6 +115,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity), "r"(kTryWaitHintNs) : "memory");
+    return ok != 0;
+}
+
+// Non-blocking test of a phase; the result comes back asynchronously, so a test issued before a block
+// of MMAs costs nothing by the time it is looked at.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
 
@@ -361,6 +374,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
                     if (lane == 0) {
                         const uint32_t slot = kv_it % kKvStages;
                         mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j0 + jj);
+                        { const int j = j0 + jj; CP_TRACE(3, j, 6 + kv); }
                         const uint32_t fbar = bars + (kBarKvFull + slot) * 8;
                         const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
                         const CUtensorMap* map = kv ? tmV : tmK;
@@ -430,6 +444,8 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
         }
         __syncwarp();
         ++kv_it;
+        bool kv_tested = false;     // V(j) and K(j+1) already seen complete by a test issued one block earlier
+        bool p_tested = false;      // same for the next P hand-over
 #pragma unroll 1
         for (int j = u.t_begin; j < n; ++j) {
             const uint32_t v_slot = kv_it % kKvStages;
@@ -438,17 +454,31 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
             const bool more = (j + 1 < n);
             const uint32_t k_slot = kv_it % kKvStages;
             const uint32_t k_par = (kv_it / kKvStages) & 1;
-            // K(j+1) and V(j) were requested long ago; check them before the P hand-over
-            MMA_WAIT(kBarKvFull + v_slot, v_par, j);
-            if (more) MMA_WAIT(kBarKvFull + k_slot, k_par, j);
+            // K(j+1) and V(j) were requested long ago
+            if (!kv_tested) {
+                MMA_WAIT(kBarKvFull + v_slot, v_par, j);
+                if (more) MMA_WAIT(kBarKvFull + k_slot, k_par, j);
+            }
+            // slots and phases of the next tile's V(j+1), K(j+2), for the early test below
+            const uint32_t it_v2 = kv_it + 1, it_k2 = kv_it + 2;
+            const uint32_t bar_v2 = bars + (kBarKvFull + it_v2 % kKvStages) * 8, par_v2 = (it_v2 / kKvStages) & 1;
+            const uint32_t bar_k2 = bars + (kBarKvFull + it_k2 % kKvStages) * 8, par_k2 = (it_k2 / kKvStages) & 1;
 #pragma unroll
             for (int wg = 0; wg < 2; ++wg) {
                 if (j == u.t_begin && round > 0) MMA_WAIT(kBarOFree + wg, (round - 1) & 1, j);
 #pragma unroll
                 for (int part = 0; part < kPieces; ++part) {
-                    MMA_WAIT(kBarPReady + wg * 4 + part, tile_cnt & 1, j);
+                    if (!p_tested) MMA_WAIT(kBarPReady + wg * 4 + part, tile_cnt & 1, j);
                     tc_fence_after();
                     if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, part); }
+                    // tests for what the next block of MMAs will need, answered while this block is issued
+                    bool next_p;
+                    if (part + 1 < kPieces) next_p = mbar_test(bars + (kBarPReady + wg * 4 + part + 1) * 8, tile_cnt & 1);
+                    else if (wg == 0) next_p = mbar_test(bars + (kBarPReady + 4) * 8, tile_cnt & 1);
+                    else next_p = more && mbar_test(bars + kBarPReady * 8, (tile_cnt + 1) & 1);
+                    bool next_kv = false;
+                    if (wg == 1 && part == kPieces - 1 && more)
+                        next_kv = mbar_test(bar_v2, par_v2) && (j + 2 >= n || mbar_test(bar_k2, par_k2));
                     if (elect_one()) {
                         mma_pv(wg, part, v_slot, j > u.t_begin);
                         if (part == kPieces - 1) {
@@ -466,6 +496,8 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
                         }
                     }
                     __syncwarp();
+                    p_tested = __all_sync(0xffffffffu, next_p);
+                    if (wg == 1 && part == kPieces - 1) kv_tested = __all_sync(0xffffffffu, next_kv);
                 }
                 if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, 5); }
             }
@@ -856,19 +888,29 @@ int encode_maps(cp_ctx* ctx, const void* q, int64_t total_rows, int32_t Hq, cons
     return CP_OK;
 }
 
-// Copies a host block into the workspace through one of the context's two pinned staging buffers
+// Moves 16-byte words from pinned host memory (read over PCIe) into device memory.  Used instead of a
+// copy-engine transfer for the schedule: a kernel stays on the compute engine, so the attention launch
+// behind it does not wait on a cross-engine hand-over.
+__global__ void stage_copy_kernel(uint4* __restrict__ dst, const uint4* __restrict__ src, int64_t n16) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (int64_t)gridDim.x * blockDim.x)
+        dst[i] = src[i];
+}
+
+// Copies a host block into the workspace through one of the context's pinned staging buffers
 // (falls back to a pageable copy for blocks that do not fit).
 int upload_block(cp_ctx* ctx, const std::vector<uint8_t>& block, void* dst, cudaStream_t s) {
     const size_t bytes = block.size();
-    if (bytes > ctx->stage_bytes)
+    if (bytes > ctx->stage_bytes || (bytes & 15) != 0)
         return check_cuda(cudaMemcpyAsync(dst, block.data(), bytes, cudaMemcpyHostToDevice, s), "schedule copy");
     const int i = ctx->stage_next;
-    ctx->stage_next ^= 1;
+    ctx->stage_next = (i + 1) % kStageBuffers;
     if (ctx->stage_used[i])
         if (int rc = check_cuda(cudaEventSynchronize(ctx->stage_event[i]), "cudaEventSynchronize(stage)")) return rc;
     memcpy(ctx->h_stage[i], block.data(), bytes);
-    if (int rc = check_cuda(cudaMemcpyAsync(dst, ctx->h_stage[i], bytes, cudaMemcpyHostToDevice, s), "schedule copy"))
-        return rc;
+    const int64_t n16 = (int64_t)(bytes / 16);
+    const int blocks = (int)std::min<int64_t>((n16 + 255) / 256, 64);
+    stage_copy_kernel<<<blocks, 256, 0, s>>>(static_cast<uint4*>(dst), static_cast<const uint4*>(ctx->h_stage[i]), n16);
+    if (int rc = check_cuda(cudaGetLastError(), "schedule copy launch")) return rc;
     ctx->stage_used[i] = true;
     return check_cuda(cudaEventRecord(ctx->stage_event[i], s), "cudaEventRecord(stage)");
 }
@@ -913,7 +955,11 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     build_tiles(B, cu_new, prefix_len, C, cu_pages, only_shard, sch.items);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (sch.items.empty()) return CP_OK;   // the shard owns no rows (only empty chunks)
-    if (int rc = build_schedule(Hq / 2, ctx->num_sms, sch)) return rc;
+    int grid_max = ctx->num_sms;
+#ifdef CPATTN_TRACE
+    if (const char* e = getenv("CPATTN_DEBUG_SMS")) grid_max = std::max(1, atoi(e));   // trace builds only
+#endif
+    if (int rc = build_schedule(Hq / 2, grid_max, sch)) return rc;
     const WorkspaceLayout lay = workspace_layout(sch.items.size(), sch.pieces.size(), sch.merges.size(),
                                                  sch.merge_slots.size(), sch.grid, sch.n_slots);
     if (lay.total > workspace_bytes)

@@ -57,11 +57,11 @@ extern "C" int cp_ctx_create(cp_ctx** out, int device) {
     memset(c, 0, sizeof *c);
     c->device = device;
     c->num_sms = prop.multiProcessorCount;
-    c->stage_bytes = 8u << 20;
+    c->stage_bytes = 2u << 20;
     int rc = check_cuda(cudaMalloc(&c->d_status, kStatusBytes), "cudaMalloc(status)");
     if (!rc) rc = check_cuda(cudaMemset(c->d_status, 0, kStatusBytes), "cudaMemset(status)");
     if (!rc) rc = check_cuda(cudaMallocHost(&c->h_status, kStatusWords * sizeof(int32_t)), "cudaMallocHost(status)");
-    for (int i = 0; i < 2 && !rc; ++i) {
+    for (int i = 0; i < kStageBuffers && !rc; ++i) {
         rc = check_cuda(cudaMallocHost(&c->h_stage[i], c->stage_bytes), "cudaMallocHost(stage)");
         if (!rc) rc = check_cuda(cudaEventCreateWithFlags(&c->stage_event[i], cudaEventDisableTiming), "cudaEventCreate");
     }
@@ -88,7 +88,7 @@ extern "C" int cp_ctx_destroy(cp_ctx* c) {
     cudaDeviceSynchronize();
     if (c->d_status) cudaFree(c->d_status);
     if (c->h_status) cudaFreeHost(c->h_status);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kStageBuffers; ++i) {
         if (c->h_stage[i]) cudaFreeHost(c->h_stage[i]);
         if (c->stage_event[i]) cudaEventDestroy(c->stage_event[i]);
     }

@@ -72,6 +72,7 @@ constexpr size_t kPartialSlotRows = 2 * 128;           // two heads x 128 query 
 constexpr size_t kWorkspaceHeader = 256;
 constexpr int kTileRows = 128;
 constexpr int kStatusWords = 4;
+constexpr int kStageBuffers = 4;
 #ifdef CPATTN_TRACE
 constexpr size_t kStatusBytes = 64 + 4 * 64 * 8 * sizeof(long long);   // status words + phase trace
 #else
@@ -106,10 +107,10 @@ struct cp_ctx {
     int num_sms;
     int32_t* d_status;                 // kStatusWords int32 on the device
     int32_t* h_status;                 // pinned mirror
-    void* h_stage[2];                  // pinned staging buffers for tile lists
+    void* h_stage[cpattn::kStageBuffers];       // pinned (device-visible) staging buffers for schedules
     size_t stage_bytes;
-    cudaEvent_t stage_event[2];
-    bool stage_used[2];
+    cudaEvent_t stage_event[cpattn::kStageBuffers];
+    bool stage_used[cpattn::kStageBuffers];
     int stage_next;
     cpattn::EncodeTiledFn encode_tiled;
     bool attn_attr_set;
