@@ -194,7 +194,7 @@ class Runner:
 
     def launches_per_step(self, e2e=False):
         """Kernels of this library per step: schedule copy + attention (+ LSE fix-up when units were split)."""
-        info, _, _ = self.binding.cp_schedule_inspect(self.cu_new, self.prefix, self.Cs, self.w.Hq,
+        info, _, _ = self.binding.cp_schedule_inspect(self.cu_new, self.prefix, self.Cs, self.w.Hq, self.w.Hkv,
                                                       self.torch.cuda.get_device_properties(0).multi_processor_count,
                                                       want_lists=False)
         self.schedule = info

@@ -32,7 +32,7 @@ extern "C" {
 enum {
     CP_OK = 0,
     CP_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, inconsistent lengths              */
-    CP_ERR_UNSUPPORTED = -2, /* D != 128, page_size != 64, odd Hq/Hkv ratio, misaligned strides    */
+    CP_ERR_UNSUPPORTED = -2, /* D != 128, page_size != 64, misaligned strides, sizes beyond limits */
     CP_ERR_WORKSPACE = -3,   /* workspace missing, misaligned or smaller than cp_workspace_bytes() */
     CP_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                                */
     CP_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (reported by poll_status)       */
@@ -105,7 +105,8 @@ size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C, i
 
 /* cp_schedule_inspect -- host only: the work distribution the attention calls would use for a batch
  * on a device with num_sms SMs (the varlen tile schedule: query tiles of at most 128 rows cut at the
- * chunk boundaries of every request's zigzag plan; one unit per tile and pair of query heads; whole
+ * chunk boundaries of every request's zigzag plan; one unit per tile and pair of query heads (per
+ * single head when Hq / Hkv is odd); whole
  * units longest first dealt to the CTAs in serpentine order, the remainder cut along KV so that every
  * CTA gets the same number of KV tile steps).  summary (8 values): CTAs, query tiles, pieces, split units,
  * partial slots, largest / smallest per-CTA load in KV tile steps, their total.  pieces (optional,
@@ -113,8 +114,8 @@ size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C, i
  * items (optional, 4 int32 per tile: first packed row, rows, keys visible to the first row, KV tiles)
  * are filled when non-NULL and large enough (CP_ERR_WORKSPACE otherwise). */
 int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
-                        int32_t Hq, int32_t num_sms, int64_t* summary, int32_t* pieces, int64_t max_pieces,
-                        int32_t* items, int64_t max_items);
+                        int32_t Hq, int32_t Hkv, int32_t num_sms, int64_t* summary, int32_t* pieces,
+                        int64_t max_pieces, int32_t* items, int64_t max_items);
 
 /* ---------------------------------------------------------------------------------------------
  * cp_prefill_attn -- all C shards of one request in one launch (Sections 2.1-2.2).
@@ -125,9 +126,10 @@ int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_
  *              original position (the "restore order" step is fused into the store)
  *   lse        device [Hq, R] fp32: natural-log sum-exp of the scaled scores of each row
  * Every shard's q-tiles are cut at chunk boundaries of cp_plan(R, P, C); the result does not
- * depend on C.  One persistent launch computes all tiles; the few units that were split along KV
- * to balance the SMs are combined by a second small launch (an LSE merge of their partials).  Requires Hq % Hkv == 0 and Hq / Hkv even (two query heads of one KV group share
- * each K/V tile).  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ * depend on C.  Requires Hq % Hkv == 0 (query head h uses KV head h / (Hq / Hkv)); with an even group
+ * size two query heads of a group share every K/V tile in shared memory, with an odd one (e.g.
+ * Hq == Hkv) every head streams K/V on its own at about half the throughput.  One persistent launch computes all tiles; the few units that were split along KV
+ * to balance the SMs are combined by a second small launch (an LSE merge of their partials).  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
  * ------------------------------------------------------------------------------------------- */
 int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
                     int64_t prefix_len, int64_t new_len, int32_t C, int32_t Hq, float scale,

@@ -81,7 +81,8 @@ struct AttnParams {
     const PieceEntry* pieces;  // NULL: implicit serpentine schedule over whole units (no KV splits)
     float* partial_o;          // [slots][2 heads][128 rows][128] fp32, normalised partial outputs
     float* partial_lse;        // [slots][2 heads][128 rows]
-    int32_t pairs_per_tile;   // Hq / 2
+    int32_t pairs_per_tile;   // units per query tile: Hq / heads_per_unit
+    int32_t heads_per_unit;   // 2: two query heads of one KV group share every K/V tile; 1: odd group size
     int32_t group;            // Hq / Hkv
     int32_t Hq;
     const int32_t* page_table;
@@ -335,7 +336,7 @@ __device__ __forceinline__ bool fetch_unit(const AttnParams& p, int round, UnitI
         u.t_end = u.it.n_kv_tiles;
         u.slot = -1;
     }
-    u.head0 = 2 * pair;
+    u.head0 = p.heads_per_unit * pair;
     u.kv_head = u.head0 / p.group;
     return true;
 }
@@ -354,8 +355,8 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
         if (lane == 0) {
             mbar_wait(bars, kBarQEmpty, (round & 1) ^ 1, abort_flag, p.status, round);
             const uint32_t qbar = bars + kBarQFull * 8;
-            mbar_expect_tx(qbar, 2 * kTileBytes);
-            for (int h = 0; h < 2; ++h)
+            mbar_expect_tx(qbar, p.heads_per_unit * kTileBytes);
+            for (int h = 0; h < p.heads_per_unit; ++h)
                 for (int half = 0; half < 2; ++half)
                     tma_load_3d(smem_base + kSmemQ + h * kTileBytes + half * kHalfBytes, tmQ, qbar, half * 64,
                                 u.head0 + h, u.it.q_row0);
@@ -402,6 +403,7 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
     const uint32_t bars = smem_base + kSmemBar;
     uint32_t kv_it = 0;        // ring slots consumed so far
     uint32_t tile_cnt = 0;     // KV tiles processed so far (phase of p_ready)
+    const int last_wg = p.heads_per_unit - 1;   // last head of a unit: its block releases the K/V slots
     const uint64_t q_desc0 = make_desc(smem_base + kSmemQ, 16, 1024);
     const uint64_t k_desc0 = make_desc(smem_base + kSmemKV, 16, 1024);           // K-major view of a ring slot
     const uint64_t v_desc0 = make_desc(smem_base + kSmemKV, kHalfBytes, 1024);   // MN-major view of a ring slot
@@ -437,8 +439,10 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
         if (elect_one()) {
             mma_s(0, slot0);
             tc_commit(bars + (kBarSReady + 0) * 8);
-            mma_s(1, slot0);
-            tc_commit(bars + (kBarSReady + 1) * 8);
+            if (last_wg == 1) {
+                mma_s(1, slot0);
+                tc_commit(bars + (kBarSReady + 1) * 8);
+            }
             tc_commit(bars + (kBarKvEmpty + slot0) * 8);
             if (u.t_begin + 1 == n) tc_commit(bars + kBarQEmpty * 8);
         }
@@ -465,6 +469,7 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
             const uint32_t bar_k2 = bars + (kBarKvFull + it_k2 % kKvStages) * 8, par_k2 = (it_k2 / kKvStages) & 1;
 #pragma unroll
             for (int wg = 0; wg < 2; ++wg) {
+                if (wg > last_wg) break;
                 if (j == u.t_begin && round > 0) MMA_WAIT(kBarOFree + wg, (round - 1) & 1, j);
 #pragma unroll
                 for (int part = 0; part < kPieces; ++part) {
@@ -474,10 +479,10 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
                     // tests for what the next block of MMAs will need, answered while this block is issued
                     bool next_p;
                     if (part + 1 < kPieces) next_p = mbar_test(bars + (kBarPReady + wg * 4 + part + 1) * 8, tile_cnt & 1);
-                    else if (wg == 0) next_p = mbar_test(bars + (kBarPReady + 4) * 8, tile_cnt & 1);
+                    else if (wg < last_wg) next_p = mbar_test(bars + (kBarPReady + 4) * 8, tile_cnt & 1);
                     else next_p = more && mbar_test(bars + kBarPReady * 8, (tile_cnt + 1) & 1);
                     bool next_kv = false;
-                    if (wg == 1 && part == kPieces - 1 && more)
+                    if (wg == last_wg && part == kPieces - 1 && more)
                         next_kv = mbar_test(bar_v2, par_v2) && (j + 2 >= n || mbar_test(bar_k2, par_k2));
                     if (elect_one()) {
                         mma_pv(wg, part, v_slot, j > u.t_begin);
@@ -488,16 +493,17 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
                             } else {
                                 tc_commit(bars + (kBarODone + wg) * 8);
                             }
-                            if (wg == 1) {
+                            if (wg == last_wg) {
                                 tc_commit(bars + (kBarKvEmpty + v_slot) * 8);
                                 if (more) tc_commit(bars + (kBarKvEmpty + k_slot) * 8);
                                 if (j + 2 == n) tc_commit(bars + kBarQEmpty * 8);
                             }
                         }
                     }
-                    __syncwarp();
-                    p_tested = __all_sync(0xffffffffu, next_p);
-                    if (wg == 1 && part == kPieces - 1) kv_tested = __all_sync(0xffffffffu, next_kv);
+                    // per-lane answers: a lane whose test came back negative waits below, the others go on
+                    // to the next elect.sync, where the warp meets again
+                    p_tested = next_p;
+                    if (wg == last_wg && part == kPieces - 1) kv_tested = next_kv;
                 }
                 if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, 5); }
             }
@@ -634,6 +640,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
     const uint32_t p_bar0 = bars + (kBarPReady + wg * 4) * 8;
     const float c = p.scale_log2;
     uint32_t tile_cnt = 0;
+    if (wg >= p.heads_per_unit) return;      // single-head units: the second softmax warpgroup has no work
 
 #define SM_WAIT(id, parity, it)                                                                  \
     mbar_wait(bars, (id), (parity), abort_flag, p.status, (it));                                 \
@@ -785,6 +792,7 @@ struct FixupParams {
     void* out;
     int32_t out_f32;
     int32_t Hq;
+    int32_t heads_per_unit;
     float* lse;
     int64_t lse_stride;
 };
@@ -803,7 +811,7 @@ __global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p)
         const int hr = blockIdx.y * kFixupRowsPerBlock + warp * 2 + r2;
         const int wg = hr / kBlockM;
         const int row = hr - wg * kBlockM;
-        if (row >= it.n_rows) continue;
+        if (row >= it.n_rows || wg >= p.heads_per_unit) continue;
         // pass 1: max of the partial LSEs (lane k of each group of 32 slots holds slot k)
         float m = -INFINITY;
         for (int base = 0; base < me.n_slots; base += 32) {
@@ -842,7 +850,7 @@ __global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p)
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
         const float inv = 1.f / wsum;     // every row of a unit sees at least key 0, so wsum > 0
-        const int head = 2 * me.pair + wg;
+        const int head = p.heads_per_unit * me.pair + wg;
         const int64_t grow = (int64_t)it.q_row0 + row;
         const int64_t off = (grow * p.Hq + head) * kD + lane * 4;
         if (p.out_f32) {
@@ -924,9 +932,8 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     if (int rc = validate_kv_cache(cache, who)) return rc;
     if (Hq < 1 || Hq % cache->Hkv != 0)
         return set_error(CP_ERR_INVALID_ARG, "%s: Hq=%d is not a multiple of Hkv=%d", who, Hq, cache->Hkv);
-    if ((Hq / cache->Hkv) % 2 != 0)
-        return set_error(CP_ERR_UNSUPPORTED, "%s: Hq/Hkv=%d must be even (two query heads share each K/V tile)", who,
-                         Hq / cache->Hkv);
+    // even group size: two query heads of one KV group share every K/V tile; odd: one head per unit
+    const int32_t heads_per_unit = ((Hq / cache->Hkv) % 2 == 0) ? 2 : 1;
     if (!(scale > 0.f)) return set_error(CP_ERR_INVALID_ARG, "%s: scale must be positive", who);
     if (((uintptr_t)q | (uintptr_t)out) & 15) return set_error(CP_ERR_INVALID_ARG, "%s: q and out must be 16-byte aligned", who);
     if (cu_new[0] != 0 || cu_pages[0] != 0) return set_error(CP_ERR_INVALID_ARG, "%s: cu_new[0] and cu_pages[0] must be 0", who);
@@ -945,7 +952,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     }
     if (cu_new[B] > 0x7fffff00ll || cu_pages[B] > 0x7fffff00ll)
         return set_error(CP_ERR_UNSUPPORTED, "%s: more than 2^31 packed rows or pages", who);
-    const size_t need_ws = cp_workspace_bytes(B, new_len.data(), C, Hq);
+    const size_t need_ws = cp_workspace_bytes(B, new_len.data(), C, Hq);   // sized for one head per unit
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need_ws)
         return set_error(CP_ERR_WORKSPACE, "%s: workspace %p of %zu bytes; need %zu bytes, 256-byte aligned", who,
                          workspace, workspace_bytes, need_ws);
@@ -959,7 +966,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
 #ifdef CPATTN_TRACE
     if (const char* e = getenv("CPATTN_DEBUG_SMS")) grid_max = std::max(1, atoi(e));   // trace builds only
 #endif
-    if (int rc = build_schedule(Hq / 2, grid_max, sch)) return rc;
+    if (int rc = build_schedule(Hq / heads_per_unit, grid_max, sch)) return rc;
     const WorkspaceLayout lay = workspace_layout(sch.items.size(), sch.pieces.size(), sch.merges.size(),
                                                  sch.merge_slots.size(), sch.grid, sch.n_slots);
     if (lay.total > workspace_bytes)
@@ -990,7 +997,8 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.pieces = reinterpret_cast<const PieceEntry*>(ws + lay.pieces);
     p.partial_o = reinterpret_cast<float*>(ws + lay.partial_o);
     p.partial_lse = reinterpret_cast<float*>(ws + lay.partial_lse);
-    p.pairs_per_tile = Hq / 2;
+    p.pairs_per_tile = Hq / heads_per_unit;
+    p.heads_per_unit = heads_per_unit;
     p.group = Hq / cache->Hkv;
     p.Hq = Hq;
     p.page_table = page_table;
@@ -1013,6 +1021,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         f.out = out;
         f.out_f32 = out_f32;
         f.Hq = Hq;
+        f.heads_per_unit = heads_per_unit;
         f.lse = lse;
         f.lse_stride = cu_new[B];
         cp_attn_fixup_kernel<<<dim3((unsigned)sch.merges.size(), 2 * kBlockM / kFixupRowsPerBlock), 256, 0, s>>>(f);
@@ -1127,8 +1136,7 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     if (int rc = validate_kv_cache(cache, who)) return rc;
     if (Hq < 1 || Hq % cache->Hkv != 0)
         return set_error(CP_ERR_INVALID_ARG, "%s: Hq=%d is not a multiple of Hkv=%d", who, Hq, cache->Hkv);
-    if ((Hq / cache->Hkv) % 2 != 0)
-        return set_error(CP_ERR_UNSUPPORTED, "%s: Hq/Hkv=%d must be even", who, Hq / cache->Hkv);
+    const int32_t heads_per_unit = ((Hq / cache->Hkv) % 2 == 0) ? 2 : 1;
     if (!(scale > 0.f)) return set_error(CP_ERR_INVALID_ARG, "%s: scale must be positive", who);
     if (((uintptr_t)q | (uintptr_t)out) & 15) return set_error(CP_ERR_INVALID_ARG, "%s: q and out must be 16-byte aligned", who);
     if (prefix_len + new_len > 0x7fffff00ll) return set_error(CP_ERR_UNSUPPORTED, "%s: request longer than 2^31 tokens", who);
@@ -1164,7 +1172,8 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     p.pieces = nullptr;
     p.partial_o = nullptr;
     p.partial_lse = nullptr;
-    p.pairs_per_tile = Hq / 2;
+    p.pairs_per_tile = Hq / heads_per_unit;
+    p.heads_per_unit = heads_per_unit;
     p.group = Hq / cache->Hkv;
     p.Hq = Hq;
     p.page_table = page_table;

@@ -198,19 +198,20 @@ extern "C" int cp_plan(int64_t new_len, int64_t prefix_len, int32_t C, cp_shard_
 }
 
 extern "C" size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C, int32_t Hq) {
-    if (B < 1 || !new_len || !C || Hq < 2) return 0;
+    if (B < 1 || !new_len || !C || Hq < 1) return 0;
     const int64_t n = max_tiles(B, new_len, C);
     if (n < 0) return 0;
-    const size_t pairs = (size_t)Hq / 2;
+    const size_t pairs = (size_t)Hq;          // one unit per head in the worst case (odd group size)
     // every unit is one piece, plus at most one extra piece per cut; the partial slots are bounded
     return workspace_layout((size_t)n, (size_t)n * pairs + kMaxSlots, kMaxSlots, kMaxSlots, kMaxGrid, kMaxSlots).total;
 }
 
 extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
-                                   int32_t Hq, int32_t num_sms, int64_t* summary, int32_t* pieces, int64_t max_pieces,
-                                   int32_t* items, int64_t max_items) {
-    if (B < 1 || !cu_new || !prefix_len || !C || Hq < 2 || Hq % 2 != 0 || num_sms < 1 || !summary)
+                                   int32_t Hq, int32_t Hkv, int32_t num_sms, int64_t* summary, int32_t* pieces,
+                                   int64_t max_pieces, int32_t* items, int64_t max_items) {
+    if (B < 1 || !cu_new || !prefix_len || !C || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || num_sms < 1 || !summary)
         return set_error(CP_ERR_INVALID_ARG, "cp_schedule_inspect: bad arguments");
+    const int32_t heads_per_unit = ((Hq / Hkv) % 2 == 0) ? 2 : 1;
     std::vector<int64_t> cu_pages(B + 1, 0);
     for (int32_t b = 0; b < B; ++b) {
         const int64_t R = cu_new[b + 1] - cu_new[b];
@@ -219,7 +220,7 @@ extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64
     }
     Schedule sch;
     build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), -1, sch.items);
-    if (int rc = build_schedule(Hq / 2, num_sms, sch)) return rc;
+    if (int rc = build_schedule(Hq / heads_per_unit, num_sms, sch)) return rc;
     int64_t max_load = 0, min_load = INT64_MAX, total = 0;
     for (int32_t c = 0; c < sch.grid; ++c) {
         int64_t load = 0;

@@ -55,7 +55,8 @@ def test_workspace_bytes(lib):
     small = binding.cp_workspace_bytes([1024], [2], 8)
     big = binding.cp_workspace_bytes([131072], [8], 32)
     assert 50e6 < small < 60e6                       # dominated by the fixed partial-result space
-    assert big - small == pytest.approx((1040 - 12) * 32 + (1040 * 16 - 12 * 4) * 16, abs=1024)
+    # 32 bytes per query tile + 16 bytes per (tile, head) unit (one head per unit in the worst case)
+    assert big - small == pytest.approx((1040 - 12) * 32 + (1040 * 32 - 12 * 8) * 16, abs=1024)
     assert small % 256 == 0 and big % 256 == 0
     assert binding.cp_workspace_bytes([0], [1], 8) == 0
     assert binding.cp_workspace_bytes([64], [1], 1) == 0

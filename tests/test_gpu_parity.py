@@ -117,6 +117,12 @@ def test_attention_small_mixed_batch(ctx):
     assert torch.equal(o1.view(torch.int16), dev.out.view(torch.int16)) and torch.equal(l1, dev.lse)
 
 
+def test_attention_odd_group_sizes(ctx):
+    # Hq / Hkv = 3 and plain multi-head attention (Hq == Hkv): one query head per work unit
+    check_batch(ctx, wl.Workload("odd_group", 41, 6, 2, [wl.Request(333, 192, 3), wl.Request(129, 0, 2)]))
+    check_batch(ctx, wl.Workload("mha", 42, 4, 4, [wl.Request(700, 64, 4)]))
+
+
 def test_attention_config1(ctx):
     check_batch(ctx, wl.config1())
 
@@ -175,8 +181,8 @@ def test_argument_validation_launches_nothing(ctx):
         binding.cp_prefill_attn(ctx, dev.q, dev.cache, dev.page_table, 0, 64, 1, w.Hq, w.scale, dev.out, dev.lse, small)
     assert e.value.code == binding.CP_ERR_WORKSPACE
     with pytest.raises(binding.CpError) as e:
-        binding.cp_prefill_attn(ctx, dev.q, dev.cache, dev.page_table, 0, 64, 1, 6, w.scale, dev.out, dev.lse, dev.ws)
-    assert e.value.code == binding.CP_ERR_UNSUPPORTED      # Hq/Hkv = 3 is odd
+        binding.cp_prefill_attn(ctx, dev.q, dev.cache, dev.page_table, 0, 64, 1, 7, w.scale, dev.out, dev.lse, dev.ws)
+    assert e.value.code == binding.CP_ERR_INVALID_ARG      # Hq = 7 is not a multiple of Hkv = 2
     with pytest.raises(binding.CpError) as e:
         binding.cp_prefill_attn(ctx, dev.q, dev.cache, dev.page_table, 0, 0, 1, w.Hq, w.scale, dev.out, dev.lse, dev.ws)
     assert e.value.code == binding.CP_ERR_INVALID_ARG

@@ -16,8 +16,8 @@ def check(w, num_sms=148):
     cu_new = w.cu_new
     prefix = [r.prefix_len for r in w.requests]
     Cs = [r.C for r in w.requests]
-    info, pieces, items = binding.cp_schedule_inspect(cu_new, prefix, Cs, w.Hq, num_sms)
-    HP = w.Hq // 2
+    info, pieces, items = binding.cp_schedule_inspect(cu_new, prefix, Cs, w.Hq, w.Hkv, num_sms)
+    HP = w.Hq // (2 if (w.Hq // w.Hkv) % 2 == 0 else 1)
     # tiles: rows tile [0, total_new) exactly, never straddle a request or a chunk, at most 128 rows
     rows = np.zeros(w.total_new, dtype=np.int32)
     for q0, n, kv0, nt in items:
@@ -71,6 +71,8 @@ def test_schedule_covers_and_balances_all_configs():
 def test_schedule_small_and_odd_shapes():
     for w in (wl.small_mixed(), wl.Workload("one_row", 1, 4, 2, [wl.Request(1, 0, 1)]),
               wl.Workload("long_prefix", 2, 8, 2, [wl.Request(7, 100000, 2)]),
-              wl.Workload("many_small", 3, 8, 2, [wl.Request(3 + i, 64 * (i % 3), 1 + i % 4) for i in range(40)])):
+              wl.Workload("many_small", 3, 8, 2, [wl.Request(3 + i, 64 * (i % 3), 1 + i % 4) for i in range(40)]),
+              wl.Workload("odd_group", 4, 6, 2, [wl.Request(300, 128, 2)]),
+              wl.Workload("mha", 5, 4, 4, [wl.Request(513, 0, 3)])):
         for sms in (1, 7, 148):
             check(w, sms)
