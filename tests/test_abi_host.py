@@ -59,7 +59,7 @@ def test_workspace_bytes(lib):
     assert big - small == pytest.approx((1040 - 12) * 32 + (1040 * 32 - 12 * 8) * 16, abs=1024)
     assert small % 256 == 0 and big % 256 == 0
     assert binding.cp_workspace_bytes([0], [1], 8) == 0
-    assert binding.cp_workspace_bytes([64], [1], 1) == 0
+    assert binding.cp_workspace_bytes([64], [1], 0) == 0
 
 
 def test_gpu_calls_fail_cleanly_without_a_device(lib):
