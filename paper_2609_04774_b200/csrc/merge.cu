@@ -11,7 +11,6 @@ namespace {
 
 constexpr int kMergeD = 128;
 constexpr int kTokPerCta = 8;    // tokens per CTA: 8 consecutive lse floats = one 32-byte sector
-constexpr int kHeadsPerWarp = 4; // consecutive heads (2 KB of every partial) handled by one warp
 constexpr int kMergeThreads = 32 * kTokPerCta;
 
 __device__ __forceinline__ float4 ld_stream(const float4* p) {
@@ -21,38 +20,43 @@ __device__ __forceinline__ float4 ld_stream(const float4* p) {
     return v;
 }
 
-// Grid: x = ceil(H / kHeadsPerWarp), y = ceil(T / kTokPerCta).  Warp w of the CTA handles token
-// y*8 + w and heads x*4 .. x*4+3.  NMAX > 0: N <= NMAX, loop fully unrolled with the loads of all
-// partials in flight before the first use.
-template <int NMAX, bool kOutBf16>
+// Grid: x = ceil(H / HPW), y = ceil(T / kTokPerCta).  Warp w of the CTA handles token y*8 + w and heads
+// x*HPW .. x*HPW+HPW-1 (HPW consecutive rows of every partial, 512 B each).  N <= NMAX; all HPW*NMAX
+// row loads of a warp are issued before the first use so that enough bytes are in flight per SM.
+template <int NMAX, int HPW, bool kOutBf16>
 __global__ void __launch_bounds__(kMergeThreads)
 merge_kernel(const float* __restrict__ partials, const float* __restrict__ lses, int N, int64_t T, int H,
              void* __restrict__ out, float* __restrict__ lse_out) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int64_t t = (int64_t)blockIdx.y * kTokPerCta + warp;
-    const int h0 = blockIdx.x * kHeadsPerWarp;
+    const int h0 = blockIdx.x * HPW;
     if (t >= T) return;
     const int64_t row_stride4 = kMergeD / 4;                          // float4 per row
     const int64_t part_stride4 = T * (int64_t)H * row_stride4;        // float4 per partial
     const float4* src = reinterpret_cast<const float4*>(partials) + (t * H + h0) * row_stride4 + lane;
 
+    float4 x[HPW][NMAX];
+    float my[HPW];
 #pragma unroll
-    for (int hh = 0; hh < kHeadsPerWarp; ++hh) {
-        const int h = h0 + hh;
-        if (h >= H) break;
-        // lane n < N holds lse of partial n; max / sum by warp shuffles
-        float my = -INFINITY;
-        if (lane < N) my = lses[((int64_t)lane * H + h) * T + t];
-        float4 x[NMAX];
+    for (int hh = 0; hh < HPW; ++hh) {
+        const bool hv = h0 + hh < H;
+        // lane n < N holds lse of partial n
+        my[hh] = (hv && lane < N) ? lses[((int64_t)lane * H + h0 + hh) * T + t] : -INFINITY;
 #pragma unroll
         for (int n = 0; n < NMAX; ++n)
-            if (n < N) x[n] = ld_stream(src + n * part_stride4 + hh * row_stride4);
-        float m = my;
+            if (hv && n < N) x[hh][n] = ld_stream(src + n * part_stride4 + hh * row_stride4);
+    }
+#pragma unroll
+    for (int hh = 0; hh < HPW; ++hh) {
+        const int h = h0 + hh;
+        if (h >= H) break;
+        // max / sum of the partial LSEs by warp shuffles
+        float m = my[hh];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
         const bool dead = (m == -INFINITY);
-        const float w = (dead || my == -INFINITY) ? 0.f : __expf(my - m);
+        const float w = (dead || my[hh] == -INFINITY) ? 0.f : __expf(my[hh] - m);
         float ws = w;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
@@ -63,10 +67,10 @@ merge_kernel(const float* __restrict__ partials, const float* __restrict__ lses,
             if (n < N) {
                 const float wn = __shfl_sync(0xffffffffu, w, n) * inv;
                 if (wn > 0.f) {   // a zero weight hides whatever the partial holds
-                    acc.x = fmaf(wn, x[n].x, acc.x);
-                    acc.y = fmaf(wn, x[n].y, acc.y);
-                    acc.z = fmaf(wn, x[n].z, acc.z);
-                    acc.w = fmaf(wn, x[n].w, acc.w);
+                    acc.x = fmaf(wn, x[hh][n].x, acc.x);
+                    acc.y = fmaf(wn, x[hh][n].y, acc.y);
+                    acc.z = fmaf(wn, x[hh][n].z, acc.z);
+                    acc.w = fmaf(wn, x[hh][n].w, acc.w);
                 }
             }
         }
@@ -85,14 +89,14 @@ merge_kernel(const float* __restrict__ partials, const float* __restrict__ lses,
     }
 }
 
-template <int NMAX>
+template <int NMAX, int HPW>
 void launch_merge(const float* partials, const float* lses, int N, int64_t T, int H, void* out, int out_dtype,
                   float* lse_out, cudaStream_t s) {
-    dim3 grid((H + kHeadsPerWarp - 1) / kHeadsPerWarp, (unsigned)((T + kTokPerCta - 1) / kTokPerCta));
+    dim3 grid((H + HPW - 1) / HPW, (unsigned)((T + kTokPerCta - 1) / kTokPerCta));
     if (out_dtype == CP_DTYPE_BF16)
-        merge_kernel<NMAX, true><<<grid, kMergeThreads, 0, s>>>(partials, lses, N, T, H, out, lse_out);
+        merge_kernel<NMAX, HPW, true><<<grid, kMergeThreads, 0, s>>>(partials, lses, N, T, H, out, lse_out);
     else
-        merge_kernel<NMAX, false><<<grid, kMergeThreads, 0, s>>>(partials, lses, N, T, H, out, lse_out);
+        merge_kernel<NMAX, HPW, false><<<grid, kMergeThreads, 0, s>>>(partials, lses, N, T, H, out, lse_out);
 }
 
 }  // namespace
@@ -111,10 +115,11 @@ extern "C" int cp_merge(cp_ctx* ctx, const float* partials, const float* lses, i
     if (((uintptr_t)partials | (uintptr_t)out) & 15)
         return set_error(CP_ERR_INVALID_ARG, "cp_merge: partials and out must be 16-byte aligned");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (N <= 2) launch_merge<2>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
-    else if (N <= 4) launch_merge<4>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
-    else if (N <= 8) launch_merge<8>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
-    else if (N <= 16) launch_merge<16>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
-    else launch_merge<32>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
+    // heads per warp chosen so that 8 to 16 row loads (128 to 256 bytes per lane) are in flight per warp
+    if (N <= 2) launch_merge<2, 4>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
+    else if (N <= 4) launch_merge<4, 2>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
+    else if (N <= 8) launch_merge<8, 1>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
+    else if (N <= 16) launch_merge<16, 1>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
+    else launch_merge<32, 1>(partials, lses, N, T, H, out, out_dtype, lse_out, s);
     return check_cuda(cudaGetLastError(), "cp_merge launch");
 }
