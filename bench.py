@@ -538,6 +538,7 @@ def run_table(args, out):
     ctx = binding.Context(0)
     Hq, Hkv, D = 32, 8, 128
     out.write("R,P,C,W,W_over_C,t_all_ms,t_shard_max_ms,t_shard_min_ms\n")
+    rows = []
     for R in args.table_R:
         for hit in (0.0, 0.25, 0.5, 0.75, 0.9):
             L = int(round(R / (1 - hit)))
@@ -553,29 +554,46 @@ def run_table(args, out):
             po = torch.empty((R, Hq, D), dtype=torch.float32, device="cuda")
             ws = torch.zeros(binding.cp_workspace_bytes([R], [8], Hq), dtype=torch.uint8, device="cuda")
 
-            def timeit(fn, reps):
+            def timeit(fn):
+                """Best of three batch means; a batch runs for about 10 ms (2 to 50 launches)."""
                 for _ in range(2):
                     fn()
                 torch.cuda.synchronize()
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-                for _ in range(reps):
-                    fn()
+                fn()
                 e1.record()
                 torch.cuda.synchronize()
-                return e0.elapsed_time(e1) / reps
+                reps = int(max(2, min(50, 10.0 / max(e0.elapsed_time(e1), 1e-3))))
+                best = float("inf")
+                for _ in range(3):
+                    e0.record()
+                    for _ in range(reps):
+                        fn()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    best = min(best, e0.elapsed_time(e1) / reps)
+                return best
 
             W = R * P + R * (R + 1) // 2
-            reps = max(2, min(20, int(2e12 / (4 * D * Hq * W))))
             for C in (1, 2, 4, 8):
-                t_all = timeit(lambda: binding.cp_prefill_attn(ctx, q, cache, pt, P, R, C, Hq, w0.scale, o, lse, ws), reps)
-                ts = [timeit(lambda: binding.cp_prefill_attn_shard(ctx, q, cache, pt, P, R, C, s, Hq, w0.scale, po, lse, ws), reps)
+                t_all = timeit(lambda: binding.cp_prefill_attn(ctx, q, cache, pt, P, R, C, Hq, w0.scale, o, lse, ws))
+                ts = [timeit(lambda: binding.cp_prefill_attn_shard(ctx, q, cache, pt, P, R, C, s, Hq, w0.scale, po, lse, ws))
                       for s in range(C)]
                 out.write("%d,%d,%d,%d,%.1f,%.4f,%.4f,%.4f\n" % (R, P, C, W, W / C, t_all, max(ts), min(ts)))
                 out.flush()
+                rows.append((R, P, C, max(ts) * 1e-3))
             ctx.poll_status()
             del q, k, v, o, po, lse
             torch.cuda.empty_cache()
+    # Eq. (2) fitted to the slowest shard of every (R, P, C): what one CP rank of degree C would take
+    from paper_2609_04774_b200 import prefill_model as pm
+    Rs, Ps, Cs, ts = (np.array(x, dtype=np.float64) for x in zip(*rows))
+    m = pm.fit(Rs, Ps, Cs, ts)
+    rel = np.abs(m.predict(Rs, Ps, Cs) / ts - 1)
+    out.write("# fit of Eq. 2 to t_shard_max (seconds): d=%.3e a=%.3e b=%.3e c=%.3e alpha=%.3e ; relative error median %.3f "
+              "p90 %.3f max %.3f\n" % (m.d, m.a, m.b, m.c, m.alpha, np.median(rel), np.quantile(rel, 0.9), rel.max()))
+    out.flush()
 
 
 def main():

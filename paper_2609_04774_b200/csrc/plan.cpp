@@ -79,7 +79,7 @@ WorkspaceLayout workspace_layout(size_t n_items, size_t n_pieces, size_t n_merge
     return w;
 }
 
-int build_schedule(int32_t pairs_per_tile, int32_t grid_max, Schedule& s) {
+static int build_schedule_impl(int32_t pairs_per_tile, int32_t grid_max, bool allow_split, Schedule& s) {
     const int32_t HP = pairs_per_tile;
     const int64_t n_items = (int64_t)s.items.size();
     const int64_t n_units = n_items * HP;
@@ -141,7 +141,7 @@ int build_schedule(int32_t pairs_per_tile, int32_t grid_max, Schedule& s) {
         while (t < n) {
             while (c < G - 1 && T - load[c] < std::min<int64_t>(minp, n - t)) ++c;          // CTA is full
             int64_t len = std::min<int64_t>(n - t, std::max<int64_t>(T - load[c], 0));
-            if (c == G - 1 || len <= 0) len = n - t;                                        // last CTA takes what is left
+            if (c == G - 1 || len <= 0 || !allow_split) len = n - t;                        // last CTA takes what is left
             if (n - t - len > 0 && n - t - len < minp) len = n - t;                           // no tiny remainder
             cuts.push_back({(int32_t)u, c, t, (int32_t)(t + len), -1});
             load[c] += len;
@@ -156,7 +156,11 @@ int build_schedule(int32_t pairs_per_tile, int32_t grid_max, Schedule& s) {
             }
         }
     }
-    if (n_slots > kMaxSlots) return set_error(CP_ERR_UNSUPPORTED, "schedule: %d partial slots", n_slots);
+    if (n_slots > kMaxSlots) {
+        // cannot happen with one cut per CTA boundary; if it ever does, fall back to whole units only
+        if (allow_split) return build_schedule_impl(pairs_per_tile, grid_max, false, s);
+        return set_error(CP_ERR_UNSUPPORTED, "schedule: %d partial slots", n_slots);
+    }
     s.n_slots = n_slots;
 
     // 3. per-CTA lists: whole units in dealing order, then the CTA's KV ranges
@@ -174,6 +178,10 @@ int build_schedule(int32_t pairs_per_tile, int32_t grid_max, Schedule& s) {
     for (const Cut& k : cuts)
         s.pieces[(size_t)fill[k.cta]++] = {tail[k.unit].item, (int16_t)tail[k.unit].pair, (int16_t)k.slot, k.t_begin, k.t_end};
     return CP_OK;
+}
+
+int build_schedule(int32_t pairs_per_tile, int32_t grid_max, Schedule& s) {
+    return build_schedule_impl(pairs_per_tile, grid_max, true, s);
 }
 
 }  // namespace cpattn
