@@ -134,19 +134,30 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t grid_max, bool al
     s.merge_slots.clear();
     int32_t n_slots = 0;
     int32_t c = 0;
+    int64_t tail_left = 0;
+    for (const TailUnit& tu : tail) tail_left += tu.n;
+    int64_t T_cur = T;       // raised when every CTA is full and work is still left (shares are rounded)
     for (size_t u = 0; u < tail.size(); ++u) {
         int32_t t = 0;
         const int32_t n = tail[u].n;
         const size_t first = cuts.size();
         while (t < n) {
-            while (c < G - 1 && T - load[c] < std::min<int64_t>(minp, n - t)) ++c;          // CTA is full
-            int64_t len = std::min<int64_t>(n - t, std::max<int64_t>(T - load[c], 0));
-            if (c == G - 1 || len <= 0 || !allow_split) len = n - t;                        // last CTA takes what is left
+            int32_t scanned = 0;
+            while (T_cur - load[c] < std::min<int64_t>(minp, n - t)) {                     // CTA is full
+                c = (c + 1 == G) ? 0 : c + 1;
+                if (++scanned >= G) {
+                    T_cur += std::max<int64_t>(minp, (tail_left + G - 1) / G);
+                    scanned = 0;
+                }
+            }
+            int64_t len = std::min<int64_t>(n - t, T_cur - load[c]);
+            if (!allow_split) len = n - t;
             if (n - t - len > 0 && n - t - len < minp) len = n - t;                           // no tiny remainder
             cuts.push_back({(int32_t)u, c, t, (int32_t)(t + len), -1});
             load[c] += len;
             ++count[c];
             t += (int32_t)len;
+            tail_left -= len;
         }
         if (cuts.size() - first > 1) {
             s.merges.push_back({tail[u].item, tail[u].pair, (int32_t)(cuts.size() - first), (int32_t)s.merge_slots.size()});

@@ -54,13 +54,17 @@ def _nnls(A: np.ndarray, y: np.ndarray, iters: int = 20000) -> np.ndarray:
     return x / scale
 
 
-def fit(R, P, C, t) -> PrefillModel:
-    """Fit (d, a, b, c, alpha) >= 0 of Eq. (2) to measured times t(R, P, C)."""
+def fit(R, P, C, t, relative: bool = True) -> PrefillModel:
+    """Fit (d, a, b, c, alpha) >= 0 of Eq. (2) to measured times t(R, P, C).  With ``relative`` every
+    sample is weighted by 1/t, so that microsecond and second scale measurements count alike."""
     R = np.asarray(R, dtype=np.float64)
     P = np.asarray(P, dtype=np.float64)
     C = np.asarray(C, dtype=np.float64)
     t = np.asarray(t, dtype=np.float64)
     A = np.stack([np.ones_like(R), R, P, R / C, remaining_workload(R, P) / C], axis=1)
+    if relative:
+        A = A / t[:, None]
+        t = np.ones_like(t)
     try:
         from scipy.optimize import nnls
         coef, _ = nnls(A / np.abs(A).max(axis=0), t)

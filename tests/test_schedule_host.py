@@ -68,6 +68,15 @@ def test_schedule_covers_and_balances_all_configs():
         assert loads.mean() >= 0.97 * info["max_load"] - 1, (cfg, info)   # the slowest CTA is within 3 % of the mean
 
 
+def test_schedule_balances_short_no_prefix_requests():
+    # many short units (no prefix): nothing may pile up on one CTA when the shares are rounded
+    for R in (1024, 2048, 4096, 8192):
+        for C in (1, 2, 8):
+            info, loads = check(wl.Workload("noprefix", 1, 32, 8, [wl.Request(R, 0, C)]))
+            share = -(-info["total"] // info["grid"])
+            assert info["max_load"] <= max(1.25 * share, share + 8), (R, C, info)
+
+
 def test_schedule_small_and_odd_shapes():
     for w in (wl.small_mixed(), wl.Workload("one_row", 1, 4, 2, [wl.Request(1, 0, 1)]),
               wl.Workload("long_prefix", 2, 8, 2, [wl.Request(7, 100000, 2)]),
