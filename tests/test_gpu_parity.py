@@ -123,6 +123,51 @@ def test_attention_odd_group_sizes(ctx):
     check_batch(ctx, wl.Workload("mha", 42, 4, 4, [wl.Request(700, 64, 4)]))
 
 
+def test_attention_kv_split_units(ctx):
+    # few query rows, long prefixes: every unit is cut along KV over many CTAs and merged by the fix-up
+    # kernel; prefix lengths that are not page multiples; a request whose rows see no key of some piece
+    w = wl.Workload("kv_split", 43, 8, 2, [wl.Request(130, 40000, 2), wl.Request(7, 100003, 1), wl.Request(64, 64, 1)])
+    info, _, _ = binding.cp_schedule_inspect(w.cu_new, [r.prefix_len for r in w.requests], [r.C for r in w.requests],
+                                             w.Hq, w.Hkv, torch.cuda.get_device_properties(0).multi_processor_count,
+                                             want_lists=False)
+    assert info["split_units"] >= 8 and info["slots"] > 2 * info["split_units"]
+    dev, out, lse, _ = check_batch(ctx, w, pair_budget=1e10)
+    o1, l1 = dev.out.clone(), dev.lse.clone()
+    dev.run_batch(ctx)                                   # the merge order is fixed: bitwise reproducible
+    assert torch.equal(o1.view(torch.int16), dev.out.view(torch.int16)) and torch.equal(l1, dev.lse)
+
+
+def test_attention_strided_cache_view(ctx):
+    # the cache is a view into a wider allocation (one unused head slot per token, an unused token row
+    # per page): only the three strides say where things are
+    w = wl.Workload("strided", 44, 8, 2, [wl.Request(300, 200, 2), wl.Request(90, 0, 1)])
+    mat = wl.materialize(w)
+    dev = DeviceWorkload(mat)
+    npg = mat.k_pages.shape[0]
+    big_k = torch.full((npg, wl.PAGE + 1, w.Hkv + 1, w.D), 3.0e38, dtype=torch.bfloat16, device="cuda")
+    big_v = torch.full_like(big_k, -3.0e38)
+    big_k[:, :wl.PAGE, :w.Hkv] = dev.k
+    big_v[:, :wl.PAGE, :w.Hkv] = dev.v
+    dev.k, dev.v = big_k[:, :wl.PAGE, :w.Hkv], big_v[:, :wl.PAGE, :w.Hkv]
+    dev.cache = binding.make_cache(dev.k, dev.v)
+    assert dev.cache.stride_tok == (w.Hkv + 1) * w.D and dev.cache.stride_page == (wl.PAGE + 1) * (w.Hkv + 1) * w.D
+    out, lse = dev.run_batch(ctx)
+    for b, r in enumerate(w.requests):
+        lo, hi = int(w.cu_new[b]), int(w.cu_new[b + 1])
+        ref_o, ref_l = oracle_request(mat, b)
+        compare(out[lo:hi], lse[:, lo:hi], ref_o, ref_l, "strided req %d" % b)
+    # gather through the same view is bit-exact too
+    r = w.requests[0]
+    kr = torch.zeros((r.total_len, w.Hkv, w.D), dtype=torch.bfloat16, device="cuda")
+    vr = torch.zeros_like(kr)
+    pt = dev.page_table[:r.n_pages]
+    binding.cp_kv_gather(ctx, dev.cache, pt, 0, r.total_len, kr, vr)
+    torch.cuda.synchronize()
+    pth = mat.page_table[:r.n_pages]
+    assert np.array_equal(kr.view(torch.int16).cpu().numpy().view(np.uint16), orc.kv_gather(mat.k_pages, pth, 0, r.total_len))
+    assert np.array_equal(vr.view(torch.int16).cpu().numpy().view(np.uint16), orc.kv_gather(mat.v_pages, pth, 0, r.total_len))
+
+
 def test_attention_config1(ctx):
     check_batch(ctx, wl.config1())
 
