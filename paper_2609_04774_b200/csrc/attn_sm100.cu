@@ -14,8 +14,8 @@
 // columns of its S tile and is consumed from TMEM as the A operand of P*V.
 // The tensor pipe executes the MMAs of the issuing thread in order, PV0(j) S0(j+1) PV1(j) S1(j+1):
 // S(j+1) follows P*V(j) of the same head (P overwrites S), and while one warpgroup runs softmax on
-// its tile the pipe works for the other head.  P is handed over in four pieces of 32 keys, so P*V
-// starts while the rest of the row is still being exponentiated.
+// its tile the pipe works for the other head.  P is handed over in two pieces (96 keys, then 32), so
+// P*V starts while the rest of the row is still being exponentiated.
 // Every wait is bounded; on expiry the CTA records where it gave up in the status word, all roles
 // drain and the kernel returns normally.
 #include <cuda_bf16.h>
@@ -71,7 +71,8 @@ constexpr uint32_t kTmemO = 256;   // + wg * 128
 constexpr uint32_t kTryWaitHintNs = 200000;             // the thread may stay suspended this long per try
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
 constexpr float kRescaleThreshold = 8.0f;
-constexpr int kPieces = 2;                            // P is handed to the MMA warp in this many pieces (1, 2 or 4)
+constexpr int kPieces = 2;                            // P is handed to the MMA warp in two pieces:
+constexpr int kSplitQ = 3;                            // the first kSplitQ quarters of the row, then the rest
 constexpr int kPolyOf4 = 1;                            // pairs out of every four whose exp2 runs on the FMA pipe              // log2 units: keep a stale row max up to 2^8
 
 struct AttnParams {
@@ -395,8 +396,8 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
 
 // The issuer warp alternates between the two heads in a fixed order, PV0(j) S0(j+1) PV1(j) S1(j+1):
 // the tensor pipe executes in issue order, which keeps the two softmax warpgroups half a period apart
-// (one exponentiates while the pipe works for the other).  P arrives in four pieces of 32 keys, so
-// P*V starts while the rest of the row is still being exponentiated.  The whole warp runs the loop
+// (one exponentiates while the pipe works for the other).  P arrives in two pieces (96 keys, then 32),
+// so P*V starts while the rest of the row is still being exponentiated.  The whole warp runs the loop
 // (waits included) so that addresses and descriptors stay warp-uniform; one elected lane issues.
 __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
                                          volatile uint32_t* abort_flag) {
@@ -417,11 +418,11 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base
                    k_desc0 + slot * (kTileBytes >> 4) + off, kIdescS, ks > 0);
         }
     };
-    // O += P V over one piece of the tile's keys: 128/kPieces keys = 8/kPieces MMAs of 16 keys
+    // O += P V over one piece of the tile's keys: MMAs of 16 keys, 2 per quarter of the row
     auto mma_pv = [&](int wg, int part, uint32_t slot, bool accumulate) {
+        const int ks0 = part == 0 ? 0 : 2 * kSplitQ, ks1 = part == 0 ? 2 * kSplitQ : 8;
 #pragma unroll
-        for (int k2 = 0; k2 < 8 / kPieces; ++k2) {
-            const int ks = part * (8 / kPieces) + k2;
+        for (int ks = ks0; ks < ks1; ++ks) {
             mma_ts(tmem_base + kTmemO + wg * 128, tmem_base + kTmemS + wg * 128 + ks * 8,
                    v_desc0 + slot * (kTileBytes >> 4) + ks * (2048 >> 4), kIdescPV, accumulate || ks > 0);
         }
@@ -558,7 +559,7 @@ __device__ __forceinline__ void exp32(const float (&s)[32], uint32_t (&pk)[16], 
 
 // One 128x128 score tile of one head: the row is read from TMEM once (four 32-column loads, one
 // wait), reduced to its max, exponentiated in four pieces of 32 keys, and P goes back to TMEM piece
-// by piece, each hand-over signalled to the MMA warp.  Straight-line code in both variants (no
+// by piece; the MMA warp is signalled after the third piece and after the last.  Straight-line code in both variants (no
 // per-element branches) so that the scheduler can overlap the MUFU, FMA and ALU pipes.
 // kMasked: the tile reaches past the causal diagonal of some rows; `lim` = visible columns of this row.
 template <bool kMasked>
@@ -614,10 +615,10 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, u
 #define CP_P_PIECE(cur, q)                                                              \
     exp32<kMasked>(cur, pk, c2, nm2, sum0, sum1, sum2, sum3);                           \
     TMEM_ST16R(s_tmem + (q) * 16, pk, 0);                                               \
-    if (((q) + 1) % (4 / kPieces) == 0) {                                               \
+    if ((q) + 1 == kSplitQ || (q) == 3) {                                               \
         tc_wait_st();                                                                   \
         tc_fence_before();                                                              \
-        mbar_arrive(p_bar0 + ((q) / (4 / kPieces)) * 8);                                \
+        mbar_arrive(p_bar0 + ((q) == 3 ? 1 : 0) * 8);                                   \
     }
     CP_P_PIECE(s0, 0)
     CP_P_PIECE(s1, 1)
