@@ -100,7 +100,8 @@ typedef struct {
  * Hq query heads: the work lists of the persistent scheduler and the fp32 partial results of the
  * (query tile, head pair) units whose KV range is split over several CTAs for load balance (about
  * 55 MB of fixed partial space plus 16 bytes per unit).  new_len, C: host arrays of B entries.
- * Returns 0 on invalid arguments. */
+ * Returns 0 on invalid arguments.  A workspace belongs to one call at a time: calls that may overlap on
+ * the GPU (different streams without an ordering between them) need separate workspaces. */
 size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C, int32_t Hq);
 
 /* cp_schedule_inspect -- host only: the work distribution the attention calls would use for a batch
@@ -120,7 +121,9 @@ int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_
 /* ---------------------------------------------------------------------------------------------
  * cp_prefill_attn -- all C shards of one request in one launch (Sections 2.1-2.2).
  *   q          device [R, Hq, D] bf16, new tokens in original order
- *   page_table device int32, ceil((P+R)/page_size) entries, each in [0, num_pages)
+ *   page_table device int32, ceil((P+R)/page_size) entries, each in [0, num_pages) (the table lives
+ *              on the device and is not validated; an entry outside the pool reads as zeros, it
+ *              cannot fault)
  *   scale      softmax scale (1/sqrt(D) in the paper's definition)
  *   out        device [R, Hq, D] bf16; row r = softmax(scale * q_r K^T + mask) V, written at its
  *              original position (the "restore order" step is fused into the store)

@@ -376,7 +376,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
                     if (lane == 0) {
                         const uint32_t slot = kv_it % kKvStages;
                         mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j0 + jj);
-                        { const int j = j0 + jj; CP_TRACE(3, j, 6 + kv); }
+                        CP_TRACE(3, j0 + jj, 6 + kv);
                         const uint32_t fbar = bars + (kBarKvFull + slot) * 8;
                         const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
                         const CUtensorMap* map = kv ? tmV : tmK;
