@@ -56,7 +56,7 @@ def load_peaks():
 
 
 def get_workload(cfg: int) -> wl.Workload:
-    return wl.CONFIGS[cfg]()
+    return (wl.CONFIGS.get(cfg) or wl.VARIANTS[cfg])()
 
 
 # ----------------------------------------------------------------------------------------------
@@ -604,7 +604,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="BASELINE config number of the headline workload")
     ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table", "kvcopy"])
-    ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5])
+    ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5],
+                    help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P")
     ap.add_argument("--merge-T", type=int, nargs="*", default=[4096, 16384, 65536, 262144])
     ap.add_argument("--merge-reps", type=int, default=20)
     ap.add_argument("--table-R", type=int, nargs="*", default=[1024, 2048, 4096, 8192, 16384, 32768, 65536, 131072])

@@ -310,7 +310,20 @@ def small_mixed(seed: int = 11) -> Workload:
     return Workload("small_mixed", seed, 8, 2, reqs)
 
 
+def variant_gqa8() -> Workload:
+    """Config 2's lengths with the head shape of a 32/4 grouped-query model (eight query heads per KV
+    head, the second model family of the paper's evaluation), seed 7."""
+    return Workload("var_gqa8_R4096_P12288_C4", 7, 32, 4, [Request(4096, 12288, 4)])
+
+
+def variant_chunked_prefill() -> Workload:
+    """One 512-token chunk of a chunked prefill behind a 64K-token cached prefix (R << P): every work
+    unit is cut along KV and merged by LSE, seed 8."""
+    return Workload("var_chunk_R512_P65536_C2", 8, 32, 8, [Request(512, 65536, 2)])
+
+
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
+VARIANTS = {6: variant_gqa8, 7: variant_chunked_prefill}
 
 
 # --------------------------------------------------------------------------------------

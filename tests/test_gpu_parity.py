@@ -248,6 +248,16 @@ def test_attention_config4_varlen(ctx):
     check_batch(ctx, wl.config4(), pair_budget=1.5e8)
 
 
+def test_attention_variant_gqa8_and_chunked_prefill(ctx):
+    # eight query heads per KV head; a short chunk behind a long cached prefix (all units KV-split)
+    check_batch(ctx, wl.variant_gqa8(), pair_budget=2e8)
+    w = wl.variant_chunked_prefill()
+    info, _, _ = binding.cp_schedule_inspect(w.cu_new, [65536], [2], w.Hq, w.Hkv,
+                                             torch.cuda.get_device_properties(0).multi_processor_count, want_lists=False)
+    assert info["split_units"] == 64 and info["max_load"] * info["grid"] <= 1.01 * info["total"]
+    check_batch(ctx, w, pair_budget=2e8)
+
+
 def test_attention_config5_sampled(ctx):
     check_batch(ctx, wl.config5(), pair_budget=1.2e9)
 
