@@ -157,6 +157,23 @@ int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, 
                           float scale, float* partial_out, float* partial_lse, void* workspace,
                           size_t workspace_bytes, void* stream);
 
+/* cp_prefill_attn_chunk -- the rows of ONE zigzag chunk (0 <= chunk < 2C) of cp_plan(R, P, C), in
+ * chunk-local buffers: what a CP rank runs twice per layer, once for its early chunk k as soon as the
+ * keys of chunks 0..k have arrived and once for its late chunk 2C-1-k (Section 2.1: rank k holds the
+ * k-th and (2C-1-k)-th chunks, gathers K/V, attends its local queries to all causally visible keys).
+ *   q_chunk    device [n, Hq, D] bf16, n = rows of the chunk (q_end - q_begin of cp_plan); row i is
+ *              new token q_begin + i, at absolute position P + q_begin + i
+ *   out_chunk  device [n, Hq, D] bf16;  lse_chunk  device [Hq, n] fp32
+ *   page_table device, ceil((P+R)/page_size) entries; only entries below ceil((P+q_end)/page_size)
+ *              are read, later pages may still be empty.  Token slots of a referenced page that lie
+ *              behind P + q_end are read and masked: they must hold finite values.
+ * An empty chunk (padding of a short request) launches nothing and returns CP_OK.  Workspace as for
+ * cp_prefill_attn with the same (R, C, Hq).  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
+int cp_prefill_attn_chunk(cp_ctx* ctx, const void* q_chunk, const cp_kv_cache* cache, const int32_t* page_table,
+                          int64_t prefix_len, int64_t new_len, int32_t C, int32_t chunk, int32_t Hq,
+                          float scale, void* out_chunk, float* lse_chunk, void* workspace,
+                          size_t workspace_bytes, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * cp_prefill_attn_static -- cp_prefill_attn for callers that must not allocate device memory.
  * (The paper has no counterpart to this call; it exists for integration reasons only.)

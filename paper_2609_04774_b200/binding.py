@@ -20,7 +20,7 @@ CP_ERR_INVALID_ARG, CP_ERR_UNSUPPORTED, CP_ERR_WORKSPACE, CP_ERR_CUDA, CP_ERR_TI
 CP_DTYPE_BF16, CP_DTYPE_F32 = 0, 1
 
 EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "cp_ctx_poll_status", "cp_plan",
-           "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_static", "cp_merge",
+           "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_chunk", "cp_prefill_attn_static", "cp_merge",
            "cp_kv_gather", "cp_kv_append"]
 
 
@@ -188,6 +188,16 @@ def cp_prefill_attn_shard(ctx, q, cache, page_table, prefix_len, new_len, C, sha
         ctypes.c_int32(C), ctypes.c_int32(shard), ctypes.c_int32(Hq), ctypes.c_float(scale), _ptr(partial_out),
         _ptr(partial_lse), _ptr(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
         _stream(stream)))
+
+
+def cp_prefill_attn_chunk(ctx, q_chunk, cache, page_table, prefix_len, new_len, C, chunk, Hq, scale, out_chunk,
+                          lse_chunk, workspace, stream=None):
+    """One zigzag chunk in chunk-local buffers: q_chunk/out_chunk [n,Hq,D] bf16, lse_chunk [Hq,n] fp32."""
+    _check(load().cp_prefill_attn_chunk(
+        ctx._h, _ptr(q_chunk), ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(prefix_len),
+        ctypes.c_int64(new_len), ctypes.c_int32(C), ctypes.c_int32(chunk), ctypes.c_int32(Hq), ctypes.c_float(scale),
+        _ptr(out_chunk), _ptr(lse_chunk), _ptr(workspace),
+        ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
 
 
 def cp_prefill_attn_static(q, cache, page_table, prefix_len, new_len, C, Hq, scale, out, lse, stream=None):

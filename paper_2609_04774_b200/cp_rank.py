@@ -1,0 +1,199 @@
+"""One rank of a degree-C context-parallel prefill worker, built on the library's single-GPU calls.
+
+Section 2.1 of the paper: rank k of C holds zigzag chunks k and 2C-1-k of the uncached suffix, computes
+Q/K/V for them, all-gathers K and V, attends its local queries to every causally visible key and the
+outputs go back to their original order.  Section 2.2: on a prefix hit the cached KV is partitioned
+across the worker's ranks, so it is gathered as well (the b*P term of Eq. 2).
+
+What runs where.  The exchange is three all-gathers (prefix blocks, early chunks, late chunks) issued
+back to back on the communicator; the attention over the early chunk needs only the first two, so it
+runs while the third is still in flight (early chunk first).  Gathered rows land in contiguous staging
+buffers and are written into this rank's own paged cache by cp_kv_append; attention reads that cache
+through cp_prefill_attn_chunk.  Remote data is therefore always copied into local HBM before a kernel
+reads it.  The module holds no arithmetic of the method: it moves rows and calls the library.
+
+Readings (the paper fixes none of these): prefix pages are owned in contiguous blocks of
+ceil(n_prefix_pages / C) pages, block r on rank r; the prefix length is a multiple of the page size
+(block-granular reuse, Section 6); chunks are padded to cl = ceil(R / 2C) rows for the collective.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+
+@dataclass(frozen=True)
+class RankLayout:
+    """Integer layout of one rank's share of a request (R new tokens behind P cached ones)."""
+    R: int
+    P: int
+    C: int
+    rank: int
+    page: int = 64
+
+    def __post_init__(self):
+        if self.R < 1 or self.P < 0 or self.C < 1 or not 0 <= self.rank < self.C:
+            raise ValueError("bad layout R=%d P=%d C=%d rank=%d" % (self.R, self.P, self.C, self.rank))
+        if self.P % self.page:
+            raise ValueError("prefix length %d is not a multiple of the page size %d" % (self.P, self.page))
+
+    @property
+    def cl(self) -> int:
+        return -(-self.R // (2 * self.C))
+
+    def chunk(self, j: int):
+        """Rows [begin, end) of zigzag chunk j (right-padded split, clipped to R)."""
+        return min(j * self.cl, self.R), min((j + 1) * self.cl, self.R)
+
+    @property
+    def early(self) -> int:
+        return self.rank
+
+    @property
+    def late(self) -> int:
+        return 2 * self.C - 1 - self.rank
+
+    def late_chunk_of(self, r: int) -> int:
+        return 2 * self.C - 1 - r
+
+    @property
+    def prefix_pages(self) -> int:
+        return self.P // self.page
+
+    @property
+    def block_pages(self) -> int:
+        """Prefix pages per rank (the last blocks may be short or empty)."""
+        return -(-self.prefix_pages // self.C) if self.prefix_pages else 0
+
+    def prefix_block(self, r: int):
+        """Token range [begin, end) of the prefix block owned by rank r."""
+        b = min(r * self.block_pages, self.prefix_pages) * self.page
+        e = min((r + 1) * self.block_pages, self.prefix_pages) * self.page
+        return b, e
+
+
+class TorchComm:
+    """All-gather of equally sized row blocks over a torch.distributed group (NCCL on GPUs, gloo on CPU)."""
+
+    def __init__(self, group=None):
+        import torch.distributed as dist
+        self.dist = dist
+        self.group = group
+        self.size = dist.get_world_size(group)
+        self.rank = dist.get_rank(group)
+
+    def all_gather(self, block):
+        """block [n, ...] -> (out [size, n, ...], handle); handle.wait() orders the caller's stream behind it."""
+        import torch
+        out = torch.empty((self.size,) + tuple(block.shape), dtype=block.dtype, device=block.device)
+        # rows travel as bytes: every backend moves uint8, whatever the row type is
+        src = block.contiguous().view(torch.uint8).reshape(-1)
+        dst = out.view(torch.uint8).reshape(self.size, -1)
+        work = self.dist.all_gather(list(dst.unbind(0)), src, group=self.group, async_op=True)
+        return out, work
+
+
+class LibraryOps:
+    """The three device steps of a rank, on this rank's paged cache, through the C-ABI library."""
+
+    def __init__(self, ctx, k_pages, v_pages, page_table, Hq, scale):
+        import torch
+        from . import binding
+        self.b, self.ctx, self.torch = binding, ctx, torch
+        self.cache = binding.make_cache(k_pages, v_pages)
+        self.k_pages, self.v_pages, self.page_table = k_pages, v_pages, page_table
+        self.Hq, self.scale = Hq, scale
+        self.Hkv, self.D = k_pages.shape[2], k_pages.shape[3]
+        self.device = k_pages.device
+        self._ws = None
+
+    def empty_rows(self, n, heads):
+        return self.torch.zeros((n, heads, self.D), dtype=self.torch.bfloat16, device=self.device)
+
+    def kv_gather(self, t_begin, n, k_rows, v_rows):
+        if n > 0:
+            self.b.cp_kv_gather(self.ctx, self.cache, self.page_table, t_begin, n, k_rows, v_rows)
+
+    def kv_append(self, t_begin, n, k_rows, v_rows):
+        if n > 0:
+            self.b.cp_kv_append(self.ctx, self.cache, self.page_table, t_begin, n, k_rows, v_rows)
+
+    def attn_chunk(self, lay: RankLayout, chunk, q_chunk):
+        n = q_chunk.shape[0]
+        out = self.torch.empty((n, self.Hq, self.D), dtype=self.torch.bfloat16, device=self.device)
+        lse = self.torch.empty((self.Hq, n), dtype=self.torch.float32, device=self.device)
+        if n == 0:
+            return out, lse
+        if self._ws is None:
+            nbytes = self.b.cp_workspace_bytes([lay.R], [lay.C], self.Hq)
+            self._ws = self.torch.empty(nbytes, dtype=self.torch.uint8, device=self.device)
+        self.b.cp_prefill_attn_chunk(self.ctx, q_chunk, self.cache, self.page_table, lay.P, lay.R, lay.C, chunk,
+                                     self.Hq, self.scale, out, lse, self._ws)
+        return out, lse
+
+
+def _padded(ops, rows, n):
+    """rows [m, H, D] -> [n, H, D] with zero rows behind (collectives need equal sizes)."""
+    if rows.shape[0] == n:
+        return rows
+    buf = ops.empty_rows(n, rows.shape[1])
+    buf[:rows.shape[0]] = rows
+    return buf
+
+
+class CpRankWorker:
+    """Runs one layer's attention for this rank's two chunks.
+
+    comm: an object with .size, .rank and all_gather(block) -> (out, handle), e.g. TorchComm.
+    ops: the device steps; LibraryOps is the only implementation in the package.
+    """
+
+    def __init__(self, layout: RankLayout, comm, ops):
+        if comm.size != layout.C or comm.rank != layout.rank:
+            raise ValueError("communicator (%d of %d) does not match the layout (%d of %d)" %
+                             (comm.rank, comm.size, layout.rank, layout.C))
+        self.lay, self.comm, self.ops = layout, comm, ops
+
+    def prefill(self, q_early, q_late, k_early, v_early, k_late, v_late):
+        """q_*: this rank's query rows [n, Hq, D]; k_*/v_*: its new K/V rows [n, Hkv, D] (n = chunk rows).
+        The rank's prefix block must already be in its cache.  Returns (out_early, lse_early, out_late, lse_late)."""
+        lay, ops, comm = self.lay, self.ops, self.comm
+        (eb, ee), (lb, le) = lay.chunk(lay.early), lay.chunk(lay.late)
+        assert q_early.shape[0] == ee - eb == k_early.shape[0] and q_late.shape[0] == le - lb == k_late.shape[0]
+
+        # 1. contributions: own prefix block read out of the cache, own chunks padded to cl rows
+        pb, pe = lay.prefix_block(lay.rank)
+        n_blk = lay.block_pages * lay.page
+        gathers = []
+        if n_blk:
+            sk, sv = ops.empty_rows(n_blk, ops.Hkv), ops.empty_rows(n_blk, ops.Hkv)
+            ops.kv_gather(pb, pe - pb, sk, sv)
+            gathers.append((comm.all_gather(sk), comm.all_gather(sv)))
+        else:
+            gathers.append(None)
+        gathers.append((comm.all_gather(_padded(ops, k_early, lay.cl)), comm.all_gather(_padded(ops, v_early, lay.cl))))
+        gathers.append((comm.all_gather(_padded(ops, k_late, lay.cl)), comm.all_gather(_padded(ops, v_late, lay.cl))))
+
+        def wait(g):
+            (k, hk), (v, hv) = g
+            hk.wait()
+            hv.wait()
+            return k, v
+
+        # 2. prefix blocks and early chunks: rank order is token order, one append each
+        if gathers[0] is not None:
+            gk, gv = wait(gathers[0])
+            ops.kv_append(0, lay.P, gk.reshape((-1,) + tuple(gk.shape[2:])), gv.reshape((-1,) + tuple(gv.shape[2:])))
+        gk, gv = wait(gathers[1])
+        n_first = min(lay.R, lay.C * lay.cl)
+        ops.kv_append(lay.P, n_first, gk.reshape((-1,) + tuple(gk.shape[2:])), gv.reshape((-1,) + tuple(gv.shape[2:])))
+
+        # 3. early chunk: its keys are all here; the late all-gather is still in flight
+        out_e, lse_e = ops.attn_chunk(lay, lay.early, q_early)
+
+        # 4. late chunks: rank r sent chunk 2C-1-r
+        gk, gv = wait(gathers[2])
+        for r in range(lay.C):
+            b, e = lay.chunk(lay.late_chunk_of(r))
+            ops.kv_append(lay.P + b, e - b, gk[r], gv[r])
+        out_l, lse_l = ops.attn_chunk(lay, lay.late, q_late)
+        return out_e, lse_e, out_l, lse_l

@@ -926,8 +926,8 @@ int upload_block(cp_ctx* ctx, const std::vector<uint8_t>& block, void* dst, cuda
 
 int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table, int32_t B,
                 const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C, const int64_t* cu_pages,
-                int32_t only_shard, int32_t Hq, float scale, void* out, int out_f32, float* lse, void* workspace,
-                size_t workspace_bytes, void* stream, const char* who) {
+                int32_t only_shard, int32_t only_chunk, int32_t Hq, float scale, void* out, int out_f32, float* lse,
+                void* workspace, size_t workspace_bytes, void* stream, const char* who) {
     if (!ctx || !q || !page_table || !out || !lse || B < 1 || !cu_new || !prefix_len || !C || !cu_pages)
         return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or B < 1", who);
     if (int rc = validate_kv_cache(cache, who)) return rc;
@@ -960,9 +960,15 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
 
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
     Schedule sch;
-    build_tiles(B, cu_new, prefix_len, C, cu_pages, only_shard, sch.items);
+    build_tiles(B, cu_new, prefix_len, C, cu_pages, only_shard, only_chunk, sch.items);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (sch.items.empty()) return CP_OK;   // the shard owns no rows (only empty chunks)
+    // rows of q / out / lse: the packed batch, or the one chunk of a chunk call
+    int64_t total_rows = cu_new[B];
+    if (only_chunk >= 0) {
+        total_rows = 0;
+        for (const TileItem& t : sch.items) total_rows = std::max<int64_t>(total_rows, (int64_t)t.q_row0 + t.n_rows);
+    }
     int grid_max = ctx->num_sms;
 #ifdef CPATTN_TRACE
     if (const char* e = getenv("CPATTN_DEBUG_SMS")) grid_max = std::max(1, atoi(e));   // trace builds only
@@ -974,7 +980,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         return set_error(CP_ERR_WORKSPACE, "%s: schedule needs %zu workspace bytes, have %zu", who, lay.total, workspace_bytes);
 
     CUtensorMap tmQ, tmK, tmV;
-    if (int rc = encode_maps(ctx, q, cu_new[B], Hq, cache, &tmQ, &tmK, &tmV)) return rc;
+    if (int rc = encode_maps(ctx, q, total_rows, Hq, cache, &tmQ, &tmK, &tmV)) return rc;
     // one contiguous block: items | cta_off | pieces | merges | merge_slots (offsets as in the layout)
     std::vector<uint8_t> block(lay.partial_o - lay.items, 0);
     memcpy(block.data() + (lay.items - lay.items), sch.items.data(), sch.items.size() * sizeof(TileItem));
@@ -1008,7 +1014,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.out = out;
     p.out_f32 = out_f32;
     p.lse = lse;
-    p.lse_stride = cu_new[B];
+    p.lse_stride = total_rows;
     p.status = ctx->d_status;
     cp_attn_kernel<<<sch.grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
     if (int rc = check_cuda(cudaGetLastError(), who)) return rc;
@@ -1024,7 +1030,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         f.Hq = Hq;
         f.heads_per_unit = heads_per_unit;
         f.lse = lse;
-        f.lse_stride = cu_new[B];
+        f.lse_stride = total_rows;
         cp_attn_fixup_kernel<<<dim3((unsigned)sch.merges.size(), 2 * kBlockM / kFixupRowsPerBlock), 256, 0, s>>>(f);
         if (int rc = check_cuda(cudaGetLastError(), "cp_attn_fixup launch")) return rc;
     }
@@ -1037,7 +1043,7 @@ extern "C" int cp_prefill_attn_batch(cp_ctx* ctx, const void* q, const cp_kv_cac
                                      int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
                                      const int64_t* cu_pages, int32_t Hq, float scale, void* out, float* lse,
                                      void* workspace, size_t workspace_bytes, void* stream) {
-    return attn_common(ctx, q, cache, page_table, B, cu_new, prefix_len, C, cu_pages, -1, Hq, scale, out, 0, lse,
+    return attn_common(ctx, q, cache, page_table, B, cu_new, prefix_len, C, cu_pages, -1, -1, Hq, scale, out, 0, lse,
                        workspace, workspace_bytes, stream, "cp_prefill_attn_batch");
 }
 
@@ -1048,7 +1054,7 @@ extern "C" int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* ca
         return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn: cache is NULL, new_len < 1 or prefix_len < 0");
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
-    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, Hq, scale, out, 0, lse,
+    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, Hq, scale, out, 0, lse,
                        workspace, workspace_bytes, stream, "cp_prefill_attn");
 }
 
@@ -1069,8 +1075,20 @@ extern "C" int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cac
     if (int rc = check_cuda(cudaGetLastError(), "fill_neg_inf launch")) return rc;
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
-    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, Hq, scale, partial_out, 1,
+    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, -1, Hq, scale, partial_out, 1,
                        partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_shard");
+}
+
+extern "C" int cp_prefill_attn_chunk(cp_ctx* ctx, const void* q_chunk, const cp_kv_cache* cache, const int32_t* page_table,
+                                     int64_t prefix_len, int64_t new_len, int32_t C, int32_t chunk, int32_t Hq,
+                                     float scale, void* out_chunk, float* lse_chunk, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+    if (!cache || new_len < 1 || prefix_len < 0 || C < 1 || chunk < 0 || chunk >= 2 * (int64_t)C)
+        return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_chunk: bad sizes or chunk %d not in [0, %d)", chunk, 2 * C);
+    const int64_t cu_new[2] = {0, new_len};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
+    return attn_common(ctx, q_chunk, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, chunk, Hq, scale,
+                       out_chunk, 0, lse_chunk, workspace, workspace_bytes, stream, "cp_prefill_attn_chunk");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1154,7 +1172,7 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
     std::vector<TileItem> tiles;
-    build_tiles(1, cu_new, &prefix_len, &C, cu_pages, -1, tiles);
+    build_tiles(1, cu_new, &prefix_len, &C, cu_pages, -1, -1, tiles);
     cp_ctx enc{};                       // only the encoder entry point is read by encode_maps
     enc.encode_tiled = st->encode_tiled;
     CUtensorMap tmQ, tmK, tmV;

@@ -89,10 +89,11 @@ int check_cuda(cudaError_t e, const char* what);
 // Host planner pieces (plan.cpp)
 int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C);
 // Builds the tile list of a batch, cut at the chunk boundaries of every request's zigzag plan and
-// sorted longest first.  only_shard < 0 keeps all shards.
+// sorted longest first.  only_shard < 0 keeps all shards; only_chunk >= 0 (B == 1) keeps that one zigzag
+// chunk and numbers its rows from the chunk's first row (q, out and lse then hold the chunk alone).
 int validate_kv_cache(const cp_kv_cache* c, const char* who);
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
-                const int64_t* cu_pages, int32_t only_shard, std::vector<TileItem>& out);
+                const int64_t* cu_pages, int32_t only_shard, int32_t only_chunk, std::vector<TileItem>& out);
 // Distributes the (tile, head pair) units of s.items over `grid_max` CTAs: whole units longest first
 // onto the least loaded CTA while they fit under the per-CTA share, the rest cut into KV ranges that
 // fill every CTA to the same number of KV tiles.  Fills cta_off / pieces / merges / merge_slots.

@@ -31,7 +31,7 @@ int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C) {
 }
 
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
-                const int64_t* cu_pages, int32_t only_shard, std::vector<TileItem>& out) {
+                const int64_t* cu_pages, int32_t only_shard, int32_t only_chunk, std::vector<TileItem>& out) {
     out.clear();
     for (int32_t b = 0; b < B; ++b) {
         const int64_t R = cu_new[b + 1] - cu_new[b];
@@ -40,15 +40,19 @@ int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, con
         for (int64_t j = 0; j < 2 * (int64_t)Cb; ++j) {
             const int32_t shard = (int32_t)(j < Cb ? j : 2 * (int64_t)Cb - 1 - j);
             if (only_shard >= 0 && shard != only_shard) continue;
+            if (only_chunk >= 0 && j != only_chunk) continue;
             int64_t cb, ce;
             chunk_range(R, Cb, j, cb, ce);
+            // a single-chunk list addresses q / out / lse rows relative to the chunk's first row
+            const int64_t row_base = only_chunk >= 0 ? cb : 0;
             for (int64_t r0 = cb; r0 < ce; r0 += kTileRows) {
                 TileItem t;
-                t.q_row0 = (int32_t)(cu_new[b] + r0);
+                t.q_row0 = (int32_t)(cu_new[b] + r0 - row_base);
                 t.n_rows = (int32_t)std::min<int64_t>(kTileRows, ce - r0);
                 t.kv_len0 = (int32_t)(P + r0 + 1);
                 t.pt_base = (int32_t)cu_pages[b];
-                t.n_pages = (int32_t)((P + R + 63) / 64);   // entries the request really uses
+                // entries the request really uses; a single chunk reads none behind its last key
+                t.n_pages = (int32_t)((P + (only_chunk >= 0 ? ce : R) + 63) / 64);
                 t.n_kv_tiles = (int32_t)((t.kv_len0 + t.n_rows - 1 + kTileRows - 1) / kTileRows);
                 t.request = b;
                 t.shard = shard;
@@ -238,7 +242,7 @@ extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64
         cu_pages[b + 1] = cu_pages[b] + (prefix_len[b] + R + 63) / 64;
     }
     Schedule sch;
-    build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), -1, sch.items);
+    build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), -1, -1, sch.items);
     if (int rc = build_schedule(Hq / heads_per_unit, num_sms, sch)) return rc;
     int64_t max_load = 0, min_load = INT64_MAX, total = 0;
     for (int32_t c = 0; c < sch.grid; ++c) {

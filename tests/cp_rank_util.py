@@ -1,0 +1,99 @@
+"""Test doubles for the CP rank worker: an in-process communicator for ranks run as threads, and the
+device steps restated on the oracle (numpy pools of bf16 bit patterns) for the CPU tests."""
+import threading
+
+import numpy as np
+import torch
+
+from oracle import reference as orc
+from paper_2609_04774_b200 import workloads as wl
+
+
+class _Done:
+    def wait(self):
+        return True
+
+
+class ThreadFabric:
+    """Shared state of C in-process ranks: the n-th all_gather of every rank meets the others'."""
+
+    def __init__(self, size):
+        self.size = size
+        self.barrier = threading.Barrier(size)
+        self.slots = {}
+        self.lock = threading.Lock()
+
+    def comm(self, rank):
+        return ThreadComm(self, rank)
+
+
+class ThreadComm:
+    def __init__(self, fabric, rank):
+        self.fabric, self.rank, self.size = fabric, rank, fabric.size
+        self.calls = 0
+
+    def all_gather(self, block):
+        f, n = self.fabric, self.calls
+        self.calls += 1
+        with f.lock:
+            f.slots.setdefault(n, [None] * f.size)[self.rank] = block
+        f.barrier.wait(timeout=120)
+        out = torch.stack([b.to(block.device) for b in f.slots[n]], 0)
+        f.barrier.wait(timeout=120)
+        return out, _Done()
+
+
+class OracleOps:
+    """kv_gather / kv_append / attn_chunk of one rank on numpy page pools, through the oracle."""
+
+    def __init__(self, k_pages, v_pages, page_table, Hq, scale):
+        self.k_pages, self.v_pages, self.page_table = k_pages, v_pages, np.asarray(page_table)
+        self.Hq, self.scale = Hq, scale
+        self.Hkv, self.D = k_pages.shape[2], k_pages.shape[3]
+
+    def empty_rows(self, n, heads):
+        return torch.zeros((n, heads, self.D), dtype=torch.int16)
+
+    @staticmethod
+    def _bits(t):
+        return t.contiguous().numpy().view(np.uint16)
+
+    def kv_gather(self, t_begin, n, k_rows, v_rows):
+        if n > 0:
+            k_rows[:n] = torch.from_numpy(orc.kv_gather(self.k_pages, self.page_table, t_begin, t_begin + n).view(np.int16))
+            v_rows[:n] = torch.from_numpy(orc.kv_gather(self.v_pages, self.page_table, t_begin, t_begin + n).view(np.int16))
+
+    def kv_append(self, t_begin, n, k_rows, v_rows):
+        if n > 0:
+            orc.kv_append(self.k_pages, self.page_table, t_begin, self._bits(k_rows)[:n])
+            orc.kv_append(self.v_pages, self.page_table, t_begin, self._bits(v_rows)[:n])
+
+    def attn_chunk(self, lay, chunk, q_chunk):
+        b, e = lay.chunk(chunk)
+        q = np.zeros((lay.R, self.Hq, self.D), dtype=np.uint16)
+        q[b:e] = self._bits(q_chunk)
+        if e == b:
+            return np.zeros((0, self.Hq, self.D)), np.zeros((self.Hq, 0))
+        return orc.attn_rows(q, self.k_pages, self.v_pages, self.page_table, lay.P, self.Hkv, self.scale, np.arange(b, e))
+
+
+def rank_inputs(mat, lay, seed):
+    """What rank `lay.rank` starts with, cut from the seeded full request: an empty page pool of its own
+    (its own page permutation) holding only the rank's prefix block, and the rank's q/k/v rows."""
+    w = mat.wl
+    pt_ref = mat.page_table
+    n_pages = len(pt_ref)
+    page_table = wl.permutation(seed + 100 * (lay.rank + 1), wl.TID_PERM, n_pages + 2)[:n_pages].astype(np.int32)
+    k_pages = np.zeros((n_pages + 2,) + mat.k_pages.shape[1:], dtype=np.uint16)
+    v_pages = np.zeros_like(k_pages)
+    pb, pe = lay.prefix_block(lay.rank)
+    if pe > pb:
+        orc.kv_append(k_pages, page_table, pb, orc.kv_gather(mat.k_pages, pt_ref, pb, pe))
+        orc.kv_append(v_pages, page_table, pb, orc.kv_gather(mat.v_pages, pt_ref, pb, pe))
+    rows = {}
+    for name, j in (("early", lay.early), ("late", lay.late)):
+        b, e = lay.chunk(j)
+        rows["q_" + name] = mat.q[b:e]
+        rows["k_" + name] = orc.kv_gather(mat.k_pages, pt_ref, lay.P + b, lay.P + e)
+        rows["v_" + name] = orc.kv_gather(mat.v_pages, pt_ref, lay.P + b, lay.P + e)
+    return k_pages, v_pages, page_table, rows

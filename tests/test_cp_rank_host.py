@@ -1,0 +1,136 @@
+"""The multi-rank CP worker on CPU: layout arithmetic against the oracle's planner, the whole exchange +
+attention orchestration with four in-process ranks, and with two gloo ranks over real collectives.
+The device steps are stood in for by the oracle (tests/cp_rank_util.py); what is checked here is the
+data movement: which rows a rank sends, where gathered rows land in its paged cache, which keys each
+chunk call may rely on."""
+import os
+import socket
+import sys
+import threading
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from oracle import reference as orc
+from paper_2609_04774_b200 import workloads as wl
+from paper_2609_04774_b200.cp_rank import CpRankWorker, RankLayout, TorchComm
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.mark.parametrize("R,P,C", [(333, 192, 3), (5, 0, 4), (4096, 12288, 4), (700, 64, 2), (1, 64, 1), (129, 448, 8)])
+def test_layout_matches_oracle_plan(R, P, C):
+    shards = orc.plan(R, P, C)
+    covered = np.zeros(P, dtype=np.int32)
+    for k in range(C):
+        lay = RankLayout(R, P, C, k)
+        assert [lay.chunk(lay.early), lay.chunk(lay.late)] == [tuple(c) for c in zip(shards[k]["q_begin"], shards[k]["q_end"])]
+        assert lay.late_chunk_of(k) == lay.late
+        b, e = lay.prefix_block(k)
+        assert b % 64 == 0 and e % 64 == 0 and e - b <= lay.block_pages * 64
+        covered[b:e] += 1
+    assert (covered == 1).all()                      # prefix blocks tile [0, P) exactly once
+    assert lay.C * lay.cl * 2 >= R
+
+
+def test_layout_rejects_bad_arguments():
+    with pytest.raises(ValueError):
+        RankLayout(10, 30, 2, 0)                     # prefix not page aligned
+    with pytest.raises(ValueError):
+        RankLayout(10, 0, 2, 2)
+
+
+def _run_rank(w, mat, lay, comm, seed, result):
+    from cp_rank_util import OracleOps, rank_inputs
+    k_pages, v_pages, page_table, rows = rank_inputs(mat, lay, seed)
+    ops = OracleOps(k_pages, v_pages, page_table, w.Hq, w.scale)
+    t = {k: torch.from_numpy(np.ascontiguousarray(v).view(np.int16)) for k, v in rows.items()}
+    worker = CpRankWorker(lay, comm, ops)
+    out_e, lse_e, out_l, lse_l = worker.prefill(t["q_early"], t["q_late"], t["k_early"], t["v_early"], t["k_late"], t["v_late"])
+    result[lay.rank] = (out_e, lse_e, out_l, lse_l, k_pages, v_pages, page_table)
+
+
+def _check_rank(w, mat, lay, res):
+    out_e, lse_e, out_l, lse_l, k_pages, v_pages, page_table = res
+    r = w.requests[0]
+    ref_o, ref_l = orc.attn_full(mat.q, mat.k_pages, mat.v_pages, mat.page_table, r.prefix_len, w.Hkv, w.scale)
+    for j, o, l in ((lay.early, out_e, lse_e), (lay.late, out_l, lse_l)):
+        b, e = lay.chunk(j)
+        assert o.shape[0] == e - b
+        if e > b:
+            assert np.abs(o - ref_o[b:e]).max() < 1e-12 and np.abs(l - ref_l[:, b:e]).max() < 1e-12
+    # after the exchange the rank's own cache holds every token of the request, bit for bit
+    L = r.prefix_len + r.new_len
+    assert np.array_equal(orc.kv_gather(k_pages, page_table, 0, L), orc.kv_gather(mat.k_pages, mat.page_table, 0, L))
+    assert np.array_equal(orc.kv_gather(v_pages, page_table, 0, L), orc.kv_gather(mat.v_pages, mat.page_table, 0, L))
+
+
+@pytest.mark.parametrize("R,P,C", [(333, 192, 4), (5, 0, 4), (200, 320, 3)])
+def test_four_ranks_in_process(R, P, C):
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from cp_rank_util import ThreadFabric
+    w = wl.Workload("cp_rank", 51, 4, 2, [wl.Request(R, P, C)])
+    mat = wl.materialize(w)
+    fabric = ThreadFabric(C)
+    result, errors = {}, []
+
+    def body(k):
+        try:
+            _run_rank(w, mat, RankLayout(R, P, C, k), fabric.comm(k), 51, result)
+        except Exception as e:               # a failing rank must not leave the others at the barrier
+            errors.append(e)
+            fabric.barrier.abort()
+
+    threads = [threading.Thread(target=body, args=(k,)) for k in range(C)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=300)
+    assert not errors, errors
+    for k in range(C):
+        _check_rank(w, mat, RankLayout(R, P, C, k), result[k])
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    p = s.getsockname()[1]
+    s.close()
+    return p
+
+
+def _gloo_rank(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        R, P = 333, 192
+        w = wl.Workload("cp_rank", 52, 4, 2, [wl.Request(R, P, world)])
+        mat = wl.materialize(w)
+        lay = RankLayout(R, P, world, rank)
+        result = {}
+        _run_rank(w, mat, lay, TorchComm(), 52, result)
+        _check_rank(w, mat, lay, result[rank])
+        q.put((rank, "ok"))
+    except Exception as e:
+        q.put((rank, repr(e)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_gloo_ranks():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_gloo_rank, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=240) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+    assert got == [(0, "ok"), (1, "ok")]

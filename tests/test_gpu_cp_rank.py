@@ -1,0 +1,158 @@
+"""The multi-rank CP worker on one GPU: C ranks run as host threads, each with its own paged cache, its
+own context and the library's kernels; rows are exchanged through an in-process communicator (a host
+barrier, no kernel waits on another).  Plus the chunk entry point on its own, and the NCCL communicator
+at world size 1 in a child process."""
+import os
+import socket
+import sys
+import threading
+
+import numpy as np
+import pytest
+import torch
+import torch.multiprocessing as mp
+
+from oracle import reference as orc
+from paper_2609_04774_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _dev(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _f64(t):
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+def _compare(o, l, ref_o, ref_l, what):
+    err = np.abs(_f64(o) - ref_o)
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3, (what, err.max(), err.mean())
+    lerr = np.abs(_f64(l) - ref_l) / np.maximum(1.0, np.abs(ref_l))
+    assert lerr.max() <= 1e-3, (what, lerr.max())
+
+
+def test_chunk_entry_point_matches_oracle_rows():
+    from paper_2609_04774_b200 import binding
+    w = wl.Workload("chunk_call", 61, 8, 2, [wl.Request(1000, 320, 3)])
+    mat = wl.materialize(w)
+    r = w.requests[0]
+    ctx = binding.Context(0)
+    k, v = _dev(mat.k_pages), _dev(mat.v_pages)
+    cache = binding.make_cache(k, v)
+    pt = torch.from_numpy(mat.page_table).cuda()
+    ws = torch.empty(binding.cp_workspace_bytes([r.new_len], [r.C], w.Hq), dtype=torch.uint8, device="cuda")
+    plan = orc.plan(r.new_len, r.prefix_len, r.C)
+    ref_o, ref_l = orc.attn_full(mat.q, mat.k_pages, mat.v_pages, mat.page_table, r.prefix_len, w.Hkv, w.scale)
+    for j in range(2 * r.C):
+        shard = j if j < r.C else 2 * r.C - 1 - j
+        half = 0 if j < r.C else 1
+        b, e = plan[shard]["q_begin"][half], plan[shard]["q_end"][half]
+        n = e - b
+        q = _dev(mat.q[b:e])
+        out = torch.full((n, w.Hq, w.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((w.Hq, n), float("nan"), dtype=torch.float32, device="cuda")
+        binding.cp_prefill_attn_chunk(ctx, q, cache, pt, r.prefix_len, r.new_len, r.C, j, w.Hq, w.scale, out, lse, ws)
+        torch.cuda.synchronize()
+        ctx.poll_status()
+        _compare(out, lse, ref_o[b:e], ref_l[:, b:e], "chunk %d" % j)
+    with pytest.raises(binding.CpError):
+        binding.cp_prefill_attn_chunk(ctx, q, cache, pt, r.prefix_len, r.new_len, r.C, 2 * r.C, w.Hq, w.scale, out, lse, ws)
+
+
+def _rank_on_gpu(w, mat, lay, comm, seed, result):
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from cp_rank_util import rank_inputs
+    from paper_2609_04774_b200 import binding
+    from paper_2609_04774_b200.cp_rank import CpRankWorker, LibraryOps
+    torch.cuda.set_device(0)
+    k_pages, v_pages, page_table, rows = rank_inputs(mat, lay, seed)
+    ops = LibraryOps(binding.Context(0), _dev(k_pages), _dev(v_pages), torch.from_numpy(page_table).cuda(), w.Hq, w.scale)
+    t = {k: _dev(x) for k, x in rows.items()}
+    out = CpRankWorker(lay, comm, ops).prefill(t["q_early"], t["q_late"], t["k_early"], t["v_early"], t["k_late"], t["v_late"])
+    torch.cuda.synchronize()
+    ops.ctx.poll_status()
+    result[lay.rank] = out + (ops.k_pages, ops.v_pages, page_table)
+
+
+def _check_rank_on_gpu(w, mat, lay, res, ref):
+    out_e, lse_e, out_l, lse_l, k_pages, v_pages, page_table = res
+    r = w.requests[0]
+    for j, o, l in ((lay.early, out_e, lse_e), (lay.late, out_l, lse_l)):
+        b, e = lay.chunk(j)
+        assert o.shape[0] == e - b
+        if e > b:
+            _compare(o, l, ref[0][b:e], ref[1][:, b:e], "rank %d chunk %d" % (lay.rank, j))
+    L = r.prefix_len + r.new_len
+    for dev_pages, ref_pages in ((k_pages, mat.k_pages), (v_pages, mat.v_pages)):
+        got = dev_pages.view(torch.int16).cpu().numpy().view(np.uint16)
+        assert np.array_equal(orc.kv_gather(got, page_table, 0, L), orc.kv_gather(ref_pages, mat.page_table, 0, L))
+
+
+@pytest.mark.parametrize("R,P,C", [(1500, 640, 4), (333, 192, 3), (5, 0, 4)])
+def test_ranks_as_threads_on_one_gpu(R, P, C):
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from cp_rank_util import ThreadFabric
+    from paper_2609_04774_b200.cp_rank import RankLayout
+    w = wl.Workload("cp_rank_gpu", 62, 8, 2, [wl.Request(R, P, C)])
+    mat = wl.materialize(w)
+    ref = orc.attn_full(mat.q, mat.k_pages, mat.v_pages, mat.page_table, P, w.Hkv, w.scale)
+    fabric = ThreadFabric(C)
+    result, errors = {}, []
+
+    def body(k):
+        try:
+            _rank_on_gpu(w, mat, RankLayout(R, P, C, k), fabric.comm(k), 62, result)
+        except Exception as e:
+            errors.append(e)
+            fabric.barrier.abort()
+
+    threads = [threading.Thread(target=body, args=(k,)) for k in range(C)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=600)
+    assert not errors, errors
+    for k in range(C):
+        _check_rank_on_gpu(w, mat, RankLayout(R, P, C, k), result[k], ref)
+
+
+def _nccl_single_rank(port, q):
+    sys.path.insert(0, ROOT)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import torch.distributed as dist
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    try:
+        torch.cuda.set_device(0)
+        dist.init_process_group("nccl", rank=0, world_size=1)
+        from paper_2609_04774_b200.cp_rank import RankLayout, TorchComm
+        R, P = 700, 256
+        w = wl.Workload("cp_rank_nccl", 63, 8, 2, [wl.Request(R, P, 1)])
+        mat = wl.materialize(w)
+        ref = orc.attn_full(mat.q, mat.k_pages, mat.v_pages, mat.page_table, P, w.Hkv, w.scale)
+        lay = RankLayout(R, P, 1, 0)
+        result = {}
+        _rank_on_gpu(w, mat, lay, TorchComm(), 63, result)
+        _check_rank_on_gpu(w, mat, lay, result[0], ref)
+        q.put("ok")
+    except Exception as e:
+        q.put(repr(e))
+    finally:
+        if dist.is_initialized():
+            dist.destroy_process_group()
+
+
+def test_nccl_communicator_world_size_one():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    p = ctx.Process(target=_nccl_single_rank, args=(port, q))
+    p.start()
+    got = q.get(timeout=600)
+    p.join(timeout=120)
+    assert got == "ok"
