@@ -9,7 +9,7 @@ original positions -> LSE merge of the units whose KV range was split across CTA
 measured with inputs resident in HBM; `e2e` goes through the same C-ABI calls from pinned HOST
 buffers (q, the new tokens' K/V rows appended into the paged cache, page table up; out and lse down).
 
-Other modes (`--mode merge|table|configs|kvcopy`) write the cp_merge sweep, the measured prefill-time
+Other modes (`--mode merge|table|configs|kvcopy|cprank`) write the cp_merge sweep, the measured prefill-time
 table over (new_len, prefix_len, C), the per-config numbers and the paged KV copy bandwidth as JSON
 lines to `--out`.
 
@@ -596,6 +596,78 @@ def run_table(args, out):
     out.flush()
 
 
+class _LoopbackComm:
+    """Stands in for the C-rank all-gather on one GPU: every peer's block is a device copy of this
+    rank's own block.  The bytes written to local HBM equal a real gather's; the values do not, so
+    this is for timing one rank's local work only."""
+
+    class _Done:
+        def wait(self):
+            return True
+
+    def __init__(self, size, rank):
+        self.size, self.rank = size, rank
+
+    def all_gather(self, block):
+        return block.unsqueeze(0).expand((self.size,) + tuple(block.shape)).contiguous(), self._Done()
+
+
+def run_cprank(args, out):
+    """Local time of every rank of a degree-C CP worker (early-chunk-first order): own prefix block read
+    out, gathered rows appended to the rank's paged cache, the two chunk attention calls.  The NVLink
+    transfer itself cannot be run on one GPU; its size and a modelled time at the measured peer-copy
+    bandwidth are printed beside the measured local time."""
+    import torch
+    from paper_2609_04774_b200 import binding, build
+    from paper_2609_04774_b200.cp_rank import CpRankWorker, LibraryOps, RankLayout
+    build.build()
+    D = 128
+    for cfg in args.configs:
+        w = get_workload(cfg)
+        if len(w.requests) != 1:
+            continue
+        r = w.requests[0]
+        R, P, C = r.new_len, r.prefix_len, r.C
+        n_pages = r.n_pages
+        k = torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
+        v = torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
+        pt = torch.from_numpy(wl.permutation(w.seed, wl.TID_PERM, n_pages)).cuda()
+        ops = LibraryOps(binding.Context(0), k, v, pt, w.Hq, w.scale)
+        per_rank = []
+        for rank in range(C):
+            lay = RankLayout(R, P, C, rank)
+            rows = {}
+            for name, j in (("early", lay.early), ("late", lay.late)):
+                b, e = lay.chunk(j)
+                rows["q_" + name] = torch.randn((e - b, w.Hq, D), device="cuda").to(torch.bfloat16)
+                rows["k_" + name] = torch.randn((e - b, w.Hkv, D), device="cuda").to(torch.bfloat16)
+                rows["v_" + name] = torch.randn((e - b, w.Hkv, D), device="cuda").to(torch.bfloat16)
+            worker = CpRankWorker(lay, _LoopbackComm(C, rank), ops)
+            fn = lambda: worker.prefill(rows["q_early"], rows["q_late"], rows["k_early"], rows["v_early"],
+                                        rows["k_late"], rows["v_late"])
+            ms = []
+            for i in range(2 + args.rank_reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                torch.cuda.synchronize()
+                if i >= 2:
+                    ms.append(e0.elapsed_time(e1))
+            ops.ctx.poll_status()
+            per_rank.append(statistics.median(ms))
+        recv = (C - 1) * 2 * 2 * w.Hkv * D * (RankLayout(R, P, C, 0).block_pages * wl.PAGE + 2 * RankLayout(R, P, C, 0).cl)
+        out.write(json.dumps({"mode": "cprank", "config": cfg, "workload": w.name, "R": R, "P": P, "C": C,
+                              "rank_local_ms": per_rank, "slowest_rank_ms": max(per_rank),
+                              "tflops_per_gpu_slowest_rank": w.flops() / C / (max(per_rank) * 1e-3) / 1e12,
+                              "nvlink_bytes_received_per_rank": recv,
+                              "nvlink_ms_modelled_at_770GBps": recv / 770e9 * 1e3,
+                              "note": "local work measured with loopback gathers; link time modelled, not measured"}) + "\n")
+        out.flush()
+        del k, v, ops
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -603,9 +675,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="BASELINE config number of the headline workload")
-    ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table", "kvcopy"])
+    ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table", "kvcopy", "cprank"])
     ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5],
                     help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P")
+    ap.add_argument("--rank-reps", type=int, default=5)
     ap.add_argument("--merge-T", type=int, nargs="*", default=[4096, 16384, 65536, 262144])
     ap.add_argument("--merge-reps", type=int, default=20)
     ap.add_argument("--table-R", type=int, nargs="*", default=[1024, 2048, 4096, 8192, 16384, 32768, 65536, 131072])
@@ -620,7 +693,7 @@ def main():
     if args.mode == "bench":
         return run_ours(args)
     out = open(args.out, "w") if args.out else sys.stdout
-    {"configs": run_configs, "merge": run_merge_sweep, "table": run_table, "kvcopy": run_kvcopy}[args.mode](args, out)
+    {"configs": run_configs, "merge": run_merge_sweep, "table": run_table, "kvcopy": run_kvcopy, "cprank": run_cprank}[args.mode](args, out)
 
 
 if __name__ == "__main__":
