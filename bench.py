@@ -668,6 +668,56 @@ def run_cprank(args, out):
         torch.cuda.empty_cache()
 
 
+def run_cachemgr(args, out):
+    """Host throughput of the prefix-cache bookkeeping on a seeded request stream: per request one
+    match per worker (ReusedPath), PreferDegree, Algorithm 1 and the new replica; a scan (Algorithm 2)
+    every 1000 requests.  The oracle runs the first tenth of the same stream for scale."""
+    from paper_2609_04774_b200 import build, cache_manager as cmgr
+    build.build()
+    model = (3e-4, 2e-7, 5e-8, 1e-6, 4e-11)
+    degrees = [1, 2, 4, 8]
+    workers = {w: degrees[w % 4] for w in range(16)}
+    ids = sorted(workers)
+    stream = wl.prefix_stream(21, args.cache_requests)
+    pick = wl.counter_uniform(21, wl.TID_STREAM, 1 << 20, len(stream))
+
+    def drive(trie, reused_fn, prefer_fn, n, wrap=lambda b: b):
+        t0 = time.perf_counter()
+        scans = 0
+        for i, (blocks, L) in enumerate(stream[:n]):
+            blocks = wrap(blocks)
+            reused = reused_fn(trie, blocks)
+            pref = prefer_fn(L, reused)
+            w = ids[int(pick[i] * len(ids))]
+            trie.update(blocks, L, w, pref, model)
+            trie.add_replica(blocks, w)
+            if i % 1000 == 999:
+                trie.scan(1e-5, 3.0, 0.4, 0.8, 16)
+                scans += 1
+        return time.perf_counter() - t0, scans
+
+    t = cmgr.Trie(degrees, 64)
+    for w, c in workers.items():
+        t.set_worker(w, c)
+    ids_arr, deg_arr = np.array(ids, dtype=np.int32), np.array([workers[w] for w in ids], dtype=np.int32)
+    dt, scans = drive(t, lambda tr, b: tr.reused_all(b, ids_arr).astype(np.int64) * 64,
+                      lambda L, reused: cmgr.cp_prefer_degree(model, L, deg_arr, reused, 1.2, 0.2)[1],
+                      len(stream), cmgr.Keys)
+    nodes = t.size()
+    sys.path.insert(0, ROOT)
+    from oracle import cache_manager as ocm
+    o = ocm.Trie(degrees, 64)
+    for w, c in workers.items():
+        o.set_worker(w, c)
+    n_o = max(1, len(stream) // 10)
+    dto, _ = drive(o, lambda tr, b: [len(tr.reused_path(b, w)) * 64 for w in ids],
+                   lambda L, reused: ocm.prefer_degree(model, L, [(workers[w], p) for w, p in zip(ids, reused)], 1.2, 0.2)[1], n_o)
+    out.write(json.dumps({"mode": "cachemgr", "requests": len(stream), "workers": len(ids), "nodes": nodes, "scans": scans,
+                          "library_requests_per_s": len(stream) / dt, "oracle_requests_per_s": n_o / dto,
+                          "oracle_sample": "first %d requests" % n_o, "note": "driven from Python through ctypes"}) + "\n")
+    out.flush()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -675,10 +725,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="BASELINE config number of the headline workload")
-    ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table", "kvcopy", "cprank"])
+    ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table", "kvcopy", "cprank", "cachemgr"])
     ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5],
                     help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P")
     ap.add_argument("--rank-reps", type=int, default=5)
+    ap.add_argument("--cache-requests", type=int, default=20000)
     ap.add_argument("--merge-T", type=int, nargs="*", default=[4096, 16384, 65536, 262144])
     ap.add_argument("--merge-reps", type=int, default=20)
     ap.add_argument("--table-R", type=int, nargs="*", default=[1024, 2048, 4096, 8192, 16384, 32768, 65536, 131072])
@@ -693,7 +744,7 @@ def main():
     if args.mode == "bench":
         return run_ours(args)
     out = open(args.out, "w") if args.out else sys.stdout
-    {"configs": run_configs, "merge": run_merge_sweep, "table": run_table, "kvcopy": run_kvcopy, "cprank": run_cprank}[args.mode](args, out)
+    {"configs": run_configs, "merge": run_merge_sweep, "table": run_table, "kvcopy": run_kvcopy, "cprank": run_cprank, "cachemgr": run_cachemgr}[args.mode](args, out)
 
 
 if __name__ == "__main__":

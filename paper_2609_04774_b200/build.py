@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libcpattn.so")
-SOURCES = ["ctx.cu", "plan.cpp", "merge.cu", "kv_copy.cu", "attn_sm100.cu"]
+SOURCES = ["ctx.cu", "plan.cpp", "cache_manager.cpp", "merge.cu", "kv_copy.cu", "attn_sm100.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
@@ -34,7 +34,8 @@ def _stale(target: str, deps) -> bool:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every source to an object in ``build/`` and link ``libcpattn.so``.  Returns its path."""
-    headers = [os.path.join(CSRC, "internal.h"), os.path.join(ROOT, "include", "cpattn.h"), os.path.abspath(__file__)]
+    headers = [os.path.join(CSRC, "internal.h"), os.path.join(ROOT, "include", "cpattn.h"),
+               os.path.join(ROOT, "include", "cpcache.h"), os.path.abspath(__file__)]
     objdir = os.path.join(_HERE, "build")
     os.makedirs(objdir, exist_ok=True)
     objs = []

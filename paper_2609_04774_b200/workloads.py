@@ -32,7 +32,7 @@ _C1 = np.uint64(0xBF58476D1CE4E5B9)
 _C2 = np.uint64(0x94D049BB133111EB)
 
 # tensor ids (second argument of the counter-based generator)
-TID_Q, TID_K, TID_V, TID_PERM, TID_LEN, TID_FRAC, TID_C, TID_PART, TID_LSE, TID_ROWS = range(10)
+TID_Q, TID_K, TID_V, TID_PERM, TID_LEN, TID_FRAC, TID_C, TID_PART, TID_LSE, TID_ROWS, TID_STREAM = range(11)
 
 
 def _mix64(x: np.ndarray) -> np.ndarray:
@@ -345,3 +345,32 @@ def sample_rows(seed: int, Hq: int, R: int, per_head: int) -> np.ndarray:
     """``per_head`` seeded random query rows for every head: int64 [Hq, per_head]."""
     u = counter_uniform(seed, TID_ROWS, 0, Hq * per_head).reshape(Hq, per_head)
     return np.minimum((u * R).astype(np.int64), R - 1)
+
+
+# --------------------------------------------------------------------------------------
+# Synthetic prefix streams for the cache-manager tests
+# --------------------------------------------------------------------------------------
+
+def prefix_stream(seed: int, n_requests: int, block_tokens: int = PAGE, max_new_blocks: int = 12):
+    """Requests as (block keys, total length L) with the reuse structure of multi-turn and shared-prompt
+    traffic: half of the requests extend an earlier request (next turn), three in ten branch off an earlier
+    request's prefix at a random depth (shared system prompt, different question), the rest start a new
+    prefix.  Block keys are distinct 64-bit integers; L = whole blocks plus a ragged tail."""
+    u = counter_uniform(seed, TID_STREAM, 0, 4 * n_requests)
+    keys = counter_u64(seed, TID_STREAM, 1 << 40, n_requests * max_new_blocks)
+    history, out, used = [], [], 0
+    for i in range(n_requests):
+        kind, pick, depth, grow = u[4 * i], u[4 * i + 1], u[4 * i + 2], u[4 * i + 3]
+        n_new = 1 + int(grow * max_new_blocks) % max_new_blocks
+        if history and kind < 0.5:
+            base = list(history[int(pick * len(history))])
+        elif history and kind < 0.8:
+            src = history[int(pick * len(history))]
+            base = list(src[:1 + int(depth * len(src)) % len(src)])
+        else:
+            base = []
+        blocks = base + [int(k) for k in keys[used:used + n_new]]
+        used += n_new
+        history.append(blocks)
+        out.append((blocks, len(blocks) * block_tokens + int(depth * block_tokens) % block_tokens))
+    return out

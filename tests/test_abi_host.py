@@ -21,13 +21,15 @@ def lib():
 
 
 def test_library_exports_every_declared_symbol(lib):
-    header = open(os.path.join(ROOT, "include", "cpattn.h")).read()
-    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(cp_[a-z_0-9]+)\s*\(", header))
-    assert declared, "no declarations found"
-    assert declared == set(binding.EXPORTS)
-    for name in declared:
-        assert hasattr(lib, name), name
+    from paper_2609_04774_b200 import cache_manager
+    for hname, exports in (("cpattn.h", binding.EXPORTS), ("cpcache.h", cache_manager.EXPORTS)):
+        header = open(os.path.join(ROOT, "include", hname)).read()
+        header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+        declared = set(re.findall(r"\b(cp_[a-z_0-9]+)\s*\(", header))
+        assert declared, "no declarations found in " + hname
+        assert declared == set(exports), hname
+        for name in declared:
+            assert hasattr(lib, name), name
 
 
 def test_struct_layouts_match_header():
