@@ -1,6 +1,8 @@
 """GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded
 inputs.  Planner and page indexing bit-exact; attention within max-abs 2e-2 / mean-abs 2e-3 and LSE
 within 1e-3; merge within fp32 round-off."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -256,6 +258,30 @@ def test_attention_variant_gqa8_and_chunked_prefill(ctx):
                                              torch.cuda.get_device_properties(0).multi_processor_count, want_lists=False)
     assert info["split_units"] == 64 and info["max_load"] * info["grid"] <= 1.01 * info["total"]
     check_batch(ctx, w, pair_budget=2e8)
+
+
+def _random_workload(seed):
+    u = wl.counter_uniform(seed, wl.TID_LEN, 0, 64)
+    heads = [(8, 2), (4, 4), (6, 2), (16, 2), (32, 4), (8, 8), (2, 1)][int(u[0] * 7)]
+    B = 1 + int(u[1] * 6)
+    reqs = []
+    for b in range(B):
+        scale = float(os.environ.get("CPATTN_FUZZ_SCALE", "1"))            # > 1: longer requests, more KV splits
+        R = max(1, int(round(scale * 2.0 ** (u[2 + 4 * b] * 11.5))))         # 1 .. ~2900, log-uniform
+        kind = u[3 + 4 * b]
+        P = 0 if kind < 0.25 else int(u[4 + 4 * b] * 8192 * scale)
+        if kind < 0.75:
+            P = P // 64 * 64                                                 # mostly page-aligned prefixes
+        C = [1, 2, 3, 4, 5, 8][int(u[5 + 4 * b] * 6)]
+        reqs.append(wl.Request(R, P, C))
+    return wl.Workload("random_%d" % seed, seed, heads[0], heads[1], reqs)
+
+
+@pytest.mark.parametrize("seed", range(1000, 1000 + int(os.environ.get("CPATTN_FUZZ_CASES", "16"))))
+def test_attention_random_batches(ctx, seed):
+    # seeded random batches: head shapes with even, odd and unit group sizes, ragged lengths from one token
+    # up, prefixes that are absent, page-aligned or not, every supported kind of C
+    check_batch(ctx, _random_workload(seed), pair_budget=6e6, seed_rows=seed)
 
 
 def test_attention_config5_sampled(ctx):
