@@ -20,17 +20,18 @@ __device__ __forceinline__ float4 ld_stream(const float4* p) {
     return v;
 }
 
-// Grid: x = ceil(H / HPW), y = ceil(T / kTokPerCta).  Warp w of the CTA handles token y*8 + w and heads
+// Grid: one-dimensional, block b = y * gx + x with gx = ceil(H / HPW), y < ceil(T / kTokPerCta) (consecutive
+// blocks read consecutive memory).  Warp w of the CTA handles token y*8 + w and heads
 // x*HPW .. x*HPW+HPW-1 (HPW consecutive rows of every partial, 512 B each).  N <= NMAX; all HPW*NMAX
 // row loads of a warp are issued before the first use so that enough bytes are in flight per SM.
 template <int NMAX, int HPW, bool kOutBf16>
 __global__ void __launch_bounds__(kMergeThreads)
-merge_kernel(const float* __restrict__ partials, const float* __restrict__ lses, int N, int64_t T, int H,
+merge_kernel(const float* __restrict__ partials, const float* __restrict__ lses, int N, int64_t T, int H, int gx,
              void* __restrict__ out, float* __restrict__ lse_out) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const int64_t t = (int64_t)blockIdx.y * kTokPerCta + warp;
-    const int h0 = blockIdx.x * HPW;
+    const int64_t t = (int64_t)(blockIdx.x / gx) * kTokPerCta + warp;
+    const int h0 = (blockIdx.x % gx) * HPW;
     if (t >= T) return;
     const int64_t row_stride4 = kMergeD / 4;                          // float4 per row
     const int64_t part_stride4 = T * (int64_t)H * row_stride4;        // float4 per partial
@@ -92,11 +93,12 @@ merge_kernel(const float* __restrict__ partials, const float* __restrict__ lses,
 template <int NMAX, int HPW>
 void launch_merge(const float* partials, const float* lses, int N, int64_t T, int H, void* out, int out_dtype,
                   float* lse_out, cudaStream_t s) {
-    dim3 grid((H + HPW - 1) / HPW, (unsigned)((T + kTokPerCta - 1) / kTokPerCta));
+    const int gx = (H + HPW - 1) / HPW;
+    const unsigned grid = (unsigned)(gx * ((T + kTokPerCta - 1) / kTokPerCta));
     if (out_dtype == CP_DTYPE_BF16)
-        merge_kernel<NMAX, HPW, true><<<grid, kMergeThreads, 0, s>>>(partials, lses, N, T, H, out, lse_out);
+        merge_kernel<NMAX, HPW, true><<<grid, kMergeThreads, 0, s>>>(partials, lses, N, T, H, gx, out, lse_out);
     else
-        merge_kernel<NMAX, HPW, false><<<grid, kMergeThreads, 0, s>>>(partials, lses, N, T, H, out, lse_out);
+        merge_kernel<NMAX, HPW, false><<<grid, kMergeThreads, 0, s>>>(partials, lses, N, T, H, gx, out, lse_out);
 }
 
 }  // namespace
@@ -110,8 +112,8 @@ extern "C" int cp_merge(cp_ctx* ctx, const float* partials, const float* lses, i
     if (N > 32) return set_error(CP_ERR_UNSUPPORTED, "cp_merge: N=%d, at most 32 partials", N);
     if (out_dtype != CP_DTYPE_BF16 && out_dtype != CP_DTYPE_F32)
         return set_error(CP_ERR_INVALID_ARG, "cp_merge: out_dtype=%d", out_dtype);
-    if ((T + kTokPerCta - 1) / kTokPerCta > 65535 * 1024ll)
-        return set_error(CP_ERR_UNSUPPORTED, "cp_merge: T=%lld too large", (long long)T);
+    if ((T + kTokPerCta - 1) / kTokPerCta * (int64_t)H > 0x7fffffffll)
+        return set_error(CP_ERR_UNSUPPORTED, "cp_merge: T=%lld x H=%d needs more than 2^31 blocks", (long long)T, H);
     if (((uintptr_t)partials | (uintptr_t)out) & 15)
         return set_error(CP_ERR_INVALID_ARG, "cp_merge: partials and out must be 16-byte aligned");
     cudaStream_t s = static_cast<cudaStream_t>(stream);

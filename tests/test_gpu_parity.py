@@ -81,6 +81,22 @@ def test_merge_parity(ctx):
         assert np.abs(l[fin] - ref_l[fin]).max() <= 1e-5 * np.abs(ref_l[fin]).max()
 
 
+def test_merge_many_tokens_one_head(ctx):
+    # more than 65535 token blocks: block indices beyond a grid's y range; last rows compared with the oracle
+    N, T, H = 2, 8 * 70000 + 3, 1
+    g = torch.Generator(device="cuda").manual_seed(9)
+    parts = torch.randn((N, T, H, 128), device="cuda", generator=g)
+    lses = 8 + 2 * torch.randn((N, H, T), device="cuda", generator=g)
+    out = torch.empty((T, H, 128), dtype=torch.float32, device="cuda")
+    lse_out = torch.empty((H, T), dtype=torch.float32, device="cuda")
+    binding.cp_merge(ctx, parts, lses, out, lse_out)
+    torch.cuda.synchronize()
+    for lo, hi in ((0, 64), (8 * 65535 - 32, 8 * 65535 + 32), (T - 64, T)):
+        ref_o, ref_l = orc.merge(parts[:, lo:hi].cpu().numpy().astype(np.float64), lses[:, :, lo:hi].cpu().numpy().astype(np.float64))
+        assert np.abs(out[lo:hi].cpu().numpy() - ref_o).max() <= 1e-5 * np.abs(ref_o).max()
+        assert np.abs(lse_out[:, lo:hi].cpu().numpy() - ref_l).max() <= 1e-5 * np.abs(ref_l).max()
+
+
 def test_kv_gather_append_bit_exact(ctx):
     w = wl.small_mixed()
     mat = wl.materialize(w)
