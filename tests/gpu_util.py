@@ -14,6 +14,28 @@ def bf16_to_f64(t: torch.Tensor) -> np.ndarray:
     return t.float().cpu().numpy().astype(np.float64)
 
 
+GUARD_BYTES = 4096
+GUARD_PATTERN = 0xA5
+
+
+class Guarded:
+    """A device tensor placed between two guard regions of a known byte pattern; check() fails if a
+    kernel wrote outside the tensor."""
+
+    def __init__(self, shape, dtype, fill=None):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        pad = (-n) % 256
+        self.raw = torch.full((GUARD_BYTES + n + pad + GUARD_BYTES,), GUARD_PATTERN, dtype=torch.uint8, device="cuda")
+        self.n = n
+        self.tensor = self.raw[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(shape)
+        if fill is not None:
+            self.tensor.fill_(fill)
+
+    def check(self, what):
+        head, tail = self.raw[:GUARD_BYTES], self.raw[GUARD_BYTES + self.n:]
+        assert bool((head == GUARD_PATTERN).all()) and bool((tail == GUARD_PATTERN).all()), "write outside " + what
+
+
 class DeviceWorkload:
     def __init__(self, mat):
         build.build()
@@ -24,11 +46,13 @@ class DeviceWorkload:
         self.v = bits_to_bf16(mat.v_pages)
         self.page_table = torch.from_numpy(mat.page_table).cuda()
         self.cache = binding.make_cache(self.k, self.v)
-        self.out = torch.full((wl.total_new, wl.Hq, wl.D), float("nan"), dtype=torch.bfloat16, device="cuda")
-        self.lse = torch.full((wl.Hq, wl.total_new), float("nan"), dtype=torch.float32, device="cuda")
+        # outputs start as NaN (every row must be written) and sit between guard regions, as does the workspace
+        self._g_out = Guarded((wl.total_new, wl.Hq, wl.D), torch.bfloat16, float("nan"))
+        self._g_lse = Guarded((wl.Hq, wl.total_new), torch.float32, float("nan"))
         nl = [r.new_len for r in wl.requests]
         cs = [r.C for r in wl.requests]
-        self.ws = torch.zeros(binding.cp_workspace_bytes(nl, cs, wl.Hq), dtype=torch.uint8, device="cuda")
+        self._g_ws = Guarded((binding.cp_workspace_bytes(nl, cs, wl.Hq),), torch.uint8, 0)
+        self.out, self.lse, self.ws = self._g_out.tensor, self._g_lse.tensor, self._g_ws.tensor
 
     def run_batch(self, ctx):
         wl = self.wl
@@ -37,6 +61,9 @@ class DeviceWorkload:
                                       wl.Hq, wl.scale, self.out, self.lse, self.ws)
         torch.cuda.synchronize()
         ctx.poll_status()
+        for g, what in ((self._g_out, "out"), (self._g_lse, "lse"), (self._g_ws, "workspace")):
+            g.check(what)
+        assert not bool(torch.isnan(self.out).any()) and not bool(torch.isnan(self.lse).any()), "a row was not written"
         return bf16_to_f64(self.out), self.lse.cpu().numpy().astype(np.float64)
 
 
