@@ -58,6 +58,13 @@ int cp_ctx_create(cp_ctx** ctx, int device);
 int cp_ctx_destroy(cp_ctx* ctx);
 int cp_ctx_poll_status(cp_ctx* ctx, int32_t* detail /* host, 4 words or NULL */);
 
+/* cp_ctx_selftest_wait_expiry -- diagnostic (the paper has no counterpart): enqueues one small block whose
+ * only act is to wait, with a limit of about a millisecond, on a barrier that nothing arrives at.  It shows
+ * on the device at hand that an expired wait ends the kernel normally and is reported: after the stream has
+ * been synchronised, cp_ctx_poll_status returns CP_ERR_TIMEOUT with detail {code, barrier 0, block 0,
+ * iteration 7} and clears the status; the context stays usable.  Errors: INVALID_ARG, CUDA. */
+int cp_ctx_selftest_wait_expiry(cp_ctx* ctx, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * cp_plan -- zigzag shard plan (paper Section 2.1, applied to the uncached suffix of Section 2.2).
  * The R new tokens are padded on the right to a multiple of 2C: chunk length cl = ceil(R / 2C);

@@ -265,7 +265,7 @@ constexpr uint32_t kIdescPV = kIdescS | (1u << 16);
 // gives up after one failed try, so all roles run off the end of their loops without blocking (the
 // results are garbage, the status word says so) and the kernel returns normally.
 __device__ __forceinline__ void mbar_wait(uint32_t bar_base, uint32_t bar_id, uint32_t parity, volatile uint32_t* abort_flag,
-                                          int32_t* status, int iter) {
+                                          int32_t* status, int iter, long long limit_cycles = kWaitLimitCycles) {
     const uint32_t bar = bar_base + bar_id * 8;
     if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
@@ -274,7 +274,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar_base, uint32_t bar_id, ui
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return;
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > limit_cycles) {
             *abort_flag = 1;
             if (atomicCAS(status, 0, CP_ERR_TIMEOUT) == 0) {
                 status[1] = (int32_t)bar_id;
@@ -777,6 +777,20 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever arrives at, with a short
+// limit.  The wait gives up, records CP_ERR_TIMEOUT in the status words and the kernel returns.
+__global__ void wait_expiry_selftest_kernel(int32_t* status, long long limit_cycles) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    mbar_wait(smem_u32(&bar), 0, 0, &abort_flag, status, 7, limit_cycles);
+}
+
 __global__ void fill_neg_inf_kernel(float* p, int64_t n) {
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         p[i] = -INFINITY;
@@ -1077,6 +1091,13 @@ extern "C" int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cac
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
     return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, -1, Hq, scale, partial_out, 1,
                        partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_shard");
+}
+
+extern "C" int cp_ctx_selftest_wait_expiry(cp_ctx* ctx, void* stream) {
+    if (!ctx) return set_error(CP_ERR_INVALID_ARG, "cp_ctx_selftest_wait_expiry: ctx is NULL");
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+    wait_expiry_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_status, 2000000ll);
+    return check_cuda(cudaGetLastError(), "cp_ctx_selftest_wait_expiry launch");
 }
 
 extern "C" int cp_prefill_attn_chunk(cp_ctx* ctx, const void* q_chunk, const cp_kv_cache* cache, const int32_t* page_table,

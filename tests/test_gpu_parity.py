@@ -258,6 +258,18 @@ def test_argument_validation_launches_nothing(ctx):
     assert torch.isnan(dev.out.float()).all()               # nothing was written
 
 
+def test_expired_wait_is_reported_and_context_survives(ctx):
+    # a block waits (about a millisecond) on a barrier nothing arrives at: the kernel returns, the status word
+    # carries the time-out, polling clears it, and the same context computes correct attention afterwards
+    ctx.selftest_wait_expiry()
+    torch.cuda.synchronize()
+    with pytest.raises(binding.CpError) as e:
+        ctx.poll_status()
+    assert e.value.code == binding.CP_ERR_TIMEOUT and "barrier 0, block 0, iteration 7" in str(e.value)
+    ctx.poll_status()                                                       # cleared
+    check_batch(ctx, wl.Workload("after_timeout", 44, 8, 2, [wl.Request(300, 128, 2)]))
+
+
 def test_attention_config2_full(ctx):
     check_batch(ctx, wl.config2(), pair_budget=1e11)
 
