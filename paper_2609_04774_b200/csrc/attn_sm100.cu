@@ -1067,7 +1067,7 @@ extern "C" int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* ca
     if (!cache || new_len < 1 || prefix_len < 0)
         return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn: cache is NULL, new_len < 1 or prefix_len < 0");
     const int64_t cu_new[2] = {0, new_len};
-    const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + kPageTokens - 1) / kPageTokens};
     return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, Hq, scale, out, 0, lse,
                        workspace, workspace_bytes, stream, "cp_prefill_attn");
 }
@@ -1088,7 +1088,7 @@ extern "C" int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cac
     fill_neg_inf_kernel<<<(int)std::min<int64_t>((n_lse + 255) / 256, 4096), 256, 0, s>>>(partial_lse, n_lse);
     if (int rc = check_cuda(cudaGetLastError(), "fill_neg_inf launch")) return rc;
     const int64_t cu_new[2] = {0, new_len};
-    const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + kPageTokens - 1) / kPageTokens};
     return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, -1, Hq, scale, partial_out, 1,
                        partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_shard");
 }
@@ -1107,7 +1107,7 @@ extern "C" int cp_prefill_attn_chunk(cp_ctx* ctx, const void* q_chunk, const cp_
     if (!cache || new_len < 1 || prefix_len < 0 || C < 1 || chunk < 0 || chunk >= 2 * (int64_t)C)
         return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_chunk: bad sizes or chunk %d not in [0, %d)", chunk, 2 * C);
     const int64_t cu_new[2] = {0, new_len};
-    const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + kPageTokens - 1) / kPageTokens};
     return attn_common(ctx, q_chunk, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, chunk, Hq, scale,
                        out_chunk, 0, lse_chunk, workspace, workspace_bytes, stream, "cp_prefill_attn_chunk");
 }
@@ -1191,7 +1191,7 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     if (int rc = static_setup(device, &st)) return rc;
 
     const int64_t cu_new[2] = {0, new_len};
-    const int64_t cu_pages[2] = {0, (prefix_len + new_len + 63) / 64};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + kPageTokens - 1) / kPageTokens};
     std::vector<TileItem> tiles;
     build_tiles(1, cu_new, &prefix_len, &C, cu_pages, -1, -1, tiles);
     cp_ctx enc{};                       // only the encoder entry point is read by encode_maps

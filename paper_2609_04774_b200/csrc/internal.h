@@ -62,6 +62,7 @@ struct WorkspaceLayout {
     size_t items, cta_off, pieces, merges, merge_slots, partial_o, partial_lse, total;
 };
 
+constexpr int kPageTokens = 64;      // tokens per cache page (the only supported page size)
 constexpr int kMaxGrid = 192;                          // upper bound on CTAs (SMs) a schedule may use
 constexpr int kMaxSlots = 2 * kMaxGrid + 32;           // partial slots a schedule may use
 constexpr int kMinShareTiles = 8;                      // smallest per-CTA share worth spreading work for

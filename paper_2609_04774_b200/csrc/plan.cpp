@@ -52,7 +52,7 @@ int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, con
                 t.kv_len0 = (int32_t)(P + r0 + 1);
                 t.pt_base = (int32_t)cu_pages[b];
                 // entries the request really uses; a single chunk reads none behind its last key
-                t.n_pages = (int32_t)((P + (only_chunk >= 0 ? ce : R) + 63) / 64);
+                t.n_pages = (int32_t)((P + (only_chunk >= 0 ? ce : R) + kPageTokens - 1) / kPageTokens);
                 t.n_kv_tiles = (int32_t)((t.kv_len0 + t.n_rows - 1 + kTileRows - 1) / kTileRows);
                 t.request = b;
                 t.shard = shard;
@@ -239,7 +239,7 @@ extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64
     for (int32_t b = 0; b < B; ++b) {
         const int64_t R = cu_new[b + 1] - cu_new[b];
         if (R < 1 || prefix_len[b] < 0 || C[b] < 1) return set_error(CP_ERR_INVALID_ARG, "cp_schedule_inspect: request %d", b);
-        cu_pages[b + 1] = cu_pages[b] + (prefix_len[b] + R + 63) / 64;
+        cu_pages[b + 1] = cu_pages[b] + (prefix_len[b] + R + kPageTokens - 1) / kPageTokens;
     }
     Schedule sch;
     build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), -1, -1, sch.items);
