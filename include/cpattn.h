@@ -32,7 +32,7 @@ extern "C" {
 enum {
     CP_OK = 0,
     CP_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, inconsistent lengths              */
-    CP_ERR_UNSUPPORTED = -2, /* D != 128, page_size != 64, misaligned strides, sizes beyond limits */
+    CP_ERR_UNSUPPORTED = -2, /* D != 128, unsupported page size, misaligned strides, sizes beyond limits */
     CP_ERR_WORKSPACE = -3,   /* workspace missing, misaligned or smaller than cp_workspace_bytes() */
     CP_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                                */
     CP_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (reported by poll_status)       */
@@ -87,7 +87,7 @@ int cp_plan(int64_t new_len, int64_t prefix_len, int32_t C, cp_shard_plan* out);
  *   page_table[t / page_size] * stride_page + (t % page_size) * stride_tok + g * stride_head + d.
  * The new tokens' K and V are already in the cache at logical positions [P, P+R) when attention is
  * called (the ranks gather K/V before attending, Section 2.1).  Default layout
- * [num_pages, 64, Hkv, 128] bf16.  Supported: page_size == 64, D == 128; the three strides must be
+ * [num_pages, 64, Hkv, 128] bf16.  Supported: page_size 16, 32, 64 or 128 tokens, D == 128; the three strides must be
  * multiples of 8 elements and k, v 16-byte aligned (tensor-map rules).  Slots that no logical
  * token maps to (tail of a last page, unreferenced pages) are never read into a result, but they
  * must hold finite bf16 values (they may pass through a multiply by an exactly zero weight).
@@ -96,7 +96,7 @@ typedef struct {
     const void* k;      /* device, bf16 */
     const void* v;      /* device, bf16 */
     int64_t num_pages;
-    int32_t page_size;  /* 64  */
+    int32_t page_size;  /* 16, 32, 64 or 128 */
     int32_t Hkv;
     int32_t D;          /* 128 */
     int32_t reserved;

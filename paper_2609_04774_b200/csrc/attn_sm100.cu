@@ -37,10 +37,13 @@ constexpr int kBlockN = 128;
 constexpr int kKvStages = 5;                       // ring of 32 KB tiles, K and V alternate
 constexpr uint32_t kTileBytes = kBlockN * kD * 2;  // 32768
 constexpr uint32_t kHalfBytes = kTileBytes / 2;    // one 64-dim half: 128 rows x 128 B
-constexpr uint32_t kPageBoxBytes = 64 * 64 * 2;    // one TMA box: 64 tokens x 64 dims
 constexpr int kThreads = 384;
-constexpr int kRegsSoftmax = 208;   // setmaxnreg budgets: 2*128*208 + 128*88 = 64512 = 384*168
-constexpr int kRegsOther = 88;
+// setmaxnreg budgets after the role split.  Their total must stay below the 64K register file by at
+// least one allocation step: with a split that used the whole file (208 / 96) the softmax warps never got
+// their registers and the kernel did not start its work.
+constexpr int kRegsSoftmax = 200;
+constexpr int kRegsOther = 104;
+static_assert(2 * 128 * kRegsSoftmax + 128 * kRegsOther <= 65536 - 1024, "leave slack in the register file");
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t kSmemQ = 0;                                  // 2 heads x 32 KB
@@ -88,6 +91,7 @@ struct AttnParams {
     int32_t Hq;
     const int32_t* page_table;
     int32_t oob_page;         // a page coordinate outside the tensor map: TMA fills zeros
+    int32_t page_tokens;      // tokens per page: 16, 32, 64 or 128 (one TMA box = one page x 64 dims)
     float scale_log2;         // scale * log2(e)
     void* out;
     int32_t out_f32;          // 0: bf16 [rows, Hq, D]; 1: fp32
@@ -364,27 +368,31 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
         }
         __syncwarp();
         const int n_tiles = u.t_end;
-        for (int j0 = u.t_begin; j0 < n_tiles; j0 += 16) {
-            // the warp fetches the page ids of 16 KV tiles (32 pages) at once
-            const int pg = 2 * j0 + lane;
+        const int ppt = kBlockN / p.page_tokens;          // pages per KV tile: 8, 4, 2 or 1
+        const int tiles_per_fetch = 32 / ppt;
+        const uint32_t box_bytes = (uint32_t)p.page_tokens * 128u;   // one page x 64 dims
+        for (int j0 = u.t_begin; j0 < n_tiles; j0 += tiles_per_fetch) {
+            // the warp fetches the page ids of the next 32 pages (32 / ppt KV tiles) at once
+            const int pg = ppt * j0 + lane;
             const int my_page = (pg < u.it.n_pages) ? __ldg(p.page_table + u.it.pt_base + pg) : p.oob_page;
-            const int jn = min(16, n_tiles - j0);
+            const int jn = min(tiles_per_fetch, n_tiles - j0);
             for (int jj = 0; jj < jn; ++jj) {
-                const int page_a = __shfl_sync(0xffffffffu, my_page, 2 * jj);
-                const int page_b = __shfl_sync(0xffffffffu, my_page, 2 * jj + 1);
                 for (int kv = 0; kv < 2; ++kv) {
+                    const uint32_t slot = kv_it % kKvStages;
+                    const uint32_t fbar = bars + (kBarKvFull + slot) * 8;
+                    const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
+                    const CUtensorMap* map = kv ? tmV : tmK;
                     if (lane == 0) {
-                        const uint32_t slot = kv_it % kKvStages;
                         mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j0 + jj);
                         CP_TRACE(3, j0 + jj, 6 + kv);
-                        const uint32_t fbar = bars + (kBarKvFull + slot) * 8;
-                        const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
-                        const CUtensorMap* map = kv ? tmV : tmK;
                         mbar_expect_tx(fbar, kTileBytes);
-                        for (int half = 0; half < 2; ++half) {
-                            tma_load_4d(dst + half * kHalfBytes, map, fbar, half * 64, u.kv_head, 0, page_a);
-                            tma_load_4d(dst + half * kHalfBytes + kPageBoxBytes, map, fbar, half * 64, u.kv_head, 0, page_b);
-                        }
+                    }
+                    __syncwarp();
+                    // lane i < ppt copies page i of the tile: both 64-dim halves of its box
+                    const int page = __shfl_sync(0xffffffffu, my_page, ppt * jj + (lane < ppt ? lane : 0));
+                    if (lane < ppt) {
+                        tma_load_4d(dst + lane * box_bytes, map, fbar, 0, u.kv_head, 0, page);
+                        tma_load_4d(dst + kHalfBytes + lane * box_bytes, map, fbar, 64, u.kv_head, 0, page);
                     }
                     __syncwarp();
                     ++kv_it;
@@ -900,7 +908,7 @@ int encode_maps(cp_ctx* ctx, const void* q, int64_t total_rows, int32_t Hq, cons
         cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)c->Hkv, (cuuint64_t)c->page_size, (cuuint64_t)c->num_pages};
         cuuint64_t strides[3] = {(cuuint64_t)c->stride_head * 2, (cuuint64_t)c->stride_tok * 2,
                                  (cuuint64_t)c->stride_page * 2};
-        cuuint32_t box[4] = {64, 1, 64, 1};
+        cuuint32_t box[4] = {64, 1, (cuuint32_t)c->page_size, 1};
         cuuint32_t es[4] = {1, 1, 1, 1};
         CUresult r = ctx->encode_tiled(kv ? tmV : tmK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
                                        const_cast<void*>(kv ? c->v : c->k), dims, strides, box, es,
@@ -938,6 +946,9 @@ int upload_block(cp_ctx* ctx, const std::vector<uint8_t>& block, void* dst, cuda
     return check_cuda(cudaEventRecord(ctx->stage_event[i], s), "cudaEventRecord(stage)");
 }
 
+// Page size for sizing a page table before the cache has been validated (a bad value is rejected later).
+inline int64_t page_tokens_of(const cp_kv_cache* c) { return (c && c->page_size > 0) ? c->page_size : kDefaultPageTokens; }
+
 int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table, int32_t B,
                 const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C, const int64_t* cu_pages,
                 int32_t only_shard, int32_t only_chunk, int32_t Hq, float scale, void* out, int out_f32, float* lse,
@@ -974,7 +985,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
 
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
     Schedule sch;
-    build_tiles(B, cu_new, prefix_len, C, cu_pages, only_shard, only_chunk, sch.items);
+    build_tiles(B, cu_new, prefix_len, C, cu_pages, cache->page_size, only_shard, only_chunk, sch.items);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (sch.items.empty()) return CP_OK;   // the shard owns no rows (only empty chunks)
     // rows of q / out / lse: the packed batch, or the one chunk of a chunk call
@@ -1024,6 +1035,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.Hq = Hq;
     p.page_table = page_table;
     p.oob_page = (int32_t)std::min<int64_t>(cache->num_pages, 0x7fffffff);
+    p.page_tokens = cache->page_size;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.out = out;
     p.out_f32 = out_f32;
@@ -1067,7 +1079,7 @@ extern "C" int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* ca
     if (!cache || new_len < 1 || prefix_len < 0)
         return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn: cache is NULL, new_len < 1 or prefix_len < 0");
     const int64_t cu_new[2] = {0, new_len};
-    const int64_t cu_pages[2] = {0, (prefix_len + new_len + kPageTokens - 1) / kPageTokens};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
     return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, Hq, scale, out, 0, lse,
                        workspace, workspace_bytes, stream, "cp_prefill_attn");
 }
@@ -1088,7 +1100,7 @@ extern "C" int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cac
     fill_neg_inf_kernel<<<(int)std::min<int64_t>((n_lse + 255) / 256, 4096), 256, 0, s>>>(partial_lse, n_lse);
     if (int rc = check_cuda(cudaGetLastError(), "fill_neg_inf launch")) return rc;
     const int64_t cu_new[2] = {0, new_len};
-    const int64_t cu_pages[2] = {0, (prefix_len + new_len + kPageTokens - 1) / kPageTokens};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
     return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, -1, Hq, scale, partial_out, 1,
                        partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_shard");
 }
@@ -1107,7 +1119,7 @@ extern "C" int cp_prefill_attn_chunk(cp_ctx* ctx, const void* q_chunk, const cp_
     if (!cache || new_len < 1 || prefix_len < 0 || C < 1 || chunk < 0 || chunk >= 2 * (int64_t)C)
         return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_chunk: bad sizes or chunk %d not in [0, %d)", chunk, 2 * C);
     const int64_t cu_new[2] = {0, new_len};
-    const int64_t cu_pages[2] = {0, (prefix_len + new_len + kPageTokens - 1) / kPageTokens};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
     return attn_common(ctx, q_chunk, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, chunk, Hq, scale,
                        out_chunk, 0, lse_chunk, workspace, workspace_bytes, stream, "cp_prefill_attn_chunk");
 }
@@ -1191,9 +1203,9 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     if (int rc = static_setup(device, &st)) return rc;
 
     const int64_t cu_new[2] = {0, new_len};
-    const int64_t cu_pages[2] = {0, (prefix_len + new_len + kPageTokens - 1) / kPageTokens};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
     std::vector<TileItem> tiles;
-    build_tiles(1, cu_new, &prefix_len, &C, cu_pages, -1, -1, tiles);
+    build_tiles(1, cu_new, &prefix_len, &C, cu_pages, cache->page_size, -1, -1, tiles);
     cp_ctx enc{};                       // only the encoder entry point is read by encode_maps
     enc.encode_tiled = st->encode_tiled;
     CUtensorMap tmQ, tmK, tmV;
@@ -1218,6 +1230,7 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     p.Hq = Hq;
     p.page_table = page_table;
     p.oob_page = (int32_t)std::min<int64_t>(cache->num_pages, 0x7fffffff);
+    p.page_tokens = cache->page_size;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.out = out;
     p.out_f32 = 0;

@@ -62,7 +62,7 @@ struct WorkspaceLayout {
     size_t items, cta_off, pieces, merges, merge_slots, partial_o, partial_lse, total;
 };
 
-constexpr int kPageTokens = 64;      // tokens per cache page (the only supported page size)
+constexpr int kDefaultPageTokens = 64;   // page size assumed where no cache is at hand (schedule inspection)
 constexpr int kMaxGrid = 192;                          // upper bound on CTAs (SMs) a schedule may use
 constexpr int kMaxSlots = 2 * kMaxGrid + 32;           // partial slots a schedule may use
 constexpr int kMinShareTiles = 8;                      // smallest per-CTA share worth spreading work for
@@ -94,7 +94,7 @@ int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C);
 // chunk and numbers its rows from the chunk's first row (q, out and lse then hold the chunk alone).
 int validate_kv_cache(const cp_kv_cache* c, const char* who);
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
-                const int64_t* cu_pages, int32_t only_shard, int32_t only_chunk, std::vector<TileItem>& out);
+                const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, std::vector<TileItem>& out);
 // Distributes the (tile, head pair) units of s.items over `grid_max` CTAs: whole units longest first
 // onto the least loaded CTA while they fit under the per-CTA share, the rest cut into KV ranges that
 // fill every CTA to the same number of KV tiles.  Fills cta_off / pieces / merges / merge_slots.

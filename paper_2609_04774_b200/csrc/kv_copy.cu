@@ -38,9 +38,9 @@ kv_copy_kernel(uint4* __restrict__ paged_k, uint4* __restrict__ paged_v, uint4* 
 int validate_cache(const cp_kv_cache* c, const char* who) {
     if (!c || !c->k || !c->v || c->num_pages < 1 || c->Hkv < 1)
         return set_error(CP_ERR_INVALID_ARG, "%s: cache is NULL or has null / non-positive fields", who);
-    if (c->page_size != 64 || c->D != 128)
-        return set_error(CP_ERR_UNSUPPORTED, "%s: page_size=%d D=%d, only 64 / 128 are supported", who, c->page_size,
-                         c->D);
+    if ((c->page_size != 16 && c->page_size != 32 && c->page_size != 64 && c->page_size != 128) || c->D != 128)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: page_size=%d D=%d; supported: pages of 16, 32, 64 or 128 tokens, D = 128", who,
+                         c->page_size, c->D);
     if ((c->stride_page | c->stride_tok | c->stride_head) & 7 || c->stride_page < 1 || c->stride_tok < 1 ||
         c->stride_head < 1)
         return set_error(CP_ERR_UNSUPPORTED, "%s: strides must be positive multiples of 8 elements", who);

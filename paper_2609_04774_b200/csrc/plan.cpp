@@ -31,7 +31,7 @@ int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C) {
 }
 
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
-                const int64_t* cu_pages, int32_t only_shard, int32_t only_chunk, std::vector<TileItem>& out) {
+                const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, std::vector<TileItem>& out) {
     out.clear();
     for (int32_t b = 0; b < B; ++b) {
         const int64_t R = cu_new[b + 1] - cu_new[b];
@@ -52,7 +52,7 @@ int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, con
                 t.kv_len0 = (int32_t)(P + r0 + 1);
                 t.pt_base = (int32_t)cu_pages[b];
                 // entries the request really uses; a single chunk reads none behind its last key
-                t.n_pages = (int32_t)((P + (only_chunk >= 0 ? ce : R) + kPageTokens - 1) / kPageTokens);
+                t.n_pages = (int32_t)((P + (only_chunk >= 0 ? ce : R) + page_size - 1) / page_size);
                 t.n_kv_tiles = (int32_t)((t.kv_len0 + t.n_rows - 1 + kTileRows - 1) / kTileRows);
                 t.request = b;
                 t.shard = shard;
@@ -239,10 +239,10 @@ extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64
     for (int32_t b = 0; b < B; ++b) {
         const int64_t R = cu_new[b + 1] - cu_new[b];
         if (R < 1 || prefix_len[b] < 0 || C[b] < 1) return set_error(CP_ERR_INVALID_ARG, "cp_schedule_inspect: request %d", b);
-        cu_pages[b + 1] = cu_pages[b] + (prefix_len[b] + R + kPageTokens - 1) / kPageTokens;
+        cu_pages[b + 1] = cu_pages[b] + (prefix_len[b] + R + kDefaultPageTokens - 1) / kDefaultPageTokens;
     }
     Schedule sch;
-    build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), -1, -1, sch.items);
+    build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), kDefaultPageTokens, -1, -1, sch.items);
     if (int rc = build_schedule(Hq / heads_per_unit, num_sms, sch)) return rc;
     int64_t max_load = 0, min_load = INT64_MAX, total = 0;
     for (int32_t c = 0; c < sch.grid; ++c) {

@@ -175,6 +175,7 @@ class Workload:
     D: int = HEAD_DIM
     spare_pages: int = 3          # physical pages never referenced by any page table
     shuffle_pages: bool = True
+    page: int = PAGE              # tokens per cache page
     meta: dict = field(default_factory=dict)
 
     @property
@@ -191,7 +192,7 @@ class Workload:
 
     @property
     def cu_pages(self) -> np.ndarray:
-        return np.concatenate([[0], np.cumsum([r.n_pages for r in self.requests])]).astype(np.int64)
+        return np.concatenate([[0], np.cumsum([-(-r.total_len // self.page) for r in self.requests])]).astype(np.int64)
 
     @property
     def num_pages(self) -> int:
@@ -236,10 +237,11 @@ def materialize(wl: Workload, need_q: bool = True) -> Materialized:
     n_logical = int(wl.cu_pages[-1])
     page_table = perm[:n_logical].astype(np.int32).copy()
 
-    k_pages = np.empty((npg, PAGE, Hkv, D), dtype=np.uint16)
-    v_pages = np.empty((npg, PAGE, Hkv, D), dtype=np.uint16)
-    garb = np.where((np.arange(PAGE * Hkv * D) % 2) == 0, GARBAGE_POS, GARBAGE_NEG).astype(np.uint16)
-    garb = garb.reshape(PAGE, Hkv, D)
+    ps = wl.page
+    k_pages = np.empty((npg, ps, Hkv, D), dtype=np.uint16)
+    v_pages = np.empty((npg, ps, Hkv, D), dtype=np.uint16)
+    garb = np.where((np.arange(ps * Hkv * D) % 2) == 0, GARBAGE_POS, GARBAGE_NEG).astype(np.uint16)
+    garb = garb.reshape(ps, Hkv, D)
     for p in perm[n_logical:]:
         k_pages[p] = garb
         v_pages[p] = garb[::-1]
@@ -251,14 +253,14 @@ def materialize(wl: Workload, need_q: bool = True) -> Materialized:
         kb = normal_bf16(wl.seed, TID_K, (L, Hkv, D), start=tok0 * row_elems)
         vb = normal_bf16(wl.seed, TID_V, (L, Hkv, D), start=tok0 * row_elems)
         pt = page_table[wl.cu_pages[b]:wl.cu_pages[b + 1]]
-        full = L // PAGE
+        full = L // ps
         if full:
-            k_pages[pt[:full]] = kb[:full * PAGE].reshape(full, PAGE, Hkv, D)
-            v_pages[pt[:full]] = vb[:full * PAGE].reshape(full, PAGE, Hkv, D)
-        rem = L - full * PAGE
+            k_pages[pt[:full]] = kb[:full * ps].reshape(full, ps, Hkv, D)
+            v_pages[pt[:full]] = vb[:full * ps].reshape(full, ps, Hkv, D)
+        rem = L - full * ps
         if rem:
-            k_pages[pt[full], :rem] = kb[full * PAGE:]
-            v_pages[pt[full], :rem] = vb[full * PAGE:]
+            k_pages[pt[full], :rem] = kb[full * ps:]
+            v_pages[pt[full], :rem] = vb[full * ps:]
             k_pages[pt[full], rem:] = garb[rem:]
             v_pages[pt[full], rem:] = garb[::-1][rem:]
         tok0 += L

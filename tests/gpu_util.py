@@ -41,6 +41,7 @@ class DeviceWorkload:
         build.build()
         wl = mat.wl
         self.wl = wl
+        self.mat = mat
         self.q = bits_to_bf16(mat.q)
         self.k = bits_to_bf16(mat.k_pages)
         self.v = bits_to_bf16(mat.v_pages)

@@ -135,6 +135,26 @@ def test_attention_small_mixed_batch(ctx):
     assert torch.equal(o1.view(torch.int16), dev.out.view(torch.int16)) and torch.equal(l1, dev.lse)
 
 
+@pytest.mark.parametrize("page", [16, 32, 128])
+def test_attention_other_page_sizes(ctx, page):
+    # cache pages of 16, 32 and 128 tokens: 8, 4 and 1 page boxes per 128-key tile; prefixes that are and are
+    # not page multiples; KV-split units; the paged copies with the same page size, bit for bit
+    reqs = [wl.Request(333, 192, 3), wl.Request(5, 0, 4), wl.Request(700, 1000, 2), wl.Request(64, 20000, 1)]
+    w = wl.Workload("page_%d" % page, 45, 8, 2, reqs, page=page)
+    dev, out, lse, _ = check_batch(ctx, w, pair_budget=3e7)
+    assert dev.cache.page_size == page
+    mat = dev.mat
+    pt_host = mat.page_table[w.cu_pages[2]:w.cu_pages[3]]
+    pt = dev.page_table[int(w.cu_pages[2]):int(w.cu_pages[3])].contiguous()
+    t0, n = 37, 1500
+    kr = torch.empty((n, w.Hkv, w.D), dtype=torch.bfloat16, device="cuda")
+    vr = torch.empty_like(kr)
+    binding.cp_kv_gather(ctx, dev.cache, pt, t0, n, kr, vr)
+    torch.cuda.synchronize()
+    assert np.array_equal(kr.view(torch.int16).cpu().numpy().view(np.uint16), orc.kv_gather(mat.k_pages, pt_host, t0, t0 + n))
+    assert np.array_equal(vr.view(torch.int16).cpu().numpy().view(np.uint16), orc.kv_gather(mat.v_pages, pt_host, t0, t0 + n))
+
+
 def test_attention_odd_group_sizes(ctx):
     # Hq / Hkv = 3 and plain multi-head attention (Hq == Hkv): one query head per work unit
     check_batch(ctx, wl.Workload("odd_group", 41, 6, 2, [wl.Request(333, 192, 3), wl.Request(129, 0, 2)]))
@@ -250,7 +270,7 @@ def test_argument_validation_launches_nothing(ctx):
         binding.cp_prefill_attn(ctx, dev.q, dev.cache, dev.page_table, 0, 0, 1, w.Hq, w.scale, dev.out, dev.lse, dev.ws)
     assert e.value.code == binding.CP_ERR_INVALID_ARG
     bad = binding.make_cache(dev.k, dev.v)
-    bad.page_size = 32
+    bad.page_size = 48                                      # pages of 16, 32, 64 or 128 tokens only
     with pytest.raises(binding.CpError) as e:
         binding.cp_prefill_attn(ctx, dev.q, bad, dev.page_table, 0, 64, 1, w.Hq, w.scale, dev.out, dev.lse, dev.ws)
     assert e.value.code == binding.CP_ERR_UNSUPPORTED
