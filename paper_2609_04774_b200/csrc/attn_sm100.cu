@@ -626,7 +626,8 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, u
     if ((q) + 1 == kSplitQ || (q) == 3) {                                               \
         tc_wait_st();                                                                   \
         tc_fence_before();                                                              \
-        mbar_arrive(p_bar0 + ((q) == 3 ? 1 : 0) * 8);                                   \
+        __syncwarp();                                                                   \
+        if ((threadIdx.x & 31) == 0) mbar_arrive(p_bar0 + ((q) == 3 ? 1 : 0) * 8);      \
     }
     CP_P_PIECE(s0, 0)
     CP_P_PIECE(s1, 1)
@@ -719,7 +720,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
             else p.lse[(int64_t)head * p.lse_stride + grow_idx] = lse_val;
         }
         tc_fence_before();
-        mbar_arrive(bars + (kBarOFree + wg) * 8);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + (kBarOFree + wg) * 8);
     }
 #undef SM_WAIT
 }
@@ -744,9 +746,9 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         for (int w = 0; w < 2; ++w) {
             mbar_init(bars + (kBarSReady + w) * 8, 1);
-            for (int q4 = 0; q4 < 4; ++q4) mbar_init(bars + (kBarPReady + 4 * w + q4) * 8, 128);
+            for (int q4 = 0; q4 < 4; ++q4) mbar_init(bars + (kBarPReady + 4 * w + q4) * 8, 4);   // one arrival per warp
             mbar_init(bars + (kBarODone + w) * 8, 1);
-            mbar_init(bars + (kBarOFree + w) * 8, 128);
+            mbar_init(bars + (kBarOFree + w) * 8, 4);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
