@@ -57,10 +57,11 @@ enum Bar : uint32_t {
     kBarQFull = 0, kBarQEmpty = 1,
     kBarKvFull = 2,                       // + stage
     kBarKvEmpty = kBarKvFull + kKvStages, // + stage
-    kBarSReady = kBarKvEmpty + kKvStages, // + wg
-    kBarPReady = kBarSReady + 2,          // + wg*4 + quarter: P columns [16*quarter, +16) written
-    kBarODone = kBarPReady + 8,           // + wg
-    kBarOFree = kBarODone + 2,            // + wg
+    kBarSReady = kBarKvEmpty + kKvStages, // + wg: the score tile in the S buffer belongs to this head and is complete
+    kBarSFree = kBarSReady + 2,           // the S buffer has been read into registers (one phase per score tile)
+    kBarPReady = kBarSFree + 1,           // + wg*4 + piece
+    kBarPvDone = kBarPReady + 8,          // + wg: P*V of a tile has finished (P and O of the head may be touched)
+    kBarOFree = kBarPvDone + 2,           // + wg
     kNumBars = kBarOFree + 2
 };
 static_assert(kNumBars * 8 + 16 <= 256, "barrier area");
@@ -68,7 +69,8 @@ constexpr uint32_t kSmemTmemPtr = kSmemBar + kNumBars * 8;      // uint32: TMEM 
 constexpr uint32_t kSmemAbort = kSmemTmemPtr + 4;               // uint32: set when a wait expired
 
 // TMEM columns
-constexpr uint32_t kTmemS = 0;     // + wg * 128
+constexpr uint32_t kTmemS = 0;     // one score tile (fp32), shared by the two heads in turn
+constexpr uint32_t kTmemP = 128;   // + wg * 64: P of a head (bf16), the TMEM A operand of P*V
 constexpr uint32_t kTmemO = 256;   // + wg * 128
 
 constexpr uint32_t kTryWaitHintNs = 200000;             // the thread may stay suspended this long per try
@@ -369,158 +371,166 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
         __syncwarp();
         const int n_tiles = u.t_end;
         const int ppt = kBlockN / p.page_tokens;          // pages per KV tile: 8, 4, 2 or 1
-        const int tiles_per_fetch = 32 / ppt;
         const uint32_t box_bytes = (uint32_t)p.page_tokens * 128u;   // one page x 64 dims
-        for (int j0 = u.t_begin; j0 < n_tiles; j0 += tiles_per_fetch) {
-            // the warp fetches the page ids of the next 32 pages (32 / ppt KV tiles) at once
-            const int pg = ppt * j0 + lane;
-            const int my_page = (pg < u.it.n_pages) ? __ldg(p.page_table + u.it.pt_base + pg) : p.oob_page;
-            const int jn = min(tiles_per_fetch, n_tiles - j0);
-            for (int jj = 0; jj < jn; ++jj) {
-                for (int kv = 0; kv < 2; ++kv) {
-                    const uint32_t slot = kv_it % kKvStages;
-                    const uint32_t fbar = bars + (kBarKvFull + slot) * 8;
-                    const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
-                    const CUtensorMap* map = kv ? tmV : tmK;
-                    if (lane == 0) {
-                        mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j0 + jj);
-                        CP_TRACE(3, j0 + jj, 6 + kv);
-                        mbar_expect_tx(fbar, kTileBytes);
-                    }
-                    __syncwarp();
-                    // lane i < ppt copies page i of the tile: both 64-dim halves of its box
-                    const int page = __shfl_sync(0xffffffffu, my_page, ppt * jj + (lane < ppt ? lane : 0));
-                    if (lane < ppt) {
-                        tma_load_4d(dst + lane * box_bytes, map, fbar, 0, u.kv_head, 0, page);
-                        tma_load_4d(dst + kHalfBytes + lane * box_bytes, map, fbar, 64, u.kv_head, 0, page);
-                    }
-                    __syncwarp();
-                    ++kv_it;
-                }
+        // load order = order of first use by the MMA warp: K(j0), then K(j+1) before V(j)
+        const int n_loads = 2 * (n_tiles - u.t_begin);
+        int pg_base = -1;       // first page whose id the lanes currently hold
+        int my_page = 0;
+        for (int ld = 0; ld < n_loads; ++ld) {
+            // ld 0: K(j0); odd ld: K(j0 + (ld+1)/2) except the last, which is V(n-1); even ld > 0: V(j0 + ld/2 - 1)
+            int j, kv;
+            if (ld == 0) { j = u.t_begin; kv = 0; }
+            else if (ld == n_loads - 1) { j = n_tiles - 1; kv = 1; }
+            else if (ld & 1) { j = u.t_begin + (ld + 1) / 2; kv = 0; }
+            else { j = u.t_begin + ld / 2 - 1; kv = 1; }
+            const int pg0 = ppt * j;
+            if (pg_base < 0 || pg0 < pg_base || pg0 + ppt > pg_base + 32) {
+                // the warp fetches 32 page ids starting at this tile (K runs one tile ahead of V, so the
+                // window is anchored at the V tile when possible)
+                pg_base = ppt * max(j - 1, u.t_begin);
+                const int pg = pg_base + lane;
+                my_page = (pg < u.it.n_pages) ? __ldg(p.page_table + u.it.pt_base + pg) : p.oob_page;
             }
+            const uint32_t slot = kv_it % kKvStages;
+            const uint32_t fbar = bars + (kBarKvFull + slot) * 8;
+            const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
+            const CUtensorMap* map = kv ? tmV : tmK;
+            if (lane == 0) {
+                mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j);
+                CP_TRACE(3, j, 6 + kv);
+                mbar_expect_tx(fbar, kTileBytes);
+            }
+            __syncwarp();
+            // lane i < ppt copies page i of the tile: both 64-dim halves of its box
+            const int page = __shfl_sync(0xffffffffu, my_page, (pg0 - pg_base + (lane < ppt ? lane : 0)) & 31);
+            if (lane < ppt) {
+                tma_load_4d(dst + lane * box_bytes, map, fbar, 0, u.kv_head, 0, page);
+                tma_load_4d(dst + kHalfBytes + lane * box_bytes, map, fbar, 64, u.kv_head, 0, page);
+            }
+            __syncwarp();
+            ++kv_it;
         }
     }
 }
 
-// The issuer warp alternates between the two heads in a fixed order, PV0(j) S0(j+1) PV1(j) S1(j+1):
-// the tensor pipe executes in issue order, which keeps the two softmax warpgroups half a period apart
-// (one exponentiates while the pipe works for the other).  P arrives in two pieces (96 keys, then 32),
-// so P*V starts while the rest of the row is still being exponentiated.  The whole warp runs the loop
-// (waits included) so that addresses and descriptors stay warp-uniform; one elected lane issues.
-__device__ __forceinline__ void mma_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
-                                         volatile uint32_t* abort_flag) {
+// The issuer warp.  One score buffer S serves both heads in turn, P and O have their own TMEM columns per
+// head.  A score tile is read into registers by its softmax warpgroup as soon as that group is free, and
+// the next score tile (of the other head, or of the same head when a unit has one) is issued the moment
+// the buffer has been read -- so the scores of a head's next tile are computed while the head is still
+// exponentiating the current one, and a softmax warpgroup never waits for the tensor pipe in steady state.
+// With H heads per unit and tiles numbered S_0, S_1, ... (head fastest), P_k = P*V of tile k, the issue
+// order is S_0 .. S_H, then P_k followed by S_(k+H+1).  P arrives in two pieces (96 keys, then 32).
+// The whole warp runs the loop (waits included) so that addresses stay warp-uniform; one elected lane issues.
+// Position in the K/V ring: slot and phase parity, advanced without divisions.
+struct RingPos {
+    uint32_t slot, par;
+    __device__ __forceinline__ RingPos plus(uint32_t n) const {   // n < kKvStages
+        RingPos r = {slot + n, par};
+        if (r.slot >= (uint32_t)kKvStages) { r.slot -= kKvStages; r.par ^= 1u; }
+        return r;
+    }
+};
+
+// Two issuer warps, one per kind of product; nothing orders them against each other, because score tiles
+// (S buffer) and P*V (P and O columns) touch disjoint TMEM and the K and V tiles have their own barriers.
+//
+// Score issuer: S tiles in the order (tile, head); each needs its K tile and the buffer back (s_free).
+__device__ __forceinline__ void mma_s_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
+                                           volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
-    uint32_t kv_it = 0;        // ring slots consumed so far
-    uint32_t tile_cnt = 0;     // KV tiles processed so far (phase of p_ready)
-    const int last_wg = p.heads_per_unit - 1;   // last head of a unit: its block releases the K/V slots
+    const int H = p.heads_per_unit;
+    RingPos unit_pos = {0, 0};         // ring position of the unit's first load, K(j0)
+    uint32_t s_par = 1;                // parity of "previous score tile was read"; 1: no tile yet (passes)
     const uint64_t q_desc0 = make_desc(smem_base + kSmemQ, 16, 1024);
     const uint64_t k_desc0 = make_desc(smem_base + kSmemKV, 16, 1024);           // K-major view of a ring slot
-    const uint64_t v_desc0 = make_desc(smem_base + kSmemKV, kHalfBytes, 1024);   // MN-major view of a ring slot
-
-    // S = Q K^T for one head: 8 MMAs of 16 dims (issued by the elected lane only)
-    auto mma_s = [&](int wg, uint32_t slot) {
-#pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) {
-            const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
-            mma_ss(tmem_base + kTmemS + wg * 128, q_desc0 + (wg * (kTileBytes >> 4)) + off,
-                   k_desc0 + slot * (kTileBytes >> 4) + off, kIdescS, ks > 0);
-        }
-    };
-    // O += P V over one piece of the tile's keys: MMAs of 16 keys, 2 per quarter of the row
-    auto mma_pv = [&](int wg, int part, uint32_t slot, bool accumulate) {
-        const int ks0 = part == 0 ? 0 : 2 * kSplitQ, ks1 = part == 0 ? 2 * kSplitQ : 8;
-#pragma unroll
-        for (int ks = ks0; ks < ks1; ++ks) {
-            mma_ts(tmem_base + kTmemO + wg * 128, tmem_base + kTmemS + wg * 128 + ks * 8,
-                   v_desc0 + slot * (kTileBytes >> 4) + ks * (2048 >> 4), kIdescPV, accumulate || ks > 0);
-        }
-    };
-#define MMA_WAIT(id, parity, it) mbar_wait(bars, (id), (parity), abort_flag, p.status, (it))
-
     for (int round = 0;; ++round) {
         UnitInfo u;
         if (!fetch_unit(p, round, u)) break;
-        const int n = u.t_end;
-        MMA_WAIT(kBarQFull, round & 1, round);
-        const uint32_t slot0 = kv_it % kKvStages;
-        MMA_WAIT(kBarKvFull + slot0, (kv_it / kKvStages) & 1, 0);
-        tc_fence_after();
-        if (elect_one()) {
-            mma_s(0, slot0);
-            tc_commit(bars + (kBarSReady + 0) * 8);
-            if (last_wg == 1) {
-                mma_s(1, slot0);
-                tc_commit(bars + (kBarSReady + 1) * 8);
-            }
-            tc_commit(bars + (kBarKvEmpty + slot0) * 8);
-            if (u.t_begin + 1 == n) tc_commit(bars + kBarQEmpty * 8);
-        }
-        __syncwarp();
-        ++kv_it;
-        bool kv_tested = false;     // V(j) and K(j+1) already seen complete by a test issued one block earlier
-        bool p_tested = false;      // same for the next P hand-over
+        const int j0 = u.t_begin, n = u.t_end;
+        mbar_wait(bars, kBarQFull, round & 1, abort_flag, p.status, round);
+        RingPos kpos = unit_pos;
 #pragma unroll 1
-        for (int j = u.t_begin; j < n; ++j) {
-            const uint32_t v_slot = kv_it % kKvStages;
-            const uint32_t v_par = (kv_it / kKvStages) & 1;
-            ++kv_it;
-            const bool more = (j + 1 < n);
-            const uint32_t k_slot = kv_it % kKvStages;
-            const uint32_t k_par = (kv_it / kKvStages) & 1;
-            // K(j+1) and V(j) were requested long ago
-            if (!kv_tested) {
-                MMA_WAIT(kBarKvFull + v_slot, v_par, j);
-                if (more) MMA_WAIT(kBarKvFull + k_slot, k_par, j);
-            }
-            // slots and phases of the next tile's V(j+1), K(j+2), for the early test below
-            const uint32_t it_v2 = kv_it + 1, it_k2 = kv_it + 2;
-            const uint32_t bar_v2 = bars + (kBarKvFull + it_v2 % kKvStages) * 8, par_v2 = (it_v2 / kKvStages) & 1;
-            const uint32_t bar_k2 = bars + (kBarKvFull + it_k2 % kKvStages) * 8, par_k2 = (it_k2 / kKvStages) & 1;
+        for (int j = j0; j < n; ++j) {
+            mbar_wait(bars, kBarKvFull + kpos.slot, kpos.par, abort_flag, p.status, j);
+            for (int h = 0; h < H; ++h) {
+                mbar_wait(bars, kBarSFree, s_par, abort_flag, p.status, j);
+                s_par ^= 1u;
+                tc_fence_after();
+                if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + h, j, 2); }
+                if (elect_one()) {
 #pragma unroll
-            for (int wg = 0; wg < 2; ++wg) {
-                if (wg > last_wg) break;
-                if (j == u.t_begin && round > 0) MMA_WAIT(kBarOFree + wg, (round - 1) & 1, j);
+                    for (int ks = 0; ks < kD / 16; ++ks) {
+                        const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+                        mma_ss(tmem_base + kTmemS, q_desc0 + (h * (kTileBytes >> 4)) + off,
+                               k_desc0 + kpos.slot * (kTileBytes >> 4) + off, kIdescS, ks > 0);
+                    }
+                    tc_commit(bars + (kBarSReady + h) * 8);
+                    if (h == H - 1) {
+                        tc_commit(bars + (kBarKvEmpty + kpos.slot) * 8);
+                        if (j == n - 1) tc_commit(bars + kBarQEmpty * 8);
+                    }
+                }
+                __syncwarp();
+                if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + h, j, 3); }
+            }
+            kpos = kpos.plus(j == j0 ? 1 : 2);     // load order: K(j0), K(j0+1), V(j0), K(j0+2), V(j0+1), ...
+        }
+        const uint32_t adv = (uint32_t)(2 * (n - j0));
+        const uint32_t q5 = adv / kKvStages, r5 = adv - q5 * kKvStages;
+        unit_pos = unit_pos.plus(r5);
+        unit_pos.par ^= (q5 & 1u);
+    }
+}
+
+// P*V issuer: O_h += P_h V_j in the order (tile, head), each in the two pieces P is handed over in.
+__device__ __forceinline__ void mma_pv_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
+                                            volatile uint32_t* abort_flag) {
+    const uint32_t bars = smem_base + kSmemBar;
+    const int H = p.heads_per_unit;
+    RingPos unit_pos = {0, 0};
+    uint32_t p_par = 0;                // phase parity of p_ready (the heads advance together)
+    const uint64_t v_desc0 = make_desc(smem_base + kSmemKV, kHalfBytes, 1024);   // MN-major view of a ring slot
+    for (int round = 0;; ++round) {
+        UnitInfo u;
+        if (!fetch_unit(p, round, u)) break;
+        const int j0 = u.t_begin, n = u.t_end;
+        RingPos vpos = unit_pos.plus(n - j0 == 1 ? 1 : 2);   // V(j0)
+#pragma unroll 1
+        for (int j = j0; j < n; ++j) {
+            mbar_wait(bars, kBarKvFull + vpos.slot, vpos.par, abort_flag, p.status, j);
+            for (int h = 0; h < H; ++h) {
+                if (j == j0 && round > 0) mbar_wait(bars, kBarOFree + h, (round - 1) & 1, abort_flag, p.status, j);
 #pragma unroll
                 for (int part = 0; part < kPieces; ++part) {
-                    if (!p_tested) MMA_WAIT(kBarPReady + wg * 4 + part, tile_cnt & 1, j);
+                    mbar_wait(bars, kBarPReady + h * 4 + part, p_par, abort_flag, p.status, j);
                     tc_fence_after();
-                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, part); }
-                    // tests for what the next block of MMAs will need, answered while this block is issued
-                    bool next_p;
-                    if (part + 1 < kPieces) next_p = mbar_test(bars + (kBarPReady + wg * 4 + part + 1) * 8, tile_cnt & 1);
-                    else if (wg < last_wg) next_p = mbar_test(bars + (kBarPReady + 4) * 8, tile_cnt & 1);
-                    else next_p = more && mbar_test(bars + kBarPReady * 8, (tile_cnt + 1) & 1);
-                    bool next_kv = false;
-                    if (wg == last_wg && part == kPieces - 1 && more)
-                        next_kv = mbar_test(bar_v2, par_v2) && (j + 2 >= n || mbar_test(bar_k2, par_k2));
+                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + h, j, part); }
                     if (elect_one()) {
-                        mma_pv(wg, part, v_slot, j > u.t_begin);
+                        const int ks0 = part == 0 ? 0 : 2 * kSplitQ, ks1 = part == 0 ? 2 * kSplitQ : 8;
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            if (ks >= ks0 && ks < ks1)
+                                mma_ts(tmem_base + kTmemO + h * 128, tmem_base + kTmemP + h * 64 + ks * 8,
+                                       v_desc0 + vpos.slot * (kTileBytes >> 4) + ks * (2048 >> 4), kIdescPV,
+                                       j > j0 || ks > 0);
+                        }
                         if (part == kPieces - 1) {
-                            if (more) {
-                                mma_s(wg, k_slot);
-                                tc_commit(bars + (kBarSReady + wg) * 8);
-                            } else {
-                                tc_commit(bars + (kBarODone + wg) * 8);
-                            }
-                            if (wg == last_wg) {
-                                tc_commit(bars + (kBarKvEmpty + v_slot) * 8);
-                                if (more) tc_commit(bars + (kBarKvEmpty + k_slot) * 8);
-                                if (j + 2 == n) tc_commit(bars + kBarQEmpty * 8);
-                            }
+                            tc_commit(bars + (kBarPvDone + h) * 8);
+                            if (h == H - 1) tc_commit(bars + (kBarKvEmpty + vpos.slot) * 8);
                         }
                     }
-                    // per-lane answers: a lane whose test came back negative waits below, the others go on
-                    // to the next elect.sync, where the warp meets again
-                    p_tested = next_p;
-                    if (wg == last_wg && part == kPieces - 1) kv_tested = next_kv;
+                    __syncwarp();
                 }
-                if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wg, j, 5); }
+                if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + h, j, 5); }
             }
-            if (more) ++kv_it;
-            ++tile_cnt;
+            p_par ^= 1u;
+            vpos = vpos.plus(j + 2 == n ? 1 : 2);
         }
+        const uint32_t adv = (uint32_t)(2 * (n - j0));
+        const uint32_t q5 = adv / kKvStages, r5 = adv - q5 * kKvStages;
+        unit_pos = unit_pos.plus(r5);
+        unit_pos.par ^= (q5 & 1u);
     }
-#undef MMA_WAIT
 }
 
 // Row max of 32 raw scores into four independent chains.
@@ -539,9 +549,10 @@ __device__ __forceinline__ void mask32(float (&s)[32], int lim) {
     for (int i = 0; i < 32; ++i)
         if (i >= lim) s[i] = -INFINITY;
 }
-// p = 2^(s*c - m) for 32 keys -> 16 packed bf16 pairs; row sums into four accumulators.  In unmasked
-// tiles kPolyOf4 of every four pairs take the FMA-pipe polynomial instead of MUFU.
-template <bool kMasked>
+// p = 2^(s*c - m) for 32 keys -> 16 packed bf16 pairs; row sums into four accumulators.  With kPoly,
+// kPolyOf4 of every four pairs take the FMA-pipe polynomial instead of MUFU; masked tiles do not (the
+// polynomial clamps a masked score, -inf, to 2^-126, which is not the exact zero a hidden key needs).
+template <bool kPoly>
 __device__ __forceinline__ void exp32(const float (&s)[32], uint32_t (&pk)[16], float2 c2, float2 nm2, float2& sum0,
                                       float2& sum1, float2& sum2, float2& sum3) {
 #pragma unroll
@@ -552,8 +563,8 @@ __device__ __forceinline__ void exp32(const float (&s)[32], uint32_t (&pk)[16], 
         const float2 x3 = __ffma2_rn(make_float2(s[2 * i + 6], s[2 * i + 7]), c2, nm2);
         const float2 p0 = make_float2(ex2(x0.x), ex2(x0.y));
         const float2 p1 = make_float2(ex2(x1.x), ex2(x1.y));
-        const float2 p2 = (kPolyOf4 >= 2 && !kMasked) ? ex2_poly2(x2) : make_float2(ex2(x2.x), ex2(x2.y));
-        const float2 p3 = (kPolyOf4 >= 1 && !kMasked) ? ex2_poly2(x3) : make_float2(ex2(x3.x), ex2(x3.y));
+        const float2 p2 = (kPoly && kPolyOf4 >= 2) ? ex2_poly2(x2) : make_float2(ex2(x2.x), ex2(x2.y));
+        const float2 p3 = (kPoly && kPolyOf4 >= 1) ? ex2_poly2(x3) : make_float2(ex2(x3.x), ex2(x3.y));
         sum0 = __fadd2_rn(sum0, p0);
         sum1 = __fadd2_rn(sum1, p1);
         sum2 = __fadd2_rn(sum2, p2);
@@ -565,43 +576,73 @@ __device__ __forceinline__ void exp32(const float (&s)[32], uint32_t (&pk)[16], 
     }
 }
 
-// One 128x128 score tile of one head: the row is read from TMEM once (four 32-column loads, one
-// wait), reduced to its max, exponentiated in four pieces of 32 keys, and P goes back to TMEM piece
-// by piece; the MMA warp is signalled after the third piece and after the last.  Straight-line code in both variants (no
-// per-element branches) so that the scheduler can overlap the MUFU, FMA and ALU pipes.
+struct SoftmaxSync {
+    uint32_t bars;                   // shared-memory address of the barrier array
+    uint32_t s_ready_id;             // barrier "a score tile of this head is in the S buffer"
+    uint32_t pv_done_id, pv_parity;  // barrier and phase of this head's previous P*V
+    volatile uint32_t* abort_flag;
+    int32_t* status;
+    int iter;
+    long long* tr;                   // trace builds: stamp row of this tile (or NULL)
+};
+
+// Reads the 128 scores of this thread's row from the S buffer (the caller has seen s_ready).
+#define CP_LOAD_S(a0, a1, a2, a3)          \
+    TMEM_LD32(s_tmem + 0, a0, 0);          \
+    TMEM_LD32(s_tmem + 32, a1, 0);         \
+    TMEM_LD32(s_tmem + 64, a2, 0);         \
+    TMEM_LD32(s_tmem + 96, a3, 0);
+
+// Hands the S buffer back once this warp's loads have landed: one arrival per warp.
+__device__ __forceinline__ void release_s(uint32_t bars) {
+    tc_wait_ld();
+    tc_fence_before();
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bars + kBarSFree * 8);
+}
+
+// One 128x128 score tile of one head; the row's scores are already in registers (c0..c3).  Row max, lazy
+// rescale, exponentials in four pieces of 32 keys, P into this head's TMEM columns piece by piece (the P*V
+// issuer is signalled after the third piece and after the last).  If the head has another tile in this
+// unit, its scores replace the current ones before the function returns: the first 96 columns already
+// after the third piece when the tile is in the S buffer by then (their registers are no longer needed,
+// so the load runs under the last exponentials), the rest -- or all of it, after a wait -- behind the
+// last piece.  The S buffer goes back to the score issuer as soon as the loads have landed.
+// Straight-line code in both variants, no per-element branches.
 // kMasked: the tile reaches past the causal diagonal of some rows; `lim` = visible columns of this row.
 template <bool kMasked>
-__device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, uint32_t p_bar0, float c, int lim,
-                                             bool first, float& m, float& l) {
-    float s0[32], s1[32], s2[32], s3[32];
-    TMEM_LD32(s_tmem + 0, s0, 0);
-    TMEM_LD32(s_tmem + 32, s1, 0);
-    TMEM_LD32(s_tmem + 64, s2, 0);
-    TMEM_LD32(s_tmem + 96, s3, 0);
-    tc_wait_ld();
+__device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], float (&c2)[32], float (&c3)[32],
+                                             bool more, uint32_t& s_par, uint32_t s_tmem, uint32_t p_tmem,
+                                             uint32_t o_tmem, uint32_t p_bar0, float c, int lim, bool first,
+                                             float& m, float& l, const SoftmaxSync& sy) {
+    if (sy.tr) sy.tr[1] = clock64();
     if (kMasked) {
-        mask32(s0, lim);
-        mask32(s1, lim - 32);
-        mask32(s2, lim - 64);
-        mask32(s3, lim - 96);
+        mask32(c0, lim);
+        mask32(c1, lim - 32);
+        mask32(c2, lim - 64);
+        mask32(c3, lim - 96);
     }
     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-    max32(s0, mx0, mx1, mx2, mx3);
-    max32(s1, mx0, mx1, mx2, mx3);
-    max32(s2, mx0, mx1, mx2, mx3);
-    max32(s3, mx0, mx1, mx2, mx3);
+    max32(c0, mx0, mx1, mx2, mx3);
+    max32(c1, mx0, mx1, mx2, mx3);
+    max32(c2, mx0, mx1, mx2, mx3);
+    max32(c3, mx0, mx1, mx2, mx3);
     const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
     const float m_new = fmaxf(m, mx * c);
     if (first) {
         m = m_new;     // O is overwritten by the first P*V: nothing to rescale
     } else {
+        // P and O of this head are free once the previous tile's P*V has finished (long ago, normally)
+        mbar_wait(sy.bars, sy.pv_done_id, sy.pv_parity, sy.abort_flag, sy.status, sy.iter);
+        __syncwarp();
+        tc_fence_after();
+        if (sy.tr) sy.tr[2] = clock64();
         const bool grow = (m_new - m) > kRescaleThreshold;
         if (__any_sync(0xffffffffu, grow)) {
             const float m_upd = grow ? m_new : m;
             const float alpha = ex2(m - m_upd);
             l *= alpha;
             m = m_upd;
-            // P*V of the previous tile finished before this S was signalled (the pipe runs in issue order)
 #pragma unroll 1
             for (int cc = 0; cc < 4; ++cc) {
                 float o[32];
@@ -613,7 +654,7 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, u
             }
         }
     }
-    const float2 c2 = make_float2(c, c);
+    const float2 c2f = make_float2(c, c);
     // a row that has seen no key yet (only possible in masked tiles of a KV-split piece) keeps m = -inf;
     // subtracting 0 instead keeps its weights at exactly 0 rather than NaN
     const float m_sub = (kMasked && m == -INFINITY) ? 0.f : m;
@@ -621,19 +662,44 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_tmem, uint32_t o_tmem, u
     float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0, sum2 = sum0, sum3 = sum0;
     uint32_t pk[16];
 #define CP_P_PIECE(cur, q)                                                              \
-    exp32<kMasked>(cur, pk, c2, nm2, sum0, sum1, sum2, sum3);                           \
-    TMEM_ST16R(s_tmem + (q) * 16, pk, 0);                                               \
+    exp32<!kMasked>(cur, pk, c2f, nm2, sum0, sum1, sum2, sum3);                         \
+    TMEM_ST16R(p_tmem + (q) * 16, pk, 0);                                               \
     if ((q) + 1 == kSplitQ || (q) == 3) {                                               \
         tc_wait_st();                                                                   \
         tc_fence_before();                                                              \
         __syncwarp();                                                                   \
         if ((threadIdx.x & 31) == 0) mbar_arrive(p_bar0 + ((q) == 3 ? 1 : 0) * 8);      \
+        if (sy.tr) sy.tr[(q) == 3 ? 4 : 3] = clock64();                                 \
     }
-    CP_P_PIECE(s0, 0)
-    CP_P_PIECE(s1, 1)
-    CP_P_PIECE(s2, 2)
-    CP_P_PIECE(s3, 3)
+    CP_P_PIECE(c0, 0)
+    CP_P_PIECE(c1, 1)
+    CP_P_PIECE(c2, 2)
+    // is the head's next score tile in the S buffer already?  (same answer in the whole warp)
+    bool early = false;
+    if (more) {
+        early = __all_sync(0xffffffffu, mbar_test(sy.bars + sy.s_ready_id * 8, s_par));
+        if (early) {
+            tc_fence_after();
+            TMEM_LD32(s_tmem + 0, c0, 0);
+            TMEM_LD32(s_tmem + 32, c1, 0);
+            TMEM_LD32(s_tmem + 64, c2, 0);
+        }
+    }
+    CP_P_PIECE(c3, 3)
 #undef CP_P_PIECE
+    if (more) {
+        if (!early) {
+            mbar_wait(sy.bars, sy.s_ready_id, s_par, sy.abort_flag, sy.status, sy.iter);
+            __syncwarp();
+            tc_fence_after();
+            TMEM_LD32(s_tmem + 0, c0, 0);
+            TMEM_LD32(s_tmem + 32, c1, 0);
+            TMEM_LD32(s_tmem + 64, c2, 0);
+        }
+        TMEM_LD32(s_tmem + 96, c3, 0);
+        release_s(sy.bars);
+        s_par ^= 1u;
+    }
     const float2 st = __fadd2_rn(__fadd2_rn(sum0, sum1), __fadd2_rn(sum2, sum3));
     l += st.x + st.y;
 }
@@ -645,7 +711,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
     const int warp_in_wg = (threadIdx.x >> 5) & 3;
     const int row = warp_in_wg * 32 + lane;                        // query row of the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)(warp_in_wg * 32) << 16;   // TMEM lane field of this warp
-    const uint32_t s_tmem = tmem_base + lane_addr + kTmemS + wg * 128;
+    const uint32_t s_tmem = tmem_base + lane_addr + kTmemS;
+    const uint32_t p_tmem = tmem_base + lane_addr + kTmemP + wg * 64;
     const uint32_t o_tmem = tmem_base + lane_addr + kTmemO + wg * 128;
     const uint32_t p_bar0 = bars + (kBarPReady + wg * 4) * 8;
     const float c = p.scale_log2;
@@ -655,6 +722,14 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
 #define SM_WAIT(id, parity, it)                                                                  \
     mbar_wait(bars, (id), (parity), abort_flag, p.status, (it));                                 \
     __syncwarp();
+#ifdef CPATTN_TRACE
+#define CP_TRACE_ROW_PTR(j_)                                                                                \
+    long long* tr = (row == CPATTN_TRACE_ROW && blockIdx.x == 0 && round == 0 && (j_) < 64)                 \
+                        ? reinterpret_cast<long long*>(p.status + 16) + (wg * 64 + (j_)) * 8 : nullptr;
+#else
+#define CP_TRACE_ROW_PTR(j_) long long* const tr = nullptr;
+#endif
+    uint32_t s_par = 0;        // phase parity of s_ready for this head
 
     for (int round = 0;; ++round) {
         UnitInfo u;
@@ -665,20 +740,30 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
         float l = 0.f;         // running row sum of 2^(s - m)
         // tiles below n_full lie entirely under the causal diagonal of every row of the q-tile
         const int n_full = u.it.kv_len0 / kBlockN;
+        float s0[32], s1[32], s2[32], s3[32];   // the row's scores of the current tile
+        // the first tile of the unit is loaded here, every later one by the tile before it
+        SM_WAIT(kBarSReady + wg, s_par, u.t_begin);
+        s_par ^= 1u;
+        tc_fence_after();
+        CP_LOAD_S(s0, s1, s2, s3)
+        release_s(bars);
 #pragma unroll 1
         for (int j = u.t_begin; j < n; ++j) {
-            SM_WAIT(kBarSReady + wg, tile_cnt & 1, j);
-            tc_fence_after();
-            if (row == CPATTN_TRACE_ROW) { CP_TRACE(wg, j, 0); }
+            CP_TRACE_ROW_PTR(j)
+            if (tr) tr[0] = clock64();
+            const SoftmaxSync sy = {bars, kBarSReady + (uint32_t)wg, kBarPvDone + (uint32_t)wg, (tile_cnt - 1) & 1,
+                                    abort_flag, p.status, j, tr};
             if (j < n_full)
-                softmax_tile<false>(s_tmem, o_tmem, p_bar0, c, 0, j == u.t_begin, m, l);
+                softmax_tile<false>(s0, s1, s2, s3, j + 1 < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c, 0,
+                                    j == u.t_begin, m, l, sy);
             else
-                softmax_tile<true>(s_tmem, o_tmem, p_bar0, c, u.it.kv_len0 + row - j * kBlockN, j == u.t_begin, m, l);
+                softmax_tile<true>(s0, s1, s2, s3, j + 1 < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c,
+                                   u.it.kv_len0 + row - j * kBlockN, j == u.t_begin, m, l, sy);
             if (row == CPATTN_TRACE_ROW) { CP_TRACE(wg, j, 6); }
             ++tile_cnt;
         }
         // epilogue: O / l -> global at the row's original position; LSE in natural log
-        SM_WAIT(kBarODone + wg, round & 1, n);
+        SM_WAIT(kBarPvDone + wg, (tile_cnt - 1) & 1, n);
         tc_fence_after();
         // a row of a KV-split piece may see none of the piece's keys: l = 0, written as O = 0, lse = -inf
         const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
@@ -744,10 +829,11 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             mbar_init(bars + (kBarKvFull + s) * 8, 1);
             mbar_init(bars + (kBarKvEmpty + s) * 8, 1);
         }
+        mbar_init(bars + kBarSFree * 8, 4);
         for (int w = 0; w < 2; ++w) {
             mbar_init(bars + (kBarSReady + w) * 8, 1);
             for (int q4 = 0; q4 < 4; ++q4) mbar_init(bars + (kBarPReady + 4 * w + q4) * 8, 4);   // one arrival per warp
-            mbar_init(bars + (kBarODone + w) * 8, 1);
+            mbar_init(bars + (kBarPvDone + w) * 8, 1);
             mbar_init(bars + (kBarOFree + w) * 8, 4);
         }
         *abort_flag = 0;
@@ -770,7 +856,9 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if (warp == 8) {
             producer_role(&tmQ, &tmK, &tmV, p, smem_base, abort_flag);
         } else if (warp == 9) {
-            mma_role(p, smem_base, tmem_base, abort_flag);
+            mma_s_role(p, smem_base, tmem_base, abort_flag);
+        } else if (warp == 10) {
+            mma_pv_role(p, smem_base, tmem_base, abort_flag);
         }
     }
 
