@@ -1088,7 +1088,9 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
 #ifdef CPATTN_TRACE
     if (const char* e = getenv("CPATTN_DEBUG_SMS")) grid_max = std::max(1, atoi(e));   // trace builds only
 #endif
-    if (int rc = build_schedule(Hq / heads_per_unit, grid_max, sch)) return rc;
+    if (int rc = build_schedule(Hq / heads_per_unit,
+                                kv_major_pairs(B, cu_new, prefix_len, cache->Hkv, (Hq / cache->Hkv) / heads_per_unit),
+                                grid_max, sch)) return rc;
     const WorkspaceLayout lay = workspace_layout(sch.items.size(), sch.pieces.size(), sch.merges.size(),
                                                  sch.merge_slots.size(), sch.grid, sch.n_slots);
     if (lay.total > workspace_bytes)

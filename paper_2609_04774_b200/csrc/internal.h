@@ -95,10 +95,13 @@ int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C);
 int validate_kv_cache(const cp_kv_cache* c, const char* who);
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
                 const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, std::vector<TileItem>& out);
-// Distributes the (tile, head pair) units of s.items over `grid_max` CTAs: whole units longest first
+// Distributes the (tile, head pair) units of s.items over `grid_max` CTAs (pairs_per_kv = units of one KV
+// head per tile): whole units, KV head by KV head and longest first within a head,
 // onto the least loaded CTA while they fit under the per-CTA share, the rest cut into KV ranges that
 // fill every CTA to the same number of KV tiles.  Fills cta_off / pieces / merges / merge_slots.
-int build_schedule(int32_t pairs_per_tile, int32_t grid_max, Schedule& s);
+int build_schedule(int32_t pairs_per_tile, int32_t pairs_per_kv, int32_t grid_max, Schedule& s);
+// pairs_per_kv to pass to build_schedule: the real value when the batch's K/V is large, else 0 (one group)
+int32_t kv_major_pairs(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, int32_t Hkv, int32_t pairs_per_kv);
 WorkspaceLayout workspace_layout(size_t n_items, size_t n_pieces, size_t n_merges, size_t n_merge_slots, size_t grid,
                                  size_t n_slots);
 

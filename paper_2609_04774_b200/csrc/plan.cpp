@@ -83,8 +83,11 @@ WorkspaceLayout workspace_layout(size_t n_items, size_t n_pieces, size_t n_merge
     return w;
 }
 
-static int build_schedule_impl(int32_t pairs_per_tile, int32_t grid_max, bool allow_split, Schedule& s) {
+static int build_schedule_impl(int32_t pairs_per_tile, int32_t pairs_per_kv, int32_t grid_max, bool allow_split,
+                               Schedule& s) {
     const int32_t HP = pairs_per_tile;
+    // units of one KV head per tile; 0 (or anything that does not divide HP): one group, longest first overall
+    const int32_t PK = (pairs_per_kv >= 1 && HP % pairs_per_kv == 0) ? pairs_per_kv : HP;
     const int64_t n_items = (int64_t)s.items.size();
     const int64_t n_units = n_items * HP;
     int64_t W = 0;
@@ -102,8 +105,11 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t grid_max, bool al
     const int32_t G = (int32_t)std::max<int64_t>(1, std::min<int64_t>(grid_max, (W + T - 1) / T));
     s.grid = G;
 
-    // 1. whole units, longest first, dealt to the CTAs in serpentine order (0..G-1, G-1..0, ...) while
-    //    they fit under the share; what does not fit goes to the tail
+    // 1. whole units dealt to the CTAs in serpentine order (0..G-1, G-1..0, ...) while they fit under the
+    //    share; what does not fit goes to the tail.  Order: longest first, either over all units or (PK < HP)
+    //    KV head by KV head.  In the second order all CTAs read the K/V of one KV head at a time (an eighth
+    //    of the cache for 8 KV heads), which keeps a long context's K/V in L2 instead of streaming it from
+    //    HBM for every query tile; the caller asks for it when the K/V of the batch is large.
     std::vector<int64_t> load(G, 0);
     std::vector<int32_t> count(G, 0);                  // pieces per CTA
     std::vector<int16_t> cta_of((size_t)n_units);      // CTA of a whole unit, -1 = tail
@@ -111,9 +117,10 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t grid_max, bool al
     std::vector<TailUnit> tail;
     {
         int64_t k = 0;   // running index over the units that were dealt
+        for (int32_t g0 = 0; g0 < HP; g0 += PK)
         for (int64_t i = 0; i < n_items; ++i) {
             const int32_t n = s.items[i].n_kv_tiles;
-            for (int32_t pr = 0; pr < HP; ++pr) {
+            for (int32_t pr = g0; pr < g0 + PK; ++pr) {
                 const int64_t r = k / G;
                 const int32_t pos = (int32_t)(k - r * G);
                 const int32_t c = (r & 1) ? G - 1 - pos : pos;
@@ -173,7 +180,7 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t grid_max, bool al
     }
     if (n_slots > kMaxSlots) {
         // cannot happen with one cut per CTA boundary; if it ever does, fall back to whole units only
-        if (allow_split) return build_schedule_impl(pairs_per_tile, grid_max, false, s);
+        if (allow_split) return build_schedule_impl(pairs_per_tile, pairs_per_kv, grid_max, false, s);
         return set_error(CP_ERR_UNSUPPORTED, "schedule: %d partial slots", n_slots);
     }
     s.n_slots = n_slots;
@@ -183,9 +190,10 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t grid_max, bool al
     for (int32_t k = 0; k < G; ++k) s.cta_off[k + 1] = s.cta_off[k] + count[k];
     s.pieces.resize((size_t)s.cta_off[G]);
     std::vector<int32_t> fill(s.cta_off.begin(), s.cta_off.end() - 1);
+    for (int32_t g0 = 0; g0 < HP; g0 += PK)
     for (int64_t i = 0; i < n_items; ++i) {
         const int32_t n = s.items[i].n_kv_tiles;
-        for (int32_t pr = 0; pr < HP; ++pr) {
+        for (int32_t pr = g0; pr < g0 + PK; ++pr) {
             const int16_t k = cta_of[(size_t)(i * HP + pr)];
             if (k >= 0) s.pieces[(size_t)fill[k]++] = {(int32_t)i, (int16_t)pr, (int16_t)-1, 0, n};
         }
@@ -195,8 +203,15 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t grid_max, bool al
     return CP_OK;
 }
 
-int build_schedule(int32_t pairs_per_tile, int32_t grid_max, Schedule& s) {
-    return build_schedule_impl(pairs_per_tile, grid_max, true, s);
+int build_schedule(int32_t pairs_per_tile, int32_t pairs_per_kv, int32_t grid_max, Schedule& s) {
+    return build_schedule_impl(pairs_per_tile, pairs_per_kv, grid_max, true, s);
+}
+
+// KV head by KV head once the batch's K and V (bf16, D = 128) exceed a quarter of a 126 MB L2.
+int32_t kv_major_pairs(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, int32_t Hkv, int32_t pairs_per_kv) {
+    int64_t tokens = 0;
+    for (int32_t b = 0; b < B; ++b) tokens += prefix_len[b] + (cu_new[b + 1] - cu_new[b]);
+    return tokens * Hkv * 128 * 4 > (32ll << 20) ? pairs_per_kv : 0;
 }
 
 }  // namespace cpattn
@@ -243,7 +258,8 @@ extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64
     }
     Schedule sch;
     build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), kDefaultPageTokens, -1, -1, sch.items);
-    if (int rc = build_schedule(Hq / heads_per_unit, num_sms, sch)) return rc;
+    if (int rc = build_schedule(Hq / heads_per_unit, kv_major_pairs(B, cu_new, prefix_len, Hkv, (Hq / Hkv) / heads_per_unit),
+                                num_sms, sch)) return rc;
     int64_t max_load = 0, min_load = INT64_MAX, total = 0;
     for (int32_t c = 0; c < sch.grid; ++c) {
         int64_t load = 0;

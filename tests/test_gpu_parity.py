@@ -304,7 +304,7 @@ def test_attention_variant_gqa8_and_chunked_prefill(ctx):
     w = wl.variant_chunked_prefill()
     info, _, _ = binding.cp_schedule_inspect(w.cu_new, [65536], [2], w.Hq, w.Hkv,
                                              torch.cuda.get_device_properties(0).multi_processor_count, want_lists=False)
-    assert info["split_units"] == 64 and info["max_load"] * info["grid"] <= 1.01 * info["total"]
+    assert info["split_units"] == 64 and info["max_load"] * info["grid"] <= 1.02 * info["total"]
     check_batch(ctx, w, pair_budget=2e8)
 
 
