@@ -78,7 +78,9 @@ constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
 constexpr float kRescaleThreshold = 8.0f;
 constexpr int kPieces = 2;                            // P is handed to the MMA warp in two pieces:
 constexpr int kSplitQ = 3;                            // the first kSplitQ quarters of the row, then the rest
-constexpr int kPolyOf4 = 1;                            // pairs out of every four whose exp2 runs on the FMA pipe              // log2 units: keep a stale row max up to 2^8
+constexpr int kPolyOf4 = 0;                            // pairs out of every four whose exp2 runs on the FMA pipe instead of MUFU:
+                                                       // 0 since both softmax warpgroups run all the time (issue slots are the
+                                                       // scarcer resource: 1 costs 3 %, 2 costs 12 %); 1 was best while they alternated
 
 struct AttnParams {
     const TileItem* items;
