@@ -39,7 +39,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one cp_attn_kernel launch, from the ncu capture
 # summarised in profiles/ (per workload name)
-ATTN_TRAFFIC_BYTES = {"cfg2_R4096_P12288_C4": 118_146_816}
+ATTN_TRAFFIC_BYTES = {"cfg2_R4096_P12288_C4": 118_038_784}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
