@@ -115,7 +115,8 @@ size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C, i
  * on a device with num_sms SMs (the varlen tile schedule: query tiles of at most 128 rows cut at the
  * chunk boundaries of every request's zigzag plan; one unit per tile and pair of query heads (per
  * single head when Hq / Hkv is odd); whole
- * units longest first dealt to the CTAs in serpentine order, the remainder cut along KV so that every
+ * units longest first -- KV head by KV head when the batch's K/V exceeds 32 MB, so that a long context's K/V
+ * stays in L2 -- dealt to the CTAs in serpentine order, the remainder cut along KV so that every
  * CTA gets the same number of KV tile steps).  summary (8 values): CTAs, query tiles, pieces, split units,
  * partial slots, largest / smallest per-CTA load in KV tile steps, their total.  pieces (optional,
  * 6 int32 per piece: cta, tile, head pair, first KV tile, end KV tile, partial slot or -1) and

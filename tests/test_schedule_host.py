@@ -85,3 +85,29 @@ def test_schedule_small_and_odd_shapes():
               wl.Workload("mha", 5, 4, 4, [wl.Request(513, 0, 3)])):
         for sms in (1, 7, 148):
             check(w, sms)
+
+
+def test_large_kv_is_scheduled_kv_head_by_kv_head():
+    # K/V beyond a quarter of L2: every CTA takes its whole units KV head by KV head (all CTAs then read one
+    # head's K/V at a time); a small batch keeps the plain longest-first order
+    def unit_sequences(w):
+        info, pieces, items = binding.cp_schedule_inspect(w.cu_new, [r.prefix_len for r in w.requests],
+                                                          [r.C for r in w.requests], w.Hq, w.Hkv, 148)
+        per_cta = {}
+        for cta, item, pair, t0, t1, slot in pieces:
+            if slot < 0:
+                per_cta.setdefault(int(cta), []).append((int(pair), int(items[item][3])))
+        return per_cta
+    big = wl.Workload("big", 1, 32, 8, [wl.Request(32768, 0, 4)])            # 134 MB of K/V
+    pairs_per_kv = (big.Hq // big.Hkv) // 2
+    for cta, seq in unit_sequences(big).items():
+        heads = [p // pairs_per_kv for p, _ in seq]
+        assert heads == sorted(heads), cta
+        assert len(set(heads)) >= 4                                           # every CTA sees most of the heads
+        for h in set(heads):                                                  # longest first within a head
+            lens = [n for p, n in seq if p // pairs_per_kv == h]
+            assert lens == sorted(lens, reverse=True)
+    small = wl.Workload("small", 1, 32, 8, [wl.Request(2048, 0, 4)])          # 8 MB of K/V
+    for cta, seq in unit_sequences(small).items():
+        lens = [n for _, n in seq]
+        assert lens == sorted(lens, reverse=True)
