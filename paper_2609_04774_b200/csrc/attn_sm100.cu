@@ -6,16 +6,19 @@
 // lands in shared memory feeds two 128x128 score tiles (GQA head sharing).  Warp roles:
 //   warps 0-3  softmax warpgroup for head 0 of the pair: one thread per query row
 //   warps 4-7  softmax warpgroup for head 1
-//   warp  8    TMA producer (lane 0 issues; the warp prefetches page ids)
-//   warp  9    tcgen05.mma issuer (warp-uniform loop, one elected lane issues)
-//   warps 10-11 idle (they complete the third warpgroup so that register budgets can be moved:
-//              the softmax warpgroups run with 208 registers per thread, the third one with 88)
-// TMEM (512 columns): S0 | S1 | O0 | O1, each 128 fp32 columns; P (bf16) overwrites the first 64
-// columns of its S tile and is consumed from TMEM as the A operand of P*V.
-// The tensor pipe executes the MMAs of the issuing thread in order, PV0(j) S0(j+1) PV1(j) S1(j+1):
-// S(j+1) follows P*V(j) of the same head (P overwrites S), and while one warpgroup runs softmax on
-// its tile the pipe works for the other head.  P is handed over in two pieces (96 keys, then 32), so
-// P*V starts while the rest of the row is still being exponentiated.
+//   warp  8    TMA producer (the warp prefetches page ids; the pages of a tile go out from several lanes)
+//   warp  9    tcgen05.mma issuer for the scores S = Q K^T (warp-uniform loop, one elected lane issues)
+//   warp  10   tcgen05.mma issuer for O += P V
+//   warp  11   idle (completes the third warpgroup so that register budgets can be moved: the softmax
+//              warpgroups run with 200 registers per thread, the third one with 104)
+// TMEM (512 columns): S | P0 | P1 | O0 | O1.  S is ONE score buffer (128 fp32 columns) that the two heads
+// use in turn; P (bf16, 64 columns per head) is the TMEM A operand of P*V; O0, O1 are the accumulators.
+// A softmax warpgroup reads its score tile into registers and hands the buffer back at once, so the next
+// score tile -- the other head's, then its own next one -- is computed while it exponentiates: in steady
+// state no softmax warpgroup waits for the tensor pipe, and both MUFU and tensor pipe stay about 74 % busy.
+// The two issuers need no ordering between them (disjoint TMEM, separate barriers for K and V tiles).
+// P is handed over in two pieces (96 keys, then 32), so P*V starts while the rest of the row is still
+// being exponentiated.
 // Every wait is bounded; on expiry the CTA records where it gave up in the status word, all roles
 // drain and the kernel returns normally.
 #include <cuda_bf16.h>
@@ -76,7 +79,7 @@ constexpr uint32_t kTmemO = 256;   // + wg * 128
 constexpr uint32_t kTryWaitHintNs = 200000;             // the thread may stay suspended this long per try
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
 constexpr float kRescaleThreshold = 8.0f;
-constexpr int kPieces = 2;                            // P is handed to the MMA warp in two pieces:
+constexpr int kPieces = 2;                            // P is handed to the P*V issuer in two pieces:
 constexpr int kSplitQ = 3;                            // the first kSplitQ quarters of the row, then the rest
 constexpr int kPolyOf4 = 0;                            // pairs out of every four whose exp2 runs on the FMA pipe instead of MUFU:
                                                        // 0 since both softmax warpgroups run all the time (issue slots are the
@@ -374,7 +377,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
         const int n_tiles = u.t_end;
         const int ppt = kBlockN / p.page_tokens;          // pages per KV tile: 8, 4, 2 or 1
         const uint32_t box_bytes = (uint32_t)p.page_tokens * 128u;   // one page x 64 dims
-        // load order = order of first use by the MMA warp: K(j0), then K(j+1) before V(j)
+        // load order = order of first use by the issuers: K(j0), then K(j+1) before V(j)
         const int n_loads = 2 * (n_tiles - u.t_begin);
         int pg_base = -1;       // first page whose id the lanes currently hold
         int my_page = 0;
