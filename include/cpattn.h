@@ -182,6 +182,20 @@ int cp_prefill_attn_chunk(cp_ctx* ctx, const void* q_chunk, const cp_kv_cache* c
                           float scale, void* out_chunk, float* lse_chunk, void* workspace,
                           size_t workspace_bytes, void* stream);
 
+/* cp_prefill_attn_kvrange -- all R queries against the keys whose absolute position lies in
+ * [kv_lo, kv_hi) only (still causal: new token r sees positions <= P + r): the partial result a CP rank
+ * produces when the K/V stays sharded over the ranks and the queries travel instead (the alternative to the
+ * all-gather of Section 2.1; the paper keeps a worker's cached KV "partitioned across its ranks",
+ * Section 2.2).  partial_out: device [R, Hq, D] fp32, normalised over the keys of the range; partial_lse:
+ * device [Hq, R] fp32; a row that sees no key of the range gets zeros and lse = -inf.  Partials over
+ * disjoint ranges that together cover [0, P + R) combine with cp_merge into cp_prefill_attn's result.
+ * Only pages holding keys of the range are read.  kv_lo, kv_hi need no alignment.  Workspace as for
+ * cp_prefill_attn with C = 1.  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
+int cp_prefill_attn_kvrange(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
+                            int64_t prefix_len, int64_t new_len, int64_t kv_lo, int64_t kv_hi, int32_t Hq,
+                            float scale, float* partial_out, float* partial_lse, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * cp_prefill_attn_static -- cp_prefill_attn for callers that must not allocate device memory.
  * (The paper has no counterpart to this call; it exists for integration reasons only.)

@@ -20,7 +20,7 @@ CP_ERR_INVALID_ARG, CP_ERR_UNSUPPORTED, CP_ERR_WORKSPACE, CP_ERR_CUDA, CP_ERR_TI
 CP_DTYPE_BF16, CP_DTYPE_F32 = 0, 1
 
 EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "cp_ctx_poll_status", "cp_ctx_selftest_wait_expiry", "cp_plan",
-           "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_chunk", "cp_prefill_attn_static", "cp_merge",
+           "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_chunk", "cp_prefill_attn_kvrange", "cp_prefill_attn_static", "cp_merge",
            "cp_kv_gather", "cp_kv_append"]
 
 
@@ -202,6 +202,16 @@ def cp_prefill_attn_chunk(ctx, q_chunk, cache, page_table, prefix_len, new_len, 
         ctypes.c_int64(new_len), ctypes.c_int32(C), ctypes.c_int32(chunk), ctypes.c_int32(Hq), ctypes.c_float(scale),
         _ptr(out_chunk), _ptr(lse_chunk), _ptr(workspace),
         ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
+
+
+def cp_prefill_attn_kvrange(ctx, q, cache, page_table, prefix_len, new_len, kv_lo, kv_hi, Hq, scale, partial_out,
+                            partial_lse, workspace, stream=None):
+    """All R queries against keys at absolute positions [kv_lo, kv_hi) only: fp32 partial + LSE for cp_merge."""
+    _check(load().cp_prefill_attn_kvrange(
+        ctx._h, _ptr(q), ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(prefix_len), ctypes.c_int64(new_len),
+        ctypes.c_int64(kv_lo), ctypes.c_int64(kv_hi), ctypes.c_int32(Hq), ctypes.c_float(scale), _ptr(partial_out),
+        _ptr(partial_lse), _ptr(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+        _stream(stream)))
 
 
 def cp_prefill_attn_static(q, cache, page_table, prefix_len, new_len, C, Hq, scale, out, lse, stream=None):

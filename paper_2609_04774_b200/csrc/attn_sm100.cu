@@ -348,6 +348,9 @@ __device__ __forceinline__ bool fetch_unit(const AttnParams& p, int round, UnitI
         u.t_end = u.it.n_kv_tiles;
         u.slot = -1;
     }
+    const int t0 = u.it.kv_lo >> 7;      // first KV tile of the unit's key range (0 for the ordinary calls)
+    u.t_begin += t0;
+    u.t_end += t0;
     u.head0 = p.heads_per_unit * pair;
     u.kv_head = u.head0 / p.group;
     return true;
@@ -549,10 +552,10 @@ __device__ __forceinline__ void max32(const float (&s)[32], float& a0, float& a1
     }
 }
 // Columns at or beyond `lim` are above the causal diagonal for this row.
-__device__ __forceinline__ void mask32(float (&s)[32], int lim) {
+__device__ __forceinline__ void mask32(float (&s)[32], int lo, int lim) {
 #pragma unroll
     for (int i = 0; i < 32; ++i)
-        if (i >= lim) s[i] = -INFINITY;
+        if (i >= lim || i < lo) s[i] = -INFINITY;
 }
 // p = 2^(s*c - m) for 32 keys -> 16 packed bf16 pairs; row sums into four accumulators.  With kPoly,
 // kPolyOf4 of every four pairs take the FMA-pipe polynomial instead of MUFU; masked tiles do not (the
@@ -614,18 +617,19 @@ __device__ __forceinline__ void release_s(uint32_t bars) {
 // so the load runs under the last exponentials), the rest -- or all of it, after a wait -- behind the
 // last piece.  The S buffer goes back to the score issuer as soon as the loads have landed.
 // Straight-line code in both variants, no per-element branches.
-// kMasked: the tile reaches past the causal diagonal of some rows; `lim` = visible columns of this row.
+// kMasked: some keys of the tile are hidden from some rows (causal diagonal, or the edge of the unit's key
+// range); this row sees columns [lo, lim).
 template <bool kMasked>
 __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], float (&c2)[32], float (&c3)[32],
                                              bool more, uint32_t& s_par, uint32_t s_tmem, uint32_t p_tmem,
-                                             uint32_t o_tmem, uint32_t p_bar0, float c, int lim, bool first,
+                                             uint32_t o_tmem, uint32_t p_bar0, float c, int lo, int lim, bool first,
                                              float& m, float& l, const SoftmaxSync& sy) {
     if (sy.tr) sy.tr[1] = clock64();
     if (kMasked) {
-        mask32(c0, lim);
-        mask32(c1, lim - 32);
-        mask32(c2, lim - 64);
-        mask32(c3, lim - 96);
+        mask32(c0, lo, lim);
+        mask32(c1, lo - 32, lim - 32);
+        mask32(c2, lo - 64, lim - 64);
+        mask32(c3, lo - 96, lim - 96);
     }
     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
     max32(c0, mx0, mx1, mx2, mx3);
@@ -743,8 +747,10 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
         const int head = u.head0 + wg;
         float m = -INFINITY;   // running row max in log2 units (possibly stale by < threshold)
         float l = 0.f;         // running row sum of 2^(s - m)
-        // tiles below n_full lie entirely under the causal diagonal of every row of the q-tile
-        const int n_full = u.it.kv_len0 / kBlockN;
+        // tiles below n_full lie entirely under the causal diagonal of every row of the q-tile and inside the
+        // unit's key range; the range's first tile is cut on the left when kv_lo is not a tile multiple
+        const int n_full = min(u.it.kv_len0, u.it.kv_hi) / kBlockN;
+        const int j_cut = (u.it.kv_lo & (kBlockN - 1)) ? (u.it.kv_lo >> 7) : -1;
         float s0[32], s1[32], s2[32], s3[32];   // the row's scores of the current tile
         // the first tile of the unit is loaded here, every later one by the tile before it
         SM_WAIT(kBarSReady + wg, s_par, u.t_begin);
@@ -758,12 +764,13 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
             if (tr) tr[0] = clock64();
             const SoftmaxSync sy = {bars, kBarSReady + (uint32_t)wg, kBarPvDone + (uint32_t)wg, (tile_cnt - 1) & 1,
                                     abort_flag, p.status, j, tr};
-            if (j < n_full)
-                softmax_tile<false>(s0, s1, s2, s3, j + 1 < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c, 0,
+            if (j < n_full && j != j_cut)
+                softmax_tile<false>(s0, s1, s2, s3, j + 1 < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c, 0, 0,
                                     j == u.t_begin, m, l, sy);
             else
                 softmax_tile<true>(s0, s1, s2, s3, j + 1 < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c,
-                                   u.it.kv_len0 + row - j * kBlockN, j == u.t_begin, m, l, sy);
+                                   u.it.kv_lo - j * kBlockN, min(u.it.kv_len0 + row, u.it.kv_hi) - j * kBlockN,
+                                   j == u.t_begin, m, l, sy);
             if (row == CPATTN_TRACE_ROW) { CP_TRACE(wg, j, 6); }
             ++tile_cnt;
         }
@@ -1046,8 +1053,8 @@ inline int64_t page_tokens_of(const cp_kv_cache* c) { return (c && c->page_size 
 
 int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table, int32_t B,
                 const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C, const int64_t* cu_pages,
-                int32_t only_shard, int32_t only_chunk, int32_t Hq, float scale, void* out, int out_f32, float* lse,
-                void* workspace, size_t workspace_bytes, void* stream, const char* who) {
+                int32_t only_shard, int32_t only_chunk, int64_t kv_lo, int64_t kv_hi, int32_t Hq, float scale, void* out,
+                int out_f32, float* lse, void* workspace, size_t workspace_bytes, void* stream, const char* who) {
     if (!ctx || !q || !page_table || !out || !lse || B < 1 || !cu_new || !prefix_len || !C || !cu_pages)
         return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or B < 1", who);
     if (int rc = validate_kv_cache(cache, who)) return rc;
@@ -1080,7 +1087,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
 
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
     Schedule sch;
-    build_tiles(B, cu_new, prefix_len, C, cu_pages, cache->page_size, only_shard, only_chunk, sch.items);
+    build_tiles(B, cu_new, prefix_len, C, cu_pages, cache->page_size, only_shard, only_chunk, kv_lo, kv_hi, sch.items);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (sch.items.empty()) return CP_OK;   // the shard owns no rows (only empty chunks)
     // rows of q / out / lse: the packed batch, or the one chunk of a chunk call
@@ -1166,8 +1173,8 @@ extern "C" int cp_prefill_attn_batch(cp_ctx* ctx, const void* q, const cp_kv_cac
                                      int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
                                      const int64_t* cu_pages, int32_t Hq, float scale, void* out, float* lse,
                                      void* workspace, size_t workspace_bytes, void* stream) {
-    return attn_common(ctx, q, cache, page_table, B, cu_new, prefix_len, C, cu_pages, -1, -1, Hq, scale, out, 0, lse,
-                       workspace, workspace_bytes, stream, "cp_prefill_attn_batch");
+    return attn_common(ctx, q, cache, page_table, B, cu_new, prefix_len, C, cu_pages, -1, -1, 0, INT32_MAX, Hq, scale, out, 0,
+                       lse, workspace, workspace_bytes, stream, "cp_prefill_attn_batch");
 }
 
 extern "C" int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
@@ -1177,8 +1184,8 @@ extern "C" int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* ca
         return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn: cache is NULL, new_len < 1 or prefix_len < 0");
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
-    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, Hq, scale, out, 0, lse,
-                       workspace, workspace_bytes, stream, "cp_prefill_attn");
+    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, 0, INT32_MAX, Hq, scale, out, 0,
+                       lse, workspace, workspace_bytes, stream, "cp_prefill_attn");
 }
 
 extern "C" int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
@@ -1198,8 +1205,33 @@ extern "C" int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cac
     if (int rc = check_cuda(cudaGetLastError(), "fill_neg_inf launch")) return rc;
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
-    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, -1, Hq, scale, partial_out, 1,
-                       partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_shard");
+    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, -1, 0, INT32_MAX, Hq, scale,
+                       partial_out, 1, partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_shard");
+}
+
+extern "C" int cp_prefill_attn_kvrange(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
+                                       int64_t prefix_len, int64_t new_len, int64_t kv_lo, int64_t kv_hi, int32_t Hq,
+                                       float scale, float* partial_out, float* partial_lse, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+    if (!cache || new_len < 1 || prefix_len < 0 || !partial_out || !partial_lse || Hq < 1)
+        return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_kvrange: null pointer or bad sizes");
+    if (kv_lo < 0 || kv_hi < kv_lo || kv_lo > 0x7fffff00ll)
+        return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_kvrange: key range [%lld, %lld)", (long long)kv_lo, (long long)kv_hi);
+    if (!ctx) return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_kvrange: ctx is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+    // rows that see no key of the range: zeros with lse = -inf (the identity element of cp_merge)
+    if (int rc = check_cuda(cudaMemsetAsync(partial_out, 0, (size_t)new_len * Hq * kD * sizeof(float), s),
+                            "cudaMemsetAsync(partial_out)")) return rc;
+    const int64_t n_lse = new_len * Hq;
+    fill_neg_inf_kernel<<<(int)std::min<int64_t>((n_lse + 255) / 256, 4096), 256, 0, s>>>(partial_lse, n_lse);
+    if (int rc = check_cuda(cudaGetLastError(), "fill_neg_inf launch")) return rc;
+    const int64_t cu_new[2] = {0, new_len};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
+    const int32_t C = 1;
+    return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, kv_lo,
+                       std::min<int64_t>(kv_hi, INT32_MAX), Hq, scale, partial_out, 1, partial_lse, workspace,
+                       workspace_bytes, stream, "cp_prefill_attn_kvrange");
 }
 
 extern "C" int cp_ctx_selftest_wait_expiry(cp_ctx* ctx, void* stream) {
@@ -1217,8 +1249,8 @@ extern "C" int cp_prefill_attn_chunk(cp_ctx* ctx, const void* q_chunk, const cp_
         return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_chunk: bad sizes or chunk %d not in [0, %d)", chunk, 2 * C);
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
-    return attn_common(ctx, q_chunk, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, chunk, Hq, scale,
-                       out_chunk, 0, lse_chunk, workspace, workspace_bytes, stream, "cp_prefill_attn_chunk");
+    return attn_common(ctx, q_chunk, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, chunk, 0, INT32_MAX, Hq,
+                       scale, out_chunk, 0, lse_chunk, workspace, workspace_bytes, stream, "cp_prefill_attn_chunk");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1302,7 +1334,7 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
     std::vector<TileItem> tiles;
-    build_tiles(1, cu_new, &prefix_len, &C, cu_pages, cache->page_size, -1, -1, tiles);
+    build_tiles(1, cu_new, &prefix_len, &C, cu_pages, cache->page_size, -1, -1, 0, INT32_MAX, tiles);
     cp_ctx enc{};                       // only the encoder entry point is read by encode_maps
     enc.encode_tiled = st->encode_tiled;
     CUtensorMap tmQ, tmK, tmV;

@@ -20,9 +20,9 @@ struct TileItem {
     int32_t kv_len0;    // keys visible to the first row: P + r0 + 1 (row i sees kv_len0 + i)
     int32_t pt_base;    // offset of the request's page table in the packed page table
     int32_t n_pages;    // entries of that page table
-    int32_t n_kv_tiles; // ceil((kv_len0 + n_rows - 1) / 128)
-    int32_t request;
-    int32_t shard;
+    int32_t n_kv_tiles; // KV tiles the unit walks: 128-key tiles from kv_lo / 128 up to its last visible key
+    int32_t kv_lo;      // keys the unit may attend: absolute positions [kv_lo, kv_hi), cut by the causal
+    int32_t kv_hi;      // limit; [0, INT32_MAX) for the ordinary calls
 };
 static_assert(sizeof(TileItem) == 32, "TileItem layout");
 
@@ -92,9 +92,11 @@ int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C);
 // Builds the tile list of a batch, cut at the chunk boundaries of every request's zigzag plan and
 // sorted longest first.  only_shard < 0 keeps all shards; only_chunk >= 0 (B == 1) keeps that one zigzag
 // chunk and numbers its rows from the chunk's first row (q, out and lse then hold the chunk alone).
+// [kv_lo, kv_hi) restricts the keys (absolute positions); tiles that see none of them are left out.
 int validate_kv_cache(const cp_kv_cache* c, const char* who);
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
-                const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, std::vector<TileItem>& out);
+                const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, int64_t kv_lo,
+                int64_t kv_hi, std::vector<TileItem>& out);
 // Distributes the (tile, head pair) units of s.items over `grid_max` CTAs (pairs_per_kv = units of one KV
 // head per tile): whole units, KV head by KV head and longest first within a head,
 // onto the least loaded CTA while they fit under the per-CTA share, the rest cut into KV ranges that

@@ -31,7 +31,8 @@ int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C) {
 }
 
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
-                const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, std::vector<TileItem>& out) {
+                const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, int64_t kv_lo,
+                int64_t kv_hi, std::vector<TileItem>& out) {
     out.clear();
     for (int32_t b = 0; b < B; ++b) {
         const int64_t R = cu_new[b + 1] - cu_new[b];
@@ -53,9 +54,13 @@ int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, con
                 t.pt_base = (int32_t)cu_pages[b];
                 // entries the request really uses; a single chunk reads none behind its last key
                 t.n_pages = (int32_t)((P + (only_chunk >= 0 ? ce : R) + page_size - 1) / page_size);
-                t.n_kv_tiles = (int32_t)((t.kv_len0 + t.n_rows - 1 + kTileRows - 1) / kTileRows);
-                t.request = b;
-                t.shard = shard;
+                // keys the tile's last row sees, cut to the allowed range; tiles that see none are left out
+                const int64_t hi = std::min<int64_t>(kv_hi, (int64_t)t.kv_len0 + t.n_rows - 1);
+                const int64_t t_lo = kv_lo / kTileRows, t_hi = (hi + kTileRows - 1) / kTileRows;
+                if (t_hi <= t_lo) continue;
+                t.n_kv_tiles = (int32_t)(t_hi - t_lo);
+                t.kv_lo = (int32_t)kv_lo;
+                t.kv_hi = (int32_t)std::min<int64_t>(kv_hi, INT32_MAX);
                 out.push_back(t);
             }
         }
@@ -257,7 +262,7 @@ extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64
         cu_pages[b + 1] = cu_pages[b] + (prefix_len[b] + R + kDefaultPageTokens - 1) / kDefaultPageTokens;
     }
     Schedule sch;
-    build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), kDefaultPageTokens, -1, -1, sch.items);
+    build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), kDefaultPageTokens, -1, -1, 0, INT32_MAX, sch.items);
     if (int rc = build_schedule(Hq / heads_per_unit, kv_major_pairs(B, cu_new, prefix_len, Hkv, (Hq / Hkv) / heads_per_unit),
                                 num_sms, sch)) return rc;
     int64_t max_load = 0, min_load = INT64_MAX, total = 0;

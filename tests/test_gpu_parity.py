@@ -256,6 +256,48 @@ def test_shard_partials_merge_to_full(ctx):
     assert np.abs(bf16_to_f64(merged) - out_full).max() <= 2.0 ** -7 * max(1.0, np.abs(out_full).max())
 
 
+def test_key_range_partials_match_oracle_and_merge_to_full(ctx):
+    # the keys of a request cut into disjoint absolute ranges with unaligned edges (inside the prefix, across
+    # the prefix / suffix border, inside the suffix, an empty one): every partial against the oracle restricted
+    # to the same keys; all of them through cp_merge against full attention
+    w = wl.Workload("kvrange", 46, 8, 2, [wl.Request(700, 1000, 1)])
+    mat = wl.materialize(w)
+    dev = DeviceWorkload(mat)
+    r = w.requests[0]
+    R, P, L = r.new_len, r.prefix_len, r.total_len
+    edges = [0, 130, 640, 1000, 1000, 1217, 1536, L]
+    parts = torch.empty((len(edges) - 1, R, w.Hq, w.D), dtype=torch.float32, device="cuda")
+    lses = torch.empty((len(edges) - 1, w.Hq, R), dtype=torch.float32, device="cuda")
+    rows = np.unique(np.concatenate([np.arange(0, 40), np.arange(200, 240), np.arange(R - 40, R), [217, 218, 535, 536]]))
+    for n, (lo, hi) in enumerate(zip(edges, edges[1:])):
+        parts[n].fill_(float("nan"))
+        lses[n].fill_(float("nan"))
+        binding.cp_prefill_attn_kvrange(ctx, dev.q, dev.cache, dev.page_table, P, R, lo, hi, w.Hq, w.scale, parts[n],
+                                        lses[n], dev.ws)
+        torch.cuda.synchronize()
+        ctx.poll_status()
+        assert not bool(torch.isnan(parts[n]).any()) and not bool(torch.isnan(lses[n]).any())
+        ref_o, ref_l = orc.attn_rows(mat.q, mat.k_pages, mat.v_pages, mat.page_table, P, w.Hkv, w.scale, rows,
+                                     key_ranges=[(lo, hi)])
+        o = parts[n][rows].cpu().numpy().astype(np.float64)
+        l = lses[n][:, rows].cpu().numpy().astype(np.float64)
+        seen = np.isfinite(ref_l)                         # rows (per head) that see a key of the range
+        assert np.array_equal(np.isneginf(l), ~seen), (lo, hi)
+        assert (o[~seen.T] == 0).all()
+        if seen.any():
+            assert np.abs(o - np.nan_to_num(ref_o)).max() <= 2e-2, (lo, hi)
+            assert (np.abs(l[seen] - ref_l[seen]) / np.maximum(1.0, np.abs(ref_l[seen]))).max() <= 1e-3, (lo, hi)
+    out = torch.empty((R, w.Hq, w.D), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((w.Hq, R), dtype=torch.float32, device="cuda")
+    binding.cp_merge(ctx, parts, lses, out, lse)
+    torch.cuda.synchronize()
+    ref_o, ref_l = oracle_request(mat, 0)
+    compare(bf16_to_f64(out), lse.cpu().numpy().astype(np.float64), ref_o, ref_l, "merged key ranges")
+    with pytest.raises(binding.CpError):
+        binding.cp_prefill_attn_kvrange(ctx, dev.q, dev.cache, dev.page_table, P, R, 10, 5, w.Hq, w.scale, parts[0],
+                                        lses[0], dev.ws)
+
+
 def test_argument_validation_launches_nothing(ctx):
     w = wl.Workload("val", 23, 8, 2, [wl.Request(64, 0, 1)])
     dev = DeviceWorkload(wl.materialize(w))
