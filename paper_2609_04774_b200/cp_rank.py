@@ -12,6 +12,12 @@ buffers and are written into this rank's own paged cache by cp_kv_append; attent
 through cp_prefill_attn_chunk.  Remote data is therefore always copied into local HBM before a kernel
 reads it.  The module holds no arithmetic of the method: it moves rows and calls the library.
 
+A second mode, prefill_pass_q, keeps the K/V sharded (a rank holds its prefix block and the K/V of its own
+two chunks) and lets the queries travel: all-gather of Q, cp_prefill_attn_kvrange over each of the rank's key
+ranges, a local cp_merge of those partials, an all-to-all that returns every row's partials to the rank that
+owns the row, and a final cp_merge over the C partials.  It moves R*Hq*D query bytes plus fp32 partials
+instead of (P+R)*Hkv*D*2 key/value bytes, which pays when the cached prefix is much longer than the suffix.
+
 Readings (the paper fixes none of these): prefix pages are owned in contiguous blocks of
 ceil(n_prefix_pages / C) pages, block r on rank r; the prefix length is a multiple of the page size
 (block-granular reuse, Section 6); chunks are padded to cl = ceil(R / 2C) rows for the collective.
@@ -92,6 +98,26 @@ class TorchComm:
         return out, work
 
 
+    def all_to_all(self, blocks):
+        """blocks [size, n, ...]: block d goes to rank d.  -> (out [size, n, ...] with out[s] = the block rank s
+        sent here, handle)."""
+        import torch
+        if self.dist.get_backend(self.group) == "gloo":
+            # gloo has no all-to-all: gather everything and keep this rank's blocks (CPU test path only)
+            gathered, work = self.all_gather(blocks)
+            work.wait()
+
+            class _Done:
+                def wait(self):
+                    return True
+            return gathered[:, self.rank].contiguous(), _Done()
+        out = torch.empty_like(blocks)
+        src = blocks.contiguous().view(torch.uint8).reshape(self.size, -1)
+        dst = out.view(torch.uint8).reshape(self.size, -1)
+        work = self.dist.all_to_all(list(dst.unbind(0)), list(src.unbind(0)), group=self.group, async_op=True)
+        return out, work
+
+
 class LibraryOps:
     """The three device steps of a rank, on this rank's paged cache, through the C-ABI library."""
 
@@ -129,6 +155,40 @@ class LibraryOps:
         self.b.cp_prefill_attn_chunk(self.ctx, q_chunk, self.cache, self.page_table, lay.P, lay.R, lay.C, chunk,
                                      self.Hq, self.scale, out, lse, self._ws)
         return out, lse
+
+
+def _library_extras():
+    """Methods of LibraryOps used by the pass-Q mode (kept together; bound below)."""
+
+    def attn_kvrange(self, lay, q_full, lo, hi):
+        torch = self.torch
+        R = lay.R
+        part = torch.empty((R, self.Hq, self.D), dtype=torch.float32, device=self.device)
+        lse = torch.empty((self.Hq, R), dtype=torch.float32, device=self.device)
+        if self._ws is None:
+            nbytes = self.b.cp_workspace_bytes([lay.R], [lay.C], self.Hq)
+            self._ws = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        self.b.cp_prefill_attn_kvrange(self.ctx, q_full, self.cache, self.page_table, lay.P, R, lo, hi, self.Hq,
+                                       self.scale, part, lse, self._ws)
+        return part, lse
+
+    def merge(self, parts, lses, final):
+        """parts [N, T, Hq, D] fp32, lses [N, Hq, T] -> (out [T, Hq, D] bf16 if final else fp32, lse [Hq, T])."""
+        torch = self.torch
+        T = parts.shape[1]
+        out = torch.empty((T, self.Hq, self.D), dtype=torch.bfloat16 if final else torch.float32, device=self.device)
+        lse = torch.empty((self.Hq, T), dtype=torch.float32, device=self.device)
+        if T:
+            self.b.cp_merge(self.ctx, parts.contiguous(), lses.contiguous(), out, lse)
+        return out, lse
+
+    def empty_f32(self, shape):
+        return self.torch.zeros(tuple(shape), dtype=self.torch.float32, device=self.device)
+
+    LibraryOps.attn_kvrange, LibraryOps.merge, LibraryOps.empty_f32 = attn_kvrange, merge, empty_f32
+
+
+_library_extras()
 
 
 def _padded(ops, rows, n):
@@ -197,3 +257,60 @@ class CpRankWorker:
             ops.kv_append(lay.P + b, e - b, gk[r], gv[r])
         out_l, lse_l = ops.attn_chunk(lay, lay.late, q_late)
         return out_e, lse_e, out_l, lse_l
+
+    def prefill_pass_q(self, q_early, q_late, k_early, v_early, k_late, v_late):
+        """Same inputs and outputs as prefill(), but the K/V never leaves its rank: the rank's cache must hold
+        its prefix block; its own chunks' K/V are appended here, nothing else is ever read from the cache."""
+        lay, ops, comm = self.lay, self.ops, self.comm
+        (eb, ee), (lb, le) = lay.chunk(lay.early), lay.chunk(lay.late)
+        assert q_early.shape[0] == ee - eb == k_early.shape[0] and q_late.shape[0] == le - lb == k_late.shape[0]
+        Hq = q_early.shape[1]
+
+        # 1. queries travel: both chunks of every rank, padded to cl rows
+        (ge, he), (gl, hl) = comm.all_gather(_padded(ops, q_early, lay.cl)), comm.all_gather(_padded(ops, q_late, lay.cl))
+        # 2. meanwhile the own new K/V goes into the own cache
+        ops.kv_append(lay.P + eb, ee - eb, k_early, v_early)
+        ops.kv_append(lay.P + lb, le - lb, k_late, v_late)
+        he.wait()
+        hl.wait()
+        q_full = ops.empty_rows(lay.R, Hq)
+        n_first = min(lay.R, lay.C * lay.cl)
+        q_full[:n_first] = ge.reshape((-1,) + tuple(ge.shape[2:]))[:n_first]
+        for r in range(lay.C):
+            b, e = lay.chunk(lay.late_chunk_of(r))
+            q_full[b:e] = gl[r][:e - b]
+
+        # 3. partial attention of all queries over each of the rank's key ranges, merged locally
+        pb, pe = lay.prefix_block(lay.rank)
+        ranges = [(lo, hi) for lo, hi in ((pb, pe), (lay.P + eb, lay.P + ee), (lay.P + lb, lay.P + le)) if hi > lo]
+        parts = [ops.attn_kvrange(lay, q_full, lo, hi) for lo, hi in ranges]
+        if len(parts) == 1:
+            mine_o, mine_l = parts[0]
+        elif parts:
+            mine_o, mine_l = ops.merge(_stack([p for p, _ in parts]), _stack([l for _, l in parts]), final=False)
+        else:                                   # the rank holds no key at all (more ranks than blocks and chunks)
+            mine_o = ops.empty_f32((lay.R, Hq, ops.D))
+            mine_l = ops.empty_f32((Hq, lay.R)) - float("inf")
+
+        # 4. every row's partial goes back to the rank that owns the row: block d = chunk d, then chunk 2C-1-d
+        send_o = ops.empty_f32((lay.C, 2 * lay.cl, Hq, ops.D))
+        send_l = ops.empty_f32((lay.C, Hq, 2 * lay.cl)) - float("inf")
+        for d in range(lay.C):
+            for half, j in enumerate((d, lay.late_chunk_of(d))):
+                b, e = lay.chunk(j)
+                send_o[d, half * lay.cl:half * lay.cl + e - b] = mine_o[b:e]
+                send_l[d, :, half * lay.cl:half * lay.cl + e - b] = mine_l[:, b:e]
+        (ro, ho), (rl, hl2) = comm.all_to_all(send_o), comm.all_to_all(send_l)
+        ho.wait()
+        hl2.wait()
+
+        # 5. the C partials of the own rows (each over a disjoint part of the keys) merge into the result
+        out, lse = ops.merge(ro, rl, final=True)
+        n_e, n_l = ee - eb, le - lb
+        return out[:n_e], lse[:, :n_e], out[lay.cl:lay.cl + n_l], lse[:, lay.cl:lay.cl + n_l]
+
+
+def _stack(tensors):
+    """Stack along a new first axis (torch.stack for tensors, the same for the test doubles' arrays)."""
+    import torch
+    return torch.stack(list(tensors), 0)

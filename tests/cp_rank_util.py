@@ -32,6 +32,11 @@ class ThreadComm:
         self.fabric, self.rank, self.size = fabric, rank, fabric.size
         self.calls = 0
 
+    def all_to_all(self, blocks):
+        # every rank's [size, n, ...] blocks meet; rank r takes block r of each
+        gathered, done = self.all_gather(blocks)
+        return gathered[:, self.rank].contiguous(), done
+
     def all_gather(self, block):
         f, n = self.fabric, self.calls
         self.calls += 1
@@ -75,6 +80,24 @@ class OracleOps:
         if e == b:
             return np.zeros((0, self.Hq, self.D)), np.zeros((self.Hq, 0))
         return orc.attn_rows(q, self.k_pages, self.v_pages, self.page_table, lay.P, self.Hkv, self.scale, np.arange(b, e))
+
+
+    # ---- pass-Q mode: partial attention over a key range, LSE merge (fp64 torch tensors) ----
+    def attn_kvrange(self, lay, q_full, lo, hi):
+        o, l = orc.attn_rows(self._bits(q_full), self.k_pages, self.v_pages, self.page_table, lay.P, self.Hkv, self.scale,
+                             np.arange(lay.R), key_ranges=[(lo, hi)])
+        dead = ~np.isfinite(l)                                   # [Hq, R]: rows that see no key of the range
+        o = np.where(dead.T[:, :, None], 0.0, o)
+        return torch.from_numpy(o), torch.from_numpy(np.where(dead, -np.inf, l))
+
+    def merge(self, parts, lses, final):
+        if parts.shape[1] == 0:
+            return torch.zeros(parts.shape[1:], dtype=torch.float64), torch.zeros(lses.shape[1:], dtype=torch.float64)
+        o, l = orc.merge(parts.numpy(), lses.numpy())
+        return torch.from_numpy(o), torch.from_numpy(l)
+
+    def empty_f32(self, shape):
+        return torch.zeros(tuple(shape), dtype=torch.float64)
 
 
 def rank_inputs(mat, lay, seed):

@@ -43,17 +43,19 @@ def test_layout_rejects_bad_arguments():
         RankLayout(10, 0, 2, 2)
 
 
-def _run_rank(w, mat, lay, comm, seed, result):
+def _run_rank(w, mat, lay, comm, seed, result, pass_q=False):
     from cp_rank_util import OracleOps, rank_inputs
     k_pages, v_pages, page_table, rows = rank_inputs(mat, lay, seed)
     ops = OracleOps(k_pages, v_pages, page_table, w.Hq, w.scale)
     t = {k: torch.from_numpy(np.ascontiguousarray(v).view(np.int16)) for k, v in rows.items()}
     worker = CpRankWorker(lay, comm, ops)
-    out_e, lse_e, out_l, lse_l = worker.prefill(t["q_early"], t["q_late"], t["k_early"], t["v_early"], t["k_late"], t["v_late"])
-    result[lay.rank] = (out_e, lse_e, out_l, lse_l, k_pages, v_pages, page_table)
+    run = worker.prefill_pass_q if pass_q else worker.prefill
+    out_e, lse_e, out_l, lse_l = run(t["q_early"], t["q_late"], t["k_early"], t["v_early"], t["k_late"], t["v_late"])
+    as_np = lambda x: x.numpy() if isinstance(x, torch.Tensor) else x
+    result[lay.rank] = (as_np(out_e), as_np(lse_e), as_np(out_l), as_np(lse_l), k_pages, v_pages, page_table)
 
 
-def _check_rank(w, mat, lay, res):
+def _check_rank(w, mat, lay, res, pass_q=False):
     out_e, lse_e, out_l, lse_l, k_pages, v_pages, page_table = res
     r = w.requests[0]
     ref_o, ref_l = orc.attn_full(mat.q, mat.k_pages, mat.v_pages, mat.page_table, r.prefix_len, w.Hkv, w.scale)
@@ -62,14 +64,27 @@ def _check_rank(w, mat, lay, res):
         assert o.shape[0] == e - b
         if e > b:
             assert np.abs(o - ref_o[b:e]).max() < 1e-12 and np.abs(l - ref_l[:, b:e]).max() < 1e-12
+    if pass_q:
+        # K/V stayed sharded: the rank's cache holds its prefix block and its own chunks, nothing else
+        own = np.zeros(r.prefix_len + r.new_len, dtype=bool)
+        pb, pe = lay.prefix_block(lay.rank)
+        own[pb:pe] = True
+        for j in (lay.early, lay.late):
+            b, e = lay.chunk(j)
+            own[r.prefix_len + b:r.prefix_len + e] = True
+        got = orc.kv_gather(k_pages, page_table, 0, own.size)
+        ref = orc.kv_gather(mat.k_pages, mat.page_table, 0, own.size)
+        assert np.array_equal(got[own], ref[own]) and not got[~own].any()
+        return
     # after the exchange the rank's own cache holds every token of the request, bit for bit
     L = r.prefix_len + r.new_len
     assert np.array_equal(orc.kv_gather(k_pages, page_table, 0, L), orc.kv_gather(mat.k_pages, mat.page_table, 0, L))
     assert np.array_equal(orc.kv_gather(v_pages, page_table, 0, L), orc.kv_gather(mat.v_pages, mat.page_table, 0, L))
 
 
+@pytest.mark.parametrize("pass_q", [False, True])
 @pytest.mark.parametrize("R,P,C", [(333, 192, 4), (5, 0, 4), (200, 320, 3)])
-def test_four_ranks_in_process(R, P, C):
+def test_four_ranks_in_process(R, P, C, pass_q):
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     from cp_rank_util import ThreadFabric
     w = wl.Workload("cp_rank", 51, 4, 2, [wl.Request(R, P, C)])
@@ -79,7 +94,7 @@ def test_four_ranks_in_process(R, P, C):
 
     def body(k):
         try:
-            _run_rank(w, mat, RankLayout(R, P, C, k), fabric.comm(k), 51, result)
+            _run_rank(w, mat, RankLayout(R, P, C, k), fabric.comm(k), 51, result, pass_q)
         except Exception as e:               # a failing rank must not leave the others at the barrier
             errors.append(e)
             fabric.barrier.abort()
@@ -91,7 +106,7 @@ def test_four_ranks_in_process(R, P, C):
         t.join(timeout=300)
     assert not errors, errors
     for k in range(C):
-        _check_rank(w, mat, RankLayout(R, P, C, k), result[k])
+        _check_rank(w, mat, RankLayout(R, P, C, k), result[k], pass_q)
 
 
 def _free_port():
@@ -116,6 +131,9 @@ def _gloo_rank(rank, world, port, q):
         result = {}
         _run_rank(w, mat, lay, TorchComm(), 52, result)
         _check_rank(w, mat, lay, result[rank])
+        result = {}
+        _run_rank(w, mat, lay, TorchComm(), 52, result, pass_q=True)
+        _check_rank(w, mat, lay, result[rank], pass_q=True)
         q.put((rank, "ok"))
     except Exception as e:
         q.put((rank, repr(e)))

@@ -62,7 +62,7 @@ def test_chunk_entry_point_matches_oracle_rows():
         binding.cp_prefill_attn_chunk(ctx, q, cache, pt, r.prefix_len, r.new_len, r.C, 2 * r.C, w.Hq, w.scale, out, lse, ws)
 
 
-def _rank_on_gpu(w, mat, lay, comm, seed, result):
+def _rank_on_gpu(w, mat, lay, comm, seed, result, pass_q=False):
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     from cp_rank_util import rank_inputs
     from paper_2609_04774_b200 import binding
@@ -71,13 +71,15 @@ def _rank_on_gpu(w, mat, lay, comm, seed, result):
     k_pages, v_pages, page_table, rows = rank_inputs(mat, lay, seed)
     ops = LibraryOps(binding.Context(0), _dev(k_pages), _dev(v_pages), torch.from_numpy(page_table).cuda(), w.Hq, w.scale)
     t = {k: _dev(x) for k, x in rows.items()}
-    out = CpRankWorker(lay, comm, ops).prefill(t["q_early"], t["q_late"], t["k_early"], t["v_early"], t["k_late"], t["v_late"])
+    worker = CpRankWorker(lay, comm, ops)
+    run = worker.prefill_pass_q if pass_q else worker.prefill
+    out = run(t["q_early"], t["q_late"], t["k_early"], t["v_early"], t["k_late"], t["v_late"])
     torch.cuda.synchronize()
     ops.ctx.poll_status()
     result[lay.rank] = out + (ops.k_pages, ops.v_pages, page_table)
 
 
-def _check_rank_on_gpu(w, mat, lay, res, ref):
+def _check_rank_on_gpu(w, mat, lay, res, ref, pass_q=False):
     out_e, lse_e, out_l, lse_l, k_pages, v_pages, page_table = res
     r = w.requests[0]
     for j, o, l in ((lay.early, out_e, lse_e), (lay.late, out_l, lse_l)):
@@ -85,14 +87,17 @@ def _check_rank_on_gpu(w, mat, lay, res, ref):
         assert o.shape[0] == e - b
         if e > b:
             _compare(o, l, ref[0][b:e], ref[1][:, b:e], "rank %d chunk %d" % (lay.rank, j))
+    if pass_q:
+        return                                   # K/V stays sharded in this mode: nothing more to find in the cache
     L = r.prefix_len + r.new_len
     for dev_pages, ref_pages in ((k_pages, mat.k_pages), (v_pages, mat.v_pages)):
         got = dev_pages.view(torch.int16).cpu().numpy().view(np.uint16)
         assert np.array_equal(orc.kv_gather(got, page_table, 0, L), orc.kv_gather(ref_pages, mat.page_table, 0, L))
 
 
+@pytest.mark.parametrize("pass_q", [False, True])
 @pytest.mark.parametrize("R,P,C", [(1500, 640, 4), (333, 192, 3), (5, 0, 4)])
-def test_ranks_as_threads_on_one_gpu(R, P, C):
+def test_ranks_as_threads_on_one_gpu(R, P, C, pass_q):
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     from cp_rank_util import ThreadFabric
     from paper_2609_04774_b200.cp_rank import RankLayout
@@ -104,7 +109,7 @@ def test_ranks_as_threads_on_one_gpu(R, P, C):
 
     def body(k):
         try:
-            _rank_on_gpu(w, mat, RankLayout(R, P, C, k), fabric.comm(k), 62, result)
+            _rank_on_gpu(w, mat, RankLayout(R, P, C, k), fabric.comm(k), 62, result, pass_q)
         except Exception as e:
             errors.append(e)
             fabric.barrier.abort()
@@ -116,7 +121,7 @@ def test_ranks_as_threads_on_one_gpu(R, P, C):
         t.join(timeout=600)
     assert not errors, errors
     for k in range(C):
-        _check_rank_on_gpu(w, mat, RankLayout(R, P, C, k), result[k], ref)
+        _check_rank_on_gpu(w, mat, RankLayout(R, P, C, k), result[k], ref, pass_q)
 
 
 def _nccl_single_rank(port, q):
@@ -136,6 +141,9 @@ def _nccl_single_rank(port, q):
         result = {}
         _rank_on_gpu(w, mat, lay, TorchComm(), 63, result)
         _check_rank_on_gpu(w, mat, lay, result[0], ref)
+        result = {}
+        _rank_on_gpu(w, mat, lay, TorchComm(), 63, result, pass_q=True)          # NCCL all-to-all at world size 1
+        _check_rank_on_gpu(w, mat, lay, result[0], ref, pass_q=True)
         q.put("ok")
     except Exception as e:
         q.put(repr(e))
