@@ -616,6 +616,9 @@ class _LoopbackComm:
     def all_gather(self, block):
         return block.unsqueeze(0).expand((self.size,) + tuple(block.shape)).contiguous(), self._Done()
 
+    def all_to_all(self, blocks):
+        return blocks.clone(), self._Done()
+
 
 def run_cprank(args, out):
     """Local time of every rank of a degree-C CP worker (early-chunk-first order): own prefix block read
@@ -648,8 +651,8 @@ def run_cprank(args, out):
                 rows["k_" + name] = torch.randn((e - b, w.Hkv, D), device="cuda").to(torch.bfloat16)
                 rows["v_" + name] = torch.randn((e - b, w.Hkv, D), device="cuda").to(torch.bfloat16)
             worker = CpRankWorker(lay, _LoopbackComm(C, rank), ops)
-            fn = lambda: worker.prefill(rows["q_early"], rows["q_late"], rows["k_early"], rows["v_early"],
-                                        rows["k_late"], rows["v_late"])
+            run = worker.prefill_pass_q if args.pass_q else worker.prefill
+            fn = lambda: run(rows["q_early"], rows["q_late"], rows["k_early"], rows["v_early"], rows["k_late"], rows["v_late"])
             ms = []
             for i in range(2 + args.rank_reps):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -661,8 +664,12 @@ def run_cprank(args, out):
                     ms.append(e0.elapsed_time(e1))
             ops.ctx.poll_status()
             per_rank.append(statistics.median(ms))
-        recv = (C - 1) * 2 * 2 * w.Hkv * D * (RankLayout(R, P, C, 0).block_pages * wl.PAGE + 2 * RankLayout(R, P, C, 0).cl)
-        out.write(json.dumps({"mode": "cprank", "config": cfg, "workload": w.name, "R": R, "P": P, "C": C,
+        lay0 = RankLayout(R, P, C, 0)
+        if args.pass_q:   # queries in (bf16), partials of the own rows back (fp32 + lse)
+            recv = (C - 1) * 2 * lay0.cl * w.Hq * (D * 2 + D * 4 + 4)
+        else:             # K and V of the other ranks' prefix blocks and chunks
+            recv = (C - 1) * 2 * 2 * w.Hkv * D * (lay0.block_pages * wl.PAGE + 2 * lay0.cl)
+        out.write(json.dumps({"mode": "cprank", "exchange": "pass-q" if args.pass_q else "all-gather-kv", "config": cfg, "workload": w.name, "R": R, "P": P, "C": C,
                               "rank_local_ms": per_rank, "slowest_rank_ms": max(per_rank),
                               "tflops_per_gpu_slowest_rank": w.flops() / C / (max(per_rank) * 1e-3) / 1e12,
                               "nvlink_bytes_received_per_rank": recv,
@@ -734,6 +741,7 @@ def main():
     ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5],
                     help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P")
     ap.add_argument("--rank-reps", type=int, default=5)
+    ap.add_argument("--pass-q", action="store_true", help="cprank mode: K/V stays sharded, queries travel")
     ap.add_argument("--cache-requests", type=int, default=20000)
     ap.add_argument("--merge-T", type=int, nargs="*", default=[4096, 16384, 65536, 262144])
     ap.add_argument("--merge-reps", type=int, default=20)
