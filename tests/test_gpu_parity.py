@@ -396,3 +396,23 @@ def test_attention_config3_sampled(ctx):
     eo, el = orc.attn_rows(mat.q, mat.k_pages, mat.v_pages, mat.page_table, 0, w.Hkv, w.scale, edge[::3])
     compare(out[edge[::3]], lse[:, edge[::3]], eo, el, "cfg3 chunk edges")
     assert np.isfinite(lse).all() and np.isfinite(out).all()
+    # the LSE-merge invariant over ALL rows at full size: the C shard partials, each computed on its own,
+    # merge into the one-launch result (every row is owned by exactly one shard)
+    del out, lse
+    R = r.new_len
+    parts = torch.empty((r.C, R, w.Hq, w.D), dtype=torch.float32, device="cuda")
+    lses = torch.empty((r.C, w.Hq, R), dtype=torch.float32, device="cuda")
+    for k in range(r.C):
+        binding.cp_prefill_attn_shard(ctx, dev.q, dev.cache, dev.page_table, 0, R, r.C, k, w.Hq, w.scale, parts[k],
+                                      lses[k], dev.ws)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    assert bool((torch.isfinite(lses).sum(0) == 1).all())
+    merged = torch.empty((R, w.Hq, w.D), dtype=torch.bfloat16, device="cuda")
+    mlse = torch.empty((w.Hq, R), dtype=torch.float32, device="cuda")
+    binding.cp_merge(ctx, parts, lses, merged, mlse)
+    torch.cuda.synchronize()
+    del parts
+    diff = (merged.float() - dev.out.float()).abs()
+    assert float(diff.max()) <= 2e-2 and float(diff.mean()) <= 1e-4
+    assert float(((mlse - dev.lse).abs() / dev.lse.abs().clamp(min=1.0)).max()) <= 1e-3
