@@ -93,6 +93,7 @@ struct AttnParams {
     float* partial_o;          // [slots][2 heads][128 rows][128] fp32, normalised partial outputs
     float* partial_lse;        // [slots][2 heads][128 rows]
     int32_t pairs_per_tile;   // units per query tile: Hq / heads_per_unit
+    int32_t pairs_per_kv;     // implicit schedule: > 0 walks the units KV head by KV head (this many units per tile and KV head)
     int32_t heads_per_unit;   // 2: two query heads of one KV group share every K/V tile; 1: odd group size
     int32_t group;            // Hq / Hkv
     int32_t Hq;
@@ -341,8 +342,17 @@ __device__ __forceinline__ bool fetch_unit(const AttnParams& p, int round, UnitI
         const int64_t idx = (int64_t)round * g + c;
         const int64_t total = (int64_t)p.n_items * p.pairs_per_tile;
         if (idx >= total) return false;
-        item = (int)(idx / p.pairs_per_tile);
-        pair = (int)(idx - (int64_t)item * p.pairs_per_tile);
+        if (p.pairs_per_kv > 0) {
+            // KV head by KV head: all CTAs read one head's K/V at a time (a long context then stays in L2)
+            const int64_t per_head = (int64_t)p.n_items * p.pairs_per_kv;
+            const int g = (int)(idx / per_head);
+            const int64_t rem = idx - (int64_t)g * per_head;
+            item = (int)(rem / p.pairs_per_kv);
+            pair = g * p.pairs_per_kv + (int)(rem - (int64_t)item * p.pairs_per_kv);
+        } else {
+            item = (int)(idx / p.pairs_per_tile);
+            pair = (int)(idx - (int64_t)item * p.pairs_per_tile);
+        }
         u.it = p.items[item];
         u.t_begin = 0;
         u.t_end = u.it.n_kv_tiles;
@@ -1134,6 +1144,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.partial_o = reinterpret_cast<float*>(ws + lay.partial_o);
     p.partial_lse = reinterpret_cast<float*>(ws + lay.partial_lse);
     p.pairs_per_tile = Hq / heads_per_unit;
+    p.pairs_per_kv = 0;
     p.heads_per_unit = heads_per_unit;
     p.group = Hq / cache->Hkv;
     p.Hq = Hq;
@@ -1354,6 +1365,7 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     p.partial_o = nullptr;
     p.partial_lse = nullptr;
     p.pairs_per_tile = Hq / heads_per_unit;
+    p.pairs_per_kv = kv_major_pairs(1, cu_new, &prefix_len, cache->Hkv, (Hq / cache->Hkv) / heads_per_unit);
     p.heads_per_unit = heads_per_unit;
     p.group = Hq / cache->Hkv;
     p.Hq = Hq;
