@@ -298,6 +298,35 @@ def test_key_range_partials_match_oracle_and_merge_to_full(ctx):
                                         lses[0], dev.ws)
 
 
+@pytest.mark.parametrize("seed", range(2000, 2008))
+def test_random_key_ranges_merge_to_full(ctx, seed):
+    # a random request, its keys cut at random positions into 2..6 ranges, other page sizes included: the range
+    # partials merged by cp_merge against the oracle
+    u = wl.counter_uniform(seed, wl.TID_LEN, 0, 16)
+    R = 1 + int(u[0] * 1500)
+    P = int(u[1] * 6000) if u[2] < 0.8 else 0
+    page = [16, 32, 64, 128][int(u[3] * 4)]
+    heads = [(8, 2), (4, 4), (16, 2)][int(u[4] * 3)]
+    w = wl.Workload("kvr_%d" % seed, seed, heads[0], heads[1], [wl.Request(R, P, 1)], page=page)
+    mat = wl.materialize(w)
+    dev = DeviceWorkload(mat)
+    L = R + P
+    n_cuts = 1 + int(u[5] * 5)
+    edges = sorted({0, L} | {int(x * L) for x in u[6:6 + n_cuts]})
+    parts = torch.empty((len(edges) - 1, R, w.Hq, w.D), dtype=torch.float32, device="cuda")
+    lses = torch.empty((len(edges) - 1, w.Hq, R), dtype=torch.float32, device="cuda")
+    for n, (lo, hi) in enumerate(zip(edges, edges[1:])):
+        binding.cp_prefill_attn_kvrange(ctx, dev.q, dev.cache, dev.page_table, P, R, lo, hi, w.Hq, w.scale, parts[n],
+                                        lses[n], dev.ws)
+    out = torch.empty((R, w.Hq, w.D), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((w.Hq, R), dtype=torch.float32, device="cuda")
+    binding.cp_merge(ctx, parts, lses, out, lse)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ref_o, ref_l = oracle_request(mat, 0)
+    compare(bf16_to_f64(out), lse.cpu().numpy().astype(np.float64), ref_o, ref_l, "random key ranges %s" % edges)
+
+
 def test_argument_validation_launches_nothing(ctx):
     w = wl.Workload("val", 23, 8, 2, [wl.Request(64, 0, 1)])
     dev = DeviceWorkload(wl.materialize(w))
