@@ -58,6 +58,15 @@ int cp_ctx_create(cp_ctx** ctx, int device);
 int cp_ctx_destroy(cp_ctx* ctx);
 int cp_ctx_poll_status(cp_ctx* ctx, int32_t* detail /* host, 4 words or NULL */);
 
+/* cp_ctx_cache_schedule -- schedule reuse, off by default.  The layers of a model call the attention entry
+ * points with the same batch over and over (same lengths, C, head counts, page-table sizes; only q, the
+ * cache contents and out differ).  With reuse on, a call whose schedule-relevant arguments AND workspace are
+ * the previous call's skips the host-side scheduling and the upload and launches on the work lists already
+ * in the workspace (about 20-100 us of host time per call and one small kernel).  While it is on, the caller
+ * must not modify the workspace between such calls, nor hand it to another context.  Turning it on or off
+ * forgets the remembered schedule.  Errors: INVALID_ARG. */
+int cp_ctx_cache_schedule(cp_ctx* ctx, int enable);
+
 /* cp_ctx_selftest_wait_expiry -- diagnostic (the paper has no counterpart): enqueues one small block whose
  * only act is to wait, with a limit of about a millisecond, on a barrier that nothing arrives at.  It shows
  * on the device at hand that an expired wait ends the kernel normally and is reported: after the stream has

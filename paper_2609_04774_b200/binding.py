@@ -19,7 +19,7 @@ CP_OK = 0
 CP_ERR_INVALID_ARG, CP_ERR_UNSUPPORTED, CP_ERR_WORKSPACE, CP_ERR_CUDA, CP_ERR_TIMEOUT, CP_ERR_BOUNDS = -1, -2, -3, -4, -5, -6
 CP_DTYPE_BF16, CP_DTYPE_F32 = 0, 1
 
-EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "cp_ctx_poll_status", "cp_ctx_selftest_wait_expiry", "cp_plan",
+EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "cp_ctx_poll_status", "cp_ctx_cache_schedule", "cp_ctx_selftest_wait_expiry", "cp_plan",
            "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_chunk", "cp_prefill_attn_kvrange", "cp_prefill_attn_static", "cp_merge",
            "cp_kv_gather", "cp_kv_append"]
 
@@ -110,6 +110,10 @@ class Context:
             self.close()
         except Exception:
             pass
+
+    def cache_schedule(self, enable: bool):
+        """Reuse the work lists left in the workspace by the previous call when the next one has the same shape."""
+        _check(load().cp_ctx_cache_schedule(self._h, ctypes.c_int(1 if enable else 0)))
 
     def selftest_wait_expiry(self, stream=None):
         """Enqueue the bounded-wait self-test; the next poll_status() after a sync raises CP_ERR_TIMEOUT."""

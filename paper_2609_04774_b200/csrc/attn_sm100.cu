@@ -1096,41 +1096,76 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
                          workspace, workspace_bytes, need_ws);
 
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    Schedule sch;
-    build_tiles(B, cu_new, prefix_len, C, cu_pages, cache->page_size, only_shard, only_chunk, kv_lo, kv_hi, sch.items);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (sch.items.empty()) return CP_OK;   // the shard owns no rows (only empty chunks)
-    // rows of q / out / lse: the packed batch, or the one chunk of a chunk call
-    int64_t total_rows = cu_new[B];
-    if (only_chunk >= 0) {
-        total_rows = 0;
-        for (const TileItem& t : sch.items) total_rows = std::max<int64_t>(total_rows, (int64_t)t.q_row0 + t.n_rows);
-    }
     int grid_max = ctx->num_sms;
 #ifdef CPATTN_TRACE
     if (const char* e = getenv("CPATTN_DEBUG_SMS")) grid_max = std::max(1, atoi(e));   // trace builds only
 #endif
-    if (int rc = build_schedule(Hq / heads_per_unit,
-                                kv_major_pairs(B, cu_new, prefix_len, cache->Hkv, (Hq / cache->Hkv) / heads_per_unit),
-                                grid_max, sch)) return rc;
-    const WorkspaceLayout lay = workspace_layout(sch.items.size(), sch.pieces.size(), sch.merges.size(),
-                                                 sch.merge_slots.size(), sch.grid, sch.n_slots);
-    if (lay.total > workspace_bytes)
-        return set_error(CP_ERR_WORKSPACE, "%s: schedule needs %zu workspace bytes, have %zu", who, lay.total, workspace_bytes);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    // With schedule reuse on, a call whose schedule-relevant arguments and workspace equal the previous call's
+    // (the next layer of the same batch) launches on the work lists that are already in the workspace.
+    uint64_t key = 0;
+    if (ctx->cache_on) {
+        key = 1469598103934665603ull;
+        auto mix = [&key](int64_t v) { key = (key ^ (uint64_t)v) * 1099511628211ull; };
+        mix(B); mix(Hq); mix(cache->Hkv); mix(cache->page_size); mix(only_shard); mix(only_chunk); mix(kv_lo); mix(kv_hi);
+        mix(grid_max); mix(out_f32);
+        for (int32_t b = 0; b < B; ++b) { mix(cu_new[b + 1]); mix(prefix_len[b]); mix(C[b]); mix(cu_pages[b + 1]); }
+    }
+    WorkspaceLayout lay;
+    int32_t grid, n_items, n_merges;
+    int64_t total_rows;
+    if (ctx->cache_on && ctx->cache_valid && ctx->cache_key == key && ctx->cache_ws == workspace) {
+        lay = ctx->cache_lay;
+        grid = ctx->cache_grid;
+        n_items = ctx->cache_items;
+        n_merges = ctx->cache_merges;
+        total_rows = ctx->cache_rows;
+    } else {
+        ctx->cache_valid = false;
+        Schedule sch;
+        build_tiles(B, cu_new, prefix_len, C, cu_pages, cache->page_size, only_shard, only_chunk, kv_lo, kv_hi, sch.items);
+        if (sch.items.empty()) return CP_OK;   // the shard owns no rows (only empty chunks)
+        // rows of q / out / lse: the packed batch, or the one chunk of a chunk call
+        total_rows = cu_new[B];
+        if (only_chunk >= 0) {
+            total_rows = 0;
+            for (const TileItem& t : sch.items) total_rows = std::max<int64_t>(total_rows, (int64_t)t.q_row0 + t.n_rows);
+        }
+        if (int rc = build_schedule(Hq / heads_per_unit,
+                                    kv_major_pairs(B, cu_new, prefix_len, cache->Hkv, (Hq / cache->Hkv) / heads_per_unit),
+                                    grid_max, sch)) return rc;
+        lay = workspace_layout(sch.items.size(), sch.pieces.size(), sch.merges.size(), sch.merge_slots.size(), sch.grid,
+                               sch.n_slots);
+        if (lay.total > workspace_bytes)
+            return set_error(CP_ERR_WORKSPACE, "%s: schedule needs %zu workspace bytes, have %zu", who, lay.total, workspace_bytes);
+        // one contiguous block: items | cta_off | pieces | merges | merge_slots (offsets as in the layout)
+        std::vector<uint8_t> block(lay.partial_o - lay.items, 0);
+        memcpy(block.data() + (lay.items - lay.items), sch.items.data(), sch.items.size() * sizeof(TileItem));
+        memcpy(block.data() + (lay.cta_off - lay.items), sch.cta_off.data(), sch.cta_off.size() * sizeof(int32_t));
+        memcpy(block.data() + (lay.pieces - lay.items), sch.pieces.data(), sch.pieces.size() * sizeof(PieceEntry));
+        if (!sch.merges.empty()) {
+            memcpy(block.data() + (lay.merges - lay.items), sch.merges.data(), sch.merges.size() * sizeof(MergeEntry));
+            memcpy(block.data() + (lay.merge_slots - lay.items), sch.merge_slots.data(), sch.merge_slots.size() * sizeof(int32_t));
+        }
+        if (int rc = upload_block(ctx, block, ws + lay.items, s)) return rc;
+        grid = sch.grid;
+        n_items = (int32_t)sch.items.size();
+        n_merges = (int32_t)sch.merges.size();
+        if (ctx->cache_on) {
+            ctx->cache_valid = true;
+            ctx->cache_key = key;
+            ctx->cache_ws = workspace;
+            ctx->cache_lay = lay;
+            ctx->cache_grid = grid;
+            ctx->cache_items = n_items;
+            ctx->cache_merges = n_merges;
+            ctx->cache_rows = total_rows;
+        }
+    }
 
     CUtensorMap tmQ, tmK, tmV;
     if (int rc = encode_maps(ctx, q, total_rows, Hq, cache, &tmQ, &tmK, &tmV)) return rc;
-    // one contiguous block: items | cta_off | pieces | merges | merge_slots (offsets as in the layout)
-    std::vector<uint8_t> block(lay.partial_o - lay.items, 0);
-    memcpy(block.data() + (lay.items - lay.items), sch.items.data(), sch.items.size() * sizeof(TileItem));
-    memcpy(block.data() + (lay.cta_off - lay.items), sch.cta_off.data(), sch.cta_off.size() * sizeof(int32_t));
-    memcpy(block.data() + (lay.pieces - lay.items), sch.pieces.data(), sch.pieces.size() * sizeof(PieceEntry));
-    if (!sch.merges.empty()) {
-        memcpy(block.data() + (lay.merges - lay.items), sch.merges.data(), sch.merges.size() * sizeof(MergeEntry));
-        memcpy(block.data() + (lay.merge_slots - lay.items), sch.merge_slots.data(), sch.merge_slots.size() * sizeof(int32_t));
-    }
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
-    if (int rc = upload_block(ctx, block, ws + lay.items, s)) return rc;
     if (!ctx->attn_attr_set) {
         if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
@@ -1138,7 +1173,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     }
     AttnParams p;
     p.items = reinterpret_cast<const TileItem*>(ws + lay.items);
-    p.n_items = (int32_t)sch.items.size();
+    p.n_items = n_items;
     p.cta_off = reinterpret_cast<const int32_t*>(ws + lay.cta_off);
     p.pieces = reinterpret_cast<const PieceEntry*>(ws + lay.pieces);
     p.partial_o = reinterpret_cast<float*>(ws + lay.partial_o);
@@ -1157,9 +1192,9 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.lse = lse;
     p.lse_stride = total_rows;
     p.status = ctx->d_status;
-    cp_attn_kernel<<<sch.grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
+    cp_attn_kernel<<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
     if (int rc = check_cuda(cudaGetLastError(), who)) return rc;
-    if (!sch.merges.empty()) {
+    if (n_merges > 0) {
         FixupParams f;
         f.items = p.items;
         f.merges = reinterpret_cast<const MergeEntry*>(ws + lay.merges);
@@ -1172,7 +1207,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         f.heads_per_unit = heads_per_unit;
         f.lse = lse;
         f.lse_stride = total_rows;
-        cp_attn_fixup_kernel<<<dim3((unsigned)sch.merges.size(), 2 * kBlockM / kFixupRowsPerBlock), 256, 0, s>>>(f);
+        cp_attn_fixup_kernel<<<dim3((unsigned)n_merges, 2 * kBlockM / kFixupRowsPerBlock), 256, 0, s>>>(f);
         if (int rc = check_cuda(cudaGetLastError(), "cp_attn_fixup launch")) return rc;
     }
     return CP_OK;

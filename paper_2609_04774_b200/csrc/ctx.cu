@@ -104,6 +104,13 @@ extern "C" int cp_debug_read_status_buffer(cp_ctx* c, void* dst, size_t bytes) {
 }
 #endif
 
+extern "C" int cp_ctx_cache_schedule(cp_ctx* c, int enable) {
+    if (!c) return set_error(CP_ERR_INVALID_ARG, "cp_ctx_cache_schedule: ctx is NULL");
+    c->cache_on = enable != 0;
+    c->cache_valid = false;
+    return CP_OK;
+}
+
 extern "C" int cp_ctx_poll_status(cp_ctx* c, int32_t* detail) {
     if (!c) return set_error(CP_ERR_INVALID_ARG, "cp_ctx_poll_status: ctx is NULL");
     if (int rc = check_cuda(cudaMemcpy(c->h_status, c->d_status, kStatusWords * sizeof(int32_t),

@@ -121,4 +121,12 @@ struct cp_ctx {
     int stage_next;
     cpattn::EncodeTiledFn encode_tiled;
     bool attn_attr_set;
+    // schedule reuse (cp_ctx_cache_schedule): what the last attention call left in its workspace
+    bool cache_on;
+    bool cache_valid;
+    uint64_t cache_key;                // hash of every argument the schedule depends on
+    const void* cache_ws;              // workspace the cached schedule lives in
+    cpattn::WorkspaceLayout cache_lay;
+    int32_t cache_grid, cache_items, cache_merges;
+    int64_t cache_rows;
 };

@@ -349,6 +349,33 @@ def test_argument_validation_launches_nothing(ctx):
     assert torch.isnan(dev.out.float()).all()               # nothing was written
 
 
+def test_schedule_reuse_gives_identical_results(ctx):
+    # the same batch three times with schedule reuse on (new q and cache contents in between), then another
+    # shape and the first one again: bit-identical to the results without reuse
+    w1, w2 = wl.small_mixed(), wl.Workload("other", 47, 8, 2, [wl.Request(500, 256, 2), wl.Request(90, 0, 1)])
+    d1, d2 = DeviceWorkload(wl.materialize(w1)), DeviceWorkload(wl.materialize(w2))
+    ref1 = [t.clone() for t in (d1.run_batch(ctx) and (d1.out, d1.lse))]
+    ref2 = [t.clone() for t in (d2.run_batch(ctx) and (d2.out, d2.lse))]
+    ctx.cache_schedule(True)
+    try:
+        for dev, ref in ((d1, ref1), (d1, ref1), (d1, ref1), (d2, ref2), (d1, ref1), (d2, ref2), (d2, ref2)):
+            dev.out.fill_(float("nan"))
+            dev.lse.fill_(float("nan"))
+            dev.run_batch(ctx)
+            assert torch.equal(dev.out.view(torch.int16), ref[0].view(torch.int16)) and torch.equal(dev.lse, ref[1])
+        # same shape, other data: the remembered work lists serve a new q
+        q_old = d1.q.clone()
+        d1.q.copy_(torch.flip(q_old, dims=[2]))
+        d1.run_batch(ctx)
+        flipped = d1.out.clone()
+        ctx.cache_schedule(False)
+        d1.run_batch(ctx)
+        assert torch.equal(flipped.view(torch.int16), d1.out.view(torch.int16))
+        assert not torch.equal(flipped.view(torch.int16), ref1[0].view(torch.int16))
+    finally:
+        ctx.cache_schedule(False)
+
+
 def test_expired_wait_is_reported_and_context_survives(ctx):
     # a block waits (about a millisecond) on a barrier nothing arrives at: the kernel returns, the status word
     # carries the time-out, polling clears it, and the same context computes correct attention afterwards
