@@ -984,7 +984,8 @@ __global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p)
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
-        const float inv = 1.f / wsum;     // every row of a unit sees at least key 0, so wsum > 0
+        // a row may see none of the unit's keys (a key range that starts behind its causal limit): zeros, -inf
+        const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
         const int head = p.heads_per_unit * me.pair + wg;
         const int64_t grow = (int64_t)it.q_row0 + row;
         const int64_t off = (grow * p.Hq + head) * kD + lane * 4;
@@ -997,7 +998,7 @@ __global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p)
             pk.y = pack_bf16(acc.z * inv, acc.w * inv);
             *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off) = pk;
         }
-        if (lane == 0) p.lse[(int64_t)head * p.lse_stride + grow] = m + __logf(wsum);
+        if (lane == 0) p.lse[(int64_t)head * p.lse_stride + grow] = wsum > 0.f ? m + __logf(wsum) : -INFINITY;
     }
 }
 
