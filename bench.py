@@ -716,6 +716,7 @@ def run_cachemgr(args, out):
                       lambda L, reused: cmgr.cp_prefer_degree(model, L, deg_arr, reused, 1.2, 0.2)[1],
                       len(stream), cmgr.Keys)
     nodes = t.size()
+    # cpu_baseline leg: the oracle on the first tenth of the stream
     sys.path.insert(0, ROOT)
     from oracle import cache_manager as ocm
     o = ocm.Trie(degrees, 64)
@@ -725,8 +726,10 @@ def run_cachemgr(args, out):
     dto, _ = drive(o, lambda tr, b: [len(tr.reused_path(b, w)) * 64 for w in ids],
                    lambda L, reused: ocm.prefer_degree(model, L, [(workers[w], p) for w, p in zip(ids, reused)], 1.2, 0.2)[1], n_o)
     out.write(json.dumps({"mode": "cachemgr", "requests": len(stream), "workers": len(ids), "nodes": nodes, "scans": scans,
-                          "library_requests_per_s": len(stream) / dt, "oracle_requests_per_s": n_o / dto,
-                          "oracle_sample": "first %d requests" % n_o, "note": "driven from Python through ctypes"}) + "\n")
+                          "library_requests_per_s": len(stream) / dt,
+                          "cpu_baseline": {"value": n_o / dto, "unit": "requests/s", "cores": 1, "kind": "oracle",
+                                           "sample": "first %d requests of the same stream" % n_o},
+                          "note": "driven from Python through ctypes"}) + "\n")
     out.flush()
 
 
