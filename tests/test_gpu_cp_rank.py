@@ -34,9 +34,10 @@ def _compare(o, l, ref_o, ref_l, what):
     assert lerr.max() <= 1e-3, (what, lerr.max())
 
 
-def test_chunk_entry_point_matches_oracle_rows():
+@pytest.mark.parametrize("page", [64, 16])
+def test_chunk_entry_point_matches_oracle_rows(page):
     from paper_2609_04774_b200 import binding
-    w = wl.Workload("chunk_call", 61, 8, 2, [wl.Request(1000, 320, 3)])
+    w = wl.Workload("chunk_call", 61, 8, 2, [wl.Request(1000, 320, 3)], page=page)
     mat = wl.materialize(w)
     r = w.requests[0]
     ctx = binding.Context(0)
