@@ -148,7 +148,9 @@ int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_
  * Every shard's q-tiles are cut at chunk boundaries of cp_plan(R, P, C); the result does not
  * depend on C.  Requires Hq % Hkv == 0 (query head h uses KV head h / (Hq / Hkv)); with an even group
  * size two query heads of a group share every K/V tile in shared memory, with an odd one (e.g.
- * Hq == Hkv) every head streams K/V on its own at about 70 % of the throughput (950 against 1360 TFLOP/s on config 2's lengths).  One persistent launch computes all tiles; the few units that were split along KV
+ * Hq == Hkv) every head streams K/V on its own: its KV tiles then alternate between the two softmax warpgroups (two
+ * online-softmax streams combined at the end), at about 80 % of the throughput (1090 against 1355 TFLOP/s on
+ * config 2's lengths).  One persistent launch computes all tiles; the few units that were split along KV
  * to balance the SMs are combined by a second small launch (an LSE merge of their partials).  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
  * ------------------------------------------------------------------------------------------- */
 int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,

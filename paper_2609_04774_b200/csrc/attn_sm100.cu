@@ -52,7 +52,8 @@ static_assert(2 * 128 * kRegsSoftmax + 128 * kRegsOther <= 65536 - 1024, "leave 
 constexpr uint32_t kSmemQ = 0;                                  // 2 heads x 32 KB
 constexpr uint32_t kSmemKV = 2 * kTileBytes;                    // kKvStages x 32 KB
 constexpr uint32_t kSmemBar = kSmemKV + kKvStages * kTileBytes; // mbarriers
-constexpr uint32_t kSmemBytes = kSmemBar + 256;
+constexpr uint32_t kSmemXchg = kSmemBar + 256;                   // 128 x (m, l) floats: second stream of a single-head unit
+constexpr uint32_t kSmemBytes = kSmemXchg + 1024;
 constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;              // slack for manual alignment
 
 // barrier indices (8 bytes each, from kSmemBar); also the ids reported on a timeout
@@ -453,10 +454,11 @@ struct RingPos {
 // (S buffer) and P*V (P and O columns) touch disjoint TMEM and the K and V tiles have their own barriers.
 //
 // Score issuer: S tiles in the order (tile, head); each needs its K tile and the buffer back (s_free).
+template <bool kDual>
 __device__ __forceinline__ void mma_s_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
                                            volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
-    const int H = p.heads_per_unit;
+    constexpr int H = kDual ? 1 : 2;
     RingPos unit_pos = {0, 0};         // ring position of the unit's first load, K(j0)
     uint32_t s_par = 1;                // parity of "previous score tile was read"; 1: no tile yet (passes)
     const uint64_t q_desc0 = make_desc(smem_base + kSmemQ, 16, 1024);
@@ -471,6 +473,8 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, uint32_t smem_ba
         for (int j = j0; j < n; ++j) {
             mbar_wait(bars, kBarKvFull + kpos.slot, kpos.par, abort_flag, p.status, j);
             for (int h = 0; h < H; ++h) {
+                // single-head unit: one Q tile, and the tiles go to the two softmax warpgroups in turn
+                const int wgt = (H == 1) ? ((j - j0) & 1) : h;
                 mbar_wait(bars, kBarSFree, s_par, abort_flag, p.status, j);
                 s_par ^= 1u;
                 tc_fence_after();
@@ -482,7 +486,7 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, uint32_t smem_ba
                         mma_ss(tmem_base + kTmemS, q_desc0 + (h * (kTileBytes >> 4)) + off,
                                k_desc0 + kpos.slot * (kTileBytes >> 4) + off, kIdescS, ks > 0);
                     }
-                    tc_commit(bars + (kBarSReady + h) * 8);
+                    tc_commit(bars + (kBarSReady + wgt) * 8);
                     if (h == H - 1) {
                         tc_commit(bars + (kBarKvEmpty + kpos.slot) * 8);
                         if (j == n - 1) tc_commit(bars + kBarQEmpty * 8);
@@ -500,13 +504,16 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, uint32_t smem_ba
     }
 }
 
-// P*V issuer: O_h += P_h V_j in the order (tile, head), each in the two pieces P is handed over in.
+// P*V issuer: O_h += P_h V_j in the order (tile, head), each in the two pieces P is handed over in.  In a
+// single-head unit the tiles alternate between the two P / O column sets (two independent online-softmax
+// streams over the even and the odd tiles of the piece, combined in the epilogue).
+template <bool kDual>
 __device__ __forceinline__ void mma_pv_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
                                             volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
-    const int H = p.heads_per_unit;
+    constexpr int H = kDual ? 1 : 2;
     RingPos unit_pos = {0, 0};
-    uint32_t p_par = 0;                // phase parity of p_ready (the heads advance together)
+    uint32_t p_par0 = 0, p_par1 = 0;   // phase parity of p_ready per softmax warpgroup
     const uint64_t v_desc0 = make_desc(smem_base + kSmemKV, kHalfBytes, 1024);   // MN-major view of a ring slot
     for (int round = 0;; ++round) {
         UnitInfo u;
@@ -517,31 +524,34 @@ __device__ __forceinline__ void mma_pv_role(const AttnParams& p, uint32_t smem_b
         for (int j = j0; j < n; ++j) {
             mbar_wait(bars, kBarKvFull + vpos.slot, vpos.par, abort_flag, p.status, j);
             for (int h = 0; h < H; ++h) {
-                if (j == j0 && round > 0) mbar_wait(bars, kBarOFree + h, (round - 1) & 1, abort_flag, p.status, j);
+                const int wgt = (H == 1) ? ((j - j0) & 1) : h;            // P / O column set and softmax warpgroup
+                const bool first = (H == 1) ? (j - j0 < 2) : (j == j0);   // first tile of this accumulator in the unit
+                if (first && round > 0) mbar_wait(bars, kBarOFree + wgt, (round - 1) & 1, abort_flag, p.status, j);
+                const uint32_t ppar = wgt ? p_par1 : p_par0;
 #pragma unroll
                 for (int part = 0; part < kPieces; ++part) {
-                    mbar_wait(bars, kBarPReady + h * 4 + part, p_par, abort_flag, p.status, j);
+                    mbar_wait(bars, kBarPReady + wgt * 4 + part, ppar, abort_flag, p.status, j);
                     tc_fence_after();
-                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + h, j, part); }
+                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wgt, j, part); }
                     if (elect_one()) {
                         const int ks0 = part == 0 ? 0 : 2 * kSplitQ, ks1 = part == 0 ? 2 * kSplitQ : 8;
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {
                             if (ks >= ks0 && ks < ks1)
-                                mma_ts(tmem_base + kTmemO + h * 128, tmem_base + kTmemP + h * 64 + ks * 8,
+                                mma_ts(tmem_base + kTmemO + wgt * 128, tmem_base + kTmemP + wgt * 64 + ks * 8,
                                        v_desc0 + vpos.slot * (kTileBytes >> 4) + ks * (2048 >> 4), kIdescPV,
-                                       j > j0 || ks > 0);
+                                       !first || ks > 0);
                         }
                         if (part == kPieces - 1) {
-                            tc_commit(bars + (kBarPvDone + h) * 8);
+                            tc_commit(bars + (kBarPvDone + wgt) * 8);
                             if (h == H - 1) tc_commit(bars + (kBarKvEmpty + vpos.slot) * 8);
                         }
                     }
                     __syncwarp();
                 }
-                if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + h, j, 5); }
+                if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wgt, j, 5); }
+                if (wgt) p_par1 ^= 1u; else p_par0 ^= 1u;
             }
-            p_par ^= 1u;
             vpos = vpos.plus(j + 2 == n ? 1 : 2);
         }
         const uint32_t adv = (uint32_t)(2 * (n - j0));
@@ -723,8 +733,9 @@ __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], f
     l += st.x + st.y;
 }
 
+template <bool kDual>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
-                                             volatile uint32_t* abort_flag, int wg) {
+                                             volatile uint32_t* abort_flag, uint8_t* smem_xchg, int wg) {
     const uint32_t bars = smem_base + kSmemBar;
     const int lane = threadIdx.x & 31;
     const int warp_in_wg = (threadIdx.x >> 5) & 3;
@@ -736,7 +747,10 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
     const uint32_t p_bar0 = bars + (kBarPReady + wg * 4) * 8;
     const float c = p.scale_log2;
     uint32_t tile_cnt = 0;
-    if (wg >= p.heads_per_unit) return;      // single-head units: the second softmax warpgroup has no work
+    // single-head units: the two warpgroups take the even and the odd KV tiles of the piece as two independent
+    // online-softmax streams (own running max, sum and O accumulator); warpgroup 0 combines them at the end
+    constexpr bool dual = kDual;
+    constexpr int step = kDual ? 2 : 1;
 
 #define SM_WAIT(id, parity, it)                                                                  \
     mbar_wait(bars, (id), (parity), abort_flag, p.status, (it));                                 \
@@ -754,7 +768,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
         UnitInfo u;
         if (!fetch_unit(p, round, u)) break;
         const int n = u.t_end;
-        const int head = u.head0 + wg;
+        const int head = u.head0 + (dual ? 0 : wg);
+        const int j_first = u.t_begin + (dual ? wg : 0);     // first tile of this warpgroup's stream
         float m = -INFINITY;   // running row max in log2 units (possibly stale by < threshold)
         float l = 0.f;         // running row sum of 2^(s - m)
         // tiles below n_full lie entirely under the causal diagonal of every row of the q-tile and inside the
@@ -762,27 +777,52 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
         const int n_full = min(u.it.kv_len0, u.it.kv_hi) / kBlockN;
         const int j_cut = (u.it.kv_lo & (kBlockN - 1)) ? (u.it.kv_lo >> 7) : -1;
         float s0[32], s1[32], s2[32], s3[32];   // the row's scores of the current tile
-        // the first tile of the unit is loaded here, every later one by the tile before it
-        SM_WAIT(kBarSReady + wg, s_par, u.t_begin);
-        s_par ^= 1u;
-        tc_fence_after();
-        CP_LOAD_S(s0, s1, s2, s3)
-        release_s(bars);
+        // the first tile of the stream is loaded here, every later one by the tile before it
+        if (!kDual || j_first < n) {
+            SM_WAIT(kBarSReady + wg, s_par, j_first);
+            s_par ^= 1u;
+            tc_fence_after();
+            CP_LOAD_S(s0, s1, s2, s3)
+            release_s(bars);
+        }
 #pragma unroll 1
-        for (int j = u.t_begin; j < n; ++j) {
+        for (int j = j_first; j < n; j += step) {
             CP_TRACE_ROW_PTR(j)
             if (tr) tr[0] = clock64();
             const SoftmaxSync sy = {bars, kBarSReady + (uint32_t)wg, kBarPvDone + (uint32_t)wg, (tile_cnt - 1) & 1,
                                     abort_flag, p.status, j, tr};
             if (j < n_full && j != j_cut)
-                softmax_tile<false>(s0, s1, s2, s3, j + 1 < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c, 0, 0,
-                                    j == u.t_begin, m, l, sy);
+                softmax_tile<false>(s0, s1, s2, s3, j + step < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c, 0, 0,
+                                    j == j_first, m, l, sy);
             else
-                softmax_tile<true>(s0, s1, s2, s3, j + 1 < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c,
+                softmax_tile<true>(s0, s1, s2, s3, j + step < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c,
                                    u.it.kv_lo - j * kBlockN, min(u.it.kv_len0 + row, u.it.kv_hi) - j * kBlockN,
-                                   j == u.t_begin, m, l, sy);
+                                   j == j_first, m, l, sy);
             if (row == CPATTN_TRACE_ROW) { CP_TRACE(wg, j, 6); }
             ++tile_cnt;
+        }
+        float a_own = 1.f, a_oth = 0.f;     // dual: weights of the two streams' accumulators in the combined row
+        if (dual) {
+            float2* xchg = reinterpret_cast<float2*>(smem_xchg);
+            if (wg == 1) {
+                // second stream: wait for its last P*V, publish (m, l), leave the rest to warpgroup 0
+                if (j_first < n) {
+                    SM_WAIT(kBarPvDone + wg, (tile_cnt - 1) & 1, n);
+                    tc_fence_before();
+                }
+                xchg[row] = make_float2(m, l);
+                asm volatile("bar.sync 1, 256;" ::: "memory");      // both streams done, (m, l) visible
+                asm volatile("bar.sync 2, 256;" ::: "memory");      // warpgroup 0 has read them
+                continue;
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            const float2 ml1 = xchg[row];
+            asm volatile("bar.arrive 2, 256;" ::: "memory");
+            const float mm = fmaxf(m, ml1.x);
+            a_own = (l > 0.f) ? ex2(m - mm) : 0.f;
+            a_oth = (ml1.y > 0.f) ? ex2(ml1.x - mm) : 0.f;
+            l = a_own * l + a_oth * ml1.y;
+            m = mm;
         }
         // epilogue: O / l -> global at the row's original position; LSE in natural log
         SM_WAIT(kBarPvDone + wg, (tile_cnt - 1) & 1, n);
@@ -794,10 +834,23 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
         const int64_t grow_idx = (int64_t)u.it.q_row0 + row;
         float* part_row = p.partial_o + (((int64_t)max(u.slot, 0) * 2 + wg) * kBlockM + row) * kD;
 #pragma unroll 1
+        const bool has_other = dual && (u.t_begin + 1 < n);     // the second stream got at least one tile
         for (int cc = 0; cc < 4; ++cc) {
             float o[32];
             TMEM_LD32(o_tmem + cc * 32, o, 0);
-            tc_wait_ld();
+            if (has_other) {
+                float o1[32];
+                TMEM_LD32(o_tmem + 128 + cc * 32, o1, 0);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] = a_own * o[i] + a_oth * o1[i];
+            } else {
+                tc_wait_ld();
+                if (dual) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] *= a_own;
+                }
+            }
             if (valid) {
                 if (partial || p.out_f32) {
                     float4* dst = partial ? reinterpret_cast<float4*>(part_row + cc * 32)
@@ -828,11 +881,17 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bars + (kBarOFree + wg) * 8);
+        if (lane == 0) {
+            mbar_arrive(bars + (kBarOFree + wg) * 8);
+            if (dual) mbar_arrive(bars + (kBarOFree + 1) * 8);     // this warpgroup has read both accumulators
+        }
     }
 #undef SM_WAIT
 }
 
+// kDual: every unit is a single query head (odd group size); its KV tiles then alternate between the two
+// softmax warpgroups.  Two separate kernels, so that neither carries the other's code in its hot loop.
+template <bool kDual>
 __global__ void __launch_bounds__(kThreads, 1)
 cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
@@ -872,15 +931,15 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-        softmax_role(p, smem_base, tmem_base, abort_flag, warp >> 2);
+        softmax_role<kDual>(p, smem_base, tmem_base, abort_flag, smem_gen + kSmemXchg, warp >> 2);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
         if (warp == 8) {
             producer_role(&tmQ, &tmK, &tmV, p, smem_base, abort_flag);
         } else if (warp == 9) {
-            mma_s_role(p, smem_base, tmem_base, abort_flag);
+            mma_s_role<kDual>(p, smem_base, tmem_base, abort_flag);
         } else if (warp == 10) {
-            mma_pv_role(p, smem_base, tmem_base, abort_flag);
+            mma_pv_role<kDual>(p, smem_base, tmem_base, abort_flag);
         }
     }
 
@@ -1168,7 +1227,9 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     CUtensorMap tmQ, tmK, tmV;
     if (int rc = encode_maps(ctx, q, total_rows, Hq, cache, &tmQ, &tmK, &tmV)) return rc;
     if (!ctx->attn_attr_set) {
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
         ctx->attn_attr_set = true;
     }
@@ -1193,7 +1254,8 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.lse = lse;
     p.lse_stride = total_rows;
     p.status = ctx->d_status;
-    cp_attn_kernel<<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
+    if (heads_per_unit == 2) cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
+    else cp_attn_kernel<true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
     if (int rc = check_cuda(cudaGetLastError(), who)) return rc;
     if (n_merges > 0) {
         FixupParams f;
@@ -1342,7 +1404,9 @@ int static_setup(int device, StaticDeviceState** out) {
                                 "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)")) return rc;
         if (q != cudaDriverEntryPointSuccess || !fn)
             return set_error(CP_ERR_CUDA, "cuTensorMapEncodeTiled is not available in this driver");
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
         st.scratch = static_cast<unsigned char*>(ptr);
         st.num_sms = prop.multiProcessorCount;
@@ -1416,6 +1480,7 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     p.status = reinterpret_cast<int32_t*>(st->scratch);
     const int64_t units = (int64_t)tiles.size() * p.pairs_per_tile;
     const int grid = (int)std::min<int64_t>(units, st->num_sms);
-    cp_attn_kernel<<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
+    if (heads_per_unit == 2) cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
+    else cp_attn_kernel<true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
     return check_cuda(cudaGetLastError(), who);
 }
