@@ -3,7 +3,9 @@
 //
 // One persistent CTA per SM walks a list of work units.  A unit is one query tile (<= 128 new
 // tokens of one zigzag chunk) for TWO query heads of the same KV group, so each K/V tile that
-// lands in shared memory feeds two 128x128 score tiles (GQA head sharing).  Warp roles:
+// lands in shared memory feeds two 128x128 score tiles (GQA head sharing).  With an odd group size a unit
+// is ONE query head, and the two softmax warpgroups take its even and odd KV tiles as two online-softmax
+// streams that are combined in the epilogue (kernel instantiation kDual).  Warp roles:
 //   warps 0-3  softmax warpgroup for head 0 of the pair: one thread per query row
 //   warps 4-7  softmax warpgroup for head 1
 //   warp  8    TMA producer (the warp prefetches page ids; the pages of a tile go out from several lanes)
