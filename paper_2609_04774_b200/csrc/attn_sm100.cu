@@ -835,8 +835,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
         const bool valid = row < u.it.n_rows;
         const int64_t grow_idx = (int64_t)u.it.q_row0 + row;
         float* part_row = p.partial_o + (((int64_t)max(u.slot, 0) * 2 + wg) * kBlockM + row) * kD;
-#pragma unroll 1
         const bool has_other = dual && (u.t_begin + 1 < n);     // the second stream got at least one tile
+#pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
             float o[32];
             TMEM_LD32(o_tmem + cc * 32, o, 0);
