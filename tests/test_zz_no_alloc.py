@@ -38,7 +38,8 @@ def test_static_entry_point_matches_regular_one_twice():
     ctx = binding.Context(0)
     try:
         for w in (wl.Workload("static_a", 31, 8, 2, [wl.Request(1500, 448, 4)]),
-                  wl.Workload("static_b", 32, 8, 2, [wl.Request(200, 64, 3)])):
+                  wl.Workload("static_b", 32, 8, 2, [wl.Request(200, 64, 3)]),
+                  wl.Workload("static_mha", 34, 4, 4, [wl.Request(900, 320, 2)])):      # single-head units
             o, l, ro, rl = _both(ctx, w)
             assert np.isfinite(o).all() and np.isfinite(l).all()
             assert np.abs(o - ro).max() <= 2e-2 and np.abs(o - ro).mean() <= 2e-3
