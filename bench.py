@@ -1,13 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of libcpattn's hot path: cache-aware causal prefill attention under zigzag CP.
 
-Default mode prints ONE JSON line for the headline workload (BASELINE config 2: Llama-3-8B-shaped
-layer, 12288 cached + 4096 new tokens, C=4, paged KV).  A step is one pass of the hot path over the
-batch: cp_plan (host) -> varlen tile schedule (host, uploaded by a copy kernel) -> one persistent
-attention launch over all C shards reading K/V through the page table and storing rows at their
-original positions -> LSE merge of the units whose KV range was split across CTAs.  `value` is
-measured with inputs resident in HBM; `e2e` goes through the same C-ABI calls from pinned HOST
-buffers (q, the new tokens' K/V rows appended into the paged cache, page table up; out and lse down).
+Default mode prints ONE JSON line.  Its headline (`value`, `roofline`, `e2e`) is configuration 2
+(Llama-3-8B-shaped layer, 12288 cached + 4096 new tokens, C=4, paged KV).  A step is one pass of the hot
+path over the batch: cp_plan (host) -> varlen tile schedule (host; small work lists ride in the launch
+parameters, large ones are uploaded by a copy kernel) -> one persistent attention launch over all C shards
+reading K/V through the page table and storing rows at their original positions -> LSE merge of the units
+whose KV range was split across CTAs.  `value` is measured with inputs resident in HBM; `e2e` goes through
+the same C-ABI calls from pinned HOST buffers (q, the new tokens' K/V rows appended into the paged cache,
+page table up; out and lse down).  At one GPU the same line also carries: `sustained` (the headline
+workload repeated for at least two seconds of GPU time, clocks sampled), `configs` (configurations 1-5,
+each with its own clocks), `merge` (cp_merge bandwidth points), `kvcopy` (paged copy bandwidth) and the
+`cpu_baseline` legs (the fp64 oracle on the host cores).
 
 Other modes (`--mode merge|table|configs|kvcopy|cprank`) write the cp_merge sweep, the measured prefill-time
 table over (new_len, prefix_len, C), the per-config numbers and the paged KV copy bandwidth as JSON
@@ -37,9 +41,9 @@ METRIC = "causal_effective_prefill_attention_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one cp_attn_kernel launch, from the ncu capture
-# summarised in profiles/ (per workload name)
-ATTN_TRAFFIC_BYTES = {"cfg2_R4096_P12288_C4": 118_038_784}
+# dram__bytes_read.sum + dram__bytes_write.sum of one cp_attn_kernel launch, from the ncu captures
+# summarised in profiles/ (per workload name; a workload without a capture reports null)
+ATTN_TRAFFIC_BYTES = {"cfg2_R4096_P12288_C4": 118_038_784, "cfg3_R131072_P0_C8": 11_500_000_000}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -57,6 +61,22 @@ def load_peaks():
 
 def get_workload(cfg: int) -> wl.Workload:
     return (wl.CONFIGS.get(cfg) or wl.VARIANTS[cfg])()
+
+
+def pairs_of(w: wl.Workload) -> int:
+    """Visible (query, key) pairs: the remaining attention workload W(R,P) = R*P + R(R+1)/2 of Eq. (1), summed over
+    the requests of the batch."""
+    return sum(r.new_len * r.prefix_len + r.new_len * (r.new_len + 1) // 2 for r in w.requests)
+
+
+def flops_of(w: wl.Workload) -> int:
+    """Causal-effective flops: 4*D per visible pair per query head (masked halves of diagonal tiles do not count)."""
+    return 4 * w.D * w.Hq * pairs_of(w)
+
+
+def algorithmic_bytes(w: wl.Workload) -> int:
+    """Q and O once, K and V once, LSE (bf16 tensors, fp32 LSE)."""
+    return 2 * w.total_new * w.Hq * w.D * 2 + 2 * sum(r.total_len for r in w.requests) * w.Hkv * w.D * 2 + 4 * w.Hq * w.total_new
 
 
 # ----------------------------------------------------------------------------------------------
@@ -228,12 +248,16 @@ class Runner:
         torch.cuda.current_stream().wait_event(self.ev_out[i])   # the timing events sit on the current stream
 
     def launches_per_step(self, e2e=False):
-        """Kernels of this library per step: schedule copy + attention (+ LSE fix-up when units were split)."""
+        """Kernels of this library per step, as the library's own schedule reports them: list copy (unless the
+        work lists ride in the launch parameters) + attention + LSE fix-up when units were split."""
         info, _, _ = self.binding.cp_schedule_inspect(self.cu_new, self.prefix, self.Cs, self.w.Hq, self.w.Hkv,
                                                       self.torch.cuda.get_device_properties(0).multi_processor_count,
                                                       want_lists=False)
         self.schedule = info
-        return 2 + (1 if info["split_units"] > 0 else 0) + (len(self.w.requests) if e2e else 0)
+        return info["launches"] + (len(self.w.requests) if e2e else 0)
+
+    def close(self):
+        self.ctx.close()
 
 
 def max_over_ranks(torch, dist, values, device):
@@ -273,8 +297,8 @@ def timed_loop(torch, fn, steps, warmup, dist=None):
 
 
 def kernel_only_ms(torch, runner, steps):
-    """Average duration of the attention launch alone: events recorded directly around each launch on the
-    launching stream, after the loop above has warmed everything up."""
+    """Average duration of one step's launches: events recorded directly around each call on the launching
+    stream, after the loop above has warmed everything up."""
     w, b = runner.w, runner.binding
     ds = []
     for _ in range(steps):
@@ -286,6 +310,147 @@ def kernel_only_ms(torch, runner, steps):
         ds.append((e0, e1))
     torch.cuda.synchronize()
     return statistics.mean(a.elapsed_time(c) for a, c in ds)
+
+
+def fractions(tflops, peaks):
+    return {"of_nominal_2250": tflops / NOMINAL_BF16_TFLOPS, "of_measured_burst": tflops / peaks["bf16_tflops"],
+            "of_measured_sustained": tflops / peaks["bf16_tflops_sustained"]}
+
+
+def sustained_leg(torch, runner, peaks, device, seconds=2.2):
+    """The headline workload back to back for at least `seconds` of GPU time (long enough for the board to reach
+    its power-capped clocks), with the clocks sampled during the loop."""
+    for _ in range(5):
+        runner.step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(20):
+        runner.step()
+    e1.record()
+    torch.cuda.synchronize()
+    steps = max(50, int(seconds * 1e3 / max(e0.elapsed_time(e1) / 20, 1e-3)) + 1)
+    sampler = ClockSampler(device)
+    sampler.start()
+    time.sleep(0.3)                     # the sampler's first sample
+    total_ms, _ = timed_loop(torch, runner.step, steps, 3)
+    clocks = sampler.stop()
+    ms = total_ms / steps
+    tf = flops_of(runner.w) / (ms * 1e-3) / 1e12
+    return {"workload": runner.w.name, "steps": steps, "gpu_seconds": total_ms * 1e-3, "ms_per_step": ms, "tflops": tf,
+            "sm_mhz_median": clocks["sm_mhz"], "ms_x_mhz": ms * clocks["sm_mhz"] if clocks["sm_mhz"] else None,
+            "frac": fractions(tf, peaks), "clocks": clocks}
+
+
+def config_leg(torch, cfg, peaks, device, budget_ms=1200.0):
+    """One configuration: 3 warm-up steps, then steps for about `budget_ms` of GPU time (at least 5), clocks sampled."""
+    w = get_workload(cfg)
+    runner = Runner(w, device)
+    sampler = ClockSampler(device)
+    sampler.start()
+    for _ in range(3):
+        runner.step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    runner.step()
+    e1.record()
+    torch.cuda.synchronize()
+    steps = int(max(5, min(2000, budget_ms / max(e0.elapsed_time(e1), 1e-3))))
+    total_ms, per = timed_loop(torch, runner.step, steps, 0)
+    clocks = sampler.stop()
+    runner.ctx.poll_status()
+    ms = total_ms / steps
+    tf = flops_of(w) / (ms * 1e-3) / 1e12
+    entry = {"config": cfg, "workload": w.name, "steps": steps, "ms": ms, "ms_best": min(per), "tflops": tf,
+             "tokens_per_s": w.total_new / (ms * 1e-3), "frac": fractions(tf, peaks), "pairs": pairs_of(w),
+             "launches_per_step": runner.launches_per_step(), "gpu_seconds": total_ms * 1e-3, "clocks": clocks,
+             "traffic": ATTN_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": algorithmic_bytes(w)}
+    runner.close()
+    del runner
+    torch.cuda.empty_cache()
+    return entry
+
+
+def merge_points(torch, peaks, points, reps=10):
+    """cp_merge bandwidth at (T, N, out dtype) points: H = 64, D = 128, partials N(0,1), lses N(8, 2^2) with every
+    16th row of partial 0 at -inf; L2 flushed between repetitions when the operands are small."""
+    from paper_2609_04774_b200 import binding
+    ctx = binding.Context(torch.cuda.current_device())
+    H, D = 64, 128
+    g = torch.Generator(device="cuda").manual_seed(6)
+    out = []
+    for T, N, dt in points:
+        in_bytes = N * T * H * (D * 4 + 4)
+        out_bytes = T * H * (D * dt.itemsize) + 4 * T * H
+        parts = torch.randn((N, T, H, D), dtype=torch.float32, device="cuda", generator=g)
+        lses = 8 + 2 * torch.randn((N, H, T), dtype=torch.float32, device="cuda", generator=g)
+        lses[0].view(-1)[::16] = float("-inf")
+        o = torch.empty((T, H, D), dtype=dt, device="cuda")
+        lo = torch.empty((H, T), dtype=torch.float32, device="cuda")
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if in_bytes < 512e6 else None
+        ds = []
+        for i in range(3 + reps):
+            if flush is not None:
+                flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            binding.cp_merge(ctx, parts, lses, o, lo)
+            e1.record()
+            if i >= 3:
+                ds.append((e0, e1))
+        torch.cuda.synchronize()
+        ms = [a.elapsed_time(b) for a, b in ds]
+        med = statistics.median(ms)
+        gbs = (in_bytes + out_bytes) / (med * 1e-3) / 1e9
+        out.append({"T": T, "N": N, "H": H, "out": str(dt).split(".")[-1], "bytes": in_bytes + out_bytes, "ms_median": med,
+                    "ms_best": min(ms), "GBps": gbs, "frac_nominal_8000": gbs / NOMINAL_HBM_GBS,
+                    "frac_measured_copy": gbs / peaks["hbm_gbs"], "l2_flush": flush is not None})
+        del parts, lses, o, lo, flush
+        torch.cuda.empty_cache()
+    ctx.close()
+    return out
+
+
+def kvcopy_points(torch, peaks, tokens=(1048576,)):
+    """cp_kv_gather / cp_kv_append bandwidth: n tokens x 8 KV heads x 128 dims, K and V, shuffled pages."""
+    from paper_2609_04774_b200 import binding
+    ctx = binding.Context(torch.cuda.current_device())
+    Hkv, D = 8, 128
+    out = []
+    for n in tokens:
+        pages = n // wl.PAGE
+        k = torch.randn((pages, wl.PAGE, Hkv, D), device="cuda").to(torch.bfloat16)
+        v = torch.randn((pages, wl.PAGE, Hkv, D), device="cuda").to(torch.bfloat16)
+        pt = torch.from_numpy(wl.permutation(9, wl.TID_PERM, pages)).cuda()
+        cache = binding.make_cache(k, v)
+        kr = torch.empty((n, Hkv, D), dtype=torch.bfloat16, device="cuda")
+        vr = torch.empty_like(kr)
+        moved = 2 * 2 * n * Hkv * D * 2 + 4 * pages          # K and V, read + written, plus the table
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if moved < 512e6 else None
+        for name, fn in (("gather", lambda: binding.cp_kv_gather(ctx, cache, pt, 0, n, kr, vr)),
+                         ("append", lambda: binding.cp_kv_append(ctx, cache, pt, 0, n, kr, vr))):
+            ds = []
+            for i in range(13):
+                if flush is not None:
+                    flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                if i >= 3:
+                    ds.append((e0, e1))
+            torch.cuda.synchronize()
+            ctx.poll_status()
+            ms = statistics.median(a.elapsed_time(b) for a, b in ds)
+            gbs = moved / (ms * 1e-3) / 1e9
+            out.append({"op": name, "tokens": n, "bytes": moved, "ms_median": ms, "GBps": gbs,
+                        "frac_nominal_8000": gbs / NOMINAL_HBM_GBS, "frac_measured_copy": gbs / peaks["hbm_gbs"],
+                        "l2_flush": flush is not None})
+        del k, v, kr, vr, flush
+        torch.cuda.empty_cache()
+    ctx.close()
+    return out
 
 
 # ----------------------------------------------------------------------------------------------
@@ -306,6 +471,64 @@ def oracle_sample(w: wl.Workload, mat, rows_per_request: int, seed: int, threads
         orc.attn_rows(q, mat.k_pages, mat.v_pages, pt, r.prefix_len, w.Hkv, w.scale, rows, n_threads=threads)
         pairs += int((r.prefix_len + rows + 1).sum()) * w.Hq
     return time.perf_counter() - t0, pairs, threads
+
+
+def cpu_model():
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def cpu_baseline_legs(headline, headline_mat, args):
+    """The oracle as it stands on the host cores, bounded to about half a minute in total: the headline
+    configuration on a seeded row sample (the `value` of the object), configuration 1 in full with one thread and
+    with all cores, the other configurations on small row samples with the full-workload time extrapolated by
+    pairs (labelled), and the merge oracle on small T scaled linearly in T."""
+    from oracle import reference as orc
+    orc.build()
+    t, pairs, threads = oracle_sample(headline, headline_mat, args.cpu_rows, 4242)
+    tf = 4 * headline.D * pairs / t / 1e12
+    base = {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "%s: %d seeded rows x %d heads (%.1f s); full pass extrapolated by pairs: %.0f s" %
+                      (headline.name, args.cpu_rows, headline.Hq, t, flops_of(headline) / (tf * 1e12)),
+            "cpu_model": cpu_model(), "nproc": os.cpu_count(), "threads": threads}
+    per = []
+    rows_for = {1: None, 2: None, 3: 48, 4: 6, 5: 40}
+    for cfg in (1, 3, 4, 5):
+        w = get_workload(cfg)
+        mat = wl.materialize(w)
+        if cfg == 1:
+            entry = {"config": cfg, "workload": w.name, "mode": "full"}
+            for label, th in (("threads_1", 1), ("threads_all", threads)):
+                r = w.requests[0]
+                t0 = time.perf_counter()
+                orc.attn_full(mat.q, mat.k_pages, mat.v_pages, mat.page_table, r.prefix_len, w.Hkv, w.scale, n_threads=th)
+                dt = time.perf_counter() - t0
+                entry[label] = {"seconds": dt, "gflops_equivalent": flops_of(w) / dt / 1e9, "tokens_per_s": w.total_new / dt}
+        else:
+            t, pairs, _ = oracle_sample(w, mat, rows_for[cfg], 4300 + cfg)
+            rate = 4 * w.D * pairs / t
+            entry = {"config": cfg, "workload": w.name, "mode": "sampled", "rows_per_request": rows_for[cfg],
+                     "sample_seconds": t, "pairs_per_s": pairs / t, "gflops_equivalent": rate / 1e9,
+                     "full_seconds_extrapolated": flops_of(w) / rate, "tokens_per_s_extrapolated": w.total_new * rate / flops_of(w)}
+        per.append(entry)
+        del mat
+    base["per_config"] = per
+    merges = []
+    for N, T in ((2, 2048), (4, 1024), (8, 512)):
+        parts, lses = wl.merge_inputs(6, N, T, 64)
+        t0 = time.perf_counter()
+        orc.merge(parts, lses)
+        dt = time.perf_counter() - t0
+        nbytes = N * T * 64 * 516 + T * 64 * 260
+        merges.append({"N": N, "T_timed": T, "seconds": dt, "GBps_equivalent": nbytes / dt / 1e9,
+                       "seconds_at_T4096_scaled": dt * 4096 / T})
+    base["merge_oracle"] = merges
+    return base
 
 
 def run_reference(args):
@@ -362,16 +585,19 @@ def run_ours(args):
     peaks = load_peaks()
     w = get_workload(args.config)
     runner = Runner(w, local, need_host=True)
-    flops = w.flops()
+    flops = flops_of(w)
 
+    # headline: exactly K steps between events, clocks sampled from the warm-up on
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+        time.sleep(0.2)
     total_ms, per = timed_loop(torch, runner.step, args.steps, args.warmup, dist)
-    e2e_ms, _ = timed_loop(torch, runner.step_e2e, max(3, args.steps // 4), 3, dist)
-    e2e_steps = max(3, args.steps // 4)
-    kern_ms = kernel_only_ms(torch, runner, min(args.steps, 50))
+    kern_steps = max(20, min(args.steps, 50))
+    kern_ms = kernel_only_ms(torch, runner, kern_steps)
     clocks = sampler.stop() if rank == 0 else None
+    e2e_steps = max(50, args.steps)
+    e2e_ms, _ = timed_loop(torch, runner.step_e2e, e2e_steps, 3, dist)
     runner.ctx.poll_status()
 
     total_ms, e2e_ms = max_over_ranks(torch, dist, [total_ms, e2e_ms], "cuda")
@@ -385,29 +611,54 @@ def run_ours(args):
     e2e_value = whole_job_value(world, flops, e2e_ms / e2e_steps)
     achieved = flops / (kern_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops"]
+    launches = runner.launches_per_step()
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "requests": len(w.requests), "new_tokens": w.total_new, "Hq": w.Hq,
-                   "Hkv": w.Hkv, "D": w.D, "page_size": wl.PAGE, "seed": w.seed, "pairs": w.pairs(),
-                   "l2": "inputs (q+kv+out = %.0f MB) exceed the 126 MB L2; no flush between steps" %
-                         ((2 * w.total_new * w.Hq * w.D * 2 + 2 * sum(r.total_len for r in w.requests) * w.Hkv * w.D * 2) / 1e6),
+                   "Hkv": w.Hkv, "D": w.D, "page_size": wl.PAGE, "seed": w.seed, "pairs": pairs_of(w),
+                   "l2": "inputs (q+kv+out = %.0f MB) exceed the 126 MB L2; no flush between steps" % (algorithmic_bytes(w) / 1e6),
                    "multi_gpu": "independent replicas of the workload per rank, no collective"},
         "tokens_per_s": world * w.total_new / (ms_per_step * 1e-3),
+        "frac": fractions(value / world, peaks),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": runner.h2d_bytes,
-                "d2h_bytes_per_step": runner.d2h_bytes, "ms_per_step": e2e_ms / e2e_steps,
+                "d2h_bytes_per_step": runner.d2h_bytes, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps,
                 "pipelining": "3 streams (copy in / compute / copy out), 2 staging buffers; every step's bytes move inside the timed region"},
-        "gpu_launches": args.steps * runner.launches_per_step(),
+        "gpu_launches": args.steps * launches,
+        "launches_per_step": launches,
         "schedule": runner.schedule,
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved / peak, "traffic": ATTN_TRAFFIC_BYTES.get(w.name), "kernel": "cp_attn_kernel",
-                     "kernel_ms": kern_ms, "kernel_ms_covers": "schedule copy + cp_attn_kernel + LSE fix-up of one step", "peak_source": "%s burst bf16 (of %s)" % (peaks["_source"], peaks["_source"]),
-                     "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                     "frac": achieved / peak, "traffic": ATTN_TRAFFIC_BYTES.get(w.name),
+                     "algorithmic_bytes": algorithmic_bytes(w), "kernel": "cp_attn_kernel",
+                     "kernel_ms": kern_ms, "kernel_launches_timed": kern_steps,
+                     "kernel_ms_covers": "the launches of one step (list copy if any + cp_attn_kernel + LSE fix-up)",
+                     "peak_source": "%s burst bf16 (of %s): the timed launches are short and run at burst clocks" % (peaks["_source"], peaks["_source"]),
                      "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS},
         "clocks": clocks,
     }
-    if not args.no_cpu_baseline and world == 1:
+    if world == 1 and not args.headline_only:
+        sus = sustained_leg(torch, runner, peaks, local)
+        line["sustained"] = sus
+        # the fraction of the power-capped peak comes from the power-capped leg only
+        line["roofline"]["frac_of_sustained"] = sus["tflops"] / peaks["bf16_tflops_sustained"]
+        line["roofline"]["frac_of_sustained_source"] = "sustained leg (%.1f s of GPU time) over the measured sustained bf16 rate" % sus["gpu_seconds"]
+        mat_headline = runner.mat
+        runner.close()
+        del runner
+        torch.cuda.empty_cache()
+        line["configs"] = [config_leg(torch, c, peaks, local) for c in (1, 2, 3, 4, 5)]
+        bf, f32 = torch.bfloat16, torch.float32
+        line["merge"] = merge_points(torch, peaks, [(T, N, bf) for T in (4096, 16384, 65536) for N in (2, 4, 8)] +
+                                     [(16384, N, f32) for N in (2, 4, 8)])
+        line["kvcopy"] = kvcopy_points(torch, peaks)
+        targets = {c["workload"]: c["ms"] for c in line["configs"]}
+        line["targets"] = {
+            "cfg2_ms_le_0.855": targets.get("cfg2_R4096_P12288_C4"), "cfg3_ms_le_125.1": targets.get("cfg3_R131072_P0_C8"),
+            "merge_points_below_5600_GBps": [(m["T"], m["N"], m["out"], round(m["GBps"])) for m in line["merge"] if m["GBps"] < 5600.0]}
+        if not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline_legs(w, mat_headline, args)
+    elif not args.no_cpu_baseline and world == 1:
         from oracle import reference as orc
         orc.build()
         t, pairs, threads = oracle_sample(w, runner.mat, args.cpu_rows, 4242)
@@ -425,112 +676,29 @@ def run_configs(args, out):
     import torch
     peaks = load_peaks()
     for cfg in args.configs:
-        w = get_workload(cfg)
-        runner = Runner(w, 0)
-        steps = max(3, min(args.steps, int(2000 / max(1.0, w.flops() / 1e12))))
-        total_ms, per = timed_loop(torch, runner.step, steps, 3)
-        runner.ctx.poll_status()
-        ms = total_ms / steps
-        tf = w.flops() / (ms * 1e-3) / 1e12
-        out.write(json.dumps({"mode": "config", "config": cfg, "workload": w.name, "ms": ms, "ms_best": min(per),
-                              "tflops": tf, "tokens_per_s": w.total_new / (ms * 1e-3),
-                              "frac_nominal_2250": tf / NOMINAL_BF16_TFLOPS, "frac_measured_burst": tf / peaks["bf16_tflops"],
-                              "frac_measured_sustained": tf / peaks["bf16_tflops_sustained"], "steps": steps}) + "\n")
+        out.write(json.dumps(dict(mode="config", **config_leg(torch, cfg, peaks, 0, budget_ms=args.config_ms))) + "\n")
         out.flush()
-        del runner
-        torch.cuda.empty_cache()
 
 
 def run_merge_sweep(args, out):
     import torch
-    from paper_2609_04774_b200 import binding, build
+    from paper_2609_04774_b200 import build
     build.build()
     peaks = load_peaks()
-    ctx = binding.Context(0)
-    H, D = 64, 128
-    for T in args.merge_T:
-        for N in (2, 4, 8):
-            for dt in (torch.bfloat16, torch.float32):
-                in_bytes = N * T * H * (D * 4 + 4)
-                out_bytes = T * H * (D * dt.itemsize) + 4 * T * H
-                if in_bytes > 100e9:
-                    continue
-                parts = torch.randn((N, T, H, D), dtype=torch.float32, device="cuda")
-                lses = 8 + 2 * torch.randn((N, H, T), dtype=torch.float32, device="cuda")
-                lses[0].view(-1)[::16] = float("-inf")
-                o = torch.empty((T, H, D), dtype=dt, device="cuda")
-                lo = torch.empty((H, T), dtype=torch.float32, device="cuda")
-                flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if in_bytes < 512e6 else None
-
-                def fn():
-                    if flush is not None:
-                        flush.zero_()
-                    binding.cp_merge(ctx, parts, lses, o, lo)
-
-                for _ in range(3):
-                    fn()
-                torch.cuda.synchronize()
-                ds = []
-                for _ in range(args.merge_reps):
-                    if flush is not None:
-                        flush.zero_()
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                    binding.cp_merge(ctx, parts, lses, o, lo)
-                    e1.record()
-                    ds.append((e0, e1))
-                torch.cuda.synchronize()
-                ms = [a.elapsed_time(b) for a, b in ds]
-                med = statistics.median(ms)
-                gbs = (in_bytes + out_bytes) / (med * 1e-3) / 1e9
-                out.write(json.dumps({"mode": "merge", "T": T, "N": N, "H": H, "out": str(dt).split(".")[-1],
-                                      "bytes": in_bytes + out_bytes, "ms_median": med, "ms_best": min(ms), "GBps": gbs,
-                                      "frac_nominal_8000": gbs / NOMINAL_HBM_GBS, "frac_measured_copy": gbs / peaks["hbm_gbs"],
-                                      "l2_flush": flush is not None}) + "\n")
-                out.flush()
-                del parts, lses, o, lo, flush
-                torch.cuda.empty_cache()
+    points = [(T, N, dt) for T in args.merge_T for N in (2, 4, 8) for dt in (torch.bfloat16, torch.float32)
+              if N * T * 64 * 516 <= 100e9]
+    for m in merge_points(torch, peaks, points, reps=args.merge_reps):
+        out.write(json.dumps(dict(mode="merge", **m)) + "\n")
+    out.flush()
 
 
 def run_kvcopy(args, out):
-    """cp_kv_gather / cp_kv_append bandwidth: n tokens x 8 KV heads x 128 dims, K and V, shuffled pages."""
     import torch
-    from paper_2609_04774_b200 import binding, build
+    from paper_2609_04774_b200 import build
     build.build()
-    peaks = load_peaks()
-    ctx = binding.Context(0)
-    Hkv, D = 8, 128
-    for n in (16384, 131072, 1048576):
-        pages = n // wl.PAGE
-        k = torch.randn((pages, wl.PAGE, Hkv, D), device="cuda").to(torch.bfloat16)
-        v = torch.randn((pages, wl.PAGE, Hkv, D), device="cuda").to(torch.bfloat16)
-        pt = torch.from_numpy(wl.permutation(9, wl.TID_PERM, pages)).cuda()
-        cache = binding.make_cache(k, v)
-        kr = torch.empty((n, Hkv, D), dtype=torch.bfloat16, device="cuda")
-        vr = torch.empty_like(kr)
-        moved = 2 * 2 * n * Hkv * D * 2 + 4 * pages          # K and V, read + written, plus the table
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if moved < 512e6 else None
-        for name, fn in (("gather", lambda: binding.cp_kv_gather(ctx, cache, pt, 0, n, kr, vr)),
-                         ("append", lambda: binding.cp_kv_append(ctx, cache, pt, 0, n, kr, vr))):
-            ds = []
-            for i in range(13):
-                if flush is not None:
-                    flush.zero_()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                fn()
-                e1.record()
-                if i >= 3:
-                    ds.append((e0, e1))
-            torch.cuda.synchronize()
-            ms = statistics.median(a.elapsed_time(b) for a, b in ds)
-            gbs = moved / (ms * 1e-3) / 1e9
-            out.write(json.dumps({"mode": "kvcopy", "op": name, "tokens": n, "bytes": moved, "ms_median": ms, "GBps": gbs,
-                                  "frac_nominal_8000": gbs / NOMINAL_HBM_GBS, "frac_measured_copy": gbs / peaks["hbm_gbs"],
-                                  "l2_flush": flush is not None}) + "\n")
-            out.flush()
-        del k, v, kr, vr, flush
-        torch.cuda.empty_cache()
+    for m in kvcopy_points(torch, load_peaks(), (16384, 131072, 1048576)):
+        out.write(json.dumps(dict(mode="kvcopy", **m)) + "\n")
+    out.flush()
 
 
 def run_table(args, out):
@@ -671,7 +839,7 @@ def run_cprank(args, out):
             recv = (C - 1) * 2 * 2 * w.Hkv * D * (lay0.block_pages * wl.PAGE + 2 * lay0.cl)
         out.write(json.dumps({"mode": "cprank", "exchange": "pass-q" if args.pass_q else "all-gather-kv", "config": cfg, "workload": w.name, "R": R, "P": P, "C": C,
                               "rank_local_ms": per_rank, "slowest_rank_ms": max(per_rank),
-                              "tflops_per_gpu_slowest_rank": w.flops() / C / (max(per_rank) * 1e-3) / 1e12,
+                              "tflops_per_gpu_slowest_rank": flops_of(w) / C / (max(per_rank) * 1e-3) / 1e12,
                               "nvlink_bytes_received_per_rank": recv,
                               "nvlink_ms_modelled_at_770GBps": recv / 770e9 * 1e3,
                               "note": "local work measured with loopback gathers; link time modelled, not measured"}) + "\n")
@@ -739,10 +907,11 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, help="BASELINE config number of the headline workload")
+    ap.add_argument("--config", type=int, default=2, help="number of the configuration used as the headline workload")
     ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table", "kvcopy", "cprank", "cachemgr"])
     ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5],
                     help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P")
+    ap.add_argument("--config-ms", type=float, default=1200.0, help="configs mode: GPU time per configuration")
     ap.add_argument("--rank-reps", type=int, default=5)
     ap.add_argument("--pass-q", action="store_true", help="cprank mode: K/V stays sharded, queries travel")
     ap.add_argument("--cache-requests", type=int, default=20000)
@@ -750,9 +919,11 @@ def main():
     ap.add_argument("--merge-reps", type=int, default=20)
     ap.add_argument("--table-R", type=int, nargs="*", default=[1024, 2048, 4096, 8192, 16384, 32768, 65536, 131072])
     ap.add_argument("--out", default=None)
-    ap.add_argument("--cpu-rows", type=int, default=1024, help="rows per request of the cpu_baseline sample")
+    ap.add_argument("--cpu-rows", type=int, default=512, help="rows per request of the cpu_baseline sample")
     ap.add_argument("--ref-rows", type=int, default=96, help="rows per request per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="bench mode: only the headline workload (no sustained / configs / merge / kvcopy legs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

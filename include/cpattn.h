@@ -15,8 +15,9 @@
  *     memory only inside cp_ctx_create().
  *   - GPU calls validate their arguments first (an invalid call launches nothing), then only
  *     ENQUEUE work on the given stream (a cudaStream_t passed as void*, NULL = default stream)
- *     and return.  Device-side failures (a bounded wait that ran out) are recorded in a status
- *     word that cp_ctx_poll_status() reads after the caller has synchronised.
+ *     and return.  Device-side failures (a bounded wait that ran out, a page id outside the pool
+ *     met by a paged copy) are recorded in a status word that cp_ctx_poll_status() reads after the
+ *     caller has synchronised.
  *   - bf16 tensors are passed as void*; element strides are in elements.
  */
 #ifndef CPATTN_H
@@ -36,7 +37,8 @@ enum {
     CP_ERR_WORKSPACE = -3,   /* workspace missing, misaligned or smaller than cp_workspace_bytes() */
     CP_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                                */
     CP_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (reported by poll_status)       */
-    CP_ERR_BOUNDS = -6       /* a host-visible index (page id, range) is out of range              */
+    CP_ERR_BOUNDS = -6       /* an index is out of range: a page-table size seen by the host, or a
+                                page id met by cp_kv_gather / cp_kv_append on the device (poll_status) */
 };
 
 enum { CP_DTYPE_BF16 = 0, CP_DTYPE_F32 = 1 };
@@ -49,8 +51,9 @@ const char* cp_last_error(void);
  * buffer for tile lists and the resolved driver entry point for tensor-map encoding.
  * cp_ctx_create() makes `device` current and allocates; cp_ctx_destroy() frees.
  * cp_ctx_poll_status() synchronises the device-to-host copy of the status word on the default
- * stream (call it after synchronising the streams you used): returns CP_OK or CP_ERR_TIMEOUT and,
- * when `detail` is non-NULL, writes 4 int32 words {code, barrier id, block, iteration}; the
+ * stream (call it after synchronising the streams you used): returns CP_OK, CP_ERR_TIMEOUT or
+ * CP_ERR_BOUNDS and, when `detail` is non-NULL, writes 4 int32 words ({code, barrier id, block,
+ * iteration} for a time-out, {code, page-table index, block, page id} for a bad page id); the
  * status word is cleared by the call.
  * ------------------------------------------------------------------------------------------- */
 typedef struct cp_ctx cp_ctx;
@@ -63,8 +66,9 @@ int cp_ctx_poll_status(cp_ctx* ctx, int32_t* detail /* host, 4 words or NULL */)
  * cache contents and out differ).  With reuse on, a call whose schedule-relevant arguments AND workspace are
  * the previous call's skips the host-side scheduling and the upload and launches on the work lists already
  * in the workspace (about 20-100 us of host time per call and one small kernel).  While it is on, the caller
- * must not modify the workspace between such calls, nor hand it to another context.  Turning it on or off
- * forgets the remembered schedule.  Errors: INVALID_ARG. */
+ * must not modify the workspace between such calls, nor hand it to another context, and must issue the
+ * calls on one stream (or order the streams behind the first call: a large schedule is uploaded on the stream
+ * of the call that built it).  Turning it on or off forgets the remembered schedule.  Errors: INVALID_ARG. */
 int cp_ctx_cache_schedule(cp_ctx* ctx, int enable);
 
 /* cp_ctx_selftest_wait_expiry -- diagnostic (the paper has no counterpart): enqueues one small block whose
@@ -121,13 +125,17 @@ typedef struct {
 size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C, int32_t Hq);
 
 /* cp_schedule_inspect -- host only: the work distribution the attention calls would use for a batch
- * on a device with num_sms SMs (the varlen tile schedule: query tiles of at most 128 rows cut at the
- * chunk boundaries of every request's zigzag plan; one unit per tile and pair of query heads (per
+ * on a device with num_sms SMs (the varlen tile schedule: query tiles of 128 rows, the last tile of a
+ * request possibly shorter -- a launch over all shards walks a request's rows as one run, so a tile may span
+ * adjacent zigzag chunks but never two requests; one unit per tile and pair of query heads (per
  * single head when Hq / Hkv is odd); whole
  * units longest first -- KV head by KV head when the batch's K/V exceeds 32 MB, so that a long context's K/V
  * stays in L2 -- dealt to the CTAs in serpentine order, the remainder cut along KV so that every
- * CTA gets the same number of KV tile steps).  summary (8 values): CTAs, query tiles, pieces, split units,
- * partial slots, largest / smallest per-CTA load in KV tile steps, their total.  pieces (optional,
+ * CTA gets the same number of KV tile steps; when there are no more units than CTAs and all are short, every
+ * unit gets a CTA of its own and nothing is cut).  summary (10 values): CTAs, query tiles, pieces, split units,
+ * partial slots, largest / smallest per-CTA load in KV tile steps, their total, 1 if the work lists are small
+ * enough to ride in the launch parameters, kernel launches the attention call makes (list copy unless they
+ * ride along + attention + merge of split units if any).  pieces (optional,
  * 6 int32 per piece: cta, tile, head pair, first KV tile, end KV tile, partial slot or -1) and
  * items (optional, 4 int32 per tile: first packed row, rows, keys visible to the first row, KV tiles)
  * are filled when non-NULL and large enough (CP_ERR_WORKSPACE otherwise). */
@@ -145,13 +153,17 @@ int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_
  *   out        device [R, Hq, D] bf16; row r = softmax(scale * q_r K^T + mask) V, written at its
  *              original position (the "restore order" step is fused into the store)
  *   lse        device [Hq, R] fp32: natural-log sum-exp of the scaled scores of each row
- * Every shard's q-tiles are cut at chunk boundaries of cp_plan(R, P, C); the result does not
- * depend on C.  Requires Hq % Hkv == 0 (query head h uses KV head h / (Hq / Hkv)); with an even group
+ * The C shards of cp_plan(R, P, C) are row-disjoint and together cover all R rows (Section 2.1), and
+ * adjacent chunks are adjacent rows with consecutive causal limits, so the launch walks the rows as one
+ * run of 128-row query tiles with a per-row limit; C is validated, and the result does not depend on it
+ * (the calls that compute ONE shard or ONE chunk cut their tiles at the chunk's boundaries).  Requires Hq % Hkv == 0 (query head h uses KV head h / (Hq / Hkv)); with an even group
  * size two query heads of a group share every K/V tile in shared memory, with an odd one (e.g.
  * Hq == Hkv) every head streams K/V on its own: its KV tiles then alternate between the two softmax warpgroups (two
  * online-softmax streams combined at the end), at about 80 % of the throughput (1090 against 1355 TFLOP/s on
  * config 2's lengths).  One persistent launch computes all tiles; the few units that were split along KV
- * to balance the SMs are combined by a second small launch (an LSE merge of their partials).  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ * to balance the SMs are combined by a second small launch (an LSE merge of their partials).  Work lists of
+ * up to 3 KB travel in the launch parameters; larger ones are first copied into the workspace by a small
+ * kernel.  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
  * ------------------------------------------------------------------------------------------- */
 int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
                     int64_t prefix_len, int64_t new_len, int32_t C, int32_t Hq, float scale,
@@ -169,8 +181,8 @@ int cp_prefill_attn_batch(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, 
 
 /* cp_prefill_attn_shard -- only the rows of shard `shard` (0 <= shard < C) of cp_plan(R, P, C):
  * what one CP rank computes.  partial_out: device [R, Hq, D] fp32, partial_lse: device [Hq, R]
- * fp32; rows the shard does not own are written 0 with lse = -inf, so that cp_merge over the C
- * shard partials reproduces cp_prefill_attn exactly. */
+ * fp32; rows the shard does not own are written 0 with lse = -inf (by a spare warp of the same
+ * launch), so that cp_merge over the C shard partials reproduces cp_prefill_attn exactly. */
 int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
                           int64_t prefix_len, int64_t new_len, int32_t C, int32_t shard, int32_t Hq,
                           float scale, float* partial_out, float* partial_lse, void* workspace,
@@ -195,9 +207,8 @@ int cp_prefill_attn_chunk(cp_ctx* ctx, const void* q_chunk, const cp_kv_cache* c
 
 /* cp_prefill_attn_kvrange -- all R queries against the keys whose absolute position lies in
  * [kv_lo, kv_hi) only (still causal: new token r sees positions <= P + r): the partial result a CP rank
- * produces when the K/V stays sharded over the ranks and the queries travel instead (the alternative to the
- * all-gather of Section 2.1; the paper keeps a worker's cached KV "partitioned across its ranks",
- * Section 2.2).  partial_out: device [R, Hq, D] fp32, normalised over the keys of the range; partial_lse:
+ * produces when the K/V stays sharded over the ranks and the queries travel instead (the alternative to
+ * Section 2.1's all-gather when a worker's cached KV stays spread over its ranks, Section 2.2).  partial_out: device [R, Hq, D] fp32, normalised over the keys of the range; partial_lse:
  * device [Hq, R] fp32; a row that sees no key of the range gets zeros and lse = -inf.  Partials over
  * disjoint ranges that together cover [0, P + R) combine with cp_merge into cp_prefill_attn's result.
  * Only pages holding keys of the range are read.  kv_lo, kv_hi need no alignment.  Workspace as for
@@ -218,8 +229,11 @@ int cp_prefill_attn_kvrange(cp_ctx* ctx, const void* q, const cp_kv_cache* cache
  * words live in a fixed device array of 65,792 bytes that is part of the library image (every GPU
  * that loads the library holds it until the process exits).
  *   - Same arguments, result and limits as cp_prefill_attn, computed on the CURRENT device.
- *   - Size limit: ceil(new_len / 128) + 2*C must not exceed 2048 query tiles (about 260K new
- *     tokens); larger requests return CP_ERR_WORKSPACE and launch nothing.
+ *   - Size limit: ceil(new_len / 128) must not exceed 2048 query tiles (262,144 new tokens);
+ *     larger requests return CP_ERR_WORKSPACE and launch nothing.
+ *   - Two launches on the given stream: a small kernel that clears the status words and writes
+ *     the tile list from (new_len, prefix_len) passed by value, then the attention kernel.  No
+ *     host buffer is read after the call returns.
  *   - The first call on each device resolves the device address of the array, the tensor-map
  *     encoder and the kernel's shared-memory attribute; make that first call before any stream
  *     capture begins.
@@ -236,7 +250,10 @@ int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, const int32_
 
 /* ---------------------------------------------------------------------------------------------
  * cp_merge -- N-way log-sum-exp combination of partial attention results over the same rows
- * (what joins per-shard or KV-split partials into full-sequence attention).
+ * (what joins per-shard or KV-split partials into full-sequence attention).  The paper states no
+ * such step: its CP outputs are row-disjoint and are concatenated (Section 2.1).  This is the general
+ * combine the library adds; row-disjoint shard partials (lse = -inf on rows a shard does not own) are
+ * the special case that reproduces the paper's concatenation.
  *   partials device [N, T, H, D] fp32;  lses device [N, H, T] fp32 (natural log; -inf = "this
  *   partial holds nothing for the row": its values are ignored even if non-finite)
  *   out      device [T, H, D], bf16 or fp32 (out_dtype = CP_DTYPE_*)
@@ -249,8 +266,13 @@ int cp_merge(cp_ctx* ctx, const float* partials, const float* lses, int32_t N, i
 
 /* ---------------------------------------------------------------------------------------------
  * Paged <-> contiguous copies of n logical tokens starting at t_begin (the prefix-KV gather path
- * as a standalone op).  k_rows / v_rows: device [n, Hkv, D] bf16, contiguous.  page_table: device.
- * Bit-exact copies.  Either of the k/v pairs may be NULL to copy only the other.
+ * as a standalone op: Section 2.2 has the cached prefix KV resident at the worker, block by block;
+ * the paper names no copy routine).  k_rows / v_rows: device [n, Hkv, D] bf16, contiguous.
+ * page_table: device, at least ceil((t_begin + n) / page_size) entries, each in [0, num_pages).
+ * Bit-exact copies.  Either of the k/v pairs may be NULL to copy only the other.  An entry outside
+ * [0, num_pages) is never used as an address: the elements behind it are skipped (not read, not
+ * written) and the first such entry is reported as CP_ERR_BOUNDS by cp_ctx_poll_status().
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
  * ------------------------------------------------------------------------------------------- */
 int cp_kv_gather(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin,
                  int64_t n, void* k_rows, void* v_rows, void* stream);

@@ -1,7 +1,7 @@
 /* cpcache.h -- prefix-cache bookkeeping of the adaptive-CP serving system: the global prefix trie with
  * its per-degree demand statistics, the per-request update (Algorithm 1), the periodic scan
  * (Algorithm 2) with the ranking rules that follow it, the prefill-time model (Eq. 2) and
- * PreferDegree (Section 6.1).  Host-only integer and double arithmetic; part of libcpattn.so.
+ * PreferDegree (Section 7.1).  Host-only integer and double arithmetic; part of libcpattn.so.
  *
  * Conventions as in cpattn.h: every call returns CP_OK (0) or a negative CP_ERR_* code and leaves a
  * message for cp_last_error(); nothing throws across the boundary; all arrays are caller-owned host
@@ -28,7 +28,7 @@ typedef struct { double d, a, b, c, alpha; } cp_prefill_model;
  * Returns NaN when model is NULL or C < 1. */
 double cp_prefill_time(const cp_prefill_model* model, int64_t R, int64_t P, int32_t C);
 
-/* PreferDegree (Section 6.1): the worker minimising the placement cost of Section 5.3 without its
+/* PreferDegree (Section 7.1): the worker minimising the placement cost of Section 5.3 without its
  * queueing term,  beta * s_w + lambda * (C_w * s_w - C_min * E_{C_min}(R_w, P_w)),  where
  * P_w = reused_len[w] is the prefix the worker can reuse, R_w = L - P_w, s_w = E_{C_w}(R_w, P_w) and
  * C_min is the smallest degree among the n workers.  The first minimum wins a tie.

@@ -2,7 +2,7 @@
 the library's cp_trie_* calls.  Nothing in the product path may import this file.
 
 What it restates, in the paper's notation:
-  * the prefix trie of Section 6.1: one node per cache block, the path from the root is the prefix; every
+  * the prefix trie of Section 7.1: one node per cache block, the path from the root is the prefix; every
     node records which workers hold the complete prefix ending there, and per supported CP degree the
     statistics access[z, C] and missed[z, C];
   * ReplicaCount(z, C), MatchedPath(i), ReusedPath(i, w);

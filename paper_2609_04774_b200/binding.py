@@ -143,12 +143,12 @@ def cp_schedule_inspect(cu_new, prefix_len, C, Hq, Hkv, num_sms=148, want_lists=
     """Host-only view of the varlen tile schedule: (summary dict, pieces [n,6] int32, items [n,4] int32)."""
     cu_new, prefix_len, C = _i64(cu_new), _i64(prefix_len), _i32(C)
     B = prefix_len.size
-    summary = np.zeros(8, dtype=np.int64)
+    summary = np.zeros(10, dtype=np.int64)
     args = [ctypes.c_int32(B), cu_new.ctypes.data_as(ctypes.c_void_p), prefix_len.ctypes.data_as(ctypes.c_void_p),
             C.ctypes.data_as(ctypes.c_void_p), ctypes.c_int32(Hq), ctypes.c_int32(Hkv), ctypes.c_int32(num_sms),
             summary.ctypes.data_as(ctypes.c_void_p)]
     _check(load().cp_schedule_inspect(*args, None, ctypes.c_int64(0), None, ctypes.c_int64(0)))
-    keys = ["grid", "tiles", "pieces", "split_units", "slots", "max_load", "min_load", "total"]
+    keys = ["grid", "tiles", "pieces", "split_units", "slots", "max_load", "min_load", "total", "inline", "launches"]
     info = dict(zip(keys, (int(x) for x in summary)))
     if not want_lists:
         return info, None, None

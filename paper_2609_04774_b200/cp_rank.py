@@ -20,11 +20,12 @@ instead of (P+R)*Hkv*D*2 key/value bytes, which pays when the cached prefix is m
 
 Readings (the paper fixes none of these): prefix pages are owned in contiguous blocks of
 ceil(n_prefix_pages / C) pages, block r on rank r; the prefix length is a multiple of the page size
-(block-granular reuse, Section 6); chunks are padded to cl = ceil(R / 2C) rows for the collective.
+(block-granular reuse, Section 7.1); chunks are padded to cl = ceil(R / 2C) rows for the collective.
 """
 from __future__ import annotations
 
 from dataclasses import dataclass
+from functools import cached_property
 
 
 @dataclass(frozen=True)
@@ -42,13 +43,22 @@ class RankLayout:
         if self.P % self.page:
             raise ValueError("prefix length %d is not a multiple of the page size %d" % (self.P, self.page))
 
+    @cached_property
+    def _plan(self):
+        """The library's shard plan of the request (cp_plan): the one place the chunk arithmetic lives."""
+        from . import binding
+        return binding.cp_plan(self.R, self.P, self.C)
+
     @property
     def cl(self) -> int:
-        return -(-self.R // (2 * self.C))
+        """Rows of a full chunk (chunk 0 is never short): what every chunk is padded to for the collectives."""
+        s0 = self._plan[0]
+        return s0["q_end"][0] - s0["q_begin"][0]
 
     def chunk(self, j: int):
-        """Rows [begin, end) of zigzag chunk j (right-padded split, clipped to R)."""
-        return min(j * self.cl, self.R), min((j + 1) * self.cl, self.R)
+        """Rows [begin, end) of zigzag chunk j: shard min(j, 2C-1-j) of the plan holds it as its early or late chunk."""
+        s, half = (self._plan[j], 0) if j < self.C else (self._plan[2 * self.C - 1 - j], 1)
+        return s["q_begin"][half], s["q_end"][half]
 
     @property
     def early(self) -> int:

@@ -11,8 +11,9 @@
 //   warp  8    TMA producer (the warp prefetches page ids; the pages of a tile go out from several lanes)
 //   warp  9    tcgen05.mma issuer for the scores S = Q K^T (warp-uniform loop, one elected lane issues)
 //   warp  10   tcgen05.mma issuer for O += P V
-//   warp  11   idle (completes the third warpgroup so that register budgets can be moved: the softmax
-//              warpgroups run with 200 registers per thread, the third one with 104)
+//   warp  11   spare (completes the third warpgroup so that register budgets can be moved: the softmax
+//              warpgroups run with 200 registers per thread, the third one with 104); in the calls that
+//              produce partial results it writes zeros / -inf into the rows the call does not compute
 // TMEM (512 columns): S | P0 | P1 | O0 | O1.  S is ONE score buffer (128 fp32 columns) that the two heads
 // use in turn; P (bf16, 64 columns per head) is the TMEM A operand of P*V; O0, O1 are the accumulators.
 // A softmax warpgroup reads its score tile into registers and hands the buffer back at once, so the next
@@ -109,6 +110,13 @@ struct AttnParams {
     float* lse;
     int64_t lse_stride;       // total rows
     int32_t* status;
+    // byte offsets of items / cta_off / pieces inside the launch-parameter copy of a small schedule; < 0: the
+    // lists are in global memory behind the pointers above
+    int32_t inl_items, inl_cta_off, inl_pieces;
+    // partial-result calls: row ranges [fill[2i], fill[2i+1]) that no tile covers get zeros (out, fp32) and
+    // lse = -inf from the kernel's spare warp
+    int32_t n_fill;
+    int32_t fill[2 * kMaxFillRanges];
 };
 
 // ------------------------------------------------------------------------------------------
@@ -301,19 +309,6 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar_base, uint32_t bar_id, ui
     }
 }
 
-// Optional phase trace (build with -DCPATTN_TRACE): block 0 stamps clock64() at fixed points of the
-// first 64 KV tiles of its first unit into the area behind the status words.
-#ifndef CPATTN_TRACE_ROW
-#define CPATTN_TRACE_ROW 0
-#endif
-#ifdef CPATTN_TRACE
-#define CP_TRACE(who, j, e)                                                                              \
-    if (blockIdx.x == 0 && round == 0 && (j) < 64)                                                       \
-        reinterpret_cast<long long*>(p.status + 16)[(((who)*64 + (j)) * 8) + (e)] = clock64();
-#else
-#define CP_TRACE(who, j, e)
-#endif
-
 // One piece of work of a CTA: KV tiles [t_begin, t_end) of one query tile for one pair of heads.
 struct UnitInfo {
     TileItem it;
@@ -327,18 +322,22 @@ struct UnitInfo {
 // ranges of units that were split to fill every CTA to the same number of KV tile steps.  Implicit:
 // serpentine over the longest-first unit list -- in even rounds CTA c takes unit round*grid + c, in
 // odd rounds round*grid + (grid-1-c), which evens out the sorted lengths; whole units only.
-__device__ __forceinline__ bool fetch_unit(const AttnParams& p, int round, UnitInfo& u) {
+__device__ __forceinline__ bool fetch_unit(const AttnParams& p, const InlineSched& inl, int round, UnitInfo& u) {
     int item, pair;
-    if (p.pieces != nullptr) {
-        const int idx = p.cta_off[blockIdx.x] + round;
-        if (idx >= p.cta_off[blockIdx.x + 1]) return false;
-        const PieceEntry e = p.pieces[idx];
+    // a small schedule sits in the launch parameters (constant bank), a large one in the workspace
+    const TileItem* items = p.inl_items >= 0 ? reinterpret_cast<const TileItem*>(inl.bytes + p.inl_items) : p.items;
+    if (p.pieces != nullptr || p.inl_pieces >= 0) {
+        const int32_t* cta_off = p.inl_cta_off >= 0 ? reinterpret_cast<const int32_t*>(inl.bytes + p.inl_cta_off) : p.cta_off;
+        const PieceEntry* pieces = p.inl_pieces >= 0 ? reinterpret_cast<const PieceEntry*>(inl.bytes + p.inl_pieces) : p.pieces;
+        const int idx = cta_off[blockIdx.x] + round;
+        if (idx >= cta_off[blockIdx.x + 1]) return false;
+        const PieceEntry e = pieces[idx];
         item = e.item;
         pair = e.pair;
         u.t_begin = e.t_begin;
         u.t_end = e.t_end;
         u.slot = e.slot;
-        u.it = p.items[item];
+        u.it = items[item];
     } else {
         const int g = gridDim.x;
         const int c = (round & 1) ? (g - 1 - (int)blockIdx.x) : (int)blockIdx.x;
@@ -356,7 +355,7 @@ __device__ __forceinline__ bool fetch_unit(const AttnParams& p, int round, UnitI
             item = (int)(idx / p.pairs_per_tile);
             pair = (int)(idx - (int64_t)item * p.pairs_per_tile);
         }
-        u.it = p.items[item];
+        u.it = items[item];
         u.t_begin = 0;
         u.t_end = u.it.n_kv_tiles;
         u.slot = -1;
@@ -373,13 +372,13 @@ __device__ __forceinline__ bool fetch_unit(const AttnParams& p, int round, UnitI
 // Roles
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV, const AttnParams& p,
-                              uint32_t smem_base, volatile uint32_t* abort_flag) {
+                              const InlineSched& inl, uint32_t smem_base, volatile uint32_t* abort_flag) {
     const int lane = threadIdx.x & 31;
     const uint32_t bars = smem_base + kSmemBar;
     uint32_t kv_it = 0;   // ring slots filled so far
     for (int round = 0;; ++round) {
         UnitInfo u;
-        if (!fetch_unit(p, round, u)) break;
+        if (!fetch_unit(p, inl, round, u)) break;
         if (lane == 0) {
             mbar_wait(bars, kBarQEmpty, (round & 1) ^ 1, abort_flag, p.status, round);
             const uint32_t qbar = bars + kBarQFull * 8;
@@ -418,7 +417,6 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
             const CUtensorMap* map = kv ? tmV : tmK;
             if (lane == 0) {
                 mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j);
-                CP_TRACE(3, j, 6 + kv);
                 mbar_expect_tx(fbar, kTileBytes);
             }
             __syncwarp();
@@ -457,7 +455,7 @@ struct RingPos {
 //
 // Score issuer: S tiles in the order (tile, head); each needs its K tile and the buffer back (s_free).
 template <bool kDual>
-__device__ __forceinline__ void mma_s_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
+__device__ __forceinline__ void mma_s_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
                                            volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
     constexpr int H = kDual ? 1 : 2;
@@ -467,7 +465,7 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, uint32_t smem_ba
     const uint64_t k_desc0 = make_desc(smem_base + kSmemKV, 16, 1024);           // K-major view of a ring slot
     for (int round = 0;; ++round) {
         UnitInfo u;
-        if (!fetch_unit(p, round, u)) break;
+        if (!fetch_unit(p, inl, round, u)) break;
         const int j0 = u.t_begin, n = u.t_end;
         mbar_wait(bars, kBarQFull, round & 1, abort_flag, p.status, round);
         RingPos kpos = unit_pos;
@@ -480,7 +478,6 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, uint32_t smem_ba
                 mbar_wait(bars, kBarSFree, s_par, abort_flag, p.status, j);
                 s_par ^= 1u;
                 tc_fence_after();
-                if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + h, j, 2); }
                 if (elect_one()) {
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
@@ -495,7 +492,6 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, uint32_t smem_ba
                     }
                 }
                 __syncwarp();
-                if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + h, j, 3); }
             }
             kpos = kpos.plus(j == j0 ? 1 : 2);     // load order: K(j0), K(j0+1), V(j0), K(j0+2), V(j0+1), ...
         }
@@ -510,7 +506,7 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, uint32_t smem_ba
 // single-head unit the tiles alternate between the two P / O column sets (two independent online-softmax
 // streams over the even and the odd tiles of the piece, combined in the epilogue).
 template <bool kDual>
-__device__ __forceinline__ void mma_pv_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
+__device__ __forceinline__ void mma_pv_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
                                             volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
     constexpr int H = kDual ? 1 : 2;
@@ -519,7 +515,7 @@ __device__ __forceinline__ void mma_pv_role(const AttnParams& p, uint32_t smem_b
     const uint64_t v_desc0 = make_desc(smem_base + kSmemKV, kHalfBytes, 1024);   // MN-major view of a ring slot
     for (int round = 0;; ++round) {
         UnitInfo u;
-        if (!fetch_unit(p, round, u)) break;
+        if (!fetch_unit(p, inl, round, u)) break;
         const int j0 = u.t_begin, n = u.t_end;
         RingPos vpos = unit_pos.plus(n - j0 == 1 ? 1 : 2);   // V(j0)
 #pragma unroll 1
@@ -534,7 +530,6 @@ __device__ __forceinline__ void mma_pv_role(const AttnParams& p, uint32_t smem_b
                 for (int part = 0; part < kPieces; ++part) {
                     mbar_wait(bars, kBarPReady + wgt * 4 + part, ppar, abort_flag, p.status, j);
                     tc_fence_after();
-                    if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wgt, j, part); }
                     if (elect_one()) {
                         const int ks0 = part == 0 ? 0 : 2 * kSplitQ, ks1 = part == 0 ? 2 * kSplitQ : 8;
 #pragma unroll
@@ -551,7 +546,6 @@ __device__ __forceinline__ void mma_pv_role(const AttnParams& p, uint32_t smem_b
                     }
                     __syncwarp();
                 }
-                if ((threadIdx.x & 31) == 0) { CP_TRACE(2 + wgt, j, 5); }
                 if (wgt) p_par1 ^= 1u; else p_par0 ^= 1u;
             }
             vpos = vpos.plus(j + 2 == n ? 1 : 2);
@@ -613,7 +607,6 @@ struct SoftmaxSync {
     volatile uint32_t* abort_flag;
     int32_t* status;
     int iter;
-    long long* tr;                   // trace builds: stamp row of this tile (or NULL)
 };
 
 // Reads the 128 scores of this thread's row from the S buffer (the caller has seen s_ready).
@@ -646,7 +639,6 @@ __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], f
                                              bool more, uint32_t& s_par, uint32_t s_tmem, uint32_t p_tmem,
                                              uint32_t o_tmem, uint32_t p_bar0, float c, int lo, int lim, bool first,
                                              float& m, float& l, const SoftmaxSync& sy) {
-    if (sy.tr) sy.tr[1] = clock64();
     if (kMasked) {
         mask32(c0, lo, lim);
         mask32(c1, lo - 32, lim - 32);
@@ -667,7 +659,6 @@ __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], f
         mbar_wait(sy.bars, sy.pv_done_id, sy.pv_parity, sy.abort_flag, sy.status, sy.iter);
         __syncwarp();
         tc_fence_after();
-        if (sy.tr) sy.tr[2] = clock64();
         const bool grow = (m_new - m) > kRescaleThreshold;
         if (__any_sync(0xffffffffu, grow)) {
             const float m_upd = grow ? m_new : m;
@@ -700,7 +691,6 @@ __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], f
         tc_fence_before();                                                              \
         __syncwarp();                                                                   \
         if ((threadIdx.x & 31) == 0) mbar_arrive(p_bar0 + ((q) == 3 ? 1 : 0) * 8);      \
-        if (sy.tr) sy.tr[(q) == 3 ? 4 : 3] = clock64();                                 \
     }
     CP_P_PIECE(c0, 0)
     CP_P_PIECE(c1, 1)
@@ -736,7 +726,7 @@ __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], f
 }
 
 template <bool kDual>
-__device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_base, uint32_t tmem_base,
+__device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
                                              volatile uint32_t* abort_flag, uint8_t* smem_xchg, int wg) {
     const uint32_t bars = smem_base + kSmemBar;
     const int lane = threadIdx.x & 31;
@@ -757,18 +747,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
 #define SM_WAIT(id, parity, it)                                                                  \
     mbar_wait(bars, (id), (parity), abort_flag, p.status, (it));                                 \
     __syncwarp();
-#ifdef CPATTN_TRACE
-#define CP_TRACE_ROW_PTR(j_)                                                                                \
-    long long* tr = (row == CPATTN_TRACE_ROW && blockIdx.x == 0 && round == 0 && (j_) < 64)                 \
-                        ? reinterpret_cast<long long*>(p.status + 16) + (wg * 64 + (j_)) * 8 : nullptr;
-#else
-#define CP_TRACE_ROW_PTR(j_) long long* const tr = nullptr;
-#endif
     uint32_t s_par = 0;        // phase parity of s_ready for this head
 
     for (int round = 0;; ++round) {
         UnitInfo u;
-        if (!fetch_unit(p, round, u)) break;
+        if (!fetch_unit(p, inl, round, u)) break;
         const int n = u.t_end;
         const int head = u.head0 + (dual ? 0 : wg);
         const int j_first = u.t_begin + (dual ? wg : 0);     // first tile of this warpgroup's stream
@@ -789,10 +772,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
         }
 #pragma unroll 1
         for (int j = j_first; j < n; j += step) {
-            CP_TRACE_ROW_PTR(j)
-            if (tr) tr[0] = clock64();
             const SoftmaxSync sy = {bars, kBarSReady + (uint32_t)wg, kBarPvDone + (uint32_t)wg, (tile_cnt - 1) & 1,
-                                    abort_flag, p.status, j, tr};
+                                    abort_flag, p.status, j};
             if (j < n_full && j != j_cut)
                 softmax_tile<false>(s0, s1, s2, s3, j + step < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c, 0, 0,
                                     j == j_first, m, l, sy);
@@ -800,7 +781,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
                 softmax_tile<true>(s0, s1, s2, s3, j + step < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c,
                                    u.it.kv_lo - j * kBlockN, min(u.it.kv_len0 + row, u.it.kv_hi) - j * kBlockN,
                                    j == j_first, m, l, sy);
-            if (row == CPATTN_TRACE_ROW) { CP_TRACE(wg, j, 6); }
             ++tile_cnt;
         }
         float a_own = 1.f, a_oth = 0.f;     // dual: weights of the two streams' accumulators in the combined row
@@ -891,12 +871,31 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, uint32_t smem_
 #undef SM_WAIT
 }
 
+// The spare warp of every CTA: rows of a partial-result call that no tile covers (rows of other shards, rows
+// that see no key of the key range) get zeros and lse = -inf here, so that the call needs no launch besides
+// this one.  out is fp32 [rows, Hq, D], so a row range is one contiguous run of floats.
+__device__ __forceinline__ void fill_role(const AttnParams& p) {
+    const int lane = threadIdx.x & 31;
+    const int64_t start = (int64_t)blockIdx.x * 32 + lane, stride = (int64_t)gridDim.x * 32;
+    for (int g = 0; g < p.n_fill; ++g) {
+        const int64_t b = p.fill[2 * g], n = p.fill[2 * g + 1] - b;
+        float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + b * p.Hq * kD);
+        const int64_t n4 = n * p.Hq * (kD / 4);
+        for (int64_t i = start; i < n4; i += stride) o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int64_t nl = n * p.Hq;
+        for (int64_t i = start; i < nl; i += stride) {
+            const int64_t h = i / n;
+            p.lse[h * p.lse_stride + b + (i - h * n)] = -INFINITY;
+        }
+    }
+}
+
 // kDual: every unit is a single query head (odd group size); its KV tiles then alternate between the two
 // softmax warpgroups.  Two separate kernels, so that neither carries the other's code in its hot loop.
 template <bool kDual>
 __global__ void __launch_bounds__(kThreads, 1)
 cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-               const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+               const __grid_constant__ CUtensorMap tmV, const AttnParams p, const __grid_constant__ InlineSched inl) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -933,15 +932,17 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-        softmax_role<kDual>(p, smem_base, tmem_base, abort_flag, smem_gen + kSmemXchg, warp >> 2);
+        softmax_role<kDual>(p, inl, smem_base, tmem_base, abort_flag, smem_gen + kSmemXchg, warp >> 2);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
         if (warp == 8) {
-            producer_role(&tmQ, &tmK, &tmV, p, smem_base, abort_flag);
+            producer_role(&tmQ, &tmK, &tmV, p, inl, smem_base, abort_flag);
         } else if (warp == 9) {
-            mma_s_role<kDual>(p, smem_base, tmem_base, abort_flag);
+            mma_s_role<kDual>(p, inl, smem_base, tmem_base, abort_flag);
         } else if (warp == 10) {
-            mma_pv_role<kDual>(p, smem_base, tmem_base, abort_flag);
+            mma_pv_role<kDual>(p, inl, smem_base, tmem_base, abort_flag);
+        } else if (p.n_fill > 0) {
+            fill_role(p);
         }
     }
 
@@ -972,9 +973,18 @@ __global__ void wait_expiry_selftest_kernel(int32_t* status, long long limit_cyc
     mbar_wait(smem_u32(&bar), 0, 0, &abort_flag, status, 7, limit_cycles);
 }
 
-__global__ void fill_neg_inf_kernel(float* p, int64_t n) {
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
-        p[i] = -INFINITY;
+// Rows [b, b + n) of a partial result that the call computes nothing for: zeros and lse = -inf.  Only used when
+// the attention kernel itself is not launched (the shard owns no row) or has more gaps than it takes.
+__global__ void fill_rows_kernel(float* out, float* lse, int64_t lse_stride, int64_t b, int64_t n, int Hq) {
+    const int64_t start = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (int64_t)gridDim.x * blockDim.x;
+    float4* o = reinterpret_cast<float4*>(out + b * Hq * kD);
+    const int64_t n4 = n * Hq * (kD / 4);
+    for (int64_t i = start; i < n4; i += stride) o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int64_t nl = n * Hq;
+    for (int64_t i = start; i < nl; i += stride) {
+        const int64_t h = i / n;
+        lse[h * lse_stride + b + (i - h * n)] = -INFINITY;
+    }
 }
 
 // LSE merge of the KV-split units: block b combines the partial slots of merges[b] into the final
@@ -991,15 +1001,19 @@ struct FixupParams {
     int32_t heads_per_unit;
     float* lse;
     int64_t lse_stride;
+    int32_t inl_items, inl_merges, inl_merge_slots;   // >= 0: the list sits at this byte offset of the launch-parameter copy
 };
 
 constexpr int kFixupRowsPerBlock = 16;    // 8 warps x 2 (head, row) combinations
 
 // grid = (split units, 256 / kFixupRowsPerBlock): each warp combines two rows; the partial LSEs of a
 // row are loaded 32 slots at a time (lane k holds slot k), max and sum by warp shuffles.
-__global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p) {
-    const MergeEntry me = p.merges[blockIdx.x];
-    const TileItem it = p.items[me.item];
+__global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p, const __grid_constant__ InlineSched inl) {
+    const TileItem* items = p.inl_items >= 0 ? reinterpret_cast<const TileItem*>(inl.bytes + p.inl_items) : p.items;
+    const MergeEntry* merges = p.inl_merges >= 0 ? reinterpret_cast<const MergeEntry*>(inl.bytes + p.inl_merges) : p.merges;
+    const int32_t* merge_slots = p.inl_merge_slots >= 0 ? reinterpret_cast<const int32_t*>(inl.bytes + p.inl_merge_slots) : p.merge_slots;
+    const MergeEntry me = merges[blockIdx.x];
+    const TileItem it = items[me.item];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
 #pragma unroll
@@ -1012,7 +1026,7 @@ __global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p)
         float m = -INFINITY;
         for (int base = 0; base < me.n_slots; base += 32) {
             if (base + lane < me.n_slots) {
-                const int slot = p.merge_slots[me.slot_off + base + lane];
+                const int slot = merge_slots[me.slot_off + base + lane];
                 m = fmaxf(m, p.partial_lse[((int64_t)slot * 2 + wg) * kBlockM + row]);
             }
         }
@@ -1025,7 +1039,7 @@ __global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p)
             int my_slot = 0;
             float w_mine = 0.f;
             if (base + lane < me.n_slots) {
-                my_slot = p.merge_slots[me.slot_off + base + lane];
+                my_slot = merge_slots[me.slot_off + base + lane];
                 const float my_lse = p.partial_lse[((int64_t)my_slot * 2 + wg) * kBlockM + row];
                 w_mine = (my_lse == -INFINITY) ? 0.f : __expf(my_lse - m);
             }
@@ -1123,10 +1137,20 @@ int upload_block(cp_ctx* ctx, const std::vector<uint8_t>& block, void* dst, cuda
 // Page size for sizing a page table before the cache has been validated (a bad value is rejected later).
 inline int64_t page_tokens_of(const cp_kv_cache* c) { return (c && c->page_size > 0) ? c->page_size : kDefaultPageTokens; }
 
+int launch_fill_rows(float* out, float* lse, int64_t lse_stride, int64_t b, int64_t n, int32_t Hq, cudaStream_t s) {
+    if (n <= 0) return CP_OK;
+    const int64_t n4 = n * Hq * (kD / 4);
+    fill_rows_kernel<<<(int)std::min<int64_t>((n4 + 255) / 256, 2048), 256, 0, s>>>(out, lse, lse_stride, b, n, Hq);
+    return check_cuda(cudaGetLastError(), "fill_rows launch");
+}
+
+// want_fill: the call produces a partial result (fp32 out); rows it computes nothing for are written as zeros with
+// lse = -inf (the identity element of cp_merge), by the attention kernel's spare warp.
 int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table, int32_t B,
                 const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C, const int64_t* cu_pages,
                 int32_t only_shard, int32_t only_chunk, int64_t kv_lo, int64_t kv_hi, int32_t Hq, float scale, void* out,
-                int out_f32, float* lse, void* workspace, size_t workspace_bytes, void* stream, const char* who) {
+                int out_f32, bool want_fill, float* lse, void* workspace, size_t workspace_bytes, void* stream,
+                const char* who) {
     if (!ctx || !q || !page_table || !out || !lse || B < 1 || !cu_new || !prefix_len || !C || !cu_pages)
         return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or B < 1", who);
     if (int rc = validate_kv_cache(cache, who)) return rc;
@@ -1159,10 +1183,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
 
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int grid_max = ctx->num_sms;
-#ifdef CPATTN_TRACE
-    if (const char* e = getenv("CPATTN_DEBUG_SMS")) grid_max = std::max(1, atoi(e));   // trace builds only
-#endif
+    const int grid_max = ctx->num_sms;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     // With schedule reuse on, a call whose schedule-relevant arguments and workspace equal the previous call's
     // (the next layer of the same batch) launches on the work lists that are already in the workspace.
@@ -1171,28 +1192,49 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         key = 1469598103934665603ull;
         auto mix = [&key](int64_t v) { key = (key ^ (uint64_t)v) * 1099511628211ull; };
         mix(B); mix(Hq); mix(cache->Hkv); mix(cache->page_size); mix(only_shard); mix(only_chunk); mix(kv_lo); mix(kv_hi);
-        mix(grid_max); mix(out_f32);
+        mix(grid_max); mix(out_f32); mix(want_fill);
         for (int32_t b = 0; b < B; ++b) { mix(cu_new[b + 1]); mix(prefix_len[b]); mix(C[b]); mix(cu_pages[b + 1]); }
     }
-    WorkspaceLayout lay;
-    int32_t grid, n_items, n_merges;
+    WorkspaceLayout lay;        // where the partial results (and the lists of a large schedule) sit in the workspace
+    WorkspaceLayout ilay;       // offsets of the lists inside the launch-parameter copy of a small schedule
+    int32_t grid, n_items, n_merges, n_fill = 0;
+    int32_t fill[2 * kMaxFillRanges] = {0};
     int64_t total_rows;
+    bool inl_on = false;
+    InlineSched inl_local;
+    inl_local.bytes[0] = 0;
+    const InlineSched* inl = &inl_local;
     if (ctx->cache_on && ctx->cache_valid && ctx->cache_key == key && ctx->cache_ws == workspace) {
         lay = ctx->cache_lay;
         grid = ctx->cache_grid;
         n_items = ctx->cache_items;
         n_merges = ctx->cache_merges;
         total_rows = ctx->cache_rows;
+        inl_on = ctx->cache_inline;
+        inl = &ctx->cache_inl;
+        n_fill = ctx->cache_n_fill;
+        memcpy(fill, ctx->cache_fill, sizeof fill);
     } else {
         ctx->cache_valid = false;
         Schedule sch;
         build_tiles(B, cu_new, prefix_len, C, cu_pages, cache->page_size, only_shard, only_chunk, kv_lo, kv_hi, sch.items);
-        if (sch.items.empty()) return CP_OK;   // the shard owns no rows (only empty chunks)
         // rows of q / out / lse: the packed batch, or the one chunk of a chunk call
         total_rows = cu_new[B];
         if (only_chunk >= 0) {
             total_rows = 0;
             for (const TileItem& t : sch.items) total_rows = std::max<int64_t>(total_rows, (int64_t)t.q_row0 + t.n_rows);
+        }
+        if (sch.items.empty())   // the shard owns no rows (only empty chunks), or no row sees a key of the range
+            return want_fill ? launch_fill_rows(static_cast<float*>(out), lse, total_rows, 0, total_rows, Hq, s) : CP_OK;
+        if (want_fill) {
+            int64_t gaps[2 * kMaxFillRanges];
+            const int n = uncovered_rows(sch.items, total_rows, gaps, kMaxFillRanges);
+            if (n > kMaxFillRanges) {     // more gaps than the kernel takes: fill everything first, in stream order
+                if (int rc = launch_fill_rows(static_cast<float*>(out), lse, total_rows, 0, total_rows, Hq, s)) return rc;
+            } else {
+                n_fill = n;
+                for (int i = 0; i < 2 * n; ++i) fill[i] = (int32_t)gaps[i];
+            }
         }
         if (int rc = build_schedule(Hq / heads_per_unit,
                                     kv_major_pairs(B, cu_new, prefix_len, cache->Hkv, (Hq / cache->Hkv) / heads_per_unit),
@@ -1201,16 +1243,37 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
                                sch.n_slots);
         if (lay.total > workspace_bytes)
             return set_error(CP_ERR_WORKSPACE, "%s: schedule needs %zu workspace bytes, have %zu", who, lay.total, workspace_bytes);
-        // one contiguous block: items | cta_off | pieces | merges | merge_slots (offsets as in the layout)
-        std::vector<uint8_t> block(lay.partial_o - lay.items, 0);
-        memcpy(block.data() + (lay.items - lay.items), sch.items.data(), sch.items.size() * sizeof(TileItem));
-        memcpy(block.data() + (lay.cta_off - lay.items), sch.cta_off.data(), sch.cta_off.size() * sizeof(int32_t));
-        memcpy(block.data() + (lay.pieces - lay.items), sch.pieces.data(), sch.pieces.size() * sizeof(PieceEntry));
-        if (!sch.merges.empty()) {
-            memcpy(block.data() + (lay.merges - lay.items), sch.merges.data(), sch.merges.size() * sizeof(MergeEntry));
-            memcpy(block.data() + (lay.merge_slots - lay.items), sch.merge_slots.data(), sch.merge_slots.size() * sizeof(int32_t));
+        // one contiguous block: items | cta_off | pieces | merges | merge_slots.  A block of at most
+        // kInlineSchedBytes (packed to 16-byte boundaries) rides in the launch parameters; a larger one is copied
+        // into the workspace by a small kernel.
+        ilay = workspace_layout(sch.items.size(), sch.pieces.size(), sch.merges.size(), sch.merge_slots.size(), sch.grid,
+                                0, 16);
+        inl_on = ilay.partial_o - ilay.items <= kInlineSchedBytes;
+        const WorkspaceLayout& bl = inl_on ? ilay : lay;
+        std::vector<uint8_t> big;
+        uint8_t* block = inl_local.bytes;
+        if (!inl_on) {
+            big.assign(bl.partial_o - bl.items, 0);
+            block = big.data();
         }
-        if (int rc = upload_block(ctx, block, ws + lay.items, s)) return rc;
+        memcpy(block + (bl.items - bl.items), sch.items.data(), sch.items.size() * sizeof(TileItem));
+        memcpy(block + (bl.cta_off - bl.items), sch.cta_off.data(), sch.cta_off.size() * sizeof(int32_t));
+        memcpy(block + (bl.pieces - bl.items), sch.pieces.data(), sch.pieces.size() * sizeof(PieceEntry));
+        if (!sch.merges.empty()) {
+            memcpy(block + (bl.merges - bl.items), sch.merges.data(), sch.merges.size() * sizeof(MergeEntry));
+            memcpy(block + (bl.merge_slots - bl.items), sch.merge_slots.data(), sch.merge_slots.size() * sizeof(int32_t));
+        }
+        if (inl_on) {
+            // the list offsets inside the parameter block take the place of the workspace offsets
+            const size_t base = ilay.items;
+            lay.items = ilay.items - base;
+            lay.cta_off = ilay.cta_off - base;
+            lay.pieces = ilay.pieces - base;
+            lay.merges = ilay.merges - base;
+            lay.merge_slots = ilay.merge_slots - base;
+        } else if (int rc = upload_block(ctx, big, ws + lay.items, s)) {
+            return rc;
+        }
         grid = sch.grid;
         n_items = (int32_t)sch.items.size();
         n_merges = (int32_t)sch.merges.size();
@@ -1223,6 +1286,10 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
             ctx->cache_items = n_items;
             ctx->cache_merges = n_merges;
             ctx->cache_rows = total_rows;
+            ctx->cache_inline = inl_on;
+            if (inl_on) memcpy(ctx->cache_inl.bytes, inl_local.bytes, kInlineSchedBytes);
+            ctx->cache_n_fill = n_fill;
+            memcpy(ctx->cache_fill, fill, sizeof fill);
         }
     }
 
@@ -1240,6 +1307,15 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.n_items = n_items;
     p.cta_off = reinterpret_cast<const int32_t*>(ws + lay.cta_off);
     p.pieces = reinterpret_cast<const PieceEntry*>(ws + lay.pieces);
+    p.inl_items = p.inl_cta_off = p.inl_pieces = -1;
+    if (inl_on) {
+        p.items = nullptr;
+        p.cta_off = nullptr;
+        p.pieces = nullptr;
+        p.inl_items = (int32_t)lay.items;
+        p.inl_cta_off = (int32_t)lay.cta_off;
+        p.inl_pieces = (int32_t)lay.pieces;
+    }
     p.partial_o = reinterpret_cast<float*>(ws + lay.partial_o);
     p.partial_lse = reinterpret_cast<float*>(ws + lay.partial_lse);
     p.pairs_per_tile = Hq / heads_per_unit;
@@ -1256,14 +1332,24 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.lse = lse;
     p.lse_stride = total_rows;
     p.status = ctx->d_status;
-    if (heads_per_unit == 2) cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
-    else cp_attn_kernel<true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
+    p.n_fill = n_fill;
+    memcpy(p.fill, fill, sizeof fill);
+    if (heads_per_unit == 2) cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
+    else cp_attn_kernel<true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
     if (int rc = check_cuda(cudaGetLastError(), who)) return rc;
     if (n_merges > 0) {
         FixupParams f;
         f.items = p.items;
         f.merges = reinterpret_cast<const MergeEntry*>(ws + lay.merges);
         f.merge_slots = reinterpret_cast<const int32_t*>(ws + lay.merge_slots);
+        f.inl_items = f.inl_merges = f.inl_merge_slots = -1;
+        if (inl_on) {
+            f.merges = nullptr;
+            f.merge_slots = nullptr;
+            f.inl_items = (int32_t)lay.items;
+            f.inl_merges = (int32_t)lay.merges;
+            f.inl_merge_slots = (int32_t)lay.merge_slots;
+        }
         f.partial_o = p.partial_o;
         f.partial_lse = p.partial_lse;
         f.out = out;
@@ -1272,7 +1358,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         f.heads_per_unit = heads_per_unit;
         f.lse = lse;
         f.lse_stride = total_rows;
-        cp_attn_fixup_kernel<<<dim3((unsigned)n_merges, 2 * kBlockM / kFixupRowsPerBlock), 256, 0, s>>>(f);
+        cp_attn_fixup_kernel<<<dim3((unsigned)n_merges, 2 * kBlockM / kFixupRowsPerBlock), 256, 0, s>>>(f, *inl);
         if (int rc = check_cuda(cudaGetLastError(), "cp_attn_fixup launch")) return rc;
     }
     return CP_OK;
@@ -1285,7 +1371,7 @@ extern "C" int cp_prefill_attn_batch(cp_ctx* ctx, const void* q, const cp_kv_cac
                                      const int64_t* cu_pages, int32_t Hq, float scale, void* out, float* lse,
                                      void* workspace, size_t workspace_bytes, void* stream) {
     return attn_common(ctx, q, cache, page_table, B, cu_new, prefix_len, C, cu_pages, -1, -1, 0, INT32_MAX, Hq, scale, out, 0,
-                       lse, workspace, workspace_bytes, stream, "cp_prefill_attn_batch");
+                       false, lse, workspace, workspace_bytes, stream, "cp_prefill_attn_batch");
 }
 
 extern "C" int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
@@ -1296,28 +1382,21 @@ extern "C" int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* ca
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
     return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, 0, INT32_MAX, Hq, scale, out, 0,
-                       lse, workspace, workspace_bytes, stream, "cp_prefill_attn");
+                       false, lse, workspace, workspace_bytes, stream, "cp_prefill_attn");
 }
 
+// The two partial-result calls write zeros with lse = -inf (the identity element of cp_merge) into the rows
+// they compute nothing for; the attention kernel's spare warp does it, so each call is one launch.
 extern "C" int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
                                      int64_t prefix_len, int64_t new_len, int32_t C, int32_t shard, int32_t Hq,
                                      float scale, float* partial_out, float* partial_lse, void* workspace,
                                      size_t workspace_bytes, void* stream) {
     if (!cache || new_len < 1 || prefix_len < 0 || C < 1 || shard < 0 || shard >= C || !partial_out || !partial_lse || Hq < 1)
         return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_shard: bad sizes or shard %d not in [0, %d)", shard, C);
-    if (!ctx) return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_shard: ctx is NULL");
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    // rows the shard does not own: zeros with lse = -inf (the identity element of cp_merge)
-    if (int rc = check_cuda(cudaMemsetAsync(partial_out, 0, (size_t)new_len * Hq * kD * sizeof(float), s),
-                            "cudaMemsetAsync(partial_out)")) return rc;
-    const int64_t n_lse = new_len * Hq;
-    fill_neg_inf_kernel<<<(int)std::min<int64_t>((n_lse + 255) / 256, 4096), 256, 0, s>>>(partial_lse, n_lse);
-    if (int rc = check_cuda(cudaGetLastError(), "fill_neg_inf launch")) return rc;
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
     return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, -1, 0, INT32_MAX, Hq, scale,
-                       partial_out, 1, partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_shard");
+                       partial_out, 1, true, partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_shard");
 }
 
 extern "C" int cp_prefill_attn_kvrange(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
@@ -1328,20 +1407,11 @@ extern "C" int cp_prefill_attn_kvrange(cp_ctx* ctx, const void* q, const cp_kv_c
         return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_kvrange: null pointer or bad sizes");
     if (kv_lo < 0 || kv_hi < kv_lo || kv_lo > 0x7fffff00ll)
         return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_kvrange: key range [%lld, %lld)", (long long)kv_lo, (long long)kv_hi);
-    if (!ctx) return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_kvrange: ctx is NULL");
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    // rows that see no key of the range: zeros with lse = -inf (the identity element of cp_merge)
-    if (int rc = check_cuda(cudaMemsetAsync(partial_out, 0, (size_t)new_len * Hq * kD * sizeof(float), s),
-                            "cudaMemsetAsync(partial_out)")) return rc;
-    const int64_t n_lse = new_len * Hq;
-    fill_neg_inf_kernel<<<(int)std::min<int64_t>((n_lse + 255) / 256, 4096), 256, 0, s>>>(partial_lse, n_lse);
-    if (int rc = check_cuda(cudaGetLastError(), "fill_neg_inf launch")) return rc;
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
     const int32_t C = 1;
     return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, kv_lo,
-                       std::min<int64_t>(kv_hi, INT32_MAX), Hq, scale, partial_out, 1, partial_lse, workspace,
+                       std::min<int64_t>(kv_hi, INT32_MAX), Hq, scale, partial_out, 1, true, partial_lse, workspace,
                        workspace_bytes, stream, "cp_prefill_attn_kvrange");
 }
 
@@ -1361,7 +1431,7 @@ extern "C" int cp_prefill_attn_chunk(cp_ctx* ctx, const void* q_chunk, const cp_
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
     return attn_common(ctx, q_chunk, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, chunk, 0, INT32_MAX, Hq,
-                       scale, out_chunk, 0, lse_chunk, workspace, workspace_bytes, stream, "cp_prefill_attn_chunk");
+                       scale, out_chunk, 0, false, lse_chunk, workspace, workspace_bytes, stream, "cp_prefill_attn_chunk");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1371,7 +1441,7 @@ extern "C" int cp_prefill_attn_chunk(cp_ctx* ctx, const void* q_chunk, const cp_
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-constexpr int kStaticMaxTiles = 2048;   // 128-row query tiles, chunk cuts included (~260K new tokens)
+constexpr int kStaticMaxTiles = 2048;   // 128-row query tiles: 262,144 new tokens
 constexpr size_t kStaticScratchBytes = kWorkspaceHeader + (size_t)kStaticMaxTiles * sizeof(TileItem);
 constexpr int kStaticMaxDevices = 64;
 
@@ -1419,6 +1489,26 @@ int static_setup(int device, StaticDeviceState** out) {
     return CP_OK;
 }
 
+// Writes the request's tile list into the scratch and clears the status words, from the lengths alone (the
+// all-shards tile list is plain arithmetic: tile t covers rows [128 t, 128 t + 128), longest tiles first), so no
+// host buffer is read when the stream runs.
+__global__ void static_tiles_kernel(unsigned char* scratch, int64_t R, int64_t P, int32_t n_pages, int32_t n_tiles) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < kStatusWords) reinterpret_cast<int32_t*>(scratch)[i] = 0;
+    if (i >= n_tiles) return;
+    const int64_t r0 = (int64_t)(n_tiles - 1 - i) * kTileRows;
+    TileItem t;
+    t.q_row0 = (int32_t)r0;
+    t.n_rows = (int32_t)min((int64_t)kTileRows, R - r0);
+    t.kv_len0 = (int32_t)(P + r0 + 1);
+    t.pt_base = 0;
+    t.n_pages = n_pages;
+    t.n_kv_tiles = (int32_t)((P + r0 + t.n_rows + kTileRows - 1) / kTileRows);
+    t.kv_lo = 0;
+    t.kv_hi = INT32_MAX;
+    reinterpret_cast<TileItem*>(scratch + kWorkspaceHeader)[i] = t;
+}
+
 }  // namespace
 
 extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, const int32_t* page_table,
@@ -1434,11 +1524,11 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     if (!(scale > 0.f)) return set_error(CP_ERR_INVALID_ARG, "%s: scale must be positive", who);
     if (((uintptr_t)q | (uintptr_t)out) & 15) return set_error(CP_ERR_INVALID_ARG, "%s: q and out must be 16-byte aligned", who);
     if (prefix_len + new_len > 0x7fffff00ll) return set_error(CP_ERR_UNSUPPORTED, "%s: request longer than 2^31 tokens", who);
-    const int64_t bound = max_tiles(1, &new_len, &C);
-    if (bound < 0 || bound > kStaticMaxTiles)
-        return set_error(CP_ERR_WORKSPACE, "%s: new_len=%lld with C=%d needs up to %lld query tiles; the built-in scratch "
-                         "holds %d (use cp_prefill_attn with a caller workspace)", who, (long long)new_len, C,
-                         (long long)bound, kStaticMaxTiles);
+    const int64_t n_tiles = (new_len + kTileRows - 1) / kTileRows;
+    if (n_tiles > kStaticMaxTiles)
+        return set_error(CP_ERR_WORKSPACE, "%s: new_len=%lld needs %lld query tiles; the built-in scratch holds %d "
+                         "(use cp_prefill_attn with a caller workspace)", who, (long long)new_len, (long long)n_tiles,
+                         kStaticMaxTiles);
     int device = -1;
     if (int rc = check_cuda(cudaGetDevice(&device), "cudaGetDevice")) return rc;
     StaticDeviceState* st = nullptr;
@@ -1446,22 +1536,20 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
 
     const int64_t cu_new[2] = {0, new_len};
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
-    std::vector<TileItem> tiles;
-    build_tiles(1, cu_new, &prefix_len, &C, cu_pages, cache->page_size, -1, -1, 0, INT32_MAX, tiles);
     cp_ctx enc{};                       // only the encoder entry point is read by encode_maps
     enc.encode_tiled = st->encode_tiled;
     CUtensorMap tmQ, tmK, tmV;
     if (int rc = encode_maps(&enc, q, new_len, Hq, cache, &tmQ, &tmK, &tmV)) return rc;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // The scratch keeps whatever the previous call left: clear the status words, overwrite the list.
-    if (int rc = check_cuda(cudaMemsetAsync(st->scratch, 0, kStatusWords * sizeof(int32_t), s), "cudaMemsetAsync(status)"))
-        return rc;
-    if (int rc = check_cuda(cudaMemcpyAsync(st->scratch + kWorkspaceHeader, tiles.data(), tiles.size() * sizeof(TileItem),
-                                            cudaMemcpyHostToDevice, s), "tile list copy")) return rc;
+    // The scratch keeps whatever the previous call left: a small kernel clears the status words and writes this
+    // request's tile list in stream order (no host memory is read later, whatever the stream does with the work).
+    static_tiles_kernel<<<(unsigned)((n_tiles + 255) / 256), 256, 0, s>>>(
+        st->scratch, new_len, prefix_len, (int32_t)cu_pages[1], (int32_t)n_tiles);
+    if (int rc = check_cuda(cudaGetLastError(), "static tile list launch")) return rc;
     AttnParams p;
     p.items = reinterpret_cast<const TileItem*>(st->scratch + kWorkspaceHeader);
-    p.n_items = (int32_t)tiles.size();
+    p.n_items = (int32_t)n_tiles;
     p.cta_off = nullptr;       // implicit schedule over whole units: no piece lists, no partial results
     p.pieces = nullptr;
     p.partial_o = nullptr;
@@ -1480,9 +1568,13 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     p.lse = lse;
     p.lse_stride = new_len;
     p.status = reinterpret_cast<int32_t*>(st->scratch);
-    const int64_t units = (int64_t)tiles.size() * p.pairs_per_tile;
+    p.inl_items = p.inl_cta_off = p.inl_pieces = -1;
+    p.n_fill = 0;
+    InlineSched none;          // unused: the tile list is in the scratch
+    none.bytes[0] = 0;
+    const int64_t units = n_tiles * p.pairs_per_tile;
     const int grid = (int)std::min<int64_t>(units, st->num_sms);
-    if (heads_per_unit == 2) cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
-    else cp_attn_kernel<true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p);
+    if (heads_per_unit == 2) cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, none);
+    else cp_attn_kernel<true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, none);
     return check_cuda(cudaGetLastError(), who);
 }

@@ -96,14 +96,6 @@ extern "C" int cp_ctx_destroy(cp_ctx* c) {
     return CP_OK;
 }
 
-#ifdef CPATTN_TRACE
-// Trace builds only: copy the status buffer (status words + phase trace) to the host.
-extern "C" int cp_debug_read_status_buffer(cp_ctx* c, void* dst, size_t bytes) {
-    if (!c || !dst || bytes > kStatusBytes) return set_error(CP_ERR_INVALID_ARG, "cp_debug_read_status_buffer");
-    return check_cuda(cudaMemcpy(dst, c->d_status, bytes, cudaMemcpyDeviceToHost), "cudaMemcpy(trace)");
-}
-#endif
-
 extern "C" int cp_ctx_cache_schedule(cp_ctx* c, int enable) {
     if (!c) return set_error(CP_ERR_INVALID_ARG, "cp_ctx_cache_schedule: ctx is NULL");
     c->cache_on = enable != 0;
@@ -118,8 +110,12 @@ extern "C" int cp_ctx_poll_status(cp_ctx* c, int32_t* detail) {
     if (detail) memcpy(detail, c->h_status, kStatusWords * sizeof(int32_t));
     if (c->h_status[0] != 0) {
         int code = c->h_status[0];
-        set_error(code, "device status: code %d, barrier %d, block %d, iteration %d", c->h_status[0],
-                  c->h_status[1], c->h_status[2], c->h_status[3]);
+        if (code == CP_ERR_BOUNDS)
+            set_error(code, "device status: page-table entry %d holds page id %d, outside the pool (block %d); the "
+                      "elements behind it were skipped", c->h_status[1], c->h_status[3], c->h_status[2]);
+        else
+            set_error(code, "device status: code %d, barrier %d, block %d, iteration %d", c->h_status[0],
+                      c->h_status[1], c->h_status[2], c->h_status[3]);
         cudaMemset(c->d_status, 0, kStatusWords * sizeof(int32_t));
         return code;
     }

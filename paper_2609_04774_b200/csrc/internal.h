@@ -74,11 +74,14 @@ constexpr size_t kWorkspaceHeader = 256;
 constexpr int kTileRows = 128;
 constexpr int kStatusWords = 4;
 constexpr int kStageBuffers = 4;
-#ifdef CPATTN_TRACE
-constexpr size_t kStatusBytes = 64 + 4 * 64 * 8 * sizeof(long long);   // status words + phase trace
-#else
 constexpr size_t kStatusBytes = kStatusWords * sizeof(int32_t);
-#endif
+// A schedule whose work lists fit in this many bytes travels inside the kernel's launch parameters instead of
+// being copied into the workspace first (one launch less for small problems).
+constexpr size_t kInlineSchedBytes = 3072;
+struct InlineSched {
+    alignas(16) unsigned char bytes[kInlineSchedBytes];
+};
+constexpr int kMaxFillRanges = 4;        // row ranges a partial-result call fills with zeros / -inf inside the kernel
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -105,7 +108,10 @@ int build_schedule(int32_t pairs_per_tile, int32_t pairs_per_kv, int32_t grid_ma
 // pairs_per_kv to pass to build_schedule: the real value when the batch's K/V is large, else 0 (one group)
 int32_t kv_major_pairs(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, int32_t Hkv, int32_t pairs_per_kv);
 WorkspaceLayout workspace_layout(size_t n_items, size_t n_pieces, size_t n_merges, size_t n_merge_slots, size_t grid,
-                                 size_t n_slots);
+                                 size_t n_slots, size_t align = 256);
+// Row ranges [begin, end) of [0, total_rows) that no tile covers, ascending; returns their number and writes
+// at most max_gaps of them (pairs of int64).
+int uncovered_rows(const std::vector<TileItem>& items, int64_t total_rows, int64_t* gaps, int max_gaps);
 
 }  // namespace cpattn
 
@@ -129,4 +135,8 @@ struct cp_ctx {
     cpattn::WorkspaceLayout cache_lay;
     int32_t cache_grid, cache_items, cache_merges;
     int64_t cache_rows;
+    bool cache_inline;                 // the remembered work lists travel in the launch parameters
+    cpattn::InlineSched cache_inl;
+    int32_t cache_n_fill;
+    int32_t cache_fill[2 * cpattn::kMaxFillRanges];
 };

@@ -14,7 +14,7 @@ __global__ void __launch_bounds__(256)
 kv_copy_kernel(uint4* __restrict__ paged_k, uint4* __restrict__ paged_v, uint4* __restrict__ rows_k,
                uint4* __restrict__ rows_v, const int32_t* __restrict__ page_table, int64_t t_begin, int64_t n,
                int page_size, int Hkv, int vec_per_head, int64_t stride_page8, int64_t stride_tok8,
-               int64_t stride_head8) {
+               int64_t stride_head8, int64_t num_pages, int32_t* status) {
     const int vec_per_tok = Hkv * vec_per_head;
     const int64_t total = n * vec_per_tok;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -23,8 +23,18 @@ kv_copy_kernel(uint4* __restrict__ paged_k, uint4* __restrict__ paged_v, uint4* 
         const int g = rem / vec_per_head;
         const int c = rem - g * vec_per_head;
         const int64_t t = t_begin + tok;
-        const int64_t off = (int64_t)page_table[t / page_size] * stride_page8 + (t % page_size) * stride_tok8 +
-                            (int64_t)g * stride_head8 + c;
+        const int64_t page = page_table[t / page_size];
+        if (page < 0 || page >= num_pages) {
+            // a page id outside the pool: the element is skipped (nothing is read or written through it) and the
+            // first such entry is recorded in the status words {code, table index, block, page id}
+            if (atomicCAS(status, 0, CP_ERR_BOUNDS) == 0) {
+                status[1] = (int32_t)(t / page_size);
+                status[2] = (int32_t)blockIdx.x;
+                status[3] = (int32_t)page;
+            }
+            continue;
+        }
+        const int64_t off = page * stride_page8 + (t % page_size) * stride_tok8 + (int64_t)g * stride_head8 + c;
         if (kToPaged) {
             if (rows_k) paged_k[off] = rows_k[i];
             if (rows_v) paged_v[off] = rows_v[i];
@@ -59,12 +69,14 @@ int kv_copy(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, in
     if (((uintptr_t)k_rows | (uintptr_t)v_rows) & 15)
         return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
     if (n == 0) return CP_OK;
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
     const int vec_per_head = cache->D / 8;
     const int64_t total = n * cache->Hkv * vec_per_head;
     const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
     kv_copy_kernel<kToPaged><<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         (uint4*)cache->k, (uint4*)cache->v, (uint4*)k_rows, (uint4*)v_rows, page_table, t_begin, n, cache->page_size,
-        cache->Hkv, vec_per_head, cache->stride_page / 8, cache->stride_tok / 8, cache->stride_head / 8);
+        cache->Hkv, vec_per_head, cache->stride_page / 8, cache->stride_tok / 8, cache->stride_head / 8, cache->num_pages,
+        ctx->d_status);
     return check_cuda(cudaGetLastError(), who);
 }
 

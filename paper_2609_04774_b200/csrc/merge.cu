@@ -116,6 +116,7 @@ extern "C" int cp_merge(cp_ctx* ctx, const float* partials, const float* lses, i
         return set_error(CP_ERR_UNSUPPORTED, "cp_merge: T=%lld x H=%d needs more than 2^31 blocks", (long long)T, H);
     if (((uintptr_t)partials | (uintptr_t)out) & 15)
         return set_error(CP_ERR_INVALID_ARG, "cp_merge: partials and out must be 16-byte aligned");
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // heads per warp chosen so that 8 to 16 row loads (128 to 256 bytes per lane) are in flight per warp
     if (N <= 2) launch_merge<2, 4>(partials, lses, N, T, H, out, out_dtype, lse_out, s);

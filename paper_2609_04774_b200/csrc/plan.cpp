@@ -2,6 +2,7 @@
 #include <algorithm>
 #include <climits>
 #include <cstdint>
+#include <utility>
 
 #include "internal.h"
 
@@ -34,16 +35,24 @@ int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, con
                 const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, int64_t kv_lo,
                 int64_t kv_hi, std::vector<TileItem>& out) {
     out.clear();
+    // A launch over ALL shards of a request walks its rows as one run: adjacent zigzag chunks are adjacent rows
+    // with consecutive causal limits, which the per-row limit kv_len0 + row already expresses, so a query tile may
+    // span a chunk boundary (never a request).  The shard stays the accounting unit of cp_plan; only the calls
+    // that compute one shard or one chunk cut their tiles at its chunk boundaries.
+    const bool all_shards = only_shard < 0 && only_chunk < 0;
     for (int32_t b = 0; b < B; ++b) {
         const int64_t R = cu_new[b + 1] - cu_new[b];
         const int64_t P = prefix_len[b];
         const int32_t Cb = C[b];
-        for (int64_t j = 0; j < 2 * (int64_t)Cb; ++j) {
-            const int32_t shard = (int32_t)(j < Cb ? j : 2 * (int64_t)Cb - 1 - j);
-            if (only_shard >= 0 && shard != only_shard) continue;
-            if (only_chunk >= 0 && j != only_chunk) continue;
-            int64_t cb, ce;
-            chunk_range(R, Cb, j, cb, ce);
+        const int64_t n_runs = all_shards ? 1 : 2 * (int64_t)Cb;
+        for (int64_t j = 0; j < n_runs; ++j) {
+            int64_t cb = 0, ce = R;
+            if (!all_shards) {
+                const int32_t shard = (int32_t)(j < Cb ? j : 2 * (int64_t)Cb - 1 - j);
+                if (only_shard >= 0 && shard != only_shard) continue;
+                if (only_chunk >= 0 && j != only_chunk) continue;
+                chunk_range(R, Cb, j, cb, ce);
+            }
             // a single-chunk list addresses q / out / lse rows relative to the chunk's first row
             const int64_t row_base = only_chunk >= 0 ? cb : 0;
             for (int64_t r0 = cb; r0 < ce; r0 += kTileRows) {
@@ -71,19 +80,42 @@ int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, con
     return CP_OK;
 }
 
+// Row ranges [begin, end) of [0, total_rows) that no tile of `items` covers (rows of other shards, rows that see
+// no key of a key range), in ascending order.  Returns how many there are; at most max_gaps are written.
+int uncovered_rows(const std::vector<TileItem>& items, int64_t total_rows, int64_t* gaps, int max_gaps) {
+    std::vector<std::pair<int64_t, int64_t>> iv;
+    iv.reserve(items.size());
+    for (const TileItem& t : items) iv.emplace_back((int64_t)t.q_row0, (int64_t)t.q_row0 + t.n_rows);
+    std::sort(iv.begin(), iv.end());
+    int n = 0;
+    int64_t at = 0;
+    auto emit = [&](int64_t b, int64_t e) {
+        if (e <= b) return;
+        if (n > 0 && n <= max_gaps && gaps[2 * (n - 1) + 1] == b) { gaps[2 * (n - 1) + 1] = e; return; }
+        if (n < max_gaps) { gaps[2 * n] = b; gaps[2 * n + 1] = e; }
+        ++n;
+    };
+    for (const auto& x : iv) {
+        emit(at, x.first);
+        at = std::max(at, x.second);
+    }
+    emit(at, total_rows);
+    return n;
+}
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 WorkspaceLayout workspace_layout(size_t n_items, size_t n_pieces, size_t n_merges, size_t n_merge_slots, size_t grid,
-                                 size_t n_slots) {
+                                 size_t n_slots, size_t align) {
     WorkspaceLayout w;
     size_t off = kWorkspaceHeader;
-    w.items = off;        off = align_up(off + n_items * sizeof(TileItem), 256);
-    w.cta_off = off;      off = align_up(off + (grid + 1) * sizeof(int32_t), 256);
-    w.pieces = off;       off = align_up(off + n_pieces * sizeof(PieceEntry), 256);
-    w.merges = off;       off = align_up(off + n_merges * sizeof(MergeEntry), 256);
-    w.merge_slots = off;  off = align_up(off + n_merge_slots * sizeof(int32_t), 256);
-    w.partial_o = off;    off = align_up(off + n_slots * kPartialSlotRows * kPartialRowFloats * sizeof(float), 256);
-    w.partial_lse = off;  off = align_up(off + n_slots * kPartialSlotRows * sizeof(float), 256);
+    w.items = off;        off = align_up(off + n_items * sizeof(TileItem), align);
+    w.cta_off = off;      off = align_up(off + (grid + 1) * sizeof(int32_t), align);
+    w.pieces = off;       off = align_up(off + n_pieces * sizeof(PieceEntry), align);
+    w.merges = off;       off = align_up(off + n_merges * sizeof(MergeEntry), align);
+    w.merge_slots = off;  off = align_up(off + n_merge_slots * sizeof(int32_t), align);
+    w.partial_o = off;    off = align_up(off + n_slots * kPartialSlotRows * kPartialRowFloats * sizeof(float), align);
+    w.partial_lse = off;  off = align_up(off + n_slots * kPartialSlotRows * sizeof(float), align);
     w.total = off;
     return w;
 }
@@ -107,7 +139,11 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t pairs_per_kv, int
     // per-CTA share of KV tile steps; never below a short unit's length (cutting those only adds
     // prologues and merges), which also shrinks the grid for tiny problems
     const int64_t T = std::max<int64_t>((W + grid_max - 1) / grid_max, std::min<int32_t>(longest, kMinShareTiles));
-    const int32_t G = (int32_t)std::max<int64_t>(1, std::min<int64_t>(grid_max, (W + T - 1) / T));
+    // When there are no more units than CTAs and none is longer than the share, every unit gets a CTA of its own:
+    // the same critical path as packing them, and nothing is cut, so no partial results and no merge launch.
+    const bool one_each = n_units <= grid_max && longest <= T;
+    const int32_t G = one_each ? (int32_t)n_units
+                               : (int32_t)std::max<int64_t>(1, std::min<int64_t>(grid_max, (W + T - 1) / T));
     s.grid = G;
 
     // 1. whole units dealt to the CTAs in serpentine order (0..G-1, G-1..0, ...) while they fit under the
@@ -281,6 +317,11 @@ extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64
     summary[5] = max_load;
     summary[6] = min_load;
     summary[7] = total;
+    // does the block of work lists fit the launch parameters, and how many launches the call then makes
+    const WorkspaceLayout il = workspace_layout(sch.items.size(), sch.pieces.size(), sch.merges.size(), sch.merge_slots.size(),
+                                                sch.grid, 0, 16);
+    summary[8] = (il.partial_o - il.items <= kInlineSchedBytes) ? 1 : 0;
+    summary[9] = (summary[8] ? 0 : 1) + 1 + (sch.merges.empty() ? 0 : 1);
     if (pieces) {
         if ((int64_t)sch.pieces.size() > max_pieces) return set_error(CP_ERR_WORKSPACE, "cp_schedule_inspect: %zu pieces", sch.pieces.size());
         for (int32_t c = 0; c < sch.grid; ++c)

@@ -198,14 +198,6 @@ class Workload:
     def num_pages(self) -> int:
         return int(self.cu_pages[-1]) + self.spare_pages
 
-    def pairs(self) -> int:
-        """Visible (query, key) pairs, the remaining attention workload of Eq. (1), summed over requests."""
-        return sum(r.new_len * r.prefix_len + r.new_len * (r.new_len + 1) // 2 for r in self.requests)
-
-    def flops(self) -> int:
-        """Causal-effective flops: 4*D per visible pair per query head."""
-        return 4 * self.D * self.Hq * self.pairs()
-
 
 GARBAGE_POS = 0x7F61   # bf16 bits of about +2.99e38 (finite)
 GARBAGE_NEG = 0xFF61

@@ -18,7 +18,9 @@ def check(w, num_sms=148):
     Cs = [r.C for r in w.requests]
     info, pieces, items = binding.cp_schedule_inspect(cu_new, prefix, Cs, w.Hq, w.Hkv, num_sms)
     HP = w.Hq // (2 if (w.Hq // w.Hkv) % 2 == 0 else 1)
-    # tiles: rows tile [0, total_new) exactly, never straddle a request or a chunk, at most 128 rows
+    # tiles: rows tile [0, total_new) exactly and never straddle a request; in a launch over all shards a tile
+    # may span the boundary of adjacent zigzag chunks (the per-row causal limit does not care), so every tile
+    # but a request's last has the full 128 rows
     rows = np.zeros(w.total_new, dtype=np.int32)
     for q0, n, kv0, nt in items:
         assert 1 <= n <= 128 and nt == -(-(kv0 + n - 1) // 128)
@@ -27,8 +29,7 @@ def check(w, num_sms=148):
         r = w.requests[b]
         r0 = q0 - cu_new[b]
         assert r0 + n <= r.new_len and kv0 == r.prefix_len + r0 + 1
-        cl = -(-r.new_len // (2 * r.C))
-        assert r0 // cl == (r0 + n - 1) // cl                      # inside one zigzag chunk
+        assert r0 % 128 == 0 and (n == 128 or r0 + n == r.new_len)
     assert (rows == 1).all()
     # pieces: per unit the KV tile ranges tile [0, n_kv_tiles) exactly; slots only on split units
     cover = {}
@@ -63,6 +64,10 @@ def test_schedule_covers_and_balances_all_configs():
     for cfg in (1, 2, 4, 5, 3):
         w = wl.CONFIGS[cfg]()
         info, loads = check(w)
+        if info["pieces"] == info["grid"] <= 148 and info["max_load"] <= 8:
+            # no more units than SMs, all short: one CTA per unit, nothing is cut (no partials, no merge launch)
+            assert cfg == 1 and info["split_units"] == 0 and info["grid"] == 32
+            continue
         share = -(-info["total"] // info["grid"])
         assert info["max_load"] <= 1.01 * share + 4, (cfg, info)   # at most one short remainder above the share
         assert loads.mean() >= 0.97 * info["max_load"] - 1, (cfg, info)   # the slowest CTA is within 3 % of the mean
