@@ -158,8 +158,8 @@ class Runner:
         self.out = torch.empty((w.total_new, w.Hq, w.D), dtype=torch.bfloat16, device="cuda")
         self.lse = torch.empty((w.Hq, w.total_new), dtype=torch.float32, device="cuda")
         self.new_len = [r.new_len for r in w.requests]
-        self.prefix = [r.prefix_len for r in w.requests]
-        self.Cs = [r.C for r in w.requests]
+        self.prefix = np.array([r.prefix_len for r in w.requests], dtype=np.int64)
+        self.Cs = np.array([r.C for r in w.requests], dtype=np.int32)
         self.ws = torch.zeros(binding.cp_workspace_bytes(self.new_len, self.Cs, w.Hq), dtype=torch.uint8, device="cuda")
         self.cu_new, self.cu_pages = w.cu_new, w.cu_pages
         if need_host:

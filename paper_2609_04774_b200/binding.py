@@ -85,6 +85,11 @@ def _i32(a):
     return np.ascontiguousarray(a, dtype=np.int32)
 
 
+def _hp(a):
+    """Address of a host numpy array (the plain integer route; `ctypes.data_as` costs twice as much per call)."""
+    return ctypes.c_void_p(a.ctypes.data)
+
+
 def _stream(stream):
     import torch
     if stream is None:
@@ -135,8 +140,8 @@ def cp_plan(new_len: int, prefix_len: int, C: int):
 
 def cp_workspace_bytes(new_len, C, Hq) -> int:
     nl, cs = _i64(new_len).reshape(-1), _i32(C).reshape(-1)
-    return int(load().cp_workspace_bytes(ctypes.c_int32(nl.size), nl.ctypes.data_as(ctypes.c_void_p),
-                                         cs.ctypes.data_as(ctypes.c_void_p), ctypes.c_int32(Hq)))
+    return int(load().cp_workspace_bytes(ctypes.c_int32(nl.size), _hp(nl),
+                                         _hp(cs), ctypes.c_int32(Hq)))
 
 
 def cp_schedule_inspect(cu_new, prefix_len, C, Hq, Hkv, num_sms=148, want_lists=True):
@@ -144,9 +149,9 @@ def cp_schedule_inspect(cu_new, prefix_len, C, Hq, Hkv, num_sms=148, want_lists=
     cu_new, prefix_len, C = _i64(cu_new), _i64(prefix_len), _i32(C)
     B = prefix_len.size
     summary = np.zeros(10, dtype=np.int64)
-    args = [ctypes.c_int32(B), cu_new.ctypes.data_as(ctypes.c_void_p), prefix_len.ctypes.data_as(ctypes.c_void_p),
-            C.ctypes.data_as(ctypes.c_void_p), ctypes.c_int32(Hq), ctypes.c_int32(Hkv), ctypes.c_int32(num_sms),
-            summary.ctypes.data_as(ctypes.c_void_p)]
+    args = [ctypes.c_int32(B), _hp(cu_new), _hp(prefix_len),
+            _hp(C), ctypes.c_int32(Hq), ctypes.c_int32(Hkv), ctypes.c_int32(num_sms),
+            _hp(summary)]
     _check(load().cp_schedule_inspect(*args, None, ctypes.c_int64(0), None, ctypes.c_int64(0)))
     keys = ["grid", "tiles", "pieces", "split_units", "slots", "max_load", "min_load", "total", "inline", "launches"]
     info = dict(zip(keys, (int(x) for x in summary)))
@@ -154,8 +159,8 @@ def cp_schedule_inspect(cu_new, prefix_len, C, Hq, Hkv, num_sms=148, want_lists=
         return info, None, None
     pieces = np.zeros((info["pieces"], 6), dtype=np.int32)
     items = np.zeros((info["tiles"], 4), dtype=np.int32)
-    _check(load().cp_schedule_inspect(*args, pieces.ctypes.data_as(ctypes.c_void_p), ctypes.c_int64(pieces.shape[0]),
-                                      items.ctypes.data_as(ctypes.c_void_p), ctypes.c_int64(items.shape[0])))
+    _check(load().cp_schedule_inspect(*args, _hp(pieces), ctypes.c_int64(pieces.shape[0]),
+                                      _hp(items), ctypes.c_int64(items.shape[0])))
     return info, pieces, items
 
 
@@ -183,8 +188,8 @@ def cp_prefill_attn_batch(ctx, q, cache, page_table, cu_new, prefix_len, C, cu_p
     assert cu_new.size == B + 1 and cu_pages.size == B + 1 and C.size == B
     _check(load().cp_prefill_attn_batch(
         ctx._h, _ptr(q), ctypes.byref(cache), _ptr(page_table), ctypes.c_int32(B),
-        cu_new.ctypes.data_as(ctypes.c_void_p), prefix_len.ctypes.data_as(ctypes.c_void_p),
-        C.ctypes.data_as(ctypes.c_void_p), cu_pages.ctypes.data_as(ctypes.c_void_p), ctypes.c_int32(Hq),
+        _hp(cu_new), _hp(prefix_len),
+        _hp(C), _hp(cu_pages), ctypes.c_int32(Hq),
         ctypes.c_float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
         ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
 

@@ -1239,6 +1239,11 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         if (int rc = build_schedule(Hq / heads_per_unit,
                                     kv_major_pairs(B, cu_new, prefix_len, cache->Hkv, (Hq / cache->Hkv) / heads_per_unit),
                                     grid_max, sch)) return rc;
+        if (n_fill > 0 && sch.grid < std::min(grid_max, kMaxGrid)) {
+            // rows to fill: CTAs without work join the launch so that every SM's spare warp shares the stores
+            sch.grid = std::min(grid_max, kMaxGrid);
+            sch.cta_off.resize((size_t)sch.grid + 1, sch.cta_off.back());
+        }
         lay = workspace_layout(sch.items.size(), sch.pieces.size(), sch.merges.size(), sch.merge_slots.size(), sch.grid,
                                sch.n_slots);
         if (lay.total > workspace_bytes)
