@@ -259,6 +259,42 @@ def materialize(wl: Workload, need_q: bool = True) -> Materialized:
     return Materialized(wl, q, k_pages, v_pages, page_table)
 
 
+@dataclass
+class MaterializedFp8:
+    wl: Workload
+    q: np.ndarray            # [sum R, Hq, D] bf16 bits, as in Materialized
+    k8_pages: np.ndarray     # [num_pages, PAGE, Hkv, D] uint8: E4M3 bytes
+    v8_pages: np.ndarray
+    k_scale: np.ndarray      # fp32 [Hkv]: value of a stored byte = scale[g] * e4m3(byte)
+    v_scale: np.ndarray
+    page_table: np.ndarray
+
+
+def materialize_fp8(wl: Workload) -> MaterializedFp8:
+    """The same logical N(0,1) K/V content as ``materialize``, stored as E4M3 bytes with one fp32 scale per
+    KV head.  The scales differ from head to head (a wrong head-to-scale mapping changes the result) and put
+    6 standard deviations at the format's largest value; the bytes are made by PyTorch's own float8 conversion
+    (round to nearest even) after clipping to +-448, so the unused slots' large garbage becomes +-448."""
+    import torch
+    mat = materialize(wl)
+    g = np.arange(wl.Hkv, dtype=np.float32)
+    k_scale = ((6.0 / 448.0) * (1.0 + g / 8.0)).astype(np.float32)
+    v_scale = ((6.0 / 448.0) * (1.5 - g / 16.0)).astype(np.float32)
+
+    def to_e4m3(pages_bits, scale):
+        out = np.empty(pages_bits.shape, dtype=np.uint8)
+        step = max(1, (1 << 24) // int(np.prod(pages_bits.shape[1:])))
+        for lo in range(0, pages_bits.shape[0], step):
+            with np.errstate(over="ignore"):              # the unused slots' garbage overflows to inf and is clipped
+                x = bf16_bits_to_f32(pages_bits[lo:lo + step]) / scale[None, None, :, None]
+            t = torch.from_numpy(np.clip(x, -448.0, 448.0).astype(np.float32)).to(torch.float8_e4m3fn)
+            out[lo:lo + step] = t.view(torch.uint8).numpy()
+        return out
+
+    return MaterializedFp8(wl, mat.q, to_e4m3(mat.k_pages, k_scale), to_e4m3(mat.v_pages, v_scale), k_scale, v_scale,
+                           mat.page_table)
+
+
 # --------------------------------------------------------------------------------------
 # The five benchmark configurations
 # --------------------------------------------------------------------------------------
