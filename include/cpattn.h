@@ -279,6 +279,51 @@ int cp_kv_gather(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_tabl
 int cp_kv_append(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin,
                  int64_t n, const void* k_rows, const void* v_rows, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * FP8 K/V variant.  The paper's main model is an FP8 model (Section 9.1) but the paper states no FP8
+ * attention recipe; the format below is this library's reading.
+ *   - K and V pages hold OCP E4M3 bytes (1-4-3 bits, bias 7, no infinities, largest finite value 448),
+ *     layout as cp_kv_cache with one byte per element (strides in bytes, multiples of 16); k_scale and
+ *     v_scale are device arrays of Hkv fp32 values: the stored byte b of KV head g stands for
+ *     scale[g] * e4m3(b).  Slots no logical token maps to must hold finite codes (not 0x7F / 0xFF).
+ *   - Queries are bf16.  Each (token, head) row is quantised by a small pre-pass kernel: amax = max |q|,
+ *     q_scale = amax / 448, code = e4m3(q * (448 / amax)), IEEE fp32 arithmetic, round to nearest even,
+ *     saturating; a row of zeros has scale 0.
+ *   - The result is the Section 2.1 formula (Section 2.2 prefix rule) on the dequantised values: Q K^T and
+ *     P V run on the tensor cores with one-byte operands and fp32 accumulation; the softmax weights are
+ *     rounded to E4M3 (after a scaling by 16) for P V, the row sum and the LSE use the unrounded weights.
+ *     LSE is as accurate as in the bf16 path; each output element is within 2^-4 * sum_j p_j |v_j| of the
+ *     exact result on the stored bytes (the rounding of the weights), typically 2-3 % of the row's norm.
+ *   - Requires an even number of query heads per KV head.  out: bf16 [R, Hq, D]; lse: fp32 [Hq, R].
+ * cp_workspace_bytes_fp8: the workspace of cp_workspace_bytes plus room for the quantised queries.
+ * cp_kv_append_fp8: writes n logical tokens starting at t_begin from bf16 rows [n, Hkv, D] into the FP8
+ * cache, each element as e4m3(x / scale[g]) (IEEE fp32 division, round to nearest even, saturating); page
+ * ids outside the pool are skipped and reported as by cp_kv_append.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    const void* k;          /* device, E4M3 bytes */
+    const void* v;
+    const float* k_scale;   /* device, [Hkv] fp32 */
+    const float* v_scale;
+    int64_t num_pages;
+    int32_t page_size;      /* 16, 32, 64 or 128 */
+    int32_t Hkv;
+    int32_t D;              /* 128 */
+    int32_t reserved;
+    int64_t stride_page, stride_tok, stride_head; /* bytes */
+} cp_kv_cache_fp8;
+size_t cp_workspace_bytes_fp8(int32_t B, const int64_t* new_len, const int32_t* C, int32_t Hq);
+int cp_prefill_attn_fp8(cp_ctx* ctx, const void* q, const cp_kv_cache_fp8* cache, const int32_t* page_table,
+                        int64_t prefix_len, int64_t new_len, int32_t C, int32_t Hq, float scale,
+                        void* out, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+int cp_prefill_attn_fp8_batch(cp_ctx* ctx, const void* q, const cp_kv_cache_fp8* cache, const int32_t* page_table,
+                              int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
+                              const int64_t* cu_pages, int32_t Hq, float scale, void* out, float* lse,
+                              void* workspace, size_t workspace_bytes, void* stream);
+int cp_kv_append_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,
+                     int64_t n, const void* k_rows, const void* v_rows, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,8 @@ CP_DTYPE_BF16, CP_DTYPE_F32 = 0, 1
 
 EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "cp_ctx_poll_status", "cp_ctx_cache_schedule", "cp_ctx_selftest_wait_expiry", "cp_plan",
            "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_chunk", "cp_prefill_attn_kvrange", "cp_prefill_attn_static", "cp_merge",
-           "cp_kv_gather", "cp_kv_append"]
+           "cp_kv_gather", "cp_kv_append", "cp_workspace_bytes_fp8", "cp_prefill_attn_fp8", "cp_prefill_attn_fp8_batch",
+           "cp_kv_append_fp8"]
 
 
 class CpError(RuntimeError):
@@ -42,6 +43,13 @@ class cp_kv_cache(ctypes.Structure):
                 ("stride_head", ctypes.c_int64)]
 
 
+class cp_kv_cache_fp8(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("k_scale", ctypes.c_void_p), ("v_scale", ctypes.c_void_p),
+                ("num_pages", ctypes.c_int64), ("page_size", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("stride_page", ctypes.c_int64), ("stride_tok", ctypes.c_int64),
+                ("stride_head", ctypes.c_int64)]
+
+
 _lib = None
 
 
@@ -57,8 +65,9 @@ def load():
         lib.cp_strerror.argtypes = [ctypes.c_int]
         lib.cp_last_error.restype = ctypes.c_char_p
         lib.cp_workspace_bytes.restype = ctypes.c_size_t
+        lib.cp_workspace_bytes_fp8.restype = ctypes.c_size_t
         for name in EXPORTS:
-            if name not in ("cp_strerror", "cp_last_error", "cp_workspace_bytes"):
+            if name not in ("cp_strerror", "cp_last_error", "cp_workspace_bytes", "cp_workspace_bytes_fp8"):
                 getattr(lib, name).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -251,3 +260,47 @@ def cp_kv_gather(ctx, cache, page_table, t_begin, n, k_rows, v_rows, stream=None
 def cp_kv_append(ctx, cache, page_table, t_begin, n, k_rows, v_rows, stream=None):
     _check(load().cp_kv_append(ctx._h, ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(t_begin),
                                ctypes.c_int64(n), _ptr(k_rows), _ptr(v_rows), _stream(stream)))
+
+
+# ------------------------------------------------------------------------------------------------
+# FP8 K/V variant
+# ------------------------------------------------------------------------------------------------
+
+def make_cache_fp8(k8_pages, v8_pages, k_scale, v_scale) -> cp_kv_cache_fp8:
+    """Describe paged E4M3 K/V tensors [num_pages, page_size, Hkv, D] (uint8) with fp32 scales [Hkv] on the device."""
+    assert k8_pages.dim() == 4 and k8_pages.stride() == v8_pages.stride() and k8_pages.stride(3) == 1
+    assert k8_pages.element_size() == 1 and k_scale.numel() == k8_pages.shape[2] == v_scale.numel()
+    c = cp_kv_cache_fp8()
+    c.k, c.v, c.k_scale, c.v_scale = k8_pages.data_ptr(), v8_pages.data_ptr(), k_scale.data_ptr(), v_scale.data_ptr()
+    c.num_pages, c.page_size, c.Hkv, c.D = k8_pages.shape
+    c.stride_page, c.stride_tok, c.stride_head = k8_pages.stride(0), k8_pages.stride(1), k8_pages.stride(2)
+    return c
+
+
+def cp_workspace_bytes_fp8(new_len, C, Hq) -> int:
+    nl, cs = _i64(new_len).reshape(-1), _i32(C).reshape(-1)
+    return int(load().cp_workspace_bytes_fp8(ctypes.c_int32(nl.size), _hp(nl), _hp(cs), ctypes.c_int32(Hq)))
+
+
+def cp_prefill_attn_fp8(ctx, q, cache, page_table, prefix_len, new_len, C, Hq, scale, out, lse, workspace, stream=None):
+    _check(load().cp_prefill_attn_fp8(ctx._h, _ptr(q), ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(prefix_len),
+                                      ctypes.c_int64(new_len), ctypes.c_int32(C), ctypes.c_int32(Hq),
+                                      ctypes.c_float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
+                                      ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
+
+
+def cp_prefill_attn_fp8_batch(ctx, q, cache, page_table, cu_new, prefix_len, C, cu_pages, Hq, scale, out, lse, workspace,
+                              stream=None):
+    cu_new, prefix_len, cu_pages, C = _i64(cu_new), _i64(prefix_len), _i64(cu_pages), _i32(C)
+    B = prefix_len.size
+    assert cu_new.size == B + 1 and cu_pages.size == B + 1 and C.size == B
+    _check(load().cp_prefill_attn_fp8_batch(
+        ctx._h, _ptr(q), ctypes.byref(cache), _ptr(page_table), ctypes.c_int32(B), _hp(cu_new), _hp(prefix_len), _hp(C),
+        _hp(cu_pages), ctypes.c_int32(Hq), ctypes.c_float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
+        ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
+
+
+def cp_kv_append_fp8(ctx, cache, page_table, t_begin, n, k_rows, v_rows, stream=None):
+    """bf16 rows [n, Hkv, D] -> E4M3 bytes of logical tokens t_begin.. of the FP8 cache (per-head scales)."""
+    _check(load().cp_kv_append_fp8(ctx._h, ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(t_begin),
+                                   ctypes.c_int64(n), _ptr(k_rows), _ptr(v_rows), _stream(stream)))

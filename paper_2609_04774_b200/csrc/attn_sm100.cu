@@ -83,6 +83,13 @@ constexpr uint32_t kTmemO = 256;   // + wg * 128
 constexpr uint32_t kTryWaitHintNs = 200000;             // the thread may stay suspended this long per try
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
 constexpr float kRescaleThreshold = 8.0f;
+// FP8 K/V variant: one K or V tile is 128 keys x 128 one-byte elements (it uses the first half of a 32 KB ring
+// slot); P is multiplied by 2^kP8Shift before it is rounded to E4M3, and the running-max reference may lag by at
+// most 2^kRescaleThreshold8, so that the scaled weights stay <= 256 (the format ends at 448) while weights down
+// to 2^-10 of the row's largest keep the full 3-bit mantissa.
+constexpr uint32_t kTileBytes8 = kBlockN * kD;     // 16384
+constexpr float kRescaleThreshold8 = 4.0f;
+constexpr float kP8Shift = 4.0f;
 constexpr int kPieces = 2;                            // P is handed to the P*V issuer in two pieces:
 constexpr int kSplitQ = 3;                            // the first kSplitQ quarters of the row, then the rest
 constexpr int kPolyOf4 = 0;                            // pairs out of every four whose exp2 runs on the FMA pipe instead of MUFU:
@@ -117,6 +124,10 @@ struct AttnParams {
     // lse = -inf from the kernel's spare warp
     int32_t n_fill;
     int32_t fill[2 * kMaxFillRanges];
+    // FP8 K/V variant: per-row query scales [rows, Hq] (written by the quantising pre-pass), per-KV-head scales
+    const float* q_scale;
+    const float* k_scale;
+    const float* v_scale;
 };
 
 // ------------------------------------------------------------------------------------------
@@ -202,6 +213,22 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
 }
 
+// the same two forms for one-byte operands (E4M3 x E4M3, fp32 accumulation; K = 32 per instruction)
+__device__ __forceinline__ void mma_ss_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_ts_f8(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+
 #define CP_R8(a, o) "=f"(a[o + 0]), "=f"(a[o + 1]), "=f"(a[o + 2]), "=f"(a[o + 3]), "=f"(a[o + 4]), "=f"(a[o + 5]), "=f"(a[o + 6]), "=f"(a[o + 7])
 #define CP_W8F(a, o) "f"(a[o + 0]), "f"(a[o + 1]), "f"(a[o + 2]), "f"(a[o + 3]), "f"(a[o + 4]), "f"(a[o + 5]), "f"(a[o + 6]), "f"(a[o + 7])
 #define CP_W8R(a, o) "r"(a[o + 0]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]), "r"(a[o + 5]), "r"(a[o + 6]), "r"(a[o + 7])
@@ -221,6 +248,9 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
     asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "                                         \
                  "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"                                 \
                  ::CP_W8R(v, o), CP_W8R(v, o + 8), "r"(taddr) : "memory")
+#define TMEM_ST8R(taddr, v, o)                                                                            \
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"                    \
+                 ::CP_W8R(v, o), "r"(taddr) : "memory")
 #define TMEM_ST32R(taddr, v, o)                                                                           \
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "                                         \
                  "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                  \
@@ -265,6 +295,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&b);
 }
 
+// Four weights -> four E4M3 bytes of one TMEM column, lowest key in the lowest byte (round to nearest even,
+// saturating at 448).  cvt packs its first source into the upper byte of the pair.
+__device__ __forceinline__ uint32_t pack_e4m3x4(float e0, float e1, float e2, float e3) {
+    uint16_t lo, hi;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(e1), "f"(e0));
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(e3), "f"(e2));
+    return (uint32_t)lo | ((uint32_t)hi << 16);
+}
+
 // tcgen05 shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
 // K-major operand (Q, K): rows of 128 B, 8-row groups 1024 B apart (SBO); LBO unused.
 // MN-major operand (V): 64 dims contiguous per key row (128 B), 8-key groups 1024 B apart (SBO),
@@ -281,6 +320,9 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 // instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = 128; bit 16 = B is MN-major
 constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((kBlockN >> 3) << 17) | ((kBlockM >> 4) << 24);
 constexpr uint32_t kIdescPV = kIdescS | (1u << 16);
+// one-byte operands: A and B format fields 0 = E4M3; same shape; K = 32 per instruction
+constexpr uint32_t kIdescS8 = (1u << 4) | ((kBlockN >> 3) << 17) | ((kBlockM >> 4) << 24);
+constexpr uint32_t kIdescPV8 = kIdescS8 | (1u << 16);
 
 // Bounded wait on an mbarrier phase.  The fast path is a single try; the slow path spins with a cycle
 // limit.  When the limit runs out the first thread to notice records {code, barrier id, block,
@@ -371,6 +413,7 @@ __device__ __forceinline__ bool fetch_unit(const AttnParams& p, const InlineSche
 // ------------------------------------------------------------------------------------------
 // Roles
 // ------------------------------------------------------------------------------------------
+template <bool kFp8>
 __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV, const AttnParams& p,
                               const InlineSched& inl, uint32_t smem_base, volatile uint32_t* abort_flag) {
     const int lane = threadIdx.x & 31;
@@ -382,16 +425,21 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
         if (lane == 0) {
             mbar_wait(bars, kBarQEmpty, (round & 1) ^ 1, abort_flag, p.status, round);
             const uint32_t qbar = bars + kBarQFull * 8;
-            mbar_expect_tx(qbar, p.heads_per_unit * kTileBytes);
-            for (int h = 0; h < p.heads_per_unit; ++h)
-                for (int half = 0; half < 2; ++half)
-                    tma_load_3d(smem_base + kSmemQ + h * kTileBytes + half * kHalfBytes, tmQ, qbar, half * 64,
-                                u.head0 + h, u.it.q_row0);
+            mbar_expect_tx(qbar, p.heads_per_unit * (kFp8 ? kTileBytes8 : kTileBytes));
+            for (int h = 0; h < p.heads_per_unit; ++h) {
+                if (kFp8) {      // one-byte queries: a row is one 128-byte swizzle line
+                    tma_load_3d(smem_base + kSmemQ + h * kTileBytes, tmQ, qbar, 0, u.head0 + h, u.it.q_row0);
+                } else {
+                    for (int half = 0; half < 2; ++half)
+                        tma_load_3d(smem_base + kSmemQ + h * kTileBytes + half * kHalfBytes, tmQ, qbar, half * 64,
+                                    u.head0 + h, u.it.q_row0);
+                }
+            }
         }
         __syncwarp();
         const int n_tiles = u.t_end;
         const int ppt = kBlockN / p.page_tokens;          // pages per KV tile: 8, 4, 2 or 1
-        const uint32_t box_bytes = (uint32_t)p.page_tokens * 128u;   // one page x 64 dims
+        const uint32_t box_bytes = (uint32_t)p.page_tokens * 128u;   // one page x 64 bf16 dims (x 128 one-byte dims)
         // load order = order of first use by the issuers: K(j0), then K(j+1) before V(j)
         const int n_loads = 2 * (n_tiles - u.t_begin);
         int pg_base = -1;       // first page whose id the lanes currently hold
@@ -417,14 +465,14 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
             const CUtensorMap* map = kv ? tmV : tmK;
             if (lane == 0) {
                 mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j);
-                mbar_expect_tx(fbar, kTileBytes);
+                mbar_expect_tx(fbar, kFp8 ? kTileBytes8 : kTileBytes);
             }
             __syncwarp();
             // lane i < ppt copies page i of the tile: both 64-dim halves of its box
             const int page = __shfl_sync(0xffffffffu, my_page, (pg0 - pg_base + (lane < ppt ? lane : 0)) & 31);
             if (lane < ppt) {
                 tma_load_4d(dst + lane * box_bytes, map, fbar, 0, u.kv_head, 0, page);
-                tma_load_4d(dst + kHalfBytes + lane * box_bytes, map, fbar, 64, u.kv_head, 0, page);
+                if (!kFp8) tma_load_4d(dst + kHalfBytes + lane * box_bytes, map, fbar, 64, u.kv_head, 0, page);
             }
             __syncwarp();
             ++kv_it;
@@ -454,7 +502,7 @@ struct RingPos {
 // (S buffer) and P*V (P and O columns) touch disjoint TMEM and the K and V tiles have their own barriers.
 //
 // Score issuer: S tiles in the order (tile, head); each needs its K tile and the buffer back (s_free).
-template <bool kDual>
+template <bool kDual, bool kFp8>
 __device__ __forceinline__ void mma_s_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
                                            volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
@@ -479,11 +527,19 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, const InlineSche
                 s_par ^= 1u;
                 tc_fence_after();
                 if (elect_one()) {
+                    if (kFp8) {
+                        // one-byte operands: the 128 dims of a row are one swizzle line, four steps of 32 bytes
 #pragma unroll
-                    for (int ks = 0; ks < kD / 16; ++ks) {
-                        const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
-                        mma_ss(tmem_base + kTmemS, q_desc0 + (h * (kTileBytes >> 4)) + off,
-                               k_desc0 + kpos.slot * (kTileBytes >> 4) + off, kIdescS, ks > 0);
+                        for (int ks = 0; ks < kD / 32; ++ks)
+                            mma_ss_f8(tmem_base + kTmemS, q_desc0 + (h * (kTileBytes >> 4)) + ks * 2,
+                                      k_desc0 + kpos.slot * (kTileBytes >> 4) + ks * 2, kIdescS8, ks > 0);
+                    } else {
+#pragma unroll
+                        for (int ks = 0; ks < kD / 16; ++ks) {
+                            const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+                            mma_ss(tmem_base + kTmemS, q_desc0 + (h * (kTileBytes >> 4)) + off,
+                                   k_desc0 + kpos.slot * (kTileBytes >> 4) + off, kIdescS, ks > 0);
+                        }
                     }
                     tc_commit(bars + (kBarSReady + wgt) * 8);
                     if (h == H - 1) {
@@ -505,7 +561,7 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, const InlineSche
 // P*V issuer: O_h += P_h V_j in the order (tile, head), each in the two pieces P is handed over in.  In a
 // single-head unit the tiles alternate between the two P / O column sets (two independent online-softmax
 // streams over the even and the odd tiles of the piece, combined in the epilogue).
-template <bool kDual>
+template <bool kDual, bool kFp8>
 __device__ __forceinline__ void mma_pv_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
                                             volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
@@ -531,6 +587,17 @@ __device__ __forceinline__ void mma_pv_role(const AttnParams& p, const InlineSch
                     mbar_wait(bars, kBarPReady + wgt * 4 + part, ppar, abort_flag, p.status, j);
                     tc_fence_after();
                     if (elect_one()) {
+                        if (kFp8) {
+                            // P in E4M3: 4 keys per TMEM column, 32 keys (8 columns, 32 V rows of 128 B) per instruction
+                            const int ks0 = part == 0 ? 0 : kSplitQ, ks1 = part == 0 ? kSplitQ : 4;
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks) {
+                                if (ks >= ks0 && ks < ks1)
+                                    mma_ts_f8(tmem_base + kTmemO + wgt * 128, tmem_base + kTmemP + wgt * 64 + ks * 8,
+                                              v_desc0 + vpos.slot * (kTileBytes >> 4) + ks * (4096 >> 4), kIdescPV8,
+                                              !first || ks > 0);
+                            }
+                        } else {
                         const int ks0 = part == 0 ? 0 : 2 * kSplitQ, ks1 = part == 0 ? 2 * kSplitQ : 8;
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {
@@ -538,6 +605,7 @@ __device__ __forceinline__ void mma_pv_role(const AttnParams& p, const InlineSch
                                 mma_ts(tmem_base + kTmemO + wgt * 128, tmem_base + kTmemP + wgt * 64 + ks * 8,
                                        v_desc0 + vpos.slot * (kTileBytes >> 4) + ks * (2048 >> 4), kIdescPV,
                                        !first || ks > 0);
+                        }
                         }
                         if (part == kPieces - 1) {
                             tc_commit(bars + (kBarPvDone + wgt) * 8);
@@ -600,6 +668,29 @@ __device__ __forceinline__ void exp32(const float (&s)[32], uint32_t (&pk)[16], 
     }
 }
 
+// The same for the FP8 variant: 32 weights -> 8 TMEM columns of four E4M3 bytes each (the caller's exponent
+// offset already holds the 2^kP8Shift scaling); the row sums take the unrounded values.
+__device__ __forceinline__ void exp32_f8(const float (&s)[32], uint32_t (&pk)[8], float2 c2, float2 nm2, float2& sum0,
+                                         float2& sum1, float2& sum2, float2& sum3) {
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+        const float2 x0 = __ffma2_rn(make_float2(s[4 * i + 0], s[4 * i + 1]), c2, nm2);
+        const float2 x1 = __ffma2_rn(make_float2(s[4 * i + 2], s[4 * i + 3]), c2, nm2);
+        const float2 x2 = __ffma2_rn(make_float2(s[4 * i + 4], s[4 * i + 5]), c2, nm2);
+        const float2 x3 = __ffma2_rn(make_float2(s[4 * i + 6], s[4 * i + 7]), c2, nm2);
+        const float2 p0 = make_float2(ex2(x0.x), ex2(x0.y));
+        const float2 p1 = make_float2(ex2(x1.x), ex2(x1.y));
+        const float2 p2 = make_float2(ex2(x2.x), ex2(x2.y));
+        const float2 p3 = make_float2(ex2(x3.x), ex2(x3.y));
+        sum0 = __fadd2_rn(sum0, p0);
+        sum1 = __fadd2_rn(sum1, p1);
+        sum2 = __fadd2_rn(sum2, p2);
+        sum3 = __fadd2_rn(sum3, p3);
+        pk[i + 0] = pack_e4m3x4(p0.x, p0.y, p1.x, p1.y);
+        pk[i + 1] = pack_e4m3x4(p2.x, p2.y, p3.x, p3.y);
+    }
+}
+
 struct SoftmaxSync {
     uint32_t bars;                   // shared-memory address of the barrier array
     uint32_t s_ready_id;             // barrier "a score tile of this head is in the S buffer"
@@ -634,7 +725,7 @@ __device__ __forceinline__ void release_s(uint32_t bars) {
 // Straight-line code in both variants, no per-element branches.
 // kMasked: some keys of the tile are hidden from some rows (causal diagonal, or the edge of the unit's key
 // range); this row sees columns [lo, lim).
-template <bool kMasked>
+template <bool kMasked, bool kFp8>
 __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], float (&c2)[32], float (&c3)[32],
                                              bool more, uint32_t& s_par, uint32_t s_tmem, uint32_t p_tmem,
                                              uint32_t o_tmem, uint32_t p_bar0, float c, int lo, int lim, bool first,
@@ -659,7 +750,7 @@ __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], f
         mbar_wait(sy.bars, sy.pv_done_id, sy.pv_parity, sy.abort_flag, sy.status, sy.iter);
         __syncwarp();
         tc_fence_after();
-        const bool grow = (m_new - m) > kRescaleThreshold;
+        const bool grow = (m_new - m) > (kFp8 ? kRescaleThreshold8 : kRescaleThreshold);
         if (__any_sync(0xffffffffu, grow)) {
             const float m_upd = grow ? m_new : m;
             const float alpha = ex2(m - m_upd);
@@ -679,13 +770,18 @@ __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], f
     const float2 c2f = make_float2(c, c);
     // a row that has seen no key yet (only possible in masked tiles of a KV-split piece) keeps m = -inf;
     // subtracting 0 instead keeps its weights at exactly 0 rather than NaN
-    const float m_sub = (kMasked && m == -INFINITY) ? 0.f : m;
+    const float m_sub = ((kMasked && m == -INFINITY) ? 0.f : m) - (kFp8 ? kP8Shift : 0.f);
     const float2 nm2 = make_float2(-m_sub, -m_sub);
     float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0, sum2 = sum0, sum3 = sum0;
-    uint32_t pk[16];
+    uint32_t pk[kFp8 ? 8 : 16];
 #define CP_P_PIECE(cur, q)                                                              \
-    exp32<!kMasked>(cur, pk, c2f, nm2, sum0, sum1, sum2, sum3);                         \
-    TMEM_ST16R(p_tmem + (q) * 16, pk, 0);                                               \
+    if constexpr (kFp8) {                                                               \
+        exp32_f8(cur, pk, c2f, nm2, sum0, sum1, sum2, sum3);                            \
+        TMEM_ST8R(p_tmem + (q) * 8, pk, 0);                                             \
+    } else {                                                                            \
+        exp32<!kMasked>(cur, pk, c2f, nm2, sum0, sum1, sum2, sum3);                     \
+        TMEM_ST16R(p_tmem + (q) * 16, pk, 0);                                           \
+    }                                                                                   \
     if ((q) + 1 == kSplitQ || (q) == 3) {                                               \
         tc_wait_st();                                                                   \
         tc_fence_before();                                                              \
@@ -725,7 +821,7 @@ __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], f
     l += st.x + st.y;
 }
 
-template <bool kDual>
+template <bool kDual, bool kFp8>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
                                              volatile uint32_t* abort_flag, uint8_t* smem_xchg, int wg) {
     const uint32_t bars = smem_base + kSmemBar;
@@ -737,7 +833,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
     const uint32_t p_tmem = tmem_base + lane_addr + kTmemP + wg * 64;
     const uint32_t o_tmem = tmem_base + lane_addr + kTmemO + wg * 128;
     const uint32_t p_bar0 = bars + (kBarPReady + wg * 4) * 8;
-    const float c = p.scale_log2;
+    float c = p.scale_log2;
     uint32_t tile_cnt = 0;
     // single-head units: the two warpgroups take the even and the odd KV tiles of the piece as two independent
     // online-softmax streams (own running max, sum and O accumulator); warpgroup 0 combines them at the end
@@ -757,6 +853,9 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
         const int j_first = u.t_begin + (dual ? wg : 0);     // first tile of this warpgroup's stream
         float m = -INFINITY;   // running row max in log2 units (possibly stale by < threshold)
         float l = 0.f;         // running row sum of 2^(s - m)
+        if (kFp8)              // raw scores are products of codes: this row's query scale and the head's key scale
+            c = p.scale_log2 * p.k_scale[u.kv_head] *
+                (row < u.it.n_rows ? p.q_scale[((int64_t)u.it.q_row0 + row) * p.Hq + head] : 0.f);
         // tiles below n_full lie entirely under the causal diagonal of every row of the q-tile and inside the
         // unit's key range; the range's first tile is cut on the left when kv_lo is not a tile multiple
         const int n_full = min(u.it.kv_len0, u.it.kv_hi) / kBlockN;
@@ -775,10 +874,10 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
             const SoftmaxSync sy = {bars, kBarSReady + (uint32_t)wg, kBarPvDone + (uint32_t)wg, (tile_cnt - 1) & 1,
                                     abort_flag, p.status, j};
             if (j < n_full && j != j_cut)
-                softmax_tile<false>(s0, s1, s2, s3, j + step < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c, 0, 0,
-                                    j == j_first, m, l, sy);
+                softmax_tile<false, kFp8>(s0, s1, s2, s3, j + step < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c, 0, 0,
+                                          j == j_first, m, l, sy);
             else
-                softmax_tile<true>(s0, s1, s2, s3, j + step < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c,
+                softmax_tile<true, kFp8>(s0, s1, s2, s3, j + step < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c,
                                    u.it.kv_lo - j * kBlockN, min(u.it.kv_len0 + row, u.it.kv_hi) - j * kBlockN,
                                    j == j_first, m, l, sy);
             ++tile_cnt;
@@ -810,7 +909,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
         SM_WAIT(kBarPvDone + wg, (tile_cnt - 1) & 1, n);
         tc_fence_after();
         // a row of a KV-split piece may see none of the piece's keys: l = 0, written as O = 0, lse = -inf
-        const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
+        // (FP8 variant: O and l both carry the 2^kP8Shift factor of the weights, which cancels; V's scale joins here)
+        const float inv_l = (l > 0.f) ? (kFp8 ? p.v_scale[u.kv_head] : 1.f) / l : 0.f;
         const bool partial = u.slot >= 0;
         const bool valid = row < u.it.n_rows;
         const int64_t grow_idx = (int64_t)u.it.q_row0 + row;
@@ -857,7 +957,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
             }
         }
         if (valid) {
-            const float lse_val = (l > 0.f) ? (m + lg2(l)) * 0.6931471805599453f : -INFINITY;
+            const float lse_val = (l > 0.f) ? (m + lg2(l) - (kFp8 ? kP8Shift : 0.f)) * 0.6931471805599453f : -INFINITY;
             if (partial) p.partial_lse[((int64_t)u.slot * 2 + wg) * kBlockM + row] = lse_val;
             else p.lse[(int64_t)head * p.lse_stride + grow_idx] = lse_val;
         }
@@ -892,7 +992,7 @@ __device__ __forceinline__ void fill_role(const AttnParams& p) {
 
 // kDual: every unit is a single query head (odd group size); its KV tiles then alternate between the two
 // softmax warpgroups.  Two separate kernels, so that neither carries the other's code in its hot loop.
-template <bool kDual>
+template <bool kDual, bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const AttnParams p, const __grid_constant__ InlineSched inl) {
@@ -932,15 +1032,15 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-        softmax_role<kDual>(p, inl, smem_base, tmem_base, abort_flag, smem_gen + kSmemXchg, warp >> 2);
+        softmax_role<kDual, kFp8>(p, inl, smem_base, tmem_base, abort_flag, smem_gen + kSmemXchg, warp >> 2);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
         if (warp == 8) {
-            producer_role(&tmQ, &tmK, &tmV, p, inl, smem_base, abort_flag);
+            producer_role<kFp8>(&tmQ, &tmK, &tmV, p, inl, smem_base, abort_flag);
         } else if (warp == 9) {
-            mma_s_role<kDual>(p, inl, smem_base, tmem_base, abort_flag);
+            mma_s_role<kDual, kFp8>(p, inl, smem_base, tmem_base, abort_flag);
         } else if (warp == 10) {
-            mma_pv_role<kDual>(p, inl, smem_base, tmem_base, abort_flag);
+            mma_pv_role<kDual, kFp8>(p, inl, smem_base, tmem_base, abort_flag);
         } else if (p.n_fill > 0) {
             fill_role(p);
         }
@@ -1107,6 +1207,54 @@ int encode_maps(cp_ctx* ctx, const void* q, int64_t total_rows, int32_t Hq, cons
     return CP_OK;
 }
 
+// Tensor maps of the FP8 variant: one-byte elements, a 128-dim row is one 128-byte swizzle line.
+int encode_maps_fp8(cp_ctx* ctx, const void* q8, int64_t total_rows, int32_t Hq, const cp_kv_cache_fp8* c, CUtensorMap* tmQ,
+                    CUtensorMap* tmK, CUtensorMap* tmV) {
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)Hq, (cuuint64_t)total_rows};
+        cuuint64_t strides[2] = {(cuuint64_t)kD, (cuuint64_t)Hq * kD};
+        cuuint32_t box[3] = {(cuuint32_t)kD, 1, (cuuint32_t)kBlockM};
+        cuuint32_t es[3] = {1, 1, 1};
+        CUresult r = ctx->encode_tiled(tmQ, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(q8), dims, strides, box,
+                                       es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return set_error(CP_ERR_CUDA, "cuTensorMapEncodeTiled(q8) failed with %d", (int)r);
+    }
+    for (int kv = 0; kv < 2; ++kv) {
+        cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)c->Hkv, (cuuint64_t)c->page_size, (cuuint64_t)c->num_pages};
+        cuuint64_t strides[3] = {(cuuint64_t)c->stride_head, (cuuint64_t)c->stride_tok, (cuuint64_t)c->stride_page};
+        cuuint32_t box[4] = {(cuuint32_t)kD, 1, (cuuint32_t)c->page_size, 1};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        CUresult r = ctx->encode_tiled(kv ? tmV : tmK, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4,
+                                       const_cast<void*>(kv ? c->v : c->k), dims, strides, box, es,
+                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return set_error(CP_ERR_CUDA, "cuTensorMapEncodeTiled(%s8) failed with %d", kv ? "v" : "k", (int)r);
+    }
+    return CP_OK;
+}
+
+// Query quantisation of the FP8 variant, one warp per (token, head) row of 128 bf16 values: amax by shuffles,
+// q_scale = amax / 448 and inv = 448 / amax (IEEE divisions), code = e4m3(q * inv) with round to nearest even and
+// saturation; a row of zeros gets scale 0 and codes 0.
+__global__ void __launch_bounds__(256)
+quantize_q_kernel(const __nv_bfloat16* __restrict__ q, uint8_t* __restrict__ q8, float* __restrict__ q_scale, int64_t n_rows) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= n_rows) return;
+    const uint2 raw = reinterpret_cast<const uint2*>(q + row * kD)[lane];
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+    const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+    const float x0 = __low2float(a), x1 = __high2float(a), x2 = __low2float(b), x3 = __high2float(b);
+    float amax = fmaxf(fmaxf(fabsf(x0), fabsf(x1)), fmaxf(fabsf(x2), fabsf(x3)));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+    reinterpret_cast<uint32_t*>(q8 + row * kD)[lane] =
+        pack_e4m3x4(__fmul_rn(x0, inv), __fmul_rn(x1, inv), __fmul_rn(x2, inv), __fmul_rn(x3, inv));
+    if (lane == 0) q_scale[row] = amax > 0.f ? __fdiv_rn(amax, 448.f) : 0.f;
+}
+
 // Moves 16-byte words from pinned host memory (read over PCIe) into device memory.  Used instead of a
 // copy-engine transfer for the schedule: a kernel stays on the compute engine, so the attention launch
 // behind it does not wait on a cross-engine hand-over.
@@ -1150,10 +1298,27 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
                 const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C, const int64_t* cu_pages,
                 int32_t only_shard, int32_t only_chunk, int64_t kv_lo, int64_t kv_hi, int32_t Hq, float scale, void* out,
                 int out_f32, bool want_fill, float* lse, void* workspace, size_t workspace_bytes, void* stream,
-                const char* who) {
+                const char* who, const cp_kv_cache_fp8* cache8 = nullptr) {
     if (!ctx || !q || !page_table || !out || !lse || B < 1 || !cu_new || !prefix_len || !C || !cu_pages)
         return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or B < 1", who);
-    if (int rc = validate_kv_cache(cache, who)) return rc;
+    cp_kv_cache shape8;         // FP8 variant: the cache's shape in the bf16 descriptor's fields, for the shared logic
+    if (cache8) {
+        if (int rc = validate_kv_cache_fp8(cache8, who)) return rc;
+        shape8.k = cache8->k;
+        shape8.v = cache8->v;
+        shape8.num_pages = cache8->num_pages;
+        shape8.page_size = cache8->page_size;
+        shape8.Hkv = cache8->Hkv;
+        shape8.D = cache8->D;
+        shape8.reserved = 0;
+        shape8.stride_page = cache8->stride_page;
+        shape8.stride_tok = cache8->stride_tok;
+        shape8.stride_head = cache8->stride_head;
+        cache = &shape8;
+        if ((cache->Hkv < 1) || (Hq / cache->Hkv) % 2 != 0)
+            return set_error(CP_ERR_UNSUPPORTED, "%s: the FP8 variant needs an even number of query heads per KV head "
+                             "(Hq=%d, Hkv=%d)", who, Hq, cache->Hkv);
+    } else if (int rc = validate_kv_cache(cache, who)) return rc;
     if (Hq < 1 || Hq % cache->Hkv != 0)
         return set_error(CP_ERR_INVALID_ARG, "%s: Hq=%d is not a multiple of Hkv=%d", who, Hq, cache->Hkv);
     // even group size: two query heads of one KV group share every K/V tile; odd: one head per unit
@@ -1176,7 +1341,9 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     }
     if (cu_new[B] > 0x7fffff00ll || cu_pages[B] > 0x7fffff00ll)
         return set_error(CP_ERR_UNSUPPORTED, "%s: more than 2^31 packed rows or pages", who);
-    const size_t need_ws = cp_workspace_bytes(B, new_len.data(), C, Hq);   // sized for one head per unit
+    const size_t base_ws = cp_workspace_bytes(B, new_len.data(), C, Hq);   // sized for one head per unit
+    // FP8 variant: the quantised queries [rows, Hq, 128] and their scales [rows, Hq] follow the schedule space
+    const size_t need_ws = cache8 ? cp_workspace_bytes_fp8(B, new_len.data(), C, Hq) : base_ws;
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need_ws)
         return set_error(CP_ERR_WORKSPACE, "%s: workspace %p of %zu bytes; need %zu bytes, 256-byte aligned", who,
                          workspace, workspace_bytes, need_ws);
@@ -1192,7 +1359,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         key = 1469598103934665603ull;
         auto mix = [&key](int64_t v) { key = (key ^ (uint64_t)v) * 1099511628211ull; };
         mix(B); mix(Hq); mix(cache->Hkv); mix(cache->page_size); mix(only_shard); mix(only_chunk); mix(kv_lo); mix(kv_hi);
-        mix(grid_max); mix(out_f32); mix(want_fill);
+        mix(grid_max); mix(out_f32); mix(want_fill); mix(cache8 != nullptr);
         for (int32_t b = 0; b < B; ++b) { mix(cu_new[b + 1]); mix(prefix_len[b]); mix(C[b]); mix(cu_pages[b + 1]); }
     }
     WorkspaceLayout lay;        // where the partial results (and the lists of a large schedule) sit in the workspace
@@ -1299,11 +1466,23 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     }
 
     CUtensorMap tmQ, tmK, tmV;
-    if (int rc = encode_maps(ctx, q, total_rows, Hq, cache, &tmQ, &tmK, &tmV)) return rc;
+    uint8_t* q8 = ws + base_ws;
+    float* q_scale = reinterpret_cast<float*>(q8 + (size_t)total_rows * Hq * kD);
+    if (cache8) {
+        // quantise the queries once per call (a unit cut along KV would otherwise repeat it per piece)
+        const int64_t n_rows = total_rows * Hq;
+        quantize_q_kernel<<<(unsigned)((n_rows + 7) / 8), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(q), q8, q_scale, n_rows);
+        if (int rc = check_cuda(cudaGetLastError(), "quantize_q launch")) return rc;
+        if (int rc = encode_maps_fp8(ctx, q8, total_rows, Hq, cache8, &tmQ, &tmK, &tmV)) return rc;
+    } else if (int rc = encode_maps(ctx, q, total_rows, Hq, cache, &tmQ, &tmK, &tmV)) {
+        return rc;
+    }
     if (!ctx->attn_attr_set) {
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
         ctx->attn_attr_set = true;
     }
@@ -1339,8 +1518,12 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.status = ctx->d_status;
     p.n_fill = n_fill;
     memcpy(p.fill, fill, sizeof fill);
-    if (heads_per_unit == 2) cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
-    else cp_attn_kernel<true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
+    p.q_scale = cache8 ? q_scale : nullptr;
+    p.k_scale = cache8 ? cache8->k_scale : nullptr;
+    p.v_scale = cache8 ? cache8->v_scale : nullptr;
+    if (cache8) cp_attn_kernel<false, true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
+    else if (heads_per_unit == 2) cp_attn_kernel<false, false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
+    else cp_attn_kernel<true, false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
     if (int rc = check_cuda(cudaGetLastError(), who)) return rc;
     if (n_merges > 0) {
         FixupParams f;
@@ -1388,6 +1571,26 @@ extern "C" int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* ca
     const int64_t cu_pages[2] = {0, (prefix_len + new_len + page_tokens_of(cache) - 1) / page_tokens_of(cache)};
     return attn_common(ctx, q, cache, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, 0, INT32_MAX, Hq, scale, out, 0,
                        false, lse, workspace, workspace_bytes, stream, "cp_prefill_attn");
+}
+
+extern "C" int cp_prefill_attn_fp8_batch(cp_ctx* ctx, const void* q, const cp_kv_cache_fp8* cache, const int32_t* page_table,
+                                         int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
+                                         const int64_t* cu_pages, int32_t Hq, float scale, void* out, float* lse,
+                                         void* workspace, size_t workspace_bytes, void* stream) {
+    if (!cache) return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_fp8_batch: cache is NULL");
+    return attn_common(ctx, q, nullptr, page_table, B, cu_new, prefix_len, C, cu_pages, -1, -1, 0, INT32_MAX, Hq, scale, out, 0,
+                       false, lse, workspace, workspace_bytes, stream, "cp_prefill_attn_fp8_batch", cache);
+}
+
+extern "C" int cp_prefill_attn_fp8(cp_ctx* ctx, const void* q, const cp_kv_cache_fp8* cache, const int32_t* page_table,
+                                   int64_t prefix_len, int64_t new_len, int32_t C, int32_t Hq, float scale, void* out,
+                                   float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!cache || new_len < 1 || prefix_len < 0 || cache->page_size < 1)
+        return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_fp8: cache is NULL, new_len < 1 or prefix_len < 0");
+    const int64_t cu_new[2] = {0, new_len};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + cache->page_size - 1) / cache->page_size};
+    return attn_common(ctx, q, nullptr, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, 0, INT32_MAX, Hq, scale, out, 0,
+                       false, lse, workspace, workspace_bytes, stream, "cp_prefill_attn_fp8", cache);
 }
 
 // The two partial-result calls write zeros with lse = -inf (the identity element of cp_merge) into the rows
@@ -1481,9 +1684,9 @@ int static_setup(int device, StaticDeviceState** out) {
                                 "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)")) return rc;
         if (q != cudaDriverEntryPointSuccess || !fn)
             return set_error(CP_ERR_CUDA, "cuTensorMapEncodeTiled is not available in this driver");
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
         st.scratch = static_cast<unsigned char*>(ptr);
         st.num_sms = prop.multiProcessorCount;
@@ -1575,11 +1778,12 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     p.status = reinterpret_cast<int32_t*>(st->scratch);
     p.inl_items = p.inl_cta_off = p.inl_pieces = -1;
     p.n_fill = 0;
+    p.q_scale = p.k_scale = p.v_scale = nullptr;
     InlineSched none;          // unused: the tile list is in the scratch
     none.bytes[0] = 0;
     const int64_t units = n_tiles * p.pairs_per_tile;
     const int grid = (int)std::min<int64_t>(units, st->num_sms);
-    if (heads_per_unit == 2) cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, none);
-    else cp_attn_kernel<true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, none);
+    if (heads_per_unit == 2) cp_attn_kernel<false, false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, none);
+    else cp_attn_kernel<true, false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, none);
     return check_cuda(cudaGetLastError(), who);
 }

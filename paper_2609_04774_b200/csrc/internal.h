@@ -97,6 +97,7 @@ int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C);
 // chunk and numbers its rows from the chunk's first row (q, out and lse then hold the chunk alone).
 // [kv_lo, kv_hi) restricts the keys (absolute positions); tiles that see none of them are left out.
 int validate_kv_cache(const cp_kv_cache* c, const char* who);
+int validate_kv_cache_fp8(const cp_kv_cache_fp8* c, const char* who);
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
                 const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, int64_t kv_lo,
                 int64_t kv_hi, std::vector<TileItem>& out);

@@ -1,5 +1,7 @@
 // cp_kv_gather / cp_kv_append: bit-exact copies between a paged KV cache and contiguous rows,
 // addressed through the page table.  One 16-byte vector per thread; HBM-bound.
+#include <cuda_bf16.h>
+
 #include <algorithm>
 
 #include "internal.h"
@@ -59,6 +61,66 @@ int validate_cache(const cp_kv_cache* c, const char* who) {
     return CP_OK;
 }
 
+// FP8 cache writer: eight bf16 values of a row -> eight E4M3 bytes, each e4m3_rne_satfinite(x / scale[g]) with
+// the quotient rounded to fp32 first.  Page ids outside the pool are skipped and reported like in the copies.
+__device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d, float sc) {
+    uint16_t lo, hi;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(__fdiv_rn(b, sc)), "f"(__fdiv_rn(a, sc)));
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(__fdiv_rn(d, sc)), "f"(__fdiv_rn(c, sc)));
+    return (uint32_t)lo | ((uint32_t)hi << 16);
+}
+
+__global__ void __launch_bounds__(256)
+kv_append_fp8_kernel(uint8_t* __restrict__ paged_k, uint8_t* __restrict__ paged_v, const uint4* __restrict__ rows_k,
+                     const uint4* __restrict__ rows_v, const float* __restrict__ k_scale, const float* __restrict__ v_scale,
+                     const int32_t* __restrict__ page_table, int64_t t_begin, int64_t n, int page_size, int Hkv,
+                     int64_t stride_page, int64_t stride_tok, int64_t stride_head, int64_t num_pages, int32_t* status) {
+    const int vec_per_tok = Hkv * 16;                 // 8 elements per thread
+    const int64_t total = n * vec_per_tok;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t tok = i / vec_per_tok;
+        const int rem = (int)(i - tok * vec_per_tok);
+        const int g = rem >> 4, c = rem & 15;
+        const int64_t t = t_begin + tok;
+        const int64_t page = page_table[t / page_size];
+        if (page < 0 || page >= num_pages) {
+            if (atomicCAS(status, 0, CP_ERR_BOUNDS) == 0) {
+                status[1] = (int32_t)(t / page_size);
+                status[2] = (int32_t)blockIdx.x;
+                status[3] = (int32_t)page;
+            }
+            continue;
+        }
+        const int64_t off = page * stride_page + (t % page_size) * stride_tok + (int64_t)g * stride_head + c * 8;
+#pragma unroll
+        for (int kv = 0; kv < 2; ++kv) {
+            const uint4* rows = kv ? rows_v : rows_k;
+            if (!rows) continue;
+            const uint4 raw = rows[i];
+            const float sc = kv ? v_scale[g] : k_scale[g];
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+            uint2 o;
+            o.x = quant4(__low2float(h[0]), __high2float(h[0]), __low2float(h[1]), __high2float(h[1]), sc);
+            o.y = quant4(__low2float(h[2]), __high2float(h[2]), __low2float(h[3]), __high2float(h[3]), sc);
+            *reinterpret_cast<uint2*>((kv ? paged_v : paged_k) + off) = o;
+        }
+    }
+}
+
+int validate_cache_fp8(const cp_kv_cache_fp8* c, const char* who) {
+    if (!c || !c->k || !c->v || !c->k_scale || !c->v_scale || c->num_pages < 1 || c->Hkv < 1)
+        return set_error(CP_ERR_INVALID_ARG, "%s: FP8 cache is NULL or has null / non-positive fields", who);
+    if ((c->page_size != 16 && c->page_size != 32 && c->page_size != 64 && c->page_size != 128) || c->D != 128)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: page_size=%d D=%d; supported: pages of 16, 32, 64 or 128 tokens, D = 128", who,
+                         c->page_size, c->D);
+    if ((c->stride_page | c->stride_tok | c->stride_head) & 15 || c->stride_page < 1 || c->stride_tok < 1 ||
+        c->stride_head < 1)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: FP8 cache strides must be positive multiples of 16 bytes", who);
+    if (((uintptr_t)c->k | (uintptr_t)c->v) & 15)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: k and v must be 16-byte aligned", who);
+    return CP_OK;
+}
+
 template <bool kToPaged>
 int kv_copy(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin, int64_t n,
             const void* k_rows, const void* v_rows, void* stream, const char* who) {
@@ -84,6 +146,27 @@ int kv_copy(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, in
 
 namespace cpattn {
 int validate_kv_cache(const cp_kv_cache* c, const char* who) { return validate_cache(c, who); }
+int validate_kv_cache_fp8(const cp_kv_cache_fp8* c, const char* who) { return validate_cache_fp8(c, who); }
+}
+
+extern "C" int cp_kv_append_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,
+                                int64_t n, const void* k_rows, const void* v_rows, void* stream) {
+    const char* who = "cp_kv_append_fp8";
+    if (!ctx || !page_table || t_begin < 0 || n < 0)
+        return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or negative range", who);
+    if (int rc = validate_cache_fp8(cache, who)) return rc;
+    if (!k_rows && !v_rows) return set_error(CP_ERR_INVALID_ARG, "%s: both row pointers are NULL", who);
+    if (((uintptr_t)k_rows | (uintptr_t)v_rows) & 15)
+        return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
+    if (n == 0) return CP_OK;
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+    const int64_t total = n * cache->Hkv * 16;
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
+    kv_append_fp8_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        (uint8_t*)cache->k, (uint8_t*)cache->v, (const uint4*)k_rows, (const uint4*)v_rows, cache->k_scale, cache->v_scale,
+        page_table, t_begin, n, cache->page_size, cache->Hkv, cache->stride_page, cache->stride_tok, cache->stride_head,
+        cache->num_pages, ctx->d_status);
+    return check_cuda(cudaGetLastError(), who);
 }
 
 extern "C" int cp_kv_gather(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin,

@@ -285,6 +285,15 @@ extern "C" size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const in
     return workspace_layout((size_t)n, (size_t)n * pairs + kMaxSlots, kMaxSlots, kMaxSlots, kMaxGrid, kMaxSlots).total;
 }
 
+extern "C" size_t cp_workspace_bytes_fp8(int32_t B, const int64_t* new_len, const int32_t* C, int32_t Hq) {
+    const size_t base = cp_workspace_bytes(B, new_len, C, Hq);
+    if (base == 0) return 0;
+    int64_t rows = 0;
+    for (int32_t b = 0; b < B; ++b) rows += new_len[b];
+    // quantised queries (one byte per element) and one fp32 scale per (token, head) row
+    return base + align_up((size_t)rows * Hq * (128 + sizeof(float)), 256);
+}
+
 extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
                                    int32_t Hq, int32_t Hkv, int32_t num_sms, int64_t* summary, int32_t* pieces,
                                    int64_t max_pieces, int32_t* items, int64_t max_items) {

@@ -1,0 +1,165 @@
+"""GPU parity of the FP8 K/V variant, through the C ABI, against the fp64 oracle on the same stored bytes.
+
+Bit-exact: the query codes and scales the library's pre-pass leaves in the workspace, and the bytes written by
+cp_kv_append_fp8.  Attention: LSE as in the bf16 path; O element by element within the bound the format gives
+for rounding the softmax weights to E4M3, 2^-4 * sum_j p_j |v_j| (the oracle returns that sum), plus 4e-3 for
+fp32 accumulation and the bf16 rounding of the output; per-row relative L2 error at most 2^-4."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fp8 as o8
+from paper_2609_04774_b200 import binding
+from paper_2609_04774_b200 import workloads as wl
+from tests.gpu_util import Guarded, bf16_to_f64, bits_to_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    c.close()
+
+
+class Device8:
+    def __init__(self, m8):
+        w = m8.wl
+        self.w, self.m8 = w, m8
+        self.q = bits_to_bf16(m8.q)
+        self.k8 = torch.from_numpy(m8.k8_pages).cuda()
+        self.v8 = torch.from_numpy(m8.v8_pages).cuda()
+        self.ks = torch.from_numpy(m8.k_scale).cuda()
+        self.vs = torch.from_numpy(m8.v_scale).cuda()
+        self.page_table = torch.from_numpy(m8.page_table).cuda()
+        self.cache = binding.make_cache_fp8(self.k8, self.v8, self.ks, self.vs)
+        self._g_out = Guarded((w.total_new, w.Hq, w.D), torch.bfloat16, float("nan"))
+        self._g_lse = Guarded((w.Hq, w.total_new), torch.float32, float("nan"))
+        nl, cs = [r.new_len for r in w.requests], [r.C for r in w.requests]
+        self.base_ws = binding.cp_workspace_bytes(nl, cs, w.Hq)
+        self._g_ws = Guarded((binding.cp_workspace_bytes_fp8(nl, cs, w.Hq),), torch.uint8, 0)
+        self.out, self.lse, self.ws = self._g_out.tensor, self._g_lse.tensor, self._g_ws.tensor
+
+    def run(self, ctx):
+        w = self.w
+        binding.cp_prefill_attn_fp8_batch(ctx, self.q, self.cache, self.page_table, w.cu_new,
+                                          [r.prefix_len for r in w.requests], [r.C for r in w.requests], w.cu_pages,
+                                          w.Hq, w.scale, self.out, self.lse, self.ws)
+        torch.cuda.synchronize()
+        ctx.poll_status()
+        for g, what in ((self._g_out, "out"), (self._g_lse, "lse"), (self._g_ws, "workspace")):
+            g.check(what)
+        assert not bool(torch.isnan(self.out).any()) and not bool(torch.isnan(self.lse).any()), "a row was not written"
+        return bf16_to_f64(self.out), self.lse.cpu().numpy().astype(np.float64)
+
+    def query_codes(self):
+        """What the quantising pre-pass left behind the schedule space: codes [rows, Hq, 128], scales [rows, Hq]."""
+        w = self.w
+        n = w.total_new * w.Hq
+        codes = self.ws[self.base_ws:self.base_ws + n * 128].cpu().numpy().reshape(w.total_new, w.Hq, 128)
+        scales = self.ws[self.base_ws + n * 128:self.base_ws + n * 132].view(torch.float32).cpu().numpy().reshape(w.total_new, w.Hq)
+        return codes, scales
+
+
+def compare8(out, lse, ref_o, ref_l, ref_a, what):
+    assert np.isfinite(out).all() and np.isfinite(lse).all(), what
+    le = np.abs(lse - ref_l) / np.maximum(1.0, np.abs(ref_l))
+    assert le.max() <= 1e-3, (what, "lse", le.max())
+    excess = np.abs(out - ref_o) - (2.0 ** -4 * ref_a + 4e-3)
+    assert excess.max() <= 0, (what, "element bound exceeded by", excess.max())
+    num = np.sqrt(((out - ref_o) ** 2).sum(-1))
+    den = np.sqrt((ref_o ** 2).sum(-1)) + 1e-30
+    assert (num / den).max() <= 2.0 ** -4, (what, "row rel-L2", (num / den).max())
+    return np.abs(out - ref_o).max(), np.abs(out - ref_o).mean(), (num / den).mean()
+
+
+def check_batch8(ctx, w, rows_per_request=None, seed=7):
+    m8 = wl.materialize_fp8(w)
+    dev = Device8(m8)
+    out, lse = dev.run(ctx)
+    codes, scales = dev.query_codes()
+    ref_codes, ref_scales = o8.quantize_q(m8.q)
+    assert np.array_equal(scales, ref_scales), "query scales differ from the oracle's"
+    assert np.array_equal(o8.e4m3_decode(codes), o8.e4m3_decode(ref_codes)), "query codes differ from the oracle's"
+    stats = []
+    for b, r in enumerate(w.requests):
+        lo, hi = int(w.cu_new[b]), int(w.cu_new[b + 1])
+        if rows_per_request is None or rows_per_request >= r.new_len:
+            rows = np.arange(r.new_len)
+        else:
+            edges = [0, 127, 128, r.new_len - 1]
+            rows = np.unique(np.clip(np.concatenate([wl.sample_rows(seed + b, 1, r.new_len, rows_per_request)[0], edges]), 0, r.new_len - 1))
+        pt = m8.page_table[w.cu_pages[b]:w.cu_pages[b + 1]]
+        ro, rl, ra = o8.attn_fp8_rows(m8.q[lo:hi], m8.k8_pages, m8.v8_pages, m8.k_scale, m8.v_scale, pt, r.prefix_len,
+                                      w.Hkv, w.scale, rows)
+        stats.append(compare8(out[lo:hi][rows], lse[:, lo:hi][:, rows], ro, rl, ra, "%s req %d" % (w.name, b)))
+    return dev, stats
+
+
+def test_fp8_append_matches_oracle_bit_for_bit(ctx):
+    w = wl.Workload("fp8_append", 51, 8, 2, [wl.Request(300, 192, 1)])
+    m8 = wl.materialize_fp8(w)
+    dev = Device8(m8)
+    r = w.requests[0]
+    t0, n = 37, r.total_len - 37
+    newk = wl.normal_bf16(52, wl.TID_K, (n, w.Hkv, w.D))
+    newv = wl.normal_bf16(52, wl.TID_V, (n, w.Hkv, w.D))
+    newk[3, 0, :8] = wl.f32_to_bf16_bits(np.array([1e4, -1e4, 0.0, 448 * m8.k_scale[0], 1e-6, -1e-6, 3e38, -3e38], dtype=np.float32))
+    binding.cp_kv_append_fp8(ctx, dev.cache, dev.page_table, t0, n, bits_to_bf16(newk), bits_to_bf16(newv))
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    kc, vc = o8.quantize_kv(newk, m8.k_scale), o8.quantize_kv(newv, m8.v_scale)
+    kp, vp = m8.k8_pages.copy(), m8.v8_pages.copy()
+    t = np.arange(t0, t0 + n)
+    kp[m8.page_table[t // wl.PAGE], t % wl.PAGE] = kc
+    vp[m8.page_table[t // wl.PAGE], t % wl.PAGE] = vc
+    got_k, got_v = dev.k8.cpu().numpy(), dev.v8.cpu().numpy()
+    assert np.array_equal(o8.e4m3_decode(got_k), o8.e4m3_decode(kp))          # (+0 and -0 codes both stand for zero)
+    assert np.array_equal(o8.e4m3_decode(got_v), o8.e4m3_decode(vp))
+    assert np.array_equal(got_k & 0x7F, kp & 0x7F) and np.array_equal(got_v & 0x7F, vp & 0x7F)
+
+
+def test_fp8_attention_small_mixed_batch(ctx):
+    w = wl.Workload("fp8_small_mixed", 53, 8, 2, [wl.Request(333, 192, 3), wl.Request(5, 0, 4), wl.Request(1, 64, 1),
+                                                  wl.Request(700, 0, 2), wl.Request(129, 448, 8), wl.Request(256, 1024, 4)])
+    dev, stats = check_batch8(ctx, w)
+    o1, l1 = dev.out.clone(), dev.lse.clone()
+    dev.run(ctx)                                                               # run-to-run bitwise determinism
+    assert torch.equal(o1.view(torch.int16), dev.out.view(torch.int16)) and torch.equal(l1, dev.lse)
+
+
+@pytest.mark.parametrize("page", [16, 32, 128])
+def test_fp8_attention_other_page_sizes_and_kv_split(ctx, page):
+    reqs = [wl.Request(333, 200, 3), wl.Request(130, 30000, 2), wl.Request(64, 20000, 1)]
+    check_batch8(ctx, wl.Workload("fp8_page_%d" % page, 54, 8, 2, reqs, page=page), rows_per_request=48)
+
+
+def test_fp8_single_request_entry_and_validation(ctx):
+    w = wl.Workload("fp8_one", 55, 16, 2, [wl.Request(517, 320, 2)])
+    m8 = wl.materialize_fp8(w)
+    dev = Device8(m8)
+    binding.cp_prefill_attn_fp8(ctx, dev.q, dev.cache, dev.page_table, 320, 517, 2, w.Hq, w.scale, dev.out, dev.lse, dev.ws)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ro, rl, ra = o8.attn_fp8_rows(m8.q, m8.k8_pages, m8.v8_pages, m8.k_scale, m8.v_scale, m8.page_table, 320, w.Hkv, w.scale,
+                                  np.arange(517))
+    compare8(bf16_to_f64(dev.out), dev.lse.cpu().numpy().astype(np.float64), ro, rl, ra, "fp8 single")
+    before = dev.out.clone()
+    with pytest.raises(binding.CpError) as e:                                  # odd group size: not supported by this variant
+        binding.cp_prefill_attn_fp8(ctx, dev.q, dev.cache, dev.page_table, 320, 517, 2, 6, w.scale, dev.out, dev.lse, dev.ws)
+    assert e.value.code == binding.CP_ERR_UNSUPPORTED
+    small = torch.zeros(dev.base_ws, dtype=torch.uint8, device="cuda")      # the bf16 path's workspace is too small
+    with pytest.raises(binding.CpError) as e:
+        binding.cp_prefill_attn_fp8(ctx, dev.q, dev.cache, dev.page_table, 320, 517, 2, w.Hq, w.scale, dev.out, dev.lse, small)
+    assert e.value.code == binding.CP_ERR_WORKSPACE
+    torch.cuda.synchronize()
+    assert torch.equal(before.view(torch.int16), dev.out.view(torch.int16))
+
+
+def test_fp8_attention_config2_shape_sampled(ctx):
+    check_batch8(ctx, wl.config2(), rows_per_request=96)
+
+
+def test_fp8_attention_config5_shape_sampled(ctx):
+    check_batch8(ctx, wl.config5(), rows_per_request=24)
