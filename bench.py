@@ -139,28 +139,35 @@ class ClockSampler:
 class Runner:
     """Holds device copies of one workload and runs steps through the C ABI."""
 
-    def __init__(self, w: wl.Workload, device: int, need_host: bool = False):
+    def __init__(self, w: wl.Workload, device: int, need_host: bool = False, fp8: bool = False):
         import torch
         from paper_2609_04774_b200 import binding, build
         build.build()
-        self.torch, self.binding, self.w = torch, binding, w
+        self.torch, self.binding, self.w, self.fp8 = torch, binding, w, fp8
         torch.cuda.set_device(device)
         self.ctx = binding.Context(device)
-        mat = wl.materialize(w)
+        mat = wl.materialize_fp8(w) if fp8 else wl.materialize(w)
         self.mat = mat
 
         def dev(bits):
             return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
 
-        self.q, self.k, self.v = dev(mat.q), dev(mat.k_pages), dev(mat.v_pages)
+        self.q = dev(mat.q)
         self.page_table = torch.from_numpy(mat.page_table).cuda()
-        self.cache = binding.make_cache(self.k, self.v)
+        if fp8:      # E4M3 pages with one fp32 scale per KV head
+            self.k, self.v = torch.from_numpy(mat.k8_pages).cuda(), torch.from_numpy(mat.v8_pages).cuda()
+            self.k_scale, self.v_scale = torch.from_numpy(mat.k_scale).cuda(), torch.from_numpy(mat.v_scale).cuda()
+            self.cache = binding.make_cache_fp8(self.k, self.v, self.k_scale, self.v_scale)
+        else:
+            self.k, self.v = dev(mat.k_pages), dev(mat.v_pages)
+            self.cache = binding.make_cache(self.k, self.v)
         self.out = torch.empty((w.total_new, w.Hq, w.D), dtype=torch.bfloat16, device="cuda")
         self.lse = torch.empty((w.Hq, w.total_new), dtype=torch.float32, device="cuda")
         self.new_len = [r.new_len for r in w.requests]
         self.prefix = np.array([r.prefix_len for r in w.requests], dtype=np.int64)
         self.Cs = np.array([r.C for r in w.requests], dtype=np.int32)
-        self.ws = torch.zeros(binding.cp_workspace_bytes(self.new_len, self.Cs, w.Hq), dtype=torch.uint8, device="cuda")
+        ws_bytes = (binding.cp_workspace_bytes_fp8 if fp8 else binding.cp_workspace_bytes)(self.new_len, self.Cs, w.Hq)
+        self.ws = torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda")
         self.cu_new, self.cu_pages = w.cu_new, w.cu_pages
         if need_host:
             self._host_buffers()
@@ -190,8 +197,9 @@ class Runner:
         b, w = self.binding, self.w
         for r in w.requests:
             b.cp_plan(r.new_len, r.prefix_len, r.C)
-        b.cp_prefill_attn_batch(self.ctx, self.q, self.cache, self.page_table, self.cu_new, self.prefix, self.Cs,
-                                self.cu_pages, w.Hq, w.scale, self.out, self.lse, self.ws)
+        call = b.cp_prefill_attn_fp8_batch if self.fp8 else b.cp_prefill_attn_batch
+        call(self.ctx, self.q, self.cache, self.page_table, self.cu_new, self.prefix, self.Cs, self.cu_pages, w.Hq, w.scale,
+             self.out, self.lse, self.ws)
 
     def _e2e_setup(self):
         """Streams and double-buffered device staging for the end-to-end leg."""
@@ -254,7 +262,7 @@ class Runner:
                                                       self.torch.cuda.get_device_properties(0).multi_processor_count,
                                                       want_lists=False)
         self.schedule = info
-        return info["launches"] + (len(self.w.requests) if e2e else 0)
+        return info["launches"] + (len(self.w.requests) if e2e else 0) + (1 if self.fp8 else 0)   # + the query quantiser
 
     def close(self):
         self.ctx.close()
@@ -342,10 +350,11 @@ def sustained_leg(torch, runner, peaks, device, seconds=2.2):
             "frac": fractions(tf, peaks), "clocks": clocks}
 
 
-def config_leg(torch, cfg, peaks, device, budget_ms=1200.0):
-    """One configuration: 3 warm-up steps, then steps for about `budget_ms` of GPU time (at least 5), clocks sampled."""
+def config_leg(torch, cfg, peaks, device, budget_ms=1200.0, fp8=False):
+    """One configuration: 3 warm-up steps, then steps for about `budget_ms` of GPU time (at least 5), clocks sampled.
+    fp8: the same lengths and heads with E4M3 K/V pages (queries quantised per step by the library's pre-pass)."""
     w = get_workload(cfg)
-    runner = Runner(w, device)
+    runner = Runner(w, device, fp8=fp8)
     sampler = ClockSampler(device)
     sampler.start()
     for _ in range(3):
@@ -366,6 +375,13 @@ def config_leg(torch, cfg, peaks, device, budget_ms=1200.0):
              "tokens_per_s": w.total_new / (ms * 1e-3), "frac": fractions(tf, peaks), "pairs": pairs_of(w),
              "launches_per_step": runner.launches_per_step(), "gpu_seconds": total_ms * 1e-3, "clocks": clocks,
              "traffic": ATTN_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": algorithmic_bytes(w)}
+    if fp8:
+        # tensor roofline of one-byte operands: the measured bf16 rates times the nominal fp8 / bf16 ratio of 2
+        entry.update(dtype="fp8_e4m3 K/V and P, bf16 q/out", traffic=None,
+                     algorithmic_bytes=2 * w.total_new * w.Hq * w.D * 2 + 2 * sum(r.total_len for r in w.requests) * w.Hkv * w.D + 4 * w.Hq * w.total_new,
+                     frac={"of_nominal_4500": tf / (2 * NOMINAL_BF16_TFLOPS), "of_2x_measured_bf16_burst": tf / (2 * peaks["bf16_tflops"]),
+                           "of_2x_measured_bf16_sustained": tf / (2 * peaks["bf16_tflops_sustained"]),
+                           "of_nominal_bf16_2250": tf / NOMINAL_BF16_TFLOPS})
     runner.close()
     del runner
     torch.cuda.empty_cache()
@@ -648,6 +664,7 @@ def run_ours(args):
         del runner
         torch.cuda.empty_cache()
         line["configs"] = [config_leg(torch, c, peaks, local) for c in (1, 2, 3, 4, 5)]
+        line["configs_fp8"] = [config_leg(torch, c, peaks, local, fp8=True) for c in (2, 5)]
         bf, f32 = torch.bfloat16, torch.float32
         line["merge"] = merge_points(torch, peaks, [(T, N, bf) for T in (4096, 16384, 65536) for N in (2, 4, 8)] +
                                      [(16384, N, f32) for N in (2, 4, 8)])
@@ -676,7 +693,7 @@ def run_configs(args, out):
     import torch
     peaks = load_peaks()
     for cfg in args.configs:
-        out.write(json.dumps(dict(mode="config", **config_leg(torch, cfg, peaks, 0, budget_ms=args.config_ms))) + "\n")
+        out.write(json.dumps(dict(mode="config", **config_leg(torch, cfg, peaks, 0, budget_ms=args.config_ms, fp8=args.fp8))) + "\n")
         out.flush()
 
 
@@ -784,6 +801,10 @@ class _LoopbackComm:
     def all_gather(self, block):
         return block.unsqueeze(0).expand((self.size,) + tuple(block.shape)).contiguous(), self._Done()
 
+    def all_gather_into(self, out, block):
+        out.view((self.size,) + tuple(block.shape)).copy_(block.unsqueeze(0).expand((self.size,) + tuple(block.shape)))
+        return self._Done()
+
     def all_to_all(self, blocks):
         return blocks.clone(), self._Done()
 
@@ -809,7 +830,7 @@ def run_cprank(args, out):
         v = torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
         pt = torch.from_numpy(wl.permutation(w.seed, wl.TID_PERM, n_pages)).cuda()
         ops = LibraryOps(binding.Context(0), k, v, pt, w.Hq, w.scale)
-        per_rank = []
+        per_rank, per_rank_graph = [], []
         for rank in range(C):
             lay = RankLayout(R, P, C, rank)
             rows = {}
@@ -832,6 +853,34 @@ def run_cprank(args, out):
                     ms.append(e0.elapsed_time(e1))
             ops.ctx.poll_status()
             per_rank.append(statistics.median(ms))
+            # the same step replayed from a CUDA graph (one launch per layer instead of ~20 calls from Python): only when
+            # both chunk calls carry their work lists in the launch parameters, so that a replay reads no host staging
+            g_ms = None
+            small = all(binding.cp_schedule_inspect([0, e - b], [P + b], [1], w.Hq, w.Hkv, want_lists=False)[0]["inline"]
+                        for b, e in (lay.chunk(lay.early), lay.chunk(lay.late)) if e > b)
+            if small and not args.pass_q:
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    fn()
+                torch.cuda.current_stream().wait_stream(side)
+                torch.cuda.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph):
+                    fn()
+                ts = []
+                for i in range(2 + args.rank_reps):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    graph.replay()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if i >= 2:
+                        ts.append(e0.elapsed_time(e1))
+                ops.ctx.poll_status()
+                g_ms = statistics.median(ts)
+                del graph
+            per_rank_graph.append(g_ms)
         lay0 = RankLayout(R, P, C, 0)
         if args.pass_q:   # queries in (bf16), partials of the own rows back (fp32 + lse)
             recv = (C - 1) * 2 * lay0.cl * w.Hq * (D * 2 + D * 4 + 4)
@@ -839,6 +888,7 @@ def run_cprank(args, out):
             recv = (C - 1) * 2 * 2 * w.Hkv * D * (lay0.block_pages * wl.PAGE + 2 * lay0.cl)
         out.write(json.dumps({"mode": "cprank", "exchange": "pass-q" if args.pass_q else "all-gather-kv", "config": cfg, "workload": w.name, "R": R, "P": P, "C": C,
                               "rank_local_ms": per_rank, "slowest_rank_ms": max(per_rank),
+                              "rank_local_ms_graph_replay": per_rank_graph,
                               "tflops_per_gpu_slowest_rank": flops_of(w) / C / (max(per_rank) * 1e-3) / 1e12,
                               "nvlink_bytes_received_per_rank": recv,
                               "nvlink_ms_modelled_at_770GBps": recv / 770e9 * 1e3,
@@ -912,6 +962,7 @@ def main():
     ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5],
                     help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P")
     ap.add_argument("--config-ms", type=float, default=1200.0, help="configs mode: GPU time per configuration")
+    ap.add_argument("--fp8", action="store_true", help="configs mode: the FP8 K/V variant of each configuration")
     ap.add_argument("--rank-reps", type=int, default=5)
     ap.add_argument("--pass-q", action="store_true", help="cprank mode: K/V stays sharded, queries travel")
     ap.add_argument("--cache-requests", type=int, default=20000)

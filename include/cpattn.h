@@ -279,6 +279,20 @@ int cp_kv_gather(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_tabl
 int cp_kv_append(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin,
                  int64_t n, const void* k_rows, const void* v_rows, void* stream);
 
+/* cp_kv_append_segments -- cp_kv_append for several runs of rows in ONE launch: segment i writes rows
+ * [row0, row0 + n) of k_rows / v_rows (device [*, Hkv, D] bf16) to logical tokens [t_begin, t_begin + n).  What a
+ * CP rank needs after an all-gather of K and V (Section 2.1): the gathered blocks of the C ranks land at C
+ * different token ranges of the rank's cache.  segments: host array; at most 64 segments per call; empty
+ * segments are skipped.  Segments must not overlap in the cache.  Page ids are checked as in cp_kv_append.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+typedef struct {
+    int64_t t_begin; /* first logical token written */
+    int64_t n;       /* tokens */
+    int64_t row0;    /* first row read from k_rows / v_rows */
+} cp_kv_segment;
+int cp_kv_append_segments(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int32_t n_segments,
+                          const cp_kv_segment* segments, const void* k_rows, const void* v_rows, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * FP8 K/V variant.  The paper's main model is an FP8 model (Section 9.1) but the paper states no FP8
  * attention recipe; the format below is this library's reading.

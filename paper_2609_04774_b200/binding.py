@@ -22,7 +22,7 @@ CP_DTYPE_BF16, CP_DTYPE_F32 = 0, 1
 EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "cp_ctx_poll_status", "cp_ctx_cache_schedule", "cp_ctx_selftest_wait_expiry", "cp_plan",
            "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_chunk", "cp_prefill_attn_kvrange", "cp_prefill_attn_static", "cp_merge",
            "cp_kv_gather", "cp_kv_append", "cp_workspace_bytes_fp8", "cp_prefill_attn_fp8", "cp_prefill_attn_fp8_batch",
-           "cp_kv_append_fp8"]
+           "cp_kv_append_fp8", "cp_kv_append_segments"]
 
 
 class CpError(RuntimeError):
@@ -260,6 +260,13 @@ def cp_kv_gather(ctx, cache, page_table, t_begin, n, k_rows, v_rows, stream=None
 def cp_kv_append(ctx, cache, page_table, t_begin, n, k_rows, v_rows, stream=None):
     _check(load().cp_kv_append(ctx._h, ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(t_begin),
                                ctypes.c_int64(n), _ptr(k_rows), _ptr(v_rows), _stream(stream)))
+
+
+def cp_kv_append_segments(ctx, cache, page_table, segments, k_rows, v_rows, stream=None):
+    """segments: iterable of (t_begin, n, row0); rows [row0, row0+n) of k_rows / v_rows go to tokens [t_begin, t_begin+n)."""
+    seg = np.ascontiguousarray(np.asarray(list(segments), dtype=np.int64).reshape(-1, 3))
+    _check(load().cp_kv_append_segments(ctx._h, ctypes.byref(cache), _ptr(page_table), ctypes.c_int32(seg.shape[0]),
+                                        _hp(seg), _ptr(k_rows), _ptr(v_rows), _stream(stream)))
 
 
 # ------------------------------------------------------------------------------------------------

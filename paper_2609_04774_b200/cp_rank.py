@@ -5,12 +5,15 @@ Q/K/V for them, all-gathers K and V, attends its local queries to every causally
 outputs go back to their original order.  Section 2.2: on a prefix hit the cached KV is partitioned
 across the worker's ranks, so it is gathered as well (the b*P term of Eq. 2).
 
-What runs where.  The exchange is three all-gathers (prefix blocks, early chunks, late chunks) issued
-back to back on the communicator; the attention over the early chunk needs only the first two, so it
-runs while the third is still in flight (early chunk first).  Gathered rows land in contiguous staging
-buffers and are written into this rank's own paged cache by cp_kv_append; attention reads that cache
-through cp_prefill_attn_chunk.  Remote data is therefore always copied into local HBM before a kernel
-reads it.  The module holds no arithmetic of the method: it moves rows and calls the library.
+What runs where.  The exchange is three all-gathers of K and of V (prefix blocks, early chunks, late
+chunks) issued back to back on the communicator; the attention over the early chunk needs only the first
+two, so it runs while the third is still in flight (early chunk first).  Every gather writes straight into
+its part of one pre-allocated arena per tensor (prefix blocks | early chunks | late chunks); two
+cp_kv_append_segments launches move the arena's rows into this rank's own paged cache (prefix blocks and early
+chunks together, then the late chunks), and attention reads that cache through cp_prefill_attn_chunk.  A rank
+step is five library launches (own prefix block read out, two appends, two attention calls) plus the merge of
+KV-split units where the schedule cuts any.  Remote data is always copied into local HBM before a kernel reads
+it.  The module holds no arithmetic of the method: it moves rows and calls the library.
 
 A second mode, prefill_pass_q, keeps the K/V sharded (a rank holds its prefix block and the K/V of its own
 two chunks) and lets the queries travel: all-gather of Q, cp_prefill_attn_kvrange over each of the rank's key
@@ -108,6 +111,14 @@ class TorchComm:
         return out, work
 
 
+    def all_gather_into(self, out, block):
+        """Gathers block [n, ...] of every rank into out [size * n, ...] (a contiguous view, e.g. a slice of an
+        arena); returns a handle."""
+        import torch
+        src = block.contiguous().view(torch.uint8).reshape(-1)
+        dst = out.view(torch.uint8).reshape(-1)
+        return self.dist.all_gather_into_tensor(dst, src, group=self.group, async_op=True)
+
     def all_to_all(self, blocks):
         """blocks [size, n, ...]: block d goes to rank d.  -> (out [size, n, ...] with out[s] = the block rank s
         sent here, handle)."""
@@ -141,9 +152,23 @@ class LibraryOps:
         self.Hkv, self.D = k_pages.shape[2], k_pages.shape[3]
         self.device = k_pages.device
         self._ws = None
+        self._buffers = {}
 
     def empty_rows(self, n, heads):
         return self.torch.zeros((n, heads, self.D), dtype=self.torch.bfloat16, device=self.device)
+
+    def buffer(self, name, shape, dtype=None):
+        """A device buffer that lives as long as this object (allocated and zeroed on first use): the staging
+        arenas, send buffers and outputs of a rank step are reused from layer to layer."""
+        key = (name, tuple(shape), dtype)
+        if key not in self._buffers:
+            self._buffers[key] = self.torch.zeros(tuple(shape), dtype=dtype or self.torch.bfloat16, device=self.device)
+        return self._buffers[key]
+
+    def kv_append_segments(self, segments, k_rows, v_rows):
+        segments = [s for s in segments if s[1] > 0]
+        if segments:
+            self.b.cp_kv_append_segments(self.ctx, self.cache, self.page_table, segments, k_rows, v_rows)
 
     def kv_gather(self, t_begin, n, k_rows, v_rows):
         if n > 0:
@@ -155,8 +180,8 @@ class LibraryOps:
 
     def attn_chunk(self, lay: RankLayout, chunk, q_chunk):
         n = q_chunk.shape[0]
-        out = self.torch.empty((n, self.Hq, self.D), dtype=self.torch.bfloat16, device=self.device)
-        lse = self.torch.empty((self.Hq, n), dtype=self.torch.float32, device=self.device)
+        out = self.buffer("out_%d" % chunk, (n, self.Hq, self.D))
+        lse = self.buffer("lse_%d" % chunk, (self.Hq, n), self.torch.float32)
         if n == 0:
             return out, lse
         if self._ws is None:
@@ -201,11 +226,12 @@ def _library_extras():
 _library_extras()
 
 
-def _padded(ops, rows, n):
-    """rows [m, H, D] -> [n, H, D] with zero rows behind (collectives need equal sizes)."""
+def _padded(ops, rows, n, name=None):
+    """rows [m, H, D] -> [n, H, D] with zero rows behind (collectives need equal sizes).  A full chunk is sent as
+    it is; a short one goes through a send buffer (a persistent one when the ops object keeps buffers)."""
     if rows.shape[0] == n:
         return rows
-    buf = ops.empty_rows(n, rows.shape[1])
+    buf = ops.buffer(name, (n,) + tuple(rows.shape[1:])) if name and hasattr(ops, "buffer") else ops.empty_rows(n, rows.shape[1])
     buf[:rows.shape[0]] = rows
     return buf
 
@@ -230,41 +256,52 @@ class CpRankWorker:
         (eb, ee), (lb, le) = lay.chunk(lay.early), lay.chunk(lay.late)
         assert q_early.shape[0] == ee - eb == k_early.shape[0] and q_late.shape[0] == le - lb == k_late.shape[0]
 
-        # 1. contributions: own prefix block read out of the cache, own chunks padded to cl rows
-        pb, pe = lay.prefix_block(lay.rank)
+        C, cl = lay.C, lay.cl
         n_blk = lay.block_pages * lay.page
-        gathers = []
+        # one arena per tensor: gathered prefix blocks | gathered early chunks | gathered late chunks (rows)
+        off_e, off_l = C * n_blk, C * (n_blk + cl)
+        ak = ops.buffer("arena_k", (C * (n_blk + 2 * cl), ops.Hkv, ops.D))
+        av = ops.buffer("arena_v", (C * (n_blk + 2 * cl), ops.Hkv, ops.D))
+
+        # 1. contributions: own prefix block read out of the cache, own chunks (padded to cl rows when short);
+        #    every gather lands in its part of the arena
+        pb, pe = lay.prefix_block(lay.rank)
+        hp = None
         if n_blk:
-            sk, sv = ops.empty_rows(n_blk, ops.Hkv), ops.empty_rows(n_blk, ops.Hkv)
+            sk, sv = ops.buffer("send_prefix_k", (n_blk, ops.Hkv, ops.D)), ops.buffer("send_prefix_v", (n_blk, ops.Hkv, ops.D))
             ops.kv_gather(pb, pe - pb, sk, sv)
-            gathers.append((comm.all_gather(sk), comm.all_gather(sv)))
-        else:
-            gathers.append(None)
-        gathers.append((comm.all_gather(_padded(ops, k_early, lay.cl)), comm.all_gather(_padded(ops, v_early, lay.cl))))
-        gathers.append((comm.all_gather(_padded(ops, k_late, lay.cl)), comm.all_gather(_padded(ops, v_late, lay.cl))))
+            hp = (comm.all_gather_into(ak[:off_e], sk), comm.all_gather_into(av[:off_e], sv))
+        he = (comm.all_gather_into(ak[off_e:off_l], _padded(ops, k_early, cl, "send_early_k")),
+              comm.all_gather_into(av[off_e:off_l], _padded(ops, v_early, cl, "send_early_v")))
+        hl = (comm.all_gather_into(ak[off_l:], _padded(ops, k_late, cl, "send_late_k")),
+              comm.all_gather_into(av[off_l:], _padded(ops, v_late, cl, "send_late_v")))
 
-        def wait(g):
-            (k, hk), (v, hv) = g
-            hk.wait()
-            hv.wait()
-            return k, v
-
-        # 2. prefix blocks and early chunks: rank order is token order, one append each
-        if gathers[0] is not None:
-            gk, gv = wait(gathers[0])
-            ops.kv_append(0, lay.P, gk.reshape((-1,) + tuple(gk.shape[2:])), gv.reshape((-1,) + tuple(gv.shape[2:])))
-        gk, gv = wait(gathers[1])
-        n_first = min(lay.R, lay.C * lay.cl)
-        ops.kv_append(lay.P, n_first, gk.reshape((-1,) + tuple(gk.shape[2:])), gv.reshape((-1,) + tuple(gv.shape[2:])))
+        # 2. prefix blocks and early chunks into the own cache, one launch: block r and chunk r came from rank r
+        segs = []
+        if hp is not None:
+            hp[0].wait()
+            hp[1].wait()
+            for r in range(C):
+                b, e = lay.prefix_block(r)
+                segs.append((b, e - b, r * n_blk))
+        he[0].wait()
+        he[1].wait()
+        for r in range(C):
+            b, e = lay.chunk(r)
+            segs.append((lay.P + b, e - b, off_e + r * cl))
+        ops.kv_append_segments(segs, ak, av)
 
         # 3. early chunk: its keys are all here; the late all-gather is still in flight
         out_e, lse_e = ops.attn_chunk(lay, lay.early, q_early)
 
-        # 4. late chunks: rank r sent chunk 2C-1-r
-        gk, gv = wait(gathers[2])
-        for r in range(lay.C):
+        # 4. late chunks (rank r sent chunk 2C-1-r), one launch, then the late chunk's attention
+        hl[0].wait()
+        hl[1].wait()
+        segs = []
+        for r in range(C):
             b, e = lay.chunk(lay.late_chunk_of(r))
-            ops.kv_append(lay.P + b, e - b, gk[r], gv[r])
+            segs.append((lay.P + b, e - b, off_l + r * cl))
+        ops.kv_append_segments(segs, ak, av)
         out_l, lse_l = ops.attn_chunk(lay, lay.late, q_late)
         return out_e, lse_e, out_l, lse_l
 

@@ -77,7 +77,7 @@ constexpr int kStageBuffers = 4;
 constexpr size_t kStatusBytes = kStatusWords * sizeof(int32_t);
 // A schedule whose work lists fit in this many bytes travels inside the kernel's launch parameters instead of
 // being copied into the workspace first (one launch less for small problems).
-constexpr size_t kInlineSchedBytes = 3072;
+constexpr size_t kInlineSchedBytes = 24576;
 struct InlineSched {
     alignas(16) unsigned char bytes[kInlineSchedBytes];
 };

@@ -61,6 +61,49 @@ int validate_cache(const cp_kv_cache* c, const char* who) {
     return CP_OK;
 }
 
+// Several runs of rows in one launch: segment i writes rows [row0, row0 + n) of the row buffers to logical tokens
+// [t_begin, t_begin + n).  The segment table travels in the launch parameters.
+constexpr int kMaxSegments = 64;
+struct SegmentTable {
+    int32_t n_segments;
+    int64_t t_begin[kMaxSegments];
+    int64_t row0[kMaxSegments];
+    int64_t cum[kMaxSegments + 1];     // prefix sums of the segment lengths
+};
+
+__global__ void __launch_bounds__(256)
+kv_append_segments_kernel(uint4* __restrict__ paged_k, uint4* __restrict__ paged_v, const uint4* __restrict__ rows_k,
+                          const uint4* __restrict__ rows_v, const int32_t* __restrict__ page_table,
+                          const __grid_constant__ SegmentTable seg, int page_size, int Hkv, int vec_per_head,
+                          int64_t stride_page8, int64_t stride_tok8, int64_t stride_head8, int64_t num_pages,
+                          int32_t* status) {
+    const int vec_per_tok = Hkv * vec_per_head;
+    const int64_t total = seg.cum[seg.n_segments] * vec_per_tok;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t tok = i / vec_per_tok;
+        const int rem = (int)(i - tok * vec_per_tok);
+        int sg = 0;
+        while (tok >= seg.cum[sg + 1]) ++sg;                       // few segments: a linear walk
+        const int64_t k = tok - seg.cum[sg];
+        const int64_t t = seg.t_begin[sg] + k;
+        const int64_t src = (seg.row0[sg] + k) * vec_per_tok + rem;
+        const int g = rem / vec_per_head;
+        const int c = rem - g * vec_per_head;
+        const int64_t page = page_table[t / page_size];
+        if (page < 0 || page >= num_pages) {
+            if (atomicCAS(status, 0, CP_ERR_BOUNDS) == 0) {
+                status[1] = (int32_t)(t / page_size);
+                status[2] = (int32_t)blockIdx.x;
+                status[3] = (int32_t)page;
+            }
+            continue;
+        }
+        const int64_t off = page * stride_page8 + (t % page_size) * stride_tok8 + (int64_t)g * stride_head8 + c;
+        if (rows_k) paged_k[off] = rows_k[src];
+        if (rows_v) paged_v[off] = rows_v[src];
+    }
+}
+
 // FP8 cache writer: eight bf16 values of a row -> eight E4M3 bytes, each e4m3_rne_satfinite(x / scale[g]) with
 // the quotient rounded to fp32 first.  Page ids outside the pool are skipped and reported like in the copies.
 __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d, float sc) {
@@ -147,6 +190,42 @@ int kv_copy(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, in
 namespace cpattn {
 int validate_kv_cache(const cp_kv_cache* c, const char* who) { return validate_cache(c, who); }
 int validate_kv_cache_fp8(const cp_kv_cache_fp8* c, const char* who) { return validate_cache_fp8(c, who); }
+}
+
+extern "C" int cp_kv_append_segments(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int32_t n_segments,
+                                     const cp_kv_segment* segments, const void* k_rows, const void* v_rows, void* stream) {
+    const char* who = "cp_kv_append_segments";
+    if (!ctx || !page_table || !segments || n_segments < 0)
+        return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or negative segment count", who);
+    if (n_segments > kMaxSegments)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: %d segments, at most %d per call", who, n_segments, kMaxSegments);
+    if (int rc = validate_cache(cache, who)) return rc;
+    if (!k_rows && !v_rows) return set_error(CP_ERR_INVALID_ARG, "%s: both row pointers are NULL", who);
+    if (((uintptr_t)k_rows | (uintptr_t)v_rows) & 15)
+        return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
+    SegmentTable tab;
+    tab.n_segments = 0;
+    tab.cum[0] = 0;
+    for (int32_t i = 0; i < n_segments; ++i) {
+        const cp_kv_segment& sg = segments[i];
+        if (sg.t_begin < 0 || sg.n < 0 || sg.row0 < 0)
+            return set_error(CP_ERR_INVALID_ARG, "%s: segment %d has a negative field", who, i);
+        if (sg.n == 0) continue;
+        const int k = tab.n_segments++;
+        tab.t_begin[k] = sg.t_begin;
+        tab.row0[k] = sg.row0;
+        tab.cum[k + 1] = tab.cum[k] + sg.n;
+    }
+    if (tab.n_segments == 0) return CP_OK;
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+    const int vec_per_head = cache->D / 8;
+    const int64_t total = tab.cum[tab.n_segments] * cache->Hkv * vec_per_head;
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
+    kv_append_segments_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        (uint4*)cache->k, (uint4*)cache->v, (const uint4*)k_rows, (const uint4*)v_rows, page_table, tab, cache->page_size,
+        cache->Hkv, vec_per_head, cache->stride_page / 8, cache->stride_tok / 8, cache->stride_head / 8, cache->num_pages,
+        ctx->d_status);
+    return check_cuda(cudaGetLastError(), who);
 }
 
 extern "C" int cp_kv_append_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,

@@ -37,6 +37,11 @@ class ThreadComm:
         gathered, done = self.all_gather(blocks)
         return gathered[:, self.rank].contiguous(), done
 
+    def all_gather_into(self, out, block):
+        gathered, done = self.all_gather(block)
+        out.copy_(gathered.reshape(out.shape))
+        return done
+
     def all_gather(self, block):
         f, n = self.fabric, self.calls
         self.calls += 1
@@ -58,6 +63,17 @@ class OracleOps:
 
     def empty_rows(self, n, heads):
         return torch.zeros((n, heads, self.D), dtype=torch.int16)
+
+    def buffer(self, name, shape, dtype=None):
+        self._buffers = getattr(self, "_buffers", {})
+        key = (name, tuple(shape))
+        if key not in self._buffers:
+            self._buffers[key] = torch.zeros(tuple(shape), dtype=torch.int16)
+        return self._buffers[key]
+
+    def kv_append_segments(self, segments, k_rows, v_rows):
+        for t_begin, n, row0 in segments:
+            self.kv_append(t_begin, n, k_rows[row0:row0 + n], v_rows[row0:row0 + n])
 
     @staticmethod
     def _bits(t):

@@ -126,6 +126,30 @@ def test_kv_gather_append_bit_exact(ctx):
     assert np.array_equal(v.view(torch.int16).cpu().numpy().view(np.uint16), vp)
 
 
+def test_kv_append_segments_bit_exact(ctx):
+    # several runs of rows in one launch, in scrambled order, with an empty segment and gaps left untouched
+    w = wl.Workload("segments", 48, 8, 2, [wl.Request(900, 448, 1)])
+    mat = wl.materialize(w)
+    k, v = bits_to_bf16(mat.k_pages), bits_to_bf16(mat.v_pages)
+    cache = binding.make_cache(k, v)
+    pt = torch.from_numpy(mat.page_table).cuda()
+    rows_k = wl.normal_bf16(49, wl.TID_K, (700, w.Hkv, w.D))
+    rows_v = wl.normal_bf16(49, wl.TID_V, (700, w.Hkv, w.D))
+    segs = [(1000, 130, 0), (5, 59, 500), (64, 0, 3), (448, 333, 150), (200, 1, 699)]
+    binding.cp_kv_append_segments(ctx, cache, pt, segs, bits_to_bf16(rows_k), bits_to_bf16(rows_v))
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    kp, vp = mat.k_pages.copy(), mat.v_pages.copy()
+    for t0, n, r0 in segs:
+        orc.kv_append(kp, mat.page_table, t0, rows_k[r0:r0 + n])
+        orc.kv_append(vp, mat.page_table, t0, rows_v[r0:r0 + n])
+    assert np.array_equal(k.view(torch.int16).cpu().numpy().view(np.uint16), kp)
+    assert np.array_equal(v.view(torch.int16).cpu().numpy().view(np.uint16), vp)
+    with pytest.raises(binding.CpError) as e:
+        binding.cp_kv_append_segments(ctx, cache, pt, [(0, 1, 0)] * 65, bits_to_bf16(rows_k), bits_to_bf16(rows_v))
+    assert e.value.code == binding.CP_ERR_UNSUPPORTED
+
+
 def test_attention_small_mixed_batch(ctx):
     dev, out, lse, _ = check_batch(ctx, wl.small_mixed())
     # run-to-run bitwise determinism
