@@ -960,7 +960,7 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="number of the configuration used as the headline workload")
     ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table", "kvcopy", "cprank", "cachemgr"])
     ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5],
-                    help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P")
+                    help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P; 8: multi-head (16/16)")
     ap.add_argument("--config-ms", type=float, default=1200.0, help="configs mode: GPU time per configuration")
     ap.add_argument("--fp8", action="store_true", help="configs mode: the FP8 K/V variant of each configuration")
     ap.add_argument("--rank-reps", type=int, default=5)

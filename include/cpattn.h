@@ -127,8 +127,8 @@ size_t cp_workspace_bytes(int32_t B, const int64_t* new_len, const int32_t* C, i
 /* cp_schedule_inspect -- host only: the work distribution the attention calls would use for a batch
  * on a device with num_sms SMs (the varlen tile schedule: query tiles of 128 rows, the last tile of a
  * request possibly shorter -- a launch over all shards walks a request's rows as one run, so a tile may span
- * adjacent zigzag chunks but never two requests; one unit per tile and pair of query heads (per
- * single head when Hq / Hkv is odd); whole
+ * adjacent zigzag chunks but never two requests; one unit per tile and pair of query heads, or, when
+ * Hq / Hkv is odd, per pair of consecutive tiles (256 rows) and single head; whole
  * units longest first -- KV head by KV head when the batch's K/V exceeds 32 MB, so that a long context's K/V
  * stays in L2 -- dealt to the CTAs in serpentine order, the remainder cut along KV so that every
  * CTA gets the same number of KV tile steps; when there are no more units than CTAs and all are short, every
@@ -156,11 +156,11 @@ int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_
  * The C shards of cp_plan(R, P, C) are row-disjoint and together cover all R rows (Section 2.1), and
  * adjacent chunks are adjacent rows with consecutive causal limits, so the launch walks the rows as one
  * run of 128-row query tiles with a per-row limit; C is validated, and the result does not depend on it
- * (the calls that compute ONE shard or ONE chunk cut their tiles at the chunk's boundaries).  Requires Hq % Hkv == 0 (query head h uses KV head h / (Hq / Hkv)); with an even group
- * size two query heads of a group share every K/V tile in shared memory, with an odd one (e.g.
- * Hq == Hkv) every head streams K/V on its own: its KV tiles then alternate between the two softmax warpgroups (two
- * online-softmax streams combined at the end), at about 80 % of the throughput (1090 against 1355 TFLOP/s on
- * config 2's lengths).  One persistent launch computes all tiles; the few units that were split along KV
+ * (the calls that compute ONE shard or ONE chunk cut their tiles at the chunk's boundaries).  Requires
+ * Hq % Hkv == 0 (query head h uses KV head h / (Hq / Hkv)).  With an even group size a work unit is one
+ * 128-row query tile for two query heads of a group, which share every K/V tile in shared memory; with an
+ * odd one (e.g. Hq == Hkv) a unit is one head and two consecutive query tiles, which share the K/V tiles
+ * the same way (measured on config 2's lengths: 1137 TFLOP/s with 16/16 heads against 1211 with 32/8).  One persistent launch computes all tiles; the few units that were split along KV
  * to balance the SMs are combined by a second small launch (an LSE merge of their partials).  Work lists of
  * up to 3 KB travel in the launch parameters; larger ones are first copied into the workspace by a small
  * kernel.  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
@@ -308,7 +308,7 @@ int cp_kv_append_segments(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* 
  *     rounded to E4M3 (after a scaling by 16) for P V, the row sum and the LSE use the unrounded weights.
  *     LSE is as accurate as in the bf16 path; each output element is within 2^-4 * sum_j p_j |v_j| of the
  *     exact result on the stored bytes (the rounding of the weights), typically 2-3 % of the row's norm.
- *   - Requires an even number of query heads per KV head.  out: bf16 [R, Hq, D]; lse: fp32 [Hq, R].
+ *   - out: bf16 [R, Hq, D]; lse: fp32 [Hq, R].
  * cp_workspace_bytes_fp8: the workspace of cp_workspace_bytes plus room for the quantised queries.
  * cp_kv_append_fp8: writes n logical tokens starting at t_begin from bf16 rows [n, Hkv, D] into the FP8
  * cache, each element as e4m3(x / scale[g]) (IEEE fp32 division, round to nearest even, saturating); page

@@ -2,12 +2,13 @@
 // TMA-staged Q/K/V tiles (K/V fetched page by page through the page table), online softmax.
 //
 // One persistent CTA per SM walks a list of work units.  A unit is one query tile (<= 128 new
-// tokens of one zigzag chunk) for TWO query heads of the same KV group, so each K/V tile that
-// lands in shared memory feeds two 128x128 score tiles (GQA head sharing).  With an odd group size a unit
-// is ONE query head, and the two softmax warpgroups take its even and odd KV tiles as two online-softmax
-// streams that are combined in the epilogue (kernel instantiation kDual).  Warp roles:
-//   warps 0-3  softmax warpgroup for head 0 of the pair: one thread per query row
-//   warps 4-7  softmax warpgroup for head 1
+// tokens) for TWO query heads of the same KV group, so each K/V tile that lands in shared memory
+// feeds two 128x128 score tiles (GQA head sharing).  With an odd group size (plain multi-head
+// attention, for instance) a unit is ONE query head and TWO consecutive query tiles (<= 256 new tokens):
+// the two tiles share every K/V tile the same way, the later one seeing one more KV tile at the end,
+// which is fully masked for the earlier one ("tile-pair" units).  Warp roles:
+//   warps 0-3  softmax warpgroup for head 0 of the pair (tile-pair units: rows 0-127): one thread per query row
+//   warps 4-7  softmax warpgroup for head 1 (tile-pair units: rows 128-255)
 //   warp  8    TMA producer (the warp prefetches page ids; the pages of a tile go out from several lanes)
 //   warp  9    tcgen05.mma issuer for the scores S = Q K^T (warp-uniform loop, one elected lane issues)
 //   warp  10   tcgen05.mma issuer for O += P V
@@ -55,8 +56,7 @@ static_assert(2 * 128 * kRegsSoftmax + 128 * kRegsOther <= 65536 - 1024, "leave 
 constexpr uint32_t kSmemQ = 0;                                  // 2 heads x 32 KB
 constexpr uint32_t kSmemKV = 2 * kTileBytes;                    // kKvStages x 32 KB
 constexpr uint32_t kSmemBar = kSmemKV + kKvStages * kTileBytes; // mbarriers
-constexpr uint32_t kSmemXchg = kSmemBar + 256;                   // 128 x (m, l) floats: second stream of a single-head unit
-constexpr uint32_t kSmemBytes = kSmemXchg + 1024;
+constexpr uint32_t kSmemBytes = kSmemBar + 256;
 constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;              // slack for manual alignment
 
 // barrier indices (8 bytes each, from kSmemBar); also the ids reported on a timeout
@@ -105,7 +105,8 @@ struct AttnParams {
     float* partial_lse;        // [slots][2 heads][128 rows]
     int32_t pairs_per_tile;   // units per query tile: Hq / heads_per_unit
     int32_t pairs_per_kv;     // implicit schedule: > 0 walks the units KV head by KV head (this many units per tile and KV head)
-    int32_t heads_per_unit;   // 2: two query heads of one KV group share every K/V tile; 1: odd group size
+    int32_t heads_per_unit;   // 2: two query heads of one KV group share every K/V tile; 1: odd group size, the unit
+                              // is one head and two consecutive 128-row query tiles (tile-pair unit)
     int32_t group;            // Hq / Hkv
     int32_t Hq;
     const int32_t* page_table;
@@ -425,14 +426,16 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
         if (lane == 0) {
             mbar_wait(bars, kBarQEmpty, (round & 1) ^ 1, abort_flag, p.status, round);
             const uint32_t qbar = bars + kBarQFull * 8;
-            mbar_expect_tx(qbar, p.heads_per_unit * (kFp8 ? kTileBytes8 : kTileBytes));
-            for (int h = 0; h < p.heads_per_unit; ++h) {
+            mbar_expect_tx(qbar, 2 * (kFp8 ? kTileBytes8 : kTileBytes));
+            for (int h = 0; h < 2; ++h) {
+                // second Q tile: the next head of the pair, or (tile-pair unit) the next 128 rows of the same head
+                const int head = u.head0 + (p.heads_per_unit == 2 ? h : 0);
+                const int row0 = u.it.q_row0 + (p.heads_per_unit == 2 ? 0 : h * kBlockM);
                 if (kFp8) {      // one-byte queries: a row is one 128-byte swizzle line
-                    tma_load_3d(smem_base + kSmemQ + h * kTileBytes, tmQ, qbar, 0, u.head0 + h, u.it.q_row0);
+                    tma_load_3d(smem_base + kSmemQ + h * kTileBytes, tmQ, qbar, 0, head, row0);
                 } else {
                     for (int half = 0; half < 2; ++half)
-                        tma_load_3d(smem_base + kSmemQ + h * kTileBytes + half * kHalfBytes, tmQ, qbar, half * 64,
-                                    u.head0 + h, u.it.q_row0);
+                        tma_load_3d(smem_base + kSmemQ + h * kTileBytes + half * kHalfBytes, tmQ, qbar, half * 64, head, row0);
                 }
             }
         }
@@ -502,11 +505,11 @@ struct RingPos {
 // (S buffer) and P*V (P and O columns) touch disjoint TMEM and the K and V tiles have their own barriers.
 //
 // Score issuer: S tiles in the order (tile, head); each needs its K tile and the buffer back (s_free).
-template <bool kDual, bool kFp8>
+template <bool kFp8>
 __device__ __forceinline__ void mma_s_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
                                            volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
-    constexpr int H = kDual ? 1 : 2;
+    constexpr int H = 2;
     RingPos unit_pos = {0, 0};         // ring position of the unit's first load, K(j0)
     uint32_t s_par = 1;                // parity of "previous score tile was read"; 1: no tile yet (passes)
     const uint64_t q_desc0 = make_desc(smem_base + kSmemQ, 16, 1024);
@@ -521,8 +524,7 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, const InlineSche
         for (int j = j0; j < n; ++j) {
             mbar_wait(bars, kBarKvFull + kpos.slot, kpos.par, abort_flag, p.status, j);
             for (int h = 0; h < H; ++h) {
-                // single-head unit: one Q tile, and the tiles go to the two softmax warpgroups in turn
-                const int wgt = (H == 1) ? ((j - j0) & 1) : h;
+                const int wgt = h;
                 mbar_wait(bars, kBarSFree, s_par, abort_flag, p.status, j);
                 s_par ^= 1u;
                 tc_fence_after();
@@ -561,11 +563,11 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, const InlineSche
 // P*V issuer: O_h += P_h V_j in the order (tile, head), each in the two pieces P is handed over in.  In a
 // single-head unit the tiles alternate between the two P / O column sets (two independent online-softmax
 // streams over the even and the odd tiles of the piece, combined in the epilogue).
-template <bool kDual, bool kFp8>
+template <bool kFp8>
 __device__ __forceinline__ void mma_pv_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
                                             volatile uint32_t* abort_flag) {
     const uint32_t bars = smem_base + kSmemBar;
-    constexpr int H = kDual ? 1 : 2;
+    constexpr int H = 2;
     RingPos unit_pos = {0, 0};
     uint32_t p_par0 = 0, p_par1 = 0;   // phase parity of p_ready per softmax warpgroup
     const uint64_t v_desc0 = make_desc(smem_base + kSmemKV, kHalfBytes, 1024);   // MN-major view of a ring slot
@@ -578,8 +580,8 @@ __device__ __forceinline__ void mma_pv_role(const AttnParams& p, const InlineSch
         for (int j = j0; j < n; ++j) {
             mbar_wait(bars, kBarKvFull + vpos.slot, vpos.par, abort_flag, p.status, j);
             for (int h = 0; h < H; ++h) {
-                const int wgt = (H == 1) ? ((j - j0) & 1) : h;            // P / O column set and softmax warpgroup
-                const bool first = (H == 1) ? (j - j0 < 2) : (j == j0);   // first tile of this accumulator in the unit
+                const int wgt = h;                 // P / O column set and softmax warpgroup
+                const bool first = j == j0;        // first tile of this accumulator in the unit
                 if (first && round > 0) mbar_wait(bars, kBarOFree + wgt, (round - 1) & 1, abort_flag, p.status, j);
                 const uint32_t ppar = wgt ? p_par1 : p_par0;
 #pragma unroll
@@ -821,24 +823,25 @@ __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], f
     l += st.x + st.y;
 }
 
-template <bool kDual, bool kFp8>
+template <bool kFp8>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
-                                             volatile uint32_t* abort_flag, uint8_t* smem_xchg, int wg) {
+                                             volatile uint32_t* abort_flag, int wg) {
     const uint32_t bars = smem_base + kSmemBar;
     const int lane = threadIdx.x & 31;
     const int warp_in_wg = (threadIdx.x >> 5) & 3;
-    const int row = warp_in_wg * 32 + lane;                        // query row of the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)(warp_in_wg * 32) << 16;   // TMEM lane field of this warp
     const uint32_t s_tmem = tmem_base + lane_addr + kTmemS;
     const uint32_t p_tmem = tmem_base + lane_addr + kTmemP + wg * 64;
     const uint32_t o_tmem = tmem_base + lane_addr + kTmemO + wg * 128;
     const uint32_t p_bar0 = bars + (kBarPReady + wg * 4) * 8;
+    // this thread's query row inside the unit: TMEM lane, plus 128 for the second tile of a tile-pair unit;
+    // its head: head wg of the pair, or the unit's only head
+    const bool tile_pair = p.heads_per_unit == 1;
+    const int row = warp_in_wg * 32 + lane + (tile_pair ? wg * kBlockM : 0);
+    const int head_sel = tile_pair ? 0 : wg;
+    const int row_base = tile_pair ? wg * kBlockM : 0;              // first row of this warpgroup's tile in the unit
     float c = p.scale_log2;
     uint32_t tile_cnt = 0;
-    // single-head units: the two warpgroups take the even and the odd KV tiles of the piece as two independent
-    // online-softmax streams (own running max, sum and O accumulator); warpgroup 0 combines them at the end
-    constexpr bool dual = kDual;
-    constexpr int step = kDual ? 2 : 1;
 
 #define SM_WAIT(id, parity, it)                                                                  \
     mbar_wait(bars, (id), (parity), abort_flag, p.status, (it));                                 \
@@ -849,61 +852,37 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
         UnitInfo u;
         if (!fetch_unit(p, inl, round, u)) break;
         const int n = u.t_end;
-        const int head = u.head0 + (dual ? 0 : wg);
-        const int j_first = u.t_begin + (dual ? wg : 0);     // first tile of this warpgroup's stream
+        const int head = u.head0 + head_sel;
+        const int j_first = u.t_begin;
         float m = -INFINITY;   // running row max in log2 units (possibly stale by < threshold)
         float l = 0.f;         // running row sum of 2^(s - m)
         if (kFp8)              // raw scores are products of codes: this row's query scale and the head's key scale
             c = p.scale_log2 * p.k_scale[u.kv_head] *
                 (row < u.it.n_rows ? p.q_scale[((int64_t)u.it.q_row0 + row) * p.Hq + head] : 0.f);
-        // tiles below n_full lie entirely under the causal diagonal of every row of the q-tile and inside the
-        // unit's key range; the range's first tile is cut on the left when kv_lo is not a tile multiple
-        const int n_full = min(u.it.kv_len0, u.it.kv_hi) / kBlockN;
+        // tiles below n_full lie entirely under the causal diagonal of every row of this warpgroup's q-tile and
+        // inside the unit's key range; the range's first tile is cut on the left when kv_lo is not a tile
+        // multiple.  (The earlier tile of a tile-pair unit finds the unit's last KV tile fully masked.)
+        const int n_full = min(u.it.kv_len0 + row_base, u.it.kv_hi) / kBlockN;
         const int j_cut = (u.it.kv_lo & (kBlockN - 1)) ? (u.it.kv_lo >> 7) : -1;
         float s0[32], s1[32], s2[32], s3[32];   // the row's scores of the current tile
-        // the first tile of the stream is loaded here, every later one by the tile before it
-        if (!kDual || j_first < n) {
-            SM_WAIT(kBarSReady + wg, s_par, j_first);
-            s_par ^= 1u;
-            tc_fence_after();
-            CP_LOAD_S(s0, s1, s2, s3)
-            release_s(bars);
-        }
+        // the first tile of the unit is loaded here, every later one by the tile before it
+        SM_WAIT(kBarSReady + wg, s_par, j_first);
+        s_par ^= 1u;
+        tc_fence_after();
+        CP_LOAD_S(s0, s1, s2, s3)
+        release_s(bars);
 #pragma unroll 1
-        for (int j = j_first; j < n; j += step) {
+        for (int j = j_first; j < n; ++j) {
             const SoftmaxSync sy = {bars, kBarSReady + (uint32_t)wg, kBarPvDone + (uint32_t)wg, (tile_cnt - 1) & 1,
                                     abort_flag, p.status, j};
             if (j < n_full && j != j_cut)
-                softmax_tile<false, kFp8>(s0, s1, s2, s3, j + step < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c, 0, 0,
+                softmax_tile<false, kFp8>(s0, s1, s2, s3, j + 1 < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c, 0, 0,
                                           j == j_first, m, l, sy);
             else
-                softmax_tile<true, kFp8>(s0, s1, s2, s3, j + step < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c,
+                softmax_tile<true, kFp8>(s0, s1, s2, s3, j + 1 < n, s_par, s_tmem, p_tmem, o_tmem, p_bar0, c,
                                    u.it.kv_lo - j * kBlockN, min(u.it.kv_len0 + row, u.it.kv_hi) - j * kBlockN,
                                    j == j_first, m, l, sy);
             ++tile_cnt;
-        }
-        float a_own = 1.f, a_oth = 0.f;     // dual: weights of the two streams' accumulators in the combined row
-        if (dual) {
-            float2* xchg = reinterpret_cast<float2*>(smem_xchg);
-            if (wg == 1) {
-                // second stream: wait for its last P*V, publish (m, l), leave the rest to warpgroup 0
-                if (j_first < n) {
-                    SM_WAIT(kBarPvDone + wg, (tile_cnt - 1) & 1, n);
-                    tc_fence_before();
-                }
-                xchg[row] = make_float2(m, l);
-                asm volatile("bar.sync 1, 256;" ::: "memory");      // both streams done, (m, l) visible
-                asm volatile("bar.sync 2, 256;" ::: "memory");      // warpgroup 0 has read them
-                continue;
-            }
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            const float2 ml1 = xchg[row];
-            asm volatile("bar.arrive 2, 256;" ::: "memory");
-            const float mm = fmaxf(m, ml1.x);
-            a_own = (l > 0.f) ? ex2(m - mm) : 0.f;
-            a_oth = (ml1.y > 0.f) ? ex2(ml1.x - mm) : 0.f;
-            l = a_own * l + a_oth * ml1.y;
-            m = mm;
         }
         // epilogue: O / l -> global at the row's original position; LSE in natural log
         SM_WAIT(kBarPvDone + wg, (tile_cnt - 1) & 1, n);
@@ -914,25 +893,12 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
         const bool partial = u.slot >= 0;
         const bool valid = row < u.it.n_rows;
         const int64_t grow_idx = (int64_t)u.it.q_row0 + row;
-        float* part_row = p.partial_o + (((int64_t)max(u.slot, 0) * 2 + wg) * kBlockM + row) * kD;
-        const bool has_other = dual && (u.t_begin + 1 < n);     // the second stream got at least one tile
+        float* part_row = p.partial_o + (((int64_t)max(u.slot, 0) * 2 + wg) * kBlockM + (row - row_base)) * kD;
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
             float o[32];
             TMEM_LD32(o_tmem + cc * 32, o, 0);
-            if (has_other) {
-                float o1[32];
-                TMEM_LD32(o_tmem + 128 + cc * 32, o1, 0);
-                tc_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) o[i] = a_own * o[i] + a_oth * o1[i];
-            } else {
-                tc_wait_ld();
-                if (dual) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] *= a_own;
-                }
-            }
+            tc_wait_ld();
             if (valid) {
                 if (partial || p.out_f32) {
                     float4* dst = partial ? reinterpret_cast<float4*>(part_row + cc * 32)
@@ -958,15 +924,12 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
         }
         if (valid) {
             const float lse_val = (l > 0.f) ? (m + lg2(l) - (kFp8 ? kP8Shift : 0.f)) * 0.6931471805599453f : -INFINITY;
-            if (partial) p.partial_lse[((int64_t)u.slot * 2 + wg) * kBlockM + row] = lse_val;
+            if (partial) p.partial_lse[((int64_t)u.slot * 2 + wg) * kBlockM + (row - row_base)] = lse_val;
             else p.lse[(int64_t)head * p.lse_stride + grow_idx] = lse_val;
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) {
-            mbar_arrive(bars + (kBarOFree + wg) * 8);
-            if (dual) mbar_arrive(bars + (kBarOFree + 1) * 8);     // this warpgroup has read both accumulators
-        }
+        if (lane == 0) mbar_arrive(bars + (kBarOFree + wg) * 8);
     }
 #undef SM_WAIT
 }
@@ -990,9 +953,8 @@ __device__ __forceinline__ void fill_role(const AttnParams& p) {
     }
 }
 
-// kDual: every unit is a single query head (odd group size); its KV tiles then alternate between the two
-// softmax warpgroups.  Two separate kernels, so that neither carries the other's code in its hot loop.
-template <bool kDual, bool kFp8>
+// kFp8: the FP8 K/V variant (one-byte Q / K / V / P operands).
+template <bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const AttnParams p, const __grid_constant__ InlineSched inl) {
@@ -1032,15 +994,15 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-        softmax_role<kDual, kFp8>(p, inl, smem_base, tmem_base, abort_flag, smem_gen + kSmemXchg, warp >> 2);
+        softmax_role<kFp8>(p, inl, smem_base, tmem_base, abort_flag, warp >> 2);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
         if (warp == 8) {
             producer_role<kFp8>(&tmQ, &tmK, &tmV, p, inl, smem_base, abort_flag);
         } else if (warp == 9) {
-            mma_s_role<kDual, kFp8>(p, inl, smem_base, tmem_base, abort_flag);
+            mma_s_role<kFp8>(p, inl, smem_base, tmem_base, abort_flag);
         } else if (warp == 10) {
-            mma_pv_role<kDual, kFp8>(p, inl, smem_base, tmem_base, abort_flag);
+            mma_pv_role<kFp8>(p, inl, smem_base, tmem_base, abort_flag);
         } else if (p.n_fill > 0) {
             fill_role(p);
         }
@@ -1119,9 +1081,10 @@ __global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p,
 #pragma unroll
     for (int r2 = 0; r2 < 2; ++r2) {
         const int hr = blockIdx.y * kFixupRowsPerBlock + warp * 2 + r2;
-        const int wg = hr / kBlockM;
+        const int wg = hr / kBlockM;                  // head wg of the pair, or (tile-pair unit) rows 128 wg .. of the one head
         const int row = hr - wg * kBlockM;
-        if (row >= it.n_rows || wg >= p.heads_per_unit) continue;
+        const int urow = p.heads_per_unit == 2 ? row : hr;     // row inside the unit
+        if (urow >= it.n_rows) continue;
         // pass 1: max of the partial LSEs (lane k of each group of 32 slots holds slot k)
         float m = -INFINITY;
         for (int base = 0; base < me.n_slots; base += 32) {
@@ -1161,8 +1124,8 @@ __global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p,
         for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
         // a row may see none of the unit's keys (a key range that starts behind its causal limit): zeros, -inf
         const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
-        const int head = p.heads_per_unit * me.pair + wg;
-        const int64_t grow = (int64_t)it.q_row0 + row;
+        const int head = p.heads_per_unit == 2 ? 2 * me.pair + wg : me.pair;
+        const int64_t grow = (int64_t)it.q_row0 + urow;
         const int64_t off = (grow * p.Hq + head) * kD + lane * 4;
         if (p.out_f32) {
             *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off) =
@@ -1315,9 +1278,6 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         shape8.stride_tok = cache8->stride_tok;
         shape8.stride_head = cache8->stride_head;
         cache = &shape8;
-        if ((cache->Hkv < 1) || (Hq / cache->Hkv) % 2 != 0)
-            return set_error(CP_ERR_UNSUPPORTED, "%s: the FP8 variant needs an even number of query heads per KV head "
-                             "(Hq=%d, Hkv=%d)", who, Hq, cache->Hkv);
     } else if (int rc = validate_kv_cache(cache, who)) return rc;
     if (Hq < 1 || Hq % cache->Hkv != 0)
         return set_error(CP_ERR_INVALID_ARG, "%s: Hq=%d is not a multiple of Hkv=%d", who, Hq, cache->Hkv);
@@ -1384,7 +1344,9 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     } else {
         ctx->cache_valid = false;
         Schedule sch;
-        build_tiles(B, cu_new, prefix_len, C, cu_pages, cache->page_size, only_shard, only_chunk, kv_lo, kv_hi, sch.items);
+        // even groups: 128-row tiles for pairs of heads; odd groups: 256-row tile pairs for single heads
+        build_tiles(B, cu_new, prefix_len, C, cu_pages, cache->page_size, only_shard, only_chunk, kv_lo, kv_hi,
+                    heads_per_unit == 2 ? kTileRows : 2 * kTileRows, sch.items);
         // rows of q / out / lse: the packed batch, or the one chunk of a chunk call
         total_rows = cu_new[B];
         if (only_chunk >= 0) {
@@ -1478,11 +1440,9 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         return rc;
     }
     if (!ctx->attn_attr_set) {
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                     (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
         ctx->attn_attr_set = true;
     }
@@ -1521,9 +1481,8 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.q_scale = cache8 ? q_scale : nullptr;
     p.k_scale = cache8 ? cache8->k_scale : nullptr;
     p.v_scale = cache8 ? cache8->v_scale : nullptr;
-    if (cache8) cp_attn_kernel<false, true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
-    else if (heads_per_unit == 2) cp_attn_kernel<false, false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
-    else cp_attn_kernel<true, false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
+    if (cache8) cp_attn_kernel<true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
+    else cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
     if (int rc = check_cuda(cudaGetLastError(), who)) return rc;
     if (n_merges > 0) {
         FixupParams f;
@@ -1684,9 +1643,7 @@ int static_setup(int device, StaticDeviceState** out) {
                                 "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)")) return rc;
         if (q != cudaDriverEntryPointSuccess || !fn)
             return set_error(CP_ERR_CUDA, "cuTensorMapEncodeTiled is not available in this driver");
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                     (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
-        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)kSmemAlloc), "cudaFuncSetAttribute(attn)")) return rc;
         st.scratch = static_cast<unsigned char*>(ptr);
         st.num_sms = prop.multiProcessorCount;
@@ -1700,14 +1657,15 @@ int static_setup(int device, StaticDeviceState** out) {
 // Writes the request's tile list into the scratch and clears the status words, from the lengths alone (the
 // all-shards tile list is plain arithmetic: tile t covers rows [128 t, 128 t + 128), longest tiles first), so no
 // host buffer is read when the stream runs.
-__global__ void static_tiles_kernel(unsigned char* scratch, int64_t R, int64_t P, int32_t n_pages, int32_t n_tiles) {
+__global__ void static_tiles_kernel(unsigned char* scratch, int64_t R, int64_t P, int32_t n_pages, int32_t n_tiles,
+                                    int32_t tile_rows) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < kStatusWords) reinterpret_cast<int32_t*>(scratch)[i] = 0;
     if (i >= n_tiles) return;
-    const int64_t r0 = (int64_t)(n_tiles - 1 - i) * kTileRows;
+    const int64_t r0 = (int64_t)(n_tiles - 1 - i) * tile_rows;
     TileItem t;
     t.q_row0 = (int32_t)r0;
-    t.n_rows = (int32_t)min((int64_t)kTileRows, R - r0);
+    t.n_rows = (int32_t)min((int64_t)tile_rows, R - r0);
     t.kv_len0 = (int32_t)(P + r0 + 1);
     t.pt_base = 0;
     t.n_pages = n_pages;
@@ -1732,11 +1690,12 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     if (!(scale > 0.f)) return set_error(CP_ERR_INVALID_ARG, "%s: scale must be positive", who);
     if (((uintptr_t)q | (uintptr_t)out) & 15) return set_error(CP_ERR_INVALID_ARG, "%s: q and out must be 16-byte aligned", who);
     if (prefix_len + new_len > 0x7fffff00ll) return set_error(CP_ERR_UNSUPPORTED, "%s: request longer than 2^31 tokens", who);
-    const int64_t n_tiles = (new_len + kTileRows - 1) / kTileRows;
-    if (n_tiles > kStaticMaxTiles)
+    const int32_t tile_rows = heads_per_unit == 2 ? kTileRows : 2 * kTileRows;      // single-head units take tile pairs
+    const int64_t n_tiles = (new_len + tile_rows - 1) / tile_rows;
+    if ((new_len + kTileRows - 1) / kTileRows > kStaticMaxTiles)
         return set_error(CP_ERR_WORKSPACE, "%s: new_len=%lld needs %lld query tiles; the built-in scratch holds %d "
-                         "(use cp_prefill_attn with a caller workspace)", who, (long long)new_len, (long long)n_tiles,
-                         kStaticMaxTiles);
+                         "(use cp_prefill_attn with a caller workspace)", who, (long long)new_len,
+                         (long long)((new_len + kTileRows - 1) / kTileRows), kStaticMaxTiles);
     int device = -1;
     if (int rc = check_cuda(cudaGetDevice(&device), "cudaGetDevice")) return rc;
     StaticDeviceState* st = nullptr;
@@ -1753,7 +1712,7 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     // The scratch keeps whatever the previous call left: a small kernel clears the status words and writes this
     // request's tile list in stream order (no host memory is read later, whatever the stream does with the work).
     static_tiles_kernel<<<(unsigned)((n_tiles + 255) / 256), 256, 0, s>>>(
-        st->scratch, new_len, prefix_len, (int32_t)cu_pages[1], (int32_t)n_tiles);
+        st->scratch, new_len, prefix_len, (int32_t)cu_pages[1], (int32_t)n_tiles, tile_rows);
     if (int rc = check_cuda(cudaGetLastError(), "static tile list launch")) return rc;
     AttnParams p;
     p.items = reinterpret_cast<const TileItem*>(st->scratch + kWorkspaceHeader);
@@ -1783,7 +1742,6 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     none.bytes[0] = 0;
     const int64_t units = n_tiles * p.pairs_per_tile;
     const int grid = (int)std::min<int64_t>(units, st->num_sms);
-    if (heads_per_unit == 2) cp_attn_kernel<false, false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, none);
-    else cp_attn_kernel<true, false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, none);
+    cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, none);
     return check_cuda(cudaGetLastError(), who);
 }

@@ -12,11 +12,12 @@
 
 namespace cpattn {
 
-// One query tile of the persistent scheduler: up to 128 consecutive new tokens of one chunk of
-// one request.  Every tile is processed once per pair of query heads.
+// One query tile of the persistent scheduler: up to 128 consecutive new tokens of one request, processed
+// once per pair of query heads; with an odd number of query heads per KV head, up to 256 tokens (two
+// consecutive tiles), processed once per head.
 struct TileItem {
     int32_t q_row0;     // first row in the packed q / out tensors
-    int32_t n_rows;     // 1..128
+    int32_t n_rows;     // 1..128 (1..256 for tile pairs)
     int32_t kv_len0;    // keys visible to the first row: P + r0 + 1 (row i sees kv_len0 + i)
     int32_t pt_base;    // offset of the request's page table in the packed page table
     int32_t n_pages;    // entries of that page table
@@ -96,11 +97,12 @@ int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C);
 // sorted longest first.  only_shard < 0 keeps all shards; only_chunk >= 0 (B == 1) keeps that one zigzag
 // chunk and numbers its rows from the chunk's first row (q, out and lse then hold the chunk alone).
 // [kv_lo, kv_hi) restricts the keys (absolute positions); tiles that see none of them are left out.
+// tile_rows: 128, or 256 when the units are single heads over tile pairs.
 int validate_kv_cache(const cp_kv_cache* c, const char* who);
 int validate_kv_cache_fp8(const cp_kv_cache_fp8* c, const char* who);
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
                 const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, int64_t kv_lo,
-                int64_t kv_hi, std::vector<TileItem>& out);
+                int64_t kv_hi, int32_t tile_rows, std::vector<TileItem>& out);
 // Distributes the (tile, head pair) units of s.items over `grid_max` CTAs (pairs_per_kv = units of one KV
 // head per tile): whole units, KV head by KV head and longest first within a head,
 // onto the least loaded CTA while they fit under the per-CTA share, the rest cut into KV ranges that

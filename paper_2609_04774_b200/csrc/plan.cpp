@@ -33,7 +33,7 @@ int64_t max_tiles(int32_t B, const int64_t* new_len, const int32_t* C) {
 
 int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
                 const int64_t* cu_pages, int32_t page_size, int32_t only_shard, int32_t only_chunk, int64_t kv_lo,
-                int64_t kv_hi, std::vector<TileItem>& out) {
+                int64_t kv_hi, int32_t tile_rows, std::vector<TileItem>& out) {
     out.clear();
     // A launch over ALL shards of a request walks its rows as one run: adjacent zigzag chunks are adjacent rows
     // with consecutive causal limits, which the per-row limit kv_len0 + row already expresses, so a query tile may
@@ -55,10 +55,10 @@ int build_tiles(int32_t B, const int64_t* cu_new, const int64_t* prefix_len, con
             }
             // a single-chunk list addresses q / out / lse rows relative to the chunk's first row
             const int64_t row_base = only_chunk >= 0 ? cb : 0;
-            for (int64_t r0 = cb; r0 < ce; r0 += kTileRows) {
+            for (int64_t r0 = cb; r0 < ce; r0 += tile_rows) {
                 TileItem t;
                 t.q_row0 = (int32_t)(cu_new[b] + r0 - row_base);
-                t.n_rows = (int32_t)std::min<int64_t>(kTileRows, ce - r0);
+                t.n_rows = (int32_t)std::min<int64_t>(tile_rows, ce - r0);
                 t.kv_len0 = (int32_t)(P + r0 + 1);
                 t.pt_base = (int32_t)cu_pages[b];
                 // entries the request really uses; a single chunk reads none behind its last key
@@ -307,7 +307,8 @@ extern "C" int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64
         cu_pages[b + 1] = cu_pages[b] + (prefix_len[b] + R + kDefaultPageTokens - 1) / kDefaultPageTokens;
     }
     Schedule sch;
-    build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), kDefaultPageTokens, -1, -1, 0, INT32_MAX, sch.items);
+    build_tiles(B, cu_new, prefix_len, C, cu_pages.data(), kDefaultPageTokens, -1, -1, 0, INT32_MAX,
+                heads_per_unit == 2 ? kTileRows : 2 * kTileRows, sch.items);
     if (int rc = build_schedule(Hq / heads_per_unit, kv_major_pairs(B, cu_new, prefix_len, Hkv, (Hq / Hkv) / heads_per_unit),
                                 num_sms, sch)) return rc;
     int64_t max_load = 0, min_load = INT64_MAX, total = 0;

@@ -352,8 +352,14 @@ def variant_chunked_prefill() -> Workload:
     return Workload("var_chunk_R512_P65536_C2", 8, 32, 8, [Request(512, 65536, 2)])
 
 
+def variant_mha() -> Workload:
+    """Config 2's lengths with plain multi-head attention (16 query heads on 16 KV heads: every work unit is a
+    single head, no K/V tile is shared), seed 9."""
+    return Workload("var_mha_R4096_P12288_C4", 9, 16, 16, [Request(4096, 12288, 4)])
+
+
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
-VARIANTS = {6: variant_gqa8, 7: variant_chunked_prefill}
+VARIANTS = {6: variant_gqa8, 7: variant_chunked_prefill, 8: variant_mha}
 
 
 # --------------------------------------------------------------------------------------

@@ -146,15 +146,18 @@ def test_fp8_single_request_entry_and_validation(ctx):
                                   np.arange(517))
     compare8(bf16_to_f64(dev.out), dev.lse.cpu().numpy().astype(np.float64), ro, rl, ra, "fp8 single")
     before = dev.out.clone()
-    with pytest.raises(binding.CpError) as e:                                  # odd group size: not supported by this variant
-        binding.cp_prefill_attn_fp8(ctx, dev.q, dev.cache, dev.page_table, 320, 517, 2, 6, w.scale, dev.out, dev.lse, dev.ws)
-    assert e.value.code == binding.CP_ERR_UNSUPPORTED
     small = torch.zeros(dev.base_ws, dtype=torch.uint8, device="cuda")      # the bf16 path's workspace is too small
     with pytest.raises(binding.CpError) as e:
         binding.cp_prefill_attn_fp8(ctx, dev.q, dev.cache, dev.page_table, 320, 517, 2, w.Hq, w.scale, dev.out, dev.lse, small)
     assert e.value.code == binding.CP_ERR_WORKSPACE
     torch.cuda.synchronize()
     assert torch.equal(before.view(torch.int16), dev.out.view(torch.int16))
+
+
+def test_fp8_attention_odd_group_sizes(ctx):
+    # three query heads per KV head and plain multi-head attention: single-head units over pairs of query tiles
+    check_batch8(ctx, wl.Workload("fp8_odd_group", 56, 6, 2, [wl.Request(333, 192, 3), wl.Request(129, 0, 2), wl.Request(700, 64, 1)]))
+    check_batch8(ctx, wl.Workload("fp8_mha", 57, 4, 4, [wl.Request(700, 64, 4), wl.Request(90, 3000, 1)]))
 
 
 def test_fp8_attention_config2_shape_sampled(ctx):

@@ -17,19 +17,21 @@ def check(w, num_sms=148):
     prefix = [r.prefix_len for r in w.requests]
     Cs = [r.C for r in w.requests]
     info, pieces, items = binding.cp_schedule_inspect(cu_new, prefix, Cs, w.Hq, w.Hkv, num_sms)
-    HP = w.Hq // (2 if (w.Hq // w.Hkv) % 2 == 0 else 1)
+    even = (w.Hq // w.Hkv) % 2 == 0
+    HP = w.Hq // (2 if even else 1)
+    TR = 128 if even else 256          # single-head units (odd group size) take two consecutive 128-row tiles
     # tiles: rows tile [0, total_new) exactly and never straddle a request; in a launch over all shards a tile
     # may span the boundary of adjacent zigzag chunks (the per-row causal limit does not care), so every tile
     # but a request's last has the full 128 rows
     rows = np.zeros(w.total_new, dtype=np.int32)
     for q0, n, kv0, nt in items:
-        assert 1 <= n <= 128 and nt == -(-(kv0 + n - 1) // 128)
+        assert 1 <= n <= TR and nt == -(-(kv0 + n - 1) // 128)
         rows[q0:q0 + n] += 1
         b = int(np.searchsorted(cu_new, q0, side="right") - 1)
         r = w.requests[b]
         r0 = q0 - cu_new[b]
         assert r0 + n <= r.new_len and kv0 == r.prefix_len + r0 + 1
-        assert r0 % 128 == 0 and (n == 128 or r0 + n == r.new_len)
+        assert r0 % TR == 0 and (n == TR or r0 + n == r.new_len)
     assert (rows == 1).all()
     # pieces: per unit the KV tile ranges tile [0, n_kv_tiles) exactly; slots only on split units
     cover = {}
