@@ -1435,9 +1435,27 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         const int64_t n_rows = total_rows * Hq;
         quantize_q_kernel<<<(unsigned)((n_rows + 7) / 8), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(q), q8, q_scale, n_rows);
         if (int rc = check_cuda(cudaGetLastError(), "quantize_q launch")) return rc;
-        if (int rc = encode_maps_fp8(ctx, q8, total_rows, Hq, cache8, &tmQ, &tmK, &tmV)) return rc;
-    } else if (int rc = encode_maps(ctx, q, total_rows, Hq, cache, &tmQ, &tmK, &tmV)) {
-        return rc;
+    }
+    // a tensor map depends only on addresses, shapes and strides: the previous call's maps serve again when
+    // those are unchanged (encoding three maps costs a few microseconds of host time)
+    const int64_t mkey[12] = {(int64_t)(uintptr_t)(cache8 ? (const void*)q8 : q), total_rows, Hq, cache8 ? 1 : 0,
+                              (int64_t)(uintptr_t)cache->k, (int64_t)(uintptr_t)cache->v, cache->num_pages, cache->page_size,
+                              cache->Hkv, cache->stride_page, cache->stride_tok, cache->stride_head};
+    if (ctx->maps_valid && memcmp(mkey, ctx->maps_key, sizeof mkey) == 0) {
+        tmQ = ctx->maps[0];
+        tmK = ctx->maps[1];
+        tmV = ctx->maps[2];
+    } else {
+        if (cache8) {
+            if (int rc = encode_maps_fp8(ctx, q8, total_rows, Hq, cache8, &tmQ, &tmK, &tmV)) return rc;
+        } else if (int rc = encode_maps(ctx, q, total_rows, Hq, cache, &tmQ, &tmK, &tmV)) {
+            return rc;
+        }
+        memcpy(ctx->maps_key, mkey, sizeof mkey);
+        ctx->maps[0] = tmQ;
+        ctx->maps[1] = tmK;
+        ctx->maps[2] = tmV;
+        ctx->maps_valid = true;
     }
     if (!ctx->attn_attr_set) {
         if (int rc = check_cuda(cudaFuncSetAttribute(cp_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,

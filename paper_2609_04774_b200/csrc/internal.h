@@ -138,6 +138,11 @@ struct cp_ctx {
     cpattn::WorkspaceLayout cache_lay;
     int32_t cache_grid, cache_items, cache_merges;
     int64_t cache_rows;
+    // the tensor maps of the last attention call, reused while the buffers and shapes they describe stay the same
+    // (the layers of a model call with the same q / cache buffers over and over)
+    bool maps_valid;
+    int64_t maps_key[12];
+    CUtensorMap maps[3];
     bool cache_inline;                 // the remembered work lists travel in the launch parameters
     cpattn::InlineSched cache_inl;
     int32_t cache_n_fill;
