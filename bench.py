@@ -48,7 +48,7 @@ NOMINAL_HBM_GBS = 8000.0
 MUFU_ROOFLINE_TFLOPS = 148 * 16 * 512 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum of one cp_attn_kernel launch, from the ncu captures
 # summarised in profiles/ (per workload name; a workload without a capture reports null)
-ATTN_TRAFFIC_BYTES = {"cfg2_R4096_P12288_C4": 118_038_784, "cfg3_R131072_P0_C8": 11_500_000_000}
+ATTN_TRAFFIC_BYTES = {"cfg2_R4096_P12288_C4": 117_532_416, "cfg3_R131072_P0_C8": 7_200_575_488}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -361,10 +361,12 @@ def sustained_leg(torch, runner, peaks, device, seconds=2.2):
             "frac": fractions(tf, peaks), "clocks": clocks}
 
 
-def config_leg(torch, cfg, peaks, device, budget_ms=1200.0, fp8=False):
+def config_leg(torch, cfg, peaks, device, budget_ms=1200.0, fp8=False, page=None):
     """One configuration: 3 warm-up steps, then steps for about `budget_ms` of GPU time (at least 5), clocks sampled.
     fp8: the same lengths and heads with E4M3 K/V pages (queries quantised per step by the library's pre-pass)."""
     w = get_workload(cfg)
+    if page:
+        w.page = page                   # tokens per cache page (16, 32, 64 or 128) instead of the configurations' 64
     runner = Runner(w, device, fp8=fp8)
     sampler = ClockSampler(device)
     sampler.start()
@@ -383,7 +385,7 @@ def config_leg(torch, cfg, peaks, device, budget_ms=1200.0, fp8=False):
     runner.ctx.poll_status()
     ms = total_ms / steps
     tf = flops_of(w) / (ms * 1e-3) / 1e12
-    entry = {"config": cfg, "workload": w.name, "steps": steps, "ms": ms, "ms_best": min(per), "tflops": tf,
+    entry = {"config": cfg, "workload": w.name, "page_tokens": w.page, "steps": steps, "ms": ms, "ms_best": min(per), "tflops": tf,
              "tokens_per_s": w.total_new / (ms * 1e-3), "frac": fractions(tf, peaks), "pairs": pairs_of(w),
              "launches_per_step": runner.launches_per_step(), "gpu_seconds": total_ms * 1e-3, "clocks": clocks,
              "traffic": ATTN_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": algorithmic_bytes(w),
@@ -712,7 +714,7 @@ def run_configs(args, out):
     import torch
     peaks = load_peaks()
     for cfg in args.configs:
-        out.write(json.dumps(dict(mode="config", **config_leg(torch, cfg, peaks, 0, budget_ms=args.config_ms, fp8=args.fp8))) + "\n")
+        out.write(json.dumps(dict(mode="config", **config_leg(torch, cfg, peaks, 0, budget_ms=args.config_ms, fp8=args.fp8, page=args.page))) + "\n")
         out.flush()
 
 
@@ -982,6 +984,7 @@ def main():
                     help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P; 8: multi-head (16/16)")
     ap.add_argument("--config-ms", type=float, default=1200.0, help="configs mode: GPU time per configuration")
     ap.add_argument("--fp8", action="store_true", help="configs mode: the FP8 K/V variant of each configuration")
+    ap.add_argument("--page", type=int, default=None, help="configs mode: tokens per cache page (16, 32, 64, 128)")
     ap.add_argument("--rank-reps", type=int, default=5)
     ap.add_argument("--pass-q", action="store_true", help="cprank mode: K/V stays sharded, queries travel")
     ap.add_argument("--cache-requests", type=int, default=20000)
