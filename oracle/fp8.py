@@ -93,7 +93,8 @@ def quantize_kv(rows_bits, scale):
     the quotient rounded to fp32 (IEEE division)."""
     x = _bf16_bits_to_f32(rows_bits)
     s = np.asarray(scale, dtype=np.float32)[None, :, None]
-    return e4m3_encode((x / s).astype(np.float32))
+    with np.errstate(over="ignore"):                      # a quotient beyond fp32 is +-inf, which saturates like any large value
+        return e4m3_encode((x / s).astype(np.float32))
 
 
 # ------------------------------------------------------------------------------------------

@@ -160,6 +160,27 @@ def test_fp8_attention_odd_group_sizes(ctx):
     check_batch8(ctx, wl.Workload("fp8_mha", 57, 4, 4, [wl.Request(700, 64, 4), wl.Request(90, 3000, 1)]))
 
 
+def _random_workload8(seed):
+    u = wl.counter_uniform(seed, wl.TID_LEN, 0, 64)
+    heads = [(8, 2), (4, 4), (6, 2), (16, 2), (32, 4), (8, 8), (2, 1)][int(u[0] * 7)]
+    page = [16, 32, 64, 128][int(u[1] * 4)]
+    reqs = []
+    for b in range(1 + int(u[2] * 5)):
+        R = max(1, int(round(2.0 ** (u[3 + 4 * b] * 10.5))))                  # 1 .. ~1450, log-uniform
+        kind = u[4 + 4 * b]
+        P = 0 if kind < 0.25 else int(u[5 + 4 * b] * 6000)
+        if kind < 0.75:
+            P = P // page * page
+        reqs.append(wl.Request(R, P, [1, 2, 3, 4, 5, 8][int(u[6 + 4 * b] * 6)]))
+    return wl.Workload("fp8_random_%d" % seed, seed, heads[0], heads[1], reqs, page=page)
+
+
+@pytest.mark.parametrize("seed", range(3000, 3008))
+def test_fp8_attention_random_batches(ctx, seed):
+    # seeded random batches: even, odd and unit group sizes, all page sizes, ragged lengths from one token up
+    check_batch8(ctx, _random_workload8(seed), rows_per_request=64, seed=seed)
+
+
 def test_fp8_attention_config2_shape_sampled(ctx):
     check_batch8(ctx, wl.config2(), rows_per_request=96)
 
