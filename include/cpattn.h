@@ -335,6 +335,21 @@ int cp_prefill_attn_fp8_batch(cp_ctx* ctx, const void* q, const cp_kv_cache_fp8*
                               int32_t B, const int64_t* cu_new, const int64_t* prefix_len, const int32_t* C,
                               const int64_t* cu_pages, int32_t Hq, float scale, void* out, float* lse,
                               void* workspace, size_t workspace_bytes, void* stream);
+/* The one-shard, one-chunk and key-range forms of the FP8 variant: arguments, tile lists, fill of uncovered rows and
+ * results as in cp_prefill_attn_shard / _chunk / _kvrange, on an FP8 cache (partials in fp32, ready for cp_merge);
+ * workspace as cp_workspace_bytes_fp8 says. */
+int cp_prefill_attn_fp8_shard(cp_ctx* ctx, const void* q, const cp_kv_cache_fp8* cache, const int32_t* page_table,
+                              int64_t prefix_len, int64_t new_len, int32_t C, int32_t shard, int32_t Hq,
+                              float scale, float* partial_out, float* partial_lse, void* workspace,
+                              size_t workspace_bytes, void* stream);
+int cp_prefill_attn_fp8_chunk(cp_ctx* ctx, const void* q_chunk, const cp_kv_cache_fp8* cache, const int32_t* page_table,
+                              int64_t prefix_len, int64_t new_len, int32_t C, int32_t chunk, int32_t Hq,
+                              float scale, void* out_chunk, float* lse_chunk, void* workspace,
+                              size_t workspace_bytes, void* stream);
+int cp_prefill_attn_fp8_kvrange(cp_ctx* ctx, const void* q, const cp_kv_cache_fp8* cache, const int32_t* page_table,
+                                int64_t prefix_len, int64_t new_len, int64_t kv_lo, int64_t kv_hi, int32_t Hq,
+                                float scale, float* partial_out, float* partial_lse, void* workspace,
+                                size_t workspace_bytes, void* stream);
 int cp_kv_append_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,
                      int64_t n, const void* k_rows, const void* v_rows, void* stream);
 

@@ -22,7 +22,8 @@ CP_DTYPE_BF16, CP_DTYPE_F32 = 0, 1
 EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "cp_ctx_poll_status", "cp_ctx_cache_schedule", "cp_ctx_selftest_wait_expiry", "cp_plan",
            "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_chunk", "cp_prefill_attn_kvrange", "cp_prefill_attn_static", "cp_merge",
            "cp_kv_gather", "cp_kv_append", "cp_workspace_bytes_fp8", "cp_prefill_attn_fp8", "cp_prefill_attn_fp8_batch",
-           "cp_kv_append_fp8", "cp_kv_append_segments"]
+           "cp_kv_append_fp8", "cp_kv_append_segments", "cp_prefill_attn_fp8_shard", "cp_prefill_attn_fp8_chunk",
+           "cp_prefill_attn_fp8_kvrange"]
 
 
 class CpError(RuntimeError):
@@ -305,6 +306,30 @@ def cp_prefill_attn_fp8_batch(ctx, q, cache, page_table, cu_new, prefix_len, C, 
         ctx._h, _ptr(q), ctypes.byref(cache), _ptr(page_table), ctypes.c_int32(B), _hp(cu_new), _hp(prefix_len), _hp(C),
         _hp(cu_pages), ctypes.c_int32(Hq), ctypes.c_float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
         ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
+
+
+def cp_prefill_attn_fp8_shard(ctx, q, cache, page_table, prefix_len, new_len, C, shard, Hq, scale, partial_out, partial_lse,
+                              workspace, stream=None):
+    _check(load().cp_prefill_attn_fp8_shard(
+        ctx._h, _ptr(q), ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(prefix_len), ctypes.c_int64(new_len),
+        ctypes.c_int32(C), ctypes.c_int32(shard), ctypes.c_int32(Hq), ctypes.c_float(scale), _ptr(partial_out),
+        _ptr(partial_lse), _ptr(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
+
+
+def cp_prefill_attn_fp8_chunk(ctx, q_chunk, cache, page_table, prefix_len, new_len, C, chunk, Hq, scale, out_chunk, lse_chunk,
+                              workspace, stream=None):
+    _check(load().cp_prefill_attn_fp8_chunk(
+        ctx._h, _ptr(q_chunk), ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(prefix_len), ctypes.c_int64(new_len),
+        ctypes.c_int32(C), ctypes.c_int32(chunk), ctypes.c_int32(Hq), ctypes.c_float(scale), _ptr(out_chunk), _ptr(lse_chunk),
+        _ptr(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
+
+
+def cp_prefill_attn_fp8_kvrange(ctx, q, cache, page_table, prefix_len, new_len, kv_lo, kv_hi, Hq, scale, partial_out,
+                                partial_lse, workspace, stream=None):
+    _check(load().cp_prefill_attn_fp8_kvrange(
+        ctx._h, _ptr(q), ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(prefix_len), ctypes.c_int64(new_len),
+        ctypes.c_int64(kv_lo), ctypes.c_int64(kv_hi), ctypes.c_int32(Hq), ctypes.c_float(scale), _ptr(partial_out),
+        _ptr(partial_lse), _ptr(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
 
 
 def cp_kv_append_fp8(ctx, cache, page_table, t_begin, n, k_rows, v_rows, stream=None):

@@ -1570,6 +1570,49 @@ extern "C" int cp_prefill_attn_fp8(cp_ctx* ctx, const void* q, const cp_kv_cache
                        false, lse, workspace, workspace_bytes, stream, "cp_prefill_attn_fp8", cache);
 }
 
+// The one-shard, one-chunk and key-range calls of the FP8 variant: the same tile lists as their bf16 forms.
+extern "C" int cp_prefill_attn_fp8_shard(cp_ctx* ctx, const void* q, const cp_kv_cache_fp8* cache, const int32_t* page_table,
+                                         int64_t prefix_len, int64_t new_len, int32_t C, int32_t shard, int32_t Hq,
+                                         float scale, float* partial_out, float* partial_lse, void* workspace,
+                                         size_t workspace_bytes, void* stream) {
+    if (!cache || cache->page_size < 1 || new_len < 1 || prefix_len < 0 || C < 1 || shard < 0 || shard >= C || !partial_out ||
+        !partial_lse || Hq < 1)
+        return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_fp8_shard: bad sizes or shard %d not in [0, %d)", shard, C);
+    const int64_t cu_new[2] = {0, new_len};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + cache->page_size - 1) / cache->page_size};
+    return attn_common(ctx, q, nullptr, page_table, 1, cu_new, &prefix_len, &C, cu_pages, shard, -1, 0, INT32_MAX, Hq, scale,
+                       partial_out, 1, true, partial_lse, workspace, workspace_bytes, stream, "cp_prefill_attn_fp8_shard", cache);
+}
+
+extern "C" int cp_prefill_attn_fp8_chunk(cp_ctx* ctx, const void* q_chunk, const cp_kv_cache_fp8* cache,
+                                         const int32_t* page_table, int64_t prefix_len, int64_t new_len, int32_t C,
+                                         int32_t chunk, int32_t Hq, float scale, void* out_chunk, float* lse_chunk,
+                                         void* workspace, size_t workspace_bytes, void* stream) {
+    if (!cache || cache->page_size < 1 || new_len < 1 || prefix_len < 0 || C < 1 || chunk < 0 || chunk >= 2 * (int64_t)C)
+        return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_fp8_chunk: bad sizes or chunk %d not in [0, %d)", chunk, 2 * C);
+    const int64_t cu_new[2] = {0, new_len};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + cache->page_size - 1) / cache->page_size};
+    return attn_common(ctx, q_chunk, nullptr, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, chunk, 0, INT32_MAX, Hq,
+                       scale, out_chunk, 0, false, lse_chunk, workspace, workspace_bytes, stream, "cp_prefill_attn_fp8_chunk",
+                       cache);
+}
+
+extern "C" int cp_prefill_attn_fp8_kvrange(cp_ctx* ctx, const void* q, const cp_kv_cache_fp8* cache, const int32_t* page_table,
+                                           int64_t prefix_len, int64_t new_len, int64_t kv_lo, int64_t kv_hi, int32_t Hq,
+                                           float scale, float* partial_out, float* partial_lse, void* workspace,
+                                           size_t workspace_bytes, void* stream) {
+    if (!cache || cache->page_size < 1 || new_len < 1 || prefix_len < 0 || !partial_out || !partial_lse || Hq < 1)
+        return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_fp8_kvrange: null pointer or bad sizes");
+    if (kv_lo < 0 || kv_hi < kv_lo || kv_lo > 0x7fffff00ll)
+        return set_error(CP_ERR_INVALID_ARG, "cp_prefill_attn_fp8_kvrange: key range [%lld, %lld)", (long long)kv_lo, (long long)kv_hi);
+    const int64_t cu_new[2] = {0, new_len};
+    const int64_t cu_pages[2] = {0, (prefix_len + new_len + cache->page_size - 1) / cache->page_size};
+    const int32_t C = 1;
+    return attn_common(ctx, q, nullptr, page_table, 1, cu_new, &prefix_len, &C, cu_pages, -1, -1, kv_lo,
+                       std::min<int64_t>(kv_hi, INT32_MAX), Hq, scale, partial_out, 1, true, partial_lse, workspace,
+                       workspace_bytes, stream, "cp_prefill_attn_fp8_kvrange", cache);
+}
+
 // The two partial-result calls write zeros with lse = -inf (the identity element of cp_merge) into the rows
 // they compute nothing for; the attention kernel's spare warp does it, so each call is one launch.
 extern "C" int cp_prefill_attn_shard(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,

@@ -160,6 +160,53 @@ def test_fp8_attention_odd_group_sizes(ctx):
     check_batch8(ctx, wl.Workload("fp8_mha", 57, 4, 4, [wl.Request(700, 64, 4), wl.Request(90, 3000, 1)]))
 
 
+def test_fp8_shard_chunk_and_key_range_calls(ctx):
+    # one request through the three partial forms of the variant: the C shard partials and a set of key-range
+    # partials each merge (cp_merge) into the oracle's full result; every chunk call reproduces its rows
+    from oracle import reference as orc
+    w = wl.Workload("fp8_partials", 58, 8, 2, [wl.Request(700, 320, 3)])
+    m8 = wl.materialize_fp8(w)
+    dev = Device8(m8)
+    r = w.requests[0]
+    R, P, C = r.new_len, r.prefix_len, r.C
+    ro, rl, ra = o8.attn_fp8_rows(m8.q, m8.k8_pages, m8.v8_pages, m8.k_scale, m8.v_scale, m8.page_table, P, w.Hkv, w.scale,
+                                  np.arange(R))
+    plan = orc.plan(R, P, C)
+    parts = torch.full((C, R, w.Hq, w.D), float("nan"), dtype=torch.float32, device="cuda")
+    lses = torch.full((C, w.Hq, R), float("nan"), dtype=torch.float32, device="cuda")
+    for k in range(C):
+        binding.cp_prefill_attn_fp8_shard(ctx, dev.q, dev.cache, dev.page_table, P, R, C, k, w.Hq, w.scale, parts[k], lses[k], dev.ws)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    for k in range(C):
+        own = np.zeros(R, dtype=bool)
+        own[orc.shard_rows(plan[k])] = True
+        lk = lses[k].cpu().numpy()
+        assert np.isfinite(lk[:, own]).all() and np.isneginf(lk[:, ~own]).all() and (parts[k].cpu().numpy()[~own] == 0).all()
+    merged = torch.empty((R, w.Hq, w.D), dtype=torch.float32, device="cuda")
+    mlse = torch.empty((w.Hq, R), dtype=torch.float32, device="cuda")
+    binding.cp_merge(ctx, parts, lses, merged, mlse)
+    torch.cuda.synchronize()
+    compare8(merged.cpu().numpy().astype(np.float64), mlse.cpu().numpy().astype(np.float64), ro, rl, ra, "fp8 merged shards")
+    edges = [0, 130, 320, 577, P + R]
+    kparts = torch.empty((len(edges) - 1, R, w.Hq, w.D), dtype=torch.float32, device="cuda")
+    klses = torch.empty((len(edges) - 1, w.Hq, R), dtype=torch.float32, device="cuda")
+    for n, (lo, hi) in enumerate(zip(edges, edges[1:])):
+        binding.cp_prefill_attn_fp8_kvrange(ctx, dev.q, dev.cache, dev.page_table, P, R, lo, hi, w.Hq, w.scale, kparts[n], klses[n], dev.ws)
+    binding.cp_merge(ctx, kparts, klses, merged, mlse)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    compare8(merged.cpu().numpy().astype(np.float64), mlse.cpu().numpy().astype(np.float64), ro, rl, ra, "fp8 merged key ranges")
+    for j in range(2 * C):
+        b, e = (plan[j]["q_begin"][0], plan[j]["q_end"][0]) if j < C else (plan[2 * C - 1 - j]["q_begin"][1], plan[2 * C - 1 - j]["q_end"][1])
+        out = torch.full((e - b, w.Hq, w.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((w.Hq, e - b), float("nan"), dtype=torch.float32, device="cuda")
+        binding.cp_prefill_attn_fp8_chunk(ctx, dev.q[b:e].contiguous(), dev.cache, dev.page_table, P, R, C, j, w.Hq, w.scale, out, lse, dev.ws)
+        torch.cuda.synchronize()
+        ctx.poll_status()
+        compare8(bf16_to_f64(out), lse.cpu().numpy().astype(np.float64), ro[b:e], rl[:, b:e], ra[b:e], "fp8 chunk %d" % j)
+
+
 def _random_workload8(seed):
     u = wl.counter_uniform(seed, wl.TID_LEN, 0, 64)
     heads = [(8, 2), (4, 4), (6, 2), (16, 2), (32, 4), (8, 8), (2, 1)][int(u[0] * 7)]
