@@ -13,9 +13,10 @@ workload repeated for at least two seconds of GPU time, clocks sampled), `config
 each with its own clocks), `merge` (cp_merge bandwidth points), `kvcopy` (paged copy bandwidth) and the
 `cpu_baseline` legs (the fp64 oracle on the host cores).
 
-Other modes (`--mode merge|table|configs|kvcopy|cprank`) write the cp_merge sweep, the measured prefill-time
-table over (new_len, prefix_len, C), the per-config numbers and the paged KV copy bandwidth as JSON
-lines to `--out`.
+Other modes (`--mode merge|table|configs|kvcopy|cprank|cachemgr|cpu`) write the cp_merge sweep, the measured
+prefill-time table over (new_len, prefix_len, C), the per-config numbers, the paged KV copy bandwidth, one CP rank's
+local time, the cache-manager throughput and the oracle's full passes over whole configurations as JSON lines to
+`--out`.
 
 `--impl reference` times the CPU fp64 oracle (host cores) on a bounded sample of the same workload.
 """
@@ -108,7 +109,7 @@ class ClockSampler:
             self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "power_w_median": None, "power_w_max": None}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -116,7 +117,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, smax, reasons = [], [], set()
+        sm, smax, power, reasons = [], [], [], set()
         try:
             for line in open(self.path):
                 f = [x.strip() for x in line.split(",")]
@@ -127,6 +128,10 @@ class ClockSampler:
                     smax.append(float(f[2]))
                 except ValueError:
                     continue
+                try:
+                    power.append(float(f[3]))
+                except ValueError:
+                    pass
                 for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                     if val.lower().startswith("active"):
                         reasons.add(name)
@@ -135,6 +140,8 @@ class ClockSampler:
             pass
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+        if power:
+            out.update(power_w_median=statistics.median(power), power_w_max=max(power))
         return out
 
 
@@ -358,6 +365,7 @@ def sustained_leg(torch, runner, peaks, device, seconds=2.2):
     tf = flops_of(runner.w) / (ms * 1e-3) / 1e12
     return {"workload": runner.w.name, "steps": steps, "gpu_seconds": total_ms * 1e-3, "ms_per_step": ms, "tflops": tf,
             "sm_mhz_median": clocks["sm_mhz"], "ms_x_mhz": ms * clocks["sm_mhz"] if clocks["sm_mhz"] else None,
+            "power_w_median": clocks["power_w_median"],
             "frac": fractions(tf, peaks), "clocks": clocks}
 
 
@@ -564,6 +572,27 @@ def cpu_baseline_legs(headline, headline_mat, args):
                        "seconds_at_T4096_scaled": dt * 4096 / T})
     base["merge_oracle"] = merges
     return base
+
+
+def run_cpu_full(args, out):
+    """The oracle as it stands over WHOLE configurations (every row, every head) on the host cores: what the bounded
+    `cpu_baseline` legs extrapolate to.  Minutes of CPU time for the larger configurations; no GPU is used."""
+    from oracle import reference as orc
+    orc.build()
+    threads = orc.host_threads()
+    for cfg in args.configs:
+        w = get_workload(cfg)
+        mat = wl.materialize(w)
+        t0 = time.perf_counter()
+        for b, r in enumerate(w.requests):
+            q = mat.q[w.cu_new[b]:w.cu_new[b + 1]]
+            pt = mat.page_table[w.cu_pages[b]:w.cu_pages[b + 1]]
+            orc.attn_full(q, mat.k_pages, mat.v_pages, pt, r.prefix_len, w.Hkv, w.scale, n_threads=threads)
+        dt = time.perf_counter() - t0
+        out.write(json.dumps({"mode": "cpu_full", "config": cfg, "workload": w.name, "threads": threads, "nproc": os.cpu_count(),
+                              "cpu_model": cpu_model(), "seconds": dt, "gflops_equivalent": flops_of(w) / dt / 1e9,
+                              "tokens_per_s": w.total_new / dt, "pairs": pairs_of(w)}) + "\n")
+        out.flush()
 
 
 def run_reference(args):
@@ -979,7 +1008,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="number of the configuration used as the headline workload")
-    ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table", "kvcopy", "cprank", "cachemgr"])
+    ap.add_argument("--mode", default="bench", choices=["bench", "configs", "merge", "table", "kvcopy", "cprank", "cachemgr", "cpu"])
     ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5],
                     help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P; 8: multi-head (16/16)")
     ap.add_argument("--config-ms", type=float, default=1200.0, help="configs mode: GPU time per configuration")
@@ -1004,7 +1033,7 @@ def main():
     if args.mode == "bench":
         return run_ours(args)
     out = open(args.out, "w") if args.out else sys.stdout
-    {"configs": run_configs, "merge": run_merge_sweep, "table": run_table, "kvcopy": run_kvcopy, "cprank": run_cprank, "cachemgr": run_cachemgr}[args.mode](args, out)
+    {"configs": run_configs, "merge": run_merge_sweep, "table": run_table, "kvcopy": run_kvcopy, "cprank": run_cprank, "cachemgr": run_cachemgr, "cpu": run_cpu_full}[args.mode](args, out)
 
 
 if __name__ == "__main__":
