@@ -10,6 +10,7 @@
 //   warps 0-3  softmax warpgroup for head 0 of the pair (tile-pair units: rows 0-127): one thread per query row
 //   warps 4-7  softmax warpgroup for head 1 (tile-pair units: rows 128-255)
 //   warp  8    TMA producer (the warp prefetches page ids; the pages of a tile go out from several lanes)
+//              (with 16-token pages the spare warp copies the second 64-dim half of every K/V tile)
 //   warp  9    tcgen05.mma issuer for the scores S = Q K^T (warp-uniform loop, one elected lane issues)
 //   warp  10   tcgen05.mma issuer for O += P V
 //   warp  11   spare (completes the third warpgroup so that register budgets can be moved: the softmax
@@ -129,6 +130,7 @@ struct AttnParams {
     const float* q_scale;
     const float* k_scale;
     const float* v_scale;
+    int32_t co_producer;      // 1: the spare warp copies the second 64-dim half of every K/V tile (16-token pages, bf16)
 };
 
 // ------------------------------------------------------------------------------------------
@@ -414,16 +416,23 @@ __device__ __forceinline__ bool fetch_unit(const AttnParams& p, const InlineSche
 // ------------------------------------------------------------------------------------------
 // Roles
 // ------------------------------------------------------------------------------------------
+// half_lo, half_hi: the 64-dim halves of every K/V tile this warp copies.  Normally warp 8 copies both; with
+// 16-token pages (sixteen 2 KB boxes per tile, whose issue cost a single warp cannot hide) the spare warp takes
+// the second half as a co-producer: it waits for the same "slot empty" phases, while the byte count of a tile is
+// announced once, by the leading warp (a copy that lands before the announcement only leaves the barrier's byte
+// count negative for a moment; the phase cannot complete before the announcing arrival).
 template <bool kFp8>
 __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV, const AttnParams& p,
-                              const InlineSched& inl, uint32_t smem_base, volatile uint32_t* abort_flag) {
+                              const InlineSched& inl, uint32_t smem_base, volatile uint32_t* abort_flag, int half_lo,
+                              int half_hi) {
     const int lane = threadIdx.x & 31;
     const uint32_t bars = smem_base + kSmemBar;
+    const bool lead = half_lo == 0;
     uint32_t kv_it = 0;   // ring slots filled so far
     for (int round = 0;; ++round) {
         UnitInfo u;
         if (!fetch_unit(p, inl, round, u)) break;
-        if (lane == 0) {
+        if (lane == 0 && lead) {
             mbar_wait(bars, kBarQEmpty, (round & 1) ^ 1, abort_flag, p.status, round);
             const uint32_t qbar = bars + kBarQFull * 8;
             mbar_expect_tx(qbar, 2 * (kFp8 ? kTileBytes8 : kTileBytes));
@@ -468,14 +477,14 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmQ, const CUte
             const CUtensorMap* map = kv ? tmV : tmK;
             if (lane == 0) {
                 mbar_wait(bars, kBarKvEmpty + slot, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, j);
-                mbar_expect_tx(fbar, kFp8 ? kTileBytes8 : kTileBytes);
+                if (lead) mbar_expect_tx(fbar, kFp8 ? kTileBytes8 : kTileBytes);
             }
             __syncwarp();
-            // lane i < ppt copies page i of the tile: both 64-dim halves of its box
+            // lane i < ppt copies page i of the tile: this warp's 64-dim halves of its box (one-byte tiles have one)
             const int page = __shfl_sync(0xffffffffu, my_page, (pg0 - pg_base + (lane < ppt ? lane : 0)) & 31);
             if (lane < ppt) {
-                tma_load_4d(dst + lane * box_bytes, map, fbar, 0, u.kv_head, 0, page);
-                if (!kFp8) tma_load_4d(dst + kHalfBytes + lane * box_bytes, map, fbar, 64, u.kv_head, 0, page);
+                for (int half = half_lo; half < (kFp8 ? 1 : half_hi); ++half)
+                    tma_load_4d(dst + half * kHalfBytes + lane * box_bytes, map, fbar, half * 64, u.kv_head, 0, page);
             }
             __syncwarp();
             ++kv_it;
@@ -998,13 +1007,15 @@ cp_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
         if (warp == 8) {
-            producer_role<kFp8>(&tmQ, &tmK, &tmV, p, inl, smem_base, abort_flag);
+            producer_role<kFp8>(&tmQ, &tmK, &tmV, p, inl, smem_base, abort_flag, 0, p.co_producer ? 1 : 2);
         } else if (warp == 9) {
             mma_s_role<kFp8>(p, inl, smem_base, tmem_base, abort_flag);
         } else if (warp == 10) {
             mma_pv_role<kFp8>(p, inl, smem_base, tmem_base, abort_flag);
         } else if (p.n_fill > 0) {
             fill_role(p);
+        } else if (!kFp8 && p.co_producer) {
+            producer_role<kFp8>(&tmQ, &tmK, &tmV, p, inl, smem_base, abort_flag, 1, 2);
         }
     }
 
@@ -1499,6 +1510,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     p.q_scale = cache8 ? q_scale : nullptr;
     p.k_scale = cache8 ? cache8->k_scale : nullptr;
     p.v_scale = cache8 ? cache8->v_scale : nullptr;
+    p.co_producer = (!cache8 && cache->page_size == 16 && n_fill == 0) ? 1 : 0;
     if (cache8) cp_attn_kernel<true><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
     else cp_attn_kernel<false><<<grid, kThreads, kSmemAlloc, s>>>(tmQ, tmK, tmV, p, *inl);
     if (int rc = check_cuda(cudaGetLastError(), who)) return rc;
@@ -1799,6 +1811,7 @@ extern "C" int cp_prefill_attn_static(const void* q, const cp_kv_cache* cache, c
     p.inl_items = p.inl_cta_off = p.inl_pieces = -1;
     p.n_fill = 0;
     p.q_scale = p.k_scale = p.v_scale = nullptr;
+    p.co_producer = cache->page_size == 16 ? 1 : 0;
     InlineSched none;          // unused: the tile list is in the scratch
     none.bytes[0] = 0;
     const int64_t units = n_tiles * p.pairs_per_tile;
