@@ -70,3 +70,50 @@ def test_reference_arm_runs_on_rank0_only():
     assert out.returncode == 0
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_flop_accounting_follows_eq1_and_timed_loop_marks():
+    # the benchmark's flop numerator is Eq. (1) summed over the batch; the sparse event marks of very short steps
+    # still bracket exactly `steps` steps
+    sys.path.insert(0, ROOT)
+    import bench
+    from oracle import reference as orc
+    from paper_2609_04774_b200 import workloads as wl
+    for cfg in (1, 2, 4, 5):
+        w = bench.get_workload(cfg)
+        assert bench.pairs_of(w) == sum(orc.remaining_workload(r.new_len, r.prefix_len) for r in w.requests)
+        assert bench.flops_of(w) == 4 * 128 * w.Hq * bench.pairs_of(w)
+    assert bench.pairs_of(wl.config2()) == 58722304 and bench.flops_of(wl.config3()) == 4 * 128 * 32 * 8590000128
+
+    class FakeEvent:
+        clock = 0.0
+
+        def __init__(self, enable_timing=True):
+            self.t = None
+
+        def record(self):
+            self.t = FakeEvent.clock
+
+        def elapsed_time(self, other):
+            return other.t - self.t
+
+    class FakeCuda:
+        Event = FakeEvent
+
+        @staticmethod
+        def synchronize():
+            pass
+
+    class FakeTorch:
+        cuda = FakeCuda
+
+    calls = []
+
+    def step():
+        calls.append(1)
+        FakeEvent.clock += 2.0
+
+    total, per = bench.timed_loop(FakeTorch, step, 37, 3, stride=16)
+    assert len(calls) == 40 and total == 74.0 and per == [2.0, 2.0, 2.0]
+    total, per = bench.timed_loop(FakeTorch, step, 5, 0)
+    assert total == 10.0 and per == [2.0] * 5
