@@ -2,8 +2,10 @@
 
 Bit-exact: the query codes and scales the library's pre-pass leaves in the workspace, and the bytes written by
 cp_kv_append_fp8.  Attention: LSE as in the bf16 path; O element by element within the bound the format gives
-for rounding the softmax weights to E4M3, 2^-4 * sum_j p_j |v_j| (the oracle returns that sum), plus 4e-3 for
-fp32 accumulation and the bf16 rounding of the output; per-row relative L2 error at most 2^-4."""
+for rounding the softmax weights to E4M3 (round to nearest: at most 2^-4 of each weight), 2^-4 * A with
+A = sum_j p_j |v_j| (the oracle returns it), plus 2^-8 * A for the bf16 rounding of the output (|O| <= A, half an
+ulp is 2^-9 of the value) and 1e-3 for the fp32 accumulation; per-row relative L2 error at most 2^-4 (expected
+2^-4 / sqrt(3) * 0.75 = 0.027 for independent rounding errors)."""
 import numpy as np
 import pytest
 import torch
@@ -66,7 +68,7 @@ def compare8(out, lse, ref_o, ref_l, ref_a, what):
     assert np.isfinite(out).all() and np.isfinite(lse).all(), what
     le = np.abs(lse - ref_l) / np.maximum(1.0, np.abs(ref_l))
     assert le.max() <= 1e-3, (what, "lse", le.max())
-    excess = np.abs(out - ref_o) - (2.0 ** -4 * ref_a + 4e-3)
+    excess = np.abs(out - ref_o) - ((2.0 ** -4 + 2.0 ** -8) * ref_a + 1e-3)
     assert excess.max() <= 0, (what, "element bound exceeded by", excess.max())
     num = np.sqrt(((out - ref_o) ** 2).sum(-1))
     den = np.sqrt((ref_o ** 2).sum(-1)) + 1e-30

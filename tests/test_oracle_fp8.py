@@ -115,6 +115,9 @@ def test_fp8_attention_equals_bf16_oracle_on_values_both_formats_hold(shape):
     assert np.abs(o - ro).max() <= 1e-12 * max(1.0, np.abs(ro).max())
     assert np.abs(l - rl).max() <= 1e-12 * max(1.0, np.abs(rl).max())
     assert (a >= np.abs(o) - 1e-12).all()                                     # |sum p v| <= sum p |v|
+    # with the sign bits of V cleared the weighted mean of |v| is the output itself
+    o2, _, a2 = o8.attn_fp8_rows(q_bits, k8, v8 & 0x7F, ks, vs, pt, P, Hkv, 0.11, rows)
+    assert np.abs(o2 - a2).max() <= 1e-13 * max(1.0, a2.max()) and np.abs(a2 - a).max() <= 1e-13 * max(1.0, a.max())
 
 
 def test_fp8_attention_closed_forms_and_scale_identities():
