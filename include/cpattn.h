@@ -19,6 +19,11 @@
  *     met by a paged copy) are recorded in a status word that cp_ctx_poll_status() reads after the
  *     caller has synchronised.
  *   - bf16 tensors are passed as void*; element strides are in elements.
+ *   - Stream capture: an attention call with a cp_ctx whose work lists ride in the launch parameters
+ *     (cp_schedule_inspect reports it; up to 24 KB of lists, i.e. a few hundred work units) reads no host
+ *     memory after it returns and may be captured into a CUDA graph and replayed; a call with a larger
+ *     schedule stages its lists through the context's pinned buffers, which later calls reuse, and must not
+ *     be replayed.  cp_merge and the paged copies take everything by value and may be captured.
  */
 #ifndef CPATTN_H
 #define CPATTN_H

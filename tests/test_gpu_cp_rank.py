@@ -165,3 +165,55 @@ def test_nccl_communicator_world_size_one():
     got = q.get(timeout=600)
     p.join(timeout=120)
     assert got == "ok"
+
+
+def test_rank_step_replays_from_a_cuda_graph():
+    # a rank step whose chunk calls carry their work lists in the launch parameters reads no host memory after the
+    # calls return, so the whole step (gathers, segment appends, both chunk attention calls) can be captured once and
+    # replayed per layer: the replay must reproduce the eager results bit for bit, also after the inputs have changed
+    # in place
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from cp_rank_util import ThreadFabric, rank_inputs
+    from paper_2609_04774_b200 import binding
+    from paper_2609_04774_b200.cp_rank import CpRankWorker, LibraryOps, RankLayout
+    R, P, C = 1000, 640, 1
+    w = wl.Workload("cp_rank_graph", 64, 8, 2, [wl.Request(R, P, C)])
+    mat = wl.materialize(w)
+    lay = RankLayout(R, P, C, 0)
+    for j in (lay.early, lay.late):
+        b, e = lay.chunk(j)
+        info, _, _ = binding.cp_schedule_inspect([0, e - b], [P + b], [1], w.Hq, w.Hkv,
+                                                 torch.cuda.get_device_properties(0).multi_processor_count, want_lists=False)
+        assert info["inline"] == 1
+    k_pages, v_pages, page_table, rows = rank_inputs(mat, lay, 64)
+    ops = LibraryOps(binding.Context(0), _dev(k_pages), _dev(v_pages), torch.from_numpy(page_table).cuda(), w.Hq, w.scale)
+    t = {k: _dev(x) for k, x in rows.items()}
+    worker = CpRankWorker(lay, ThreadFabric(1).comm(0), ops)
+    run = lambda: worker.prefill(t["q_early"], t["q_late"], t["k_early"], t["v_early"], t["k_late"], t["v_late"])
+    eager = [x.clone() for x in run()]
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        run()                                               # warm-up on a side stream, as graph capture wants
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        captured = run()
+    graph.replay()
+    torch.cuda.synchronize()
+    ops.ctx.poll_status()
+    for a, b in zip(eager, captured):
+        assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a, b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
+    ref = orc.attn_full(mat.q, mat.k_pages, mat.v_pages, mat.page_table, P, w.Hkv, w.scale)
+    _check_rank_on_gpu(w, mat, lay, tuple(captured) + (ops.k_pages, ops.v_pages, page_table), ref)
+    # new queries in the same buffers: the replay computes on them
+    t["q_early"].copy_(torch.flip(t["q_early"], dims=[2]))
+    graph.replay()
+    torch.cuda.synchronize()
+    replayed = [x.clone() for x in captured]
+    again = [x.clone() for x in run()]
+    torch.cuda.synchronize()
+    assert torch.equal(replayed[0].view(torch.int16), again[0].view(torch.int16)) and torch.equal(replayed[1], again[1])
+    assert not torch.equal(replayed[0].view(torch.int16), eager[0].view(torch.int16))
