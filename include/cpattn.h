@@ -22,8 +22,8 @@
  *   - Stream capture: an attention call with a cp_ctx whose work lists ride in the launch parameters
  *     (cp_schedule_inspect reports it; up to 24 KB of lists, i.e. a few hundred work units) reads no host
  *     memory after it returns and may be captured into a CUDA graph and replayed; a call with a larger
- *     schedule stages its lists through the context's pinned buffers, which later calls reuse, and must not
- *     be replayed.  cp_merge and the paged copies take everything by value and may be captured.
+ *     schedule stages its lists through the context's pinned buffers, which later calls reuse: such a
+ *     call on a capturing stream returns CP_ERR_UNSUPPORTED and enqueues nothing.  cp_merge and the paged copies take everything by value and may be captured.
  */
 #ifndef CPATTN_H
 #define CPATTN_H

@@ -1416,8 +1416,14 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
             lay.pieces = ilay.pieces - base;
             lay.merges = ilay.merges - base;
             lay.merge_slots = ilay.merge_slots - base;
-        } else if (int rc = upload_block(ctx, big, ws + lay.items, s)) {
-            return rc;
+        } else {
+            // the staged upload reads a pinned buffer that later calls reuse: a captured copy would replay stale lists
+            cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+            if (int rc = check_cuda(cudaStreamIsCapturing(s, &cap), "cudaStreamIsCapturing")) return rc;
+            if (cap != cudaStreamCaptureStatusNone)
+                return set_error(CP_ERR_UNSUPPORTED, "%s: the work lists (%zu bytes) do not fit the launch parameters (%zu); "
+                                 "a call of this size cannot be captured into a CUDA graph", who, big.size(), kInlineSchedBytes);
+            if (int rc = upload_block(ctx, big, ws + lay.items, s)) return rc;
         }
         grid = sch.grid;
         n_items = (int32_t)sch.items.size();

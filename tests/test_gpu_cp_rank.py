@@ -217,3 +217,36 @@ def test_rank_step_replays_from_a_cuda_graph():
     torch.cuda.synchronize()
     assert torch.equal(replayed[0].view(torch.int16), again[0].view(torch.int16)) and torch.equal(replayed[1], again[1])
     assert not torch.equal(replayed[0].view(torch.int16), eager[0].view(torch.int16))
+
+
+def test_large_schedule_refuses_capture():
+    # a call whose work lists do not fit the launch parameters stages them through pinned buffers; on a capturing
+    # stream it must refuse (nothing enqueued) instead of recording a copy that would replay stale lists
+    from paper_2609_04774_b200 import binding
+    R = 40000
+    w = wl.Workload("big_sched", 65, 8, 2, [wl.Request(R, 0, 1)])
+    info, _, _ = binding.cp_schedule_inspect([0, R], [0], [1], w.Hq, w.Hkv,
+                                             torch.cuda.get_device_properties(0).multi_processor_count, want_lists=False)
+    assert info["inline"] == 0
+    ctx = binding.Context(0)
+    pages = -(-R // 64)
+    k = torch.zeros((pages, 64, w.Hkv, 128), dtype=torch.bfloat16, device="cuda")
+    cache = binding.make_cache(k, k)
+    pt = torch.arange(pages, dtype=torch.int32, device="cuda")
+    q = torch.zeros((R, w.Hq, 128), dtype=torch.bfloat16, device="cuda")
+    out = torch.full_like(q, float("nan"))
+    lse = torch.empty((w.Hq, R), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(binding.cp_workspace_bytes([R], [1], w.Hq), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with pytest.raises(binding.CpError) as e:
+        with torch.cuda.graph(graph):
+            binding.cp_prefill_attn(ctx, q, cache, pt, 0, R, 1, w.Hq, w.scale, out, lse, ws)
+    assert e.value.code == binding.CP_ERR_UNSUPPORTED and "captured" in str(e.value)
+    torch.cuda.synchronize()
+    assert bool(torch.isnan(out.float()).all())             # nothing ran
+    binding.cp_prefill_attn(ctx, q, cache, pt, 0, R, 1, w.Hq, w.scale, out, lse, ws)      # outside capture it runs
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    assert not bool(torch.isnan(out.float()).any())
+    ctx.close()
