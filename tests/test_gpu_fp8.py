@@ -162,6 +162,41 @@ def test_fp8_attention_odd_group_sizes(ctx):
     check_batch8(ctx, wl.Workload("fp8_mha", 57, 4, 4, [wl.Request(700, 64, 4), wl.Request(90, 3000, 1)]))
 
 
+def test_fp8_strided_cache_view_and_tile_pair_splits(ctx):
+    # the FP8 cache as a view into a wider allocation (an unused head slot per token, an unused token row per page);
+    # then single-head units with prefixes long enough for KV cuts
+    w = wl.Workload("fp8_strided", 59, 8, 2, [wl.Request(300, 200, 2), wl.Request(90, 0, 1)])
+    m8 = wl.materialize_fp8(w)
+    dev = Device8(m8)
+    npg = m8.k8_pages.shape[0]
+    big_k = torch.full((npg, wl.PAGE + 1, w.Hkv + 1, w.D), 0x7E, dtype=torch.uint8, device="cuda")
+    big_v = torch.full_like(big_k, 0xFE)
+    big_k[:, :wl.PAGE, :w.Hkv] = dev.k8
+    big_v[:, :wl.PAGE, :w.Hkv] = dev.v8
+    dev.k8, dev.v8 = big_k[:, :wl.PAGE, :w.Hkv], big_v[:, :wl.PAGE, :w.Hkv]
+    dev.cache = binding.make_cache_fp8(dev.k8, dev.v8, dev.ks, dev.vs)
+    assert dev.cache.stride_tok == (w.Hkv + 1) * w.D and dev.cache.stride_page == (wl.PAGE + 1) * (w.Hkv + 1) * w.D
+    out, lse = dev.run(ctx)
+    for b, r in enumerate(w.requests):
+        lo, hi = int(w.cu_new[b]), int(w.cu_new[b + 1])
+        pt = m8.page_table[w.cu_pages[b]:w.cu_pages[b + 1]]
+        ro, rl, ra = o8.attn_fp8_rows(m8.q[lo:hi], m8.k8_pages, m8.v8_pages, m8.k_scale, m8.v_scale, pt, r.prefix_len, w.Hkv,
+                                      w.scale, np.arange(r.new_len))
+        compare8(out[lo:hi], lse[:, lo:hi], ro, rl, ra, "fp8 strided req %d" % b)
+    # quantising append through the same view
+    newk = wl.normal_bf16(60, wl.TID_K, (64, w.Hkv, w.D))
+    binding.cp_kv_append_fp8(ctx, dev.cache, dev.page_table, 10, 64, bits_to_bf16(newk), None)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    kc = o8.quantize_kv(newk, m8.k_scale)
+    t = np.arange(10, 74)
+    got = dev.k8.cpu().numpy()[m8.page_table[t // wl.PAGE], t % wl.PAGE]
+    assert np.array_equal(o8.e4m3_decode(got), o8.e4m3_decode(kc))
+    assert bool((big_k[:, wl.PAGE] == 0x7E).all()) and bool((big_k[:, :, w.Hkv] == 0x7E).all())     # nothing outside the view
+    reqs = [wl.Request(128, 30000, 1), wl.Request(257, 5003, 3), wl.Request(1, 40001, 1)]
+    check_batch8(ctx, wl.Workload("fp8_pair_split", 61, 6, 2, reqs), rows_per_request=40)
+
+
 def test_fp8_shard_chunk_and_key_range_calls(ctx):
     # one request through the three partial forms of the variant: the C shard partials and a set of key-range
     # partials each merge (cp_merge) into the oracle's full result; every chunk call reproduces its rows

@@ -185,6 +185,30 @@ def test_attention_odd_group_sizes(ctx):
     check_batch(ctx, wl.Workload("mha", 42, 4, 4, [wl.Request(700, 64, 4)]))
 
 
+def test_attention_tile_pair_edges(ctx):
+    # single-head units (three heads per KV head; plain multi-head) over pairs of query tiles: requests of exactly
+    # one tile, one row more, two tiles, two tiles and a row, a single row; long prefixes so that the units are cut
+    # along KV (a piece may lie wholly behind the earlier tile's causal limit); unaligned prefixes
+    reqs = [wl.Request(128, 40000, 1), wl.Request(129, 5003, 2), wl.Request(256, 0, 1), wl.Request(257, 64, 3),
+            wl.Request(1, 70001, 1), wl.Request(385, 20000, 4)]
+    for name, heads in (("pair_g3", (6, 2)), ("pair_mha", (4, 4))):
+        w = wl.Workload(name, 49, heads[0], heads[1], reqs)
+        info, _, _ = binding.cp_schedule_inspect(w.cu_new, [r.prefix_len for r in reqs], [r.C for r in reqs], w.Hq, w.Hkv,
+                                                 torch.cuda.get_device_properties(0).multi_processor_count, want_lists=False)
+        assert info["split_units"] > 0
+        dev, out, lse, _ = check_batch(ctx, w, pair_budget=4e7)
+        o1, l1 = dev.out.clone(), dev.lse.clone()
+        dev.run_batch(ctx)
+        assert torch.equal(o1.view(torch.int16), dev.out.view(torch.int16)) and torch.equal(l1, dev.lse)
+
+
+def test_attention_many_small_requests(ctx):
+    # forty requests of 3 to 42 new tokens behind 0, 64 or 128 cached ones: every tile is ragged, most units one KV tile
+    reqs = [wl.Request(3 + i, 64 * (i % 3), 1 + i % 4) for i in range(40)]
+    check_batch(ctx, wl.Workload("many_small", 50, 8, 2, reqs))
+    check_batch(ctx, wl.Workload("many_small_mha", 50, 2, 2, reqs))
+
+
 def test_attention_kv_split_units(ctx):
     # few query rows, long prefixes: every unit is cut along KV over many CTAs and merged by the fix-up
     # kernel; prefix lengths that are not page multiples; a request whose rows see no key of some piece
