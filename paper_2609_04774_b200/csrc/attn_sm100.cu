@@ -1077,10 +1077,12 @@ struct FixupParams {
     int32_t inl_items, inl_merges, inl_merge_slots;   // >= 0: the list sits at this byte offset of the launch-parameter copy
 };
 
-constexpr int kFixupRowsPerBlock = 16;    // 8 warps x 2 (head, row) combinations
+constexpr int kFixupRowsPerBlock = 8;     // one (head, row) combination per warp
 
-// grid = (split units, 256 / kFixupRowsPerBlock): each warp combines two rows; the partial LSEs of a
-// row are loaded 32 slots at a time (lane k holds slot k), max and sum by warp shuffles.
+// grid = (split units, 256 / kFixupRowsPerBlock): each warp combines one row.  The partial LSEs of the row are
+// loaded 32 slots at a time (lane k holds slot k), max and sum by warp shuffles; units cut into at most 32 pieces
+// (all but pathological schedules) read every LSE once.  The partial rows are fetched four at a time, all loads
+// issued before the first use.
 __global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p, const __grid_constant__ InlineSched inl) {
     const TileItem* items = p.inl_items >= 0 ? reinterpret_cast<const TileItem*>(inl.bytes + p.inl_items) : p.items;
     const MergeEntry* merges = p.inl_merges >= 0 ? reinterpret_cast<const MergeEntry*>(inl.bytes + p.inl_merges) : p.merges;
@@ -1089,66 +1091,80 @@ __global__ void __launch_bounds__(256) cp_attn_fixup_kernel(const FixupParams p,
     const TileItem it = items[me.item];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int r2 = 0; r2 < 2; ++r2) {
-        const int hr = blockIdx.y * kFixupRowsPerBlock + warp * 2 + r2;
-        const int wg = hr / kBlockM;                  // head wg of the pair, or (tile-pair unit) rows 128 wg .. of the one head
-        const int row = hr - wg * kBlockM;
-        const int urow = p.heads_per_unit == 2 ? row : hr;     // row inside the unit
-        if (urow >= it.n_rows) continue;
-        // pass 1: max of the partial LSEs (lane k of each group of 32 slots holds slot k)
-        float m = -INFINITY;
-        for (int base = 0; base < me.n_slots; base += 32) {
-            if (base + lane < me.n_slots) {
-                const int slot = merge_slots[me.slot_off + base + lane];
-                m = fmaxf(m, p.partial_lse[((int64_t)slot * 2 + wg) * kBlockM + row]);
-            }
+    const int hr = blockIdx.y * kFixupRowsPerBlock + warp;
+    const int wg = hr / kBlockM;                  // head wg of the pair, or (tile-pair unit) rows 128 wg .. of the one head
+    const int row = hr - wg * kBlockM;
+    const int urow = p.heads_per_unit == 2 ? row : hr;     // row inside the unit
+    if (urow >= it.n_rows) return;
+    // pass 1: max of the partial LSEs (lane k of each group of 32 slots holds slot k)
+    float m = -INFINITY;
+    int slot0 = 0;
+    float lse0 = -INFINITY;        // the first group's values stay in registers for pass 2
+    for (int base = 0; base < me.n_slots; base += 32) {
+        if (base + lane < me.n_slots) {
+            const int slot = merge_slots[me.slot_off + base + lane];
+            const float v = p.partial_lse[((int64_t)slot * 2 + wg) * kBlockM + row];
+            if (base == 0) { slot0 = slot; lse0 = v; }
+            m = fmaxf(m, v);
         }
+    }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        // pass 2: weights exp(lse_k - m) and the weighted sum of the partial rows
-        float wsum = 0.f;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int base = 0; base < me.n_slots; base += 32) {
-            int my_slot = 0;
-            float w_mine = 0.f;
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    // pass 2: weights exp(lse_k - m) and the weighted sum of the partial rows
+    float wsum = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int base = 0; base < me.n_slots; base += 32) {
+        int my_slot = slot0;
+        float my_lse = lse0;
+        if (base > 0) {
+            my_lse = -INFINITY;
             if (base + lane < me.n_slots) {
                 my_slot = merge_slots[me.slot_off + base + lane];
-                const float my_lse = p.partial_lse[((int64_t)my_slot * 2 + wg) * kBlockM + row];
-                w_mine = (my_lse == -INFINITY) ? 0.f : __expf(my_lse - m);
-            }
-            wsum += w_mine;
-            const int cnt = min(32, me.n_slots - base);
-            for (int k = 0; k < cnt; ++k) {
-                const float w = __shfl_sync(0xffffffffu, w_mine, k);
-                const int slot = __shfl_sync(0xffffffffu, my_slot, k);
-                if (w > 0.f) {     // a zero weight hides whatever the slot holds for this row
-                    const float4 x = reinterpret_cast<const float4*>(p.partial_o + (((int64_t)slot * 2 + wg) * kBlockM + row) * kD)[lane];
-                    acc.x = fmaf(w, x.x, acc.x);
-                    acc.y = fmaf(w, x.y, acc.y);
-                    acc.z = fmaf(w, x.z, acc.z);
-                    acc.w = fmaf(w, x.w, acc.w);
-                }
+                my_lse = p.partial_lse[((int64_t)my_slot * 2 + wg) * kBlockM + row];
             }
         }
+        const float w_mine = (my_lse == -INFINITY) ? 0.f : __expf(my_lse - m);
+        wsum += w_mine;
+        const int cnt = min(32, me.n_slots - base);
+        for (int k0 = 0; k0 < cnt; k0 += 4) {
+            float w[4];
+            float4 x[4];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
-        // a row may see none of the unit's keys (a key range that starts behind its causal limit): zeros, -inf
-        const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
-        const int head = p.heads_per_unit == 2 ? 2 * me.pair + wg : me.pair;
-        const int64_t grow = (int64_t)it.q_row0 + urow;
-        const int64_t off = (grow * p.Hq + head) * kD + lane * 4;
-        if (p.out_f32) {
-            *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off) =
-                make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-        } else {
-            uint2 pk;
-            pk.x = pack_bf16(acc.x * inv, acc.y * inv);
-            pk.y = pack_bf16(acc.z * inv, acc.w * inv);
-            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off) = pk;
+            for (int k = 0; k < 4; ++k) {
+                // lanes beyond the group hold weight 0; their slot index (0 or a real one) is a valid slot to read
+                w[k] = __shfl_sync(0xffffffffu, w_mine, (k0 + k) & 31);
+                const int slot = __shfl_sync(0xffffffffu, my_slot, (k0 + k) & 31);
+                x[k] = (k0 + k < cnt && w[k] > 0.f)
+                           ? reinterpret_cast<const float4*>(p.partial_o + (((int64_t)slot * 2 + wg) * kBlockM + row) * kD)[lane]
+                           : make_float4(0.f, 0.f, 0.f, 0.f);     // a zero weight hides whatever the slot holds for this row
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float wk = (k0 + k < cnt) ? w[k] : 0.f;
+                acc.x = fmaf(wk, x[k].x, acc.x);
+                acc.y = fmaf(wk, x[k].y, acc.y);
+                acc.z = fmaf(wk, x[k].z, acc.z);
+                acc.w = fmaf(wk, x[k].w, acc.w);
+            }
         }
-        if (lane == 0) p.lse[(int64_t)head * p.lse_stride + grow] = wsum > 0.f ? m + __logf(wsum) : -INFINITY;
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+    // a row may see none of the unit's keys (a key range that starts behind its causal limit): zeros, -inf
+    const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
+    const int head = p.heads_per_unit == 2 ? 2 * me.pair + wg : me.pair;
+    const int64_t grow = (int64_t)it.q_row0 + urow;
+    const int64_t off = (grow * p.Hq + head) * kD + lane * 4;
+    if (p.out_f32) {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off) =
+            make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+    } else {
+        uint2 pk;
+        pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+        pk.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off) = pk;
+    }
+    if (lane == 0) p.lse[(int64_t)head * p.lse_stride + grow] = wsum > 0.f ? m + __logf(wsum) : -INFINITY;
 }
 
 // ------------------------------------------------------------------------------------------
