@@ -873,7 +873,7 @@ def run_cprank(args, out):
     bandwidth are printed beside the measured local time."""
     import torch
     from paper_2609_04774_b200 import binding, build
-    from paper_2609_04774_b200.cp_rank import CpRankWorker, LibraryOps, RankLayout
+    from paper_2609_04774_b200.cp_rank import CpRankWorker, LibraryOps, LibraryOps8, RankLayout
     build.build()
     D = 128
     for cfg in args.configs:
@@ -883,10 +883,16 @@ def run_cprank(args, out):
         r = w.requests[0]
         R, P, C = r.new_len, r.prefix_len, r.C
         n_pages = r.n_pages
-        k = torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
-        v = torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
         pt = torch.from_numpy(wl.permutation(w.seed, wl.TID_PERM, n_pages)).cuda()
-        ops = LibraryOps(binding.Context(0), k, v, pt, w.Hq, w.scale)
+        if args.fp8:      # E4M3 pages (finite codes), per-head scales shared by all ranks; stored bytes travel
+            k = (torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda") * 70).to(torch.float8_e4m3fn).view(torch.uint8)
+            v = (torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda") * 70).to(torch.float8_e4m3fn).view(torch.uint8)
+            sc = torch.full((w.Hkv,), 6.0 / 448.0, dtype=torch.float32, device="cuda")
+            ops = LibraryOps8(binding.Context(0), k, v, sc, sc.clone(), pt, w.Hq, w.scale)
+        else:
+            k = torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
+            v = torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
+            ops = LibraryOps(binding.Context(0), k, v, pt, w.Hq, w.scale)
         per_rank, per_rank_graph = [], []
         for rank in range(C):
             lay = RankLayout(R, P, C, rank)
@@ -942,8 +948,8 @@ def run_cprank(args, out):
         if args.pass_q:   # queries in (bf16), partials of the own rows back (fp32 + lse)
             recv = (C - 1) * 2 * lay0.cl * w.Hq * (D * 2 + D * 4 + 4)
         else:             # K and V of the other ranks' prefix blocks and chunks
-            recv = (C - 1) * 2 * 2 * w.Hkv * D * (lay0.block_pages * wl.PAGE + 2 * lay0.cl)
-        out.write(json.dumps({"mode": "cprank", "exchange": "pass-q" if args.pass_q else "all-gather-kv", "config": cfg, "workload": w.name, "R": R, "P": P, "C": C,
+            recv = (C - 1) * 2 * (1 if args.fp8 else 2) * w.Hkv * D * (lay0.block_pages * wl.PAGE + 2 * lay0.cl)
+        out.write(json.dumps({"mode": "cprank", "exchange": "pass-q" if args.pass_q else ("all-gather-kv, fp8 bytes" if args.fp8 else "all-gather-kv"), "config": cfg, "workload": w.name, "R": R, "P": P, "C": C,
                               "rank_local_ms": per_rank, "slowest_rank_ms": max(per_rank),
                               "rank_local_ms_graph_replay": per_rank_graph,
                               "tflops_per_gpu_slowest_rank": flops_of(w) / C / (max(per_rank) * 1e-3) / 1e12,
@@ -1019,7 +1025,7 @@ def main():
     ap.add_argument("--configs", type=int, nargs="*", default=[1, 2, 3, 4, 5],
                     help="1-5: the benchmark configurations; 6: 32/4 grouped-query head shape; 7: chunked prefill, R << P; 8: multi-head (16/16)")
     ap.add_argument("--config-ms", type=float, default=1200.0, help="configs mode: GPU time per configuration")
-    ap.add_argument("--fp8", action="store_true", help="configs mode: the FP8 K/V variant of each configuration")
+    ap.add_argument("--fp8", action="store_true", help="configs / cprank modes: the FP8 K/V variant")
     ap.add_argument("--page", type=int, default=None, help="configs mode: tokens per cache page (16, 32, 64, 128)")
     ap.add_argument("--rank-reps", type=int, default=5)
     ap.add_argument("--pass-q", action="store_true", help="cprank mode: K/V stays sharded, queries travel")

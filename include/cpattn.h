@@ -357,6 +357,15 @@ int cp_prefill_attn_fp8_kvrange(cp_ctx* ctx, const void* q, const cp_kv_cache_fp
                                 size_t workspace_bytes, void* stream);
 int cp_kv_append_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,
                      int64_t n, const void* k_rows, const void* v_rows, void* stream);
+/* Raw byte copies of an FP8 cache, no conversion: cp_kv_gather_fp8 reads n logical tokens from t_begin into
+ * k_bytes / v_bytes (device [n, Hkv, D] E4M3 bytes); cp_kv_append_segments_fp8 writes runs of such rows like
+ * cp_kv_append_segments.  For the exchange between CP ranks whose caches share the per-head scales: the stored
+ * bytes travel (half of what bf16 rows cost on the link) and are appended as they are.  Bit-exact; page ids are
+ * checked as in cp_kv_append.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+int cp_kv_gather_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,
+                     int64_t n, void* k_bytes, void* v_bytes, void* stream);
+int cp_kv_append_segments_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int32_t n_segments,
+                              const cp_kv_segment* segments, const void* k_bytes, const void* v_bytes, void* stream);
 
 #ifdef __cplusplus
 }

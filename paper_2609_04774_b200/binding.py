@@ -23,7 +23,7 @@ EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "c
            "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_chunk", "cp_prefill_attn_kvrange", "cp_prefill_attn_static", "cp_merge",
            "cp_kv_gather", "cp_kv_append", "cp_workspace_bytes_fp8", "cp_prefill_attn_fp8", "cp_prefill_attn_fp8_batch",
            "cp_kv_append_fp8", "cp_kv_append_segments", "cp_prefill_attn_fp8_shard", "cp_prefill_attn_fp8_chunk",
-           "cp_prefill_attn_fp8_kvrange"]
+           "cp_prefill_attn_fp8_kvrange", "cp_kv_gather_fp8", "cp_kv_append_segments_fp8"]
 
 
 class CpError(RuntimeError):
@@ -336,3 +336,16 @@ def cp_kv_append_fp8(ctx, cache, page_table, t_begin, n, k_rows, v_rows, stream=
     """bf16 rows [n, Hkv, D] -> E4M3 bytes of logical tokens t_begin.. of the FP8 cache (per-head scales)."""
     _check(load().cp_kv_append_fp8(ctx._h, ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(t_begin),
                                    ctypes.c_int64(n), _ptr(k_rows), _ptr(v_rows), _stream(stream)))
+
+
+def cp_kv_gather_fp8(ctx, cache, page_table, t_begin, n, k_bytes, v_bytes, stream=None):
+    """Raw E4M3 bytes of logical tokens [t_begin, t_begin + n) -> k_bytes / v_bytes [n, Hkv, D] uint8."""
+    _check(load().cp_kv_gather_fp8(ctx._h, ctypes.byref(cache), _ptr(page_table), ctypes.c_int64(t_begin),
+                                   ctypes.c_int64(n), _ptr(k_bytes), _ptr(v_bytes), _stream(stream)))
+
+
+def cp_kv_append_segments_fp8(ctx, cache, page_table, segments, k_bytes, v_bytes, stream=None):
+    """cp_kv_append_segments for an FP8 cache: rows of stored bytes, copied as they are."""
+    seg = np.ascontiguousarray(np.asarray(list(segments), dtype=np.int64).reshape(-1, 3))
+    _check(load().cp_kv_append_segments_fp8(ctx._h, ctypes.byref(cache), _ptr(page_table), ctypes.c_int32(seg.shape[0]),
+                                            _hp(seg), _ptr(k_bytes), _ptr(v_bytes), _stream(stream)))

@@ -21,6 +21,10 @@ ranges, a local cp_merge of those partials, an all-to-all that returns every row
 owns the row, and a final cp_merge over the C partials.  It moves R*Hq*D query bytes plus fp32 partials
 instead of (P+R)*Hkv*D*2 key/value bytes, which pays when the cached prefix is much longer than the suffix.
 
+With an FP8 cache (LibraryOps8) the exchange carries the stored E4M3 bytes: a rank first writes its own new K/V
+into its cache through the quantising append, reads the bytes back as its contribution, and appends the other ranks'
+bytes as they are (all ranks share the per-head scales), so the link carries half of what bf16 rows cost.
+
 Readings (the paper fixes none of these): prefix pages are owned in contiguous blocks of
 ceil(n_prefix_pages / C) pages, block r on rank r; the prefix length is a multiple of the page size
 (block-granular reuse, Section 7.1); chunks are padded to cl = ceil(R / 2C) rows for the collective.
@@ -159,11 +163,22 @@ class LibraryOps:
 
     def buffer(self, name, shape, dtype=None):
         """A device buffer that lives as long as this object (allocated and zeroed on first use): the staging
-        arenas, send buffers and outputs of a rank step are reused from layer to layer."""
+        arenas, send buffers and outputs of a rank step are reused from layer to layer.  Default type: that of the
+        rows on the wire."""
+        dtype = dtype or self.wire_dtype
         key = (name, tuple(shape), dtype)
         if key not in self._buffers:
-            self._buffers[key] = self.torch.zeros(tuple(shape), dtype=dtype or self.torch.bfloat16, device=self.device)
+            self._buffers[key] = self.torch.zeros(tuple(shape), dtype=dtype, device=self.device)
         return self._buffers[key]
+
+    @property
+    def wire_dtype(self):
+        """Element type of K/V rows as they travel between ranks and sit in the arenas."""
+        return self.torch.bfloat16
+
+    def to_wire(self, name, t_begin, k_rows, v_rows):
+        """This rank's new K/V rows (bf16, logical tokens t_begin..) in the form they travel in: as they are."""
+        return k_rows, v_rows
 
     def kv_append_segments(self, segments, k_rows, v_rows):
         segments = [s for s in segments if s[1] > 0]
@@ -180,7 +195,7 @@ class LibraryOps:
 
     def attn_chunk(self, lay: RankLayout, chunk, q_chunk):
         n = q_chunk.shape[0]
-        out = self.buffer("out_%d" % chunk, (n, self.Hq, self.D))
+        out = self.buffer("out_%d" % chunk, (n, self.Hq, self.D), self.torch.bfloat16)
         lse = self.buffer("lse_%d" % chunk, (self.Hq, n), self.torch.float32)
         if n == 0:
             return out, lse
@@ -189,6 +204,62 @@ class LibraryOps:
             self._ws = self.torch.empty(nbytes, dtype=self.torch.uint8, device=self.device)
         self.b.cp_prefill_attn_chunk(self.ctx, q_chunk, self.cache, self.page_table, lay.P, lay.R, lay.C, chunk,
                                      self.Hq, self.scale, out, lse, self._ws)
+        return out, lse
+
+
+class LibraryOps8(LibraryOps):
+    """The device steps of a rank on an FP8 K/V cache (E4M3 pages, one fp32 scale per KV head shared by all ranks)."""
+
+    def __init__(self, ctx, k8_pages, v8_pages, k_scale, v_scale, page_table, Hq, scale):
+        import torch
+        from . import binding
+        self.b, self.ctx, self.torch = binding, ctx, torch
+        self.cache = binding.make_cache_fp8(k8_pages, v8_pages, k_scale, v_scale)
+        self.k_pages, self.v_pages, self.page_table = k8_pages, v8_pages, page_table
+        self.k_scale, self.v_scale = k_scale, v_scale
+        self.Hq, self.scale = Hq, scale
+        self.Hkv, self.D = k8_pages.shape[2], k8_pages.shape[3]
+        self.device = k8_pages.device
+        self._ws = None
+        self._buffers = {}
+
+    @property
+    def wire_dtype(self):
+        return self.torch.uint8
+
+    def empty_rows(self, n, heads):
+        return self.torch.zeros((n, heads, self.D), dtype=self.torch.uint8, device=self.device)
+
+    def to_wire(self, name, t_begin, k_rows, v_rows):
+        """Quantise the rank's own new rows into its cache (they belong there anyway) and read the stored bytes
+        back: what the other ranks receive is exactly what this rank attends to."""
+        n = k_rows.shape[0]
+        kb, vb = self.buffer("wire_k_" + name, (n, self.Hkv, self.D)), self.buffer("wire_v_" + name, (n, self.Hkv, self.D))
+        if n > 0:
+            self.b.cp_kv_append_fp8(self.ctx, self.cache, self.page_table, t_begin, n, k_rows, v_rows)
+            self.b.cp_kv_gather_fp8(self.ctx, self.cache, self.page_table, t_begin, n, kb, vb)
+        return kb, vb
+
+    def kv_gather(self, t_begin, n, k_rows, v_rows):
+        if n > 0:
+            self.b.cp_kv_gather_fp8(self.ctx, self.cache, self.page_table, t_begin, n, k_rows, v_rows)
+
+    def kv_append_segments(self, segments, k_rows, v_rows):
+        segments = [s for s in segments if s[1] > 0]
+        if segments:
+            self.b.cp_kv_append_segments_fp8(self.ctx, self.cache, self.page_table, segments, k_rows, v_rows)
+
+    def attn_chunk(self, lay: RankLayout, chunk, q_chunk):
+        n = q_chunk.shape[0]
+        out = self.buffer("out_%d" % chunk, (n, self.Hq, self.D), self.torch.bfloat16)
+        lse = self.buffer("lse_%d" % chunk, (self.Hq, n), self.torch.float32)
+        if n == 0:
+            return out, lse
+        if self._ws is None:
+            nbytes = self.b.cp_workspace_bytes_fp8([lay.R], [lay.C], self.Hq)
+            self._ws = self.torch.empty(nbytes, dtype=self.torch.uint8, device=self.device)
+        self.b.cp_prefill_attn_fp8_chunk(self.ctx, q_chunk, self.cache, self.page_table, lay.P, lay.R, lay.C, chunk,
+                                         self.Hq, self.scale, out, lse, self._ws)
         return out, lse
 
 
@@ -271,6 +342,9 @@ class CpRankWorker:
             sk, sv = ops.buffer("send_prefix_k", (n_blk, ops.Hkv, ops.D)), ops.buffer("send_prefix_v", (n_blk, ops.Hkv, ops.D))
             ops.kv_gather(pb, pe - pb, sk, sv)
             hp = (comm.all_gather_into(ak[:off_e], sk), comm.all_gather_into(av[:off_e], sv))
+        if hasattr(ops, "to_wire"):       # an FP8 cache sends stored bytes; a bf16 cache the rows as they are
+            k_early, v_early = ops.to_wire("early", lay.P + eb, k_early, v_early)
+            k_late, v_late = ops.to_wire("late", lay.P + lb, k_late, v_late)
         he = (comm.all_gather_into(ak[off_e:off_l], _padded(ops, k_early, cl, "send_early_k")),
               comm.all_gather_into(av[off_e:off_l], _padded(ops, v_early, cl, "send_early_v")))
         hl = (comm.all_gather_into(ak[off_l:], _padded(ops, k_late, cl, "send_late_k")),

@@ -228,6 +228,67 @@ extern "C" int cp_kv_append_segments(cp_ctx* ctx, const cp_kv_cache* cache, cons
     return check_cuda(cudaGetLastError(), who);
 }
 
+// Raw byte copies of an FP8 cache (no conversion): the same kernels with one-byte elements, i.e. 8 vectors of 16
+// bytes per head row.  What a CP rank exchanges when the cache is FP8: stored bytes travel, and because all ranks
+// share the per-head scales they can be appended as they are.
+extern "C" int cp_kv_gather_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,
+                                int64_t n, void* k_bytes, void* v_bytes, void* stream) {
+    const char* who = "cp_kv_gather_fp8";
+    if (!ctx || !page_table || t_begin < 0 || n < 0)
+        return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or negative range", who);
+    if (int rc = validate_cache_fp8(cache, who)) return rc;
+    if (!k_bytes && !v_bytes) return set_error(CP_ERR_INVALID_ARG, "%s: both row pointers are NULL", who);
+    if (((uintptr_t)k_bytes | (uintptr_t)v_bytes) & 15)
+        return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
+    if (n == 0) return CP_OK;
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+    const int vec_per_head = cache->D / 16;
+    const int64_t total = n * cache->Hkv * vec_per_head;
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
+    kv_copy_kernel<false><<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        (uint4*)cache->k, (uint4*)cache->v, (uint4*)k_bytes, (uint4*)v_bytes, page_table, t_begin, n, cache->page_size,
+        cache->Hkv, vec_per_head, cache->stride_page / 16, cache->stride_tok / 16, cache->stride_head / 16, cache->num_pages,
+        ctx->d_status);
+    return check_cuda(cudaGetLastError(), who);
+}
+
+extern "C" int cp_kv_append_segments_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table,
+                                         int32_t n_segments, const cp_kv_segment* segments, const void* k_bytes,
+                                         const void* v_bytes, void* stream) {
+    const char* who = "cp_kv_append_segments_fp8";
+    if (!ctx || !page_table || !segments || n_segments < 0)
+        return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or negative segment count", who);
+    if (n_segments > kMaxSegments)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: %d segments, at most %d per call", who, n_segments, kMaxSegments);
+    if (int rc = validate_cache_fp8(cache, who)) return rc;
+    if (!k_bytes && !v_bytes) return set_error(CP_ERR_INVALID_ARG, "%s: both row pointers are NULL", who);
+    if (((uintptr_t)k_bytes | (uintptr_t)v_bytes) & 15)
+        return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
+    SegmentTable tab;
+    tab.n_segments = 0;
+    tab.cum[0] = 0;
+    for (int32_t i = 0; i < n_segments; ++i) {
+        const cp_kv_segment& sg = segments[i];
+        if (sg.t_begin < 0 || sg.n < 0 || sg.row0 < 0)
+            return set_error(CP_ERR_INVALID_ARG, "%s: segment %d has a negative field", who, i);
+        if (sg.n == 0) continue;
+        const int k = tab.n_segments++;
+        tab.t_begin[k] = sg.t_begin;
+        tab.row0[k] = sg.row0;
+        tab.cum[k + 1] = tab.cum[k] + sg.n;
+    }
+    if (tab.n_segments == 0) return CP_OK;
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+    const int vec_per_head = cache->D / 16;
+    const int64_t total = tab.cum[tab.n_segments] * cache->Hkv * vec_per_head;
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
+    kv_append_segments_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        (uint4*)cache->k, (uint4*)cache->v, (const uint4*)k_bytes, (const uint4*)v_bytes, page_table, tab, cache->page_size,
+        cache->Hkv, vec_per_head, cache->stride_page / 16, cache->stride_tok / 16, cache->stride_head / 16, cache->num_pages,
+        ctx->d_status);
+    return check_cuda(cudaGetLastError(), who);
+}
+
 extern "C" int cp_kv_append_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,
                                 int64_t n, const void* k_rows, const void* v_rows, void* stream) {
     const char* who = "cp_kv_append_fp8";

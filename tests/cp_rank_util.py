@@ -116,6 +116,74 @@ class OracleOps:
         return torch.zeros(tuple(shape), dtype=torch.float64)
 
 
+class OracleOps8(OracleOps):
+    """The same steps on E4M3 byte pools with per-head scales, through the FP8 oracle."""
+
+    def __init__(self, k8_pages, v8_pages, k_scale, v_scale, page_table, Hq, scale):
+        super().__init__(k8_pages, v8_pages, page_table, Hq, scale)
+        self.k_scale, self.v_scale = k_scale, v_scale
+
+    def empty_rows(self, n, heads):
+        return torch.zeros((n, heads, self.D), dtype=torch.uint8)
+
+    def buffer(self, name, shape, dtype=None):
+        self._buffers = getattr(self, "_buffers", {})
+        key = (name, tuple(shape))
+        if key not in self._buffers:
+            self._buffers[key] = torch.zeros(tuple(shape), dtype=torch.uint8)
+        return self._buffers[key]
+
+    @staticmethod
+    def _bits(t):
+        return t.contiguous().numpy()
+
+    def to_wire(self, name, t_begin, k_rows, v_rows):
+        from oracle import fp8 as o8
+        kc = o8.quantize_kv(k_rows.contiguous().numpy().view(np.uint16), self.k_scale)
+        vc = o8.quantize_kv(v_rows.contiguous().numpy().view(np.uint16), self.v_scale)
+        if kc.shape[0]:
+            orc.kv_append(self.k_pages, self.page_table, t_begin, kc)
+            orc.kv_append(self.v_pages, self.page_table, t_begin, vc)
+        return torch.from_numpy(kc), torch.from_numpy(vc)
+
+    def kv_gather(self, t_begin, n, k_rows, v_rows):
+        if n > 0:
+            k_rows[:n] = torch.from_numpy(orc.kv_gather(self.k_pages, self.page_table, t_begin, t_begin + n))
+            v_rows[:n] = torch.from_numpy(orc.kv_gather(self.v_pages, self.page_table, t_begin, t_begin + n))
+
+    def attn_chunk(self, lay, chunk, q_chunk):
+        from oracle import fp8 as o8
+        b, e = lay.chunk(chunk)
+        q = np.zeros((lay.R, self.Hq, self.D), dtype=np.uint16)
+        q[b:e] = q_chunk.contiguous().numpy().view(np.uint16)
+        if e == b:
+            return np.zeros((0, self.Hq, self.D)), np.zeros((self.Hq, 0))
+        o, l, _ = o8.attn_fp8_rows(q, self.k_pages, self.v_pages, self.k_scale, self.v_scale, self.page_table, lay.P, self.Hkv,
+                                   self.scale, np.arange(b, e))
+        return o, l
+
+
+def rank_inputs8(m8, mat, lay, seed):
+    """FP8 form of rank_inputs: the rank's own byte pool holds only its prefix block (the stored bytes of the seeded
+    request); its q / k / v rows are the bf16 rows the bytes were made from."""
+    pt_ref = m8.page_table
+    n_pages = len(pt_ref)
+    page_table = wl.permutation(seed + 100 * (lay.rank + 1), wl.TID_PERM, n_pages + 2)[:n_pages].astype(np.int32)
+    k_pages = np.zeros((n_pages + 2,) + m8.k8_pages.shape[1:], dtype=np.uint8)
+    v_pages = np.zeros_like(k_pages)
+    pb, pe = lay.prefix_block(lay.rank)
+    if pe > pb:
+        orc.kv_append(k_pages, page_table, pb, orc.kv_gather(m8.k8_pages, pt_ref, pb, pe))
+        orc.kv_append(v_pages, page_table, pb, orc.kv_gather(m8.v8_pages, pt_ref, pb, pe))
+    rows = {}
+    for name, j in (("early", lay.early), ("late", lay.late)):
+        b, e = lay.chunk(j)
+        rows["q_" + name] = mat.q[b:e]
+        rows["k_" + name] = orc.kv_gather(mat.k_pages, mat.page_table, lay.P + b, lay.P + e)
+        rows["v_" + name] = orc.kv_gather(mat.v_pages, mat.page_table, lay.P + b, lay.P + e)
+    return k_pages, v_pages, page_table, rows
+
+
 def rank_inputs(mat, lay, seed):
     """What rank `lay.rank` starts with, cut from the seeded full request: an empty page pool of its own
     (its own page permutation) holding only the rank's prefix block, and the rank's q/k/v rows."""

@@ -152,3 +152,49 @@ def test_two_gloo_ranks():
     for p in procs:
         p.join(timeout=60)
     assert got == [(0, "ok"), (1, "ok")]
+
+
+@pytest.mark.parametrize("R,P,C", [(333, 192, 4), (5, 0, 4), (200, 320, 3)])
+def test_four_ranks_in_process_fp8_cache(R, P, C):
+    # the same exchange with FP8 caches: stored bytes travel, every rank's cache ends up holding the whole request's
+    # bytes, and each chunk's result is the FP8 oracle's on those bytes
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from cp_rank_util import OracleOps8, ThreadFabric, rank_inputs8
+    from oracle import fp8 as o8
+    w = wl.Workload("cp_rank8", 53, 4, 2, [wl.Request(R, P, C)])
+    m8, mat = wl.materialize_fp8(w), wl.materialize(w)
+    fabric = ThreadFabric(C)
+    result, errors = {}, []
+
+    def body(k):
+        try:
+            lay = RankLayout(R, P, C, k)
+            k_pages, v_pages, page_table, rows = rank_inputs8(m8, mat, lay, 53)
+            ops = OracleOps8(k_pages, v_pages, m8.k_scale, m8.v_scale, page_table, w.Hq, w.scale)
+            t = {n: torch.from_numpy(np.ascontiguousarray(v).view(np.int16)) for n, v in rows.items()}
+            out = CpRankWorker(lay, fabric.comm(k), ops).prefill(t["q_early"], t["q_late"], t["k_early"], t["v_early"],
+                                                                   t["k_late"], t["v_late"])
+            result[k] = out + (k_pages, v_pages, page_table)
+        except Exception as e:
+            errors.append(e)
+            fabric.barrier.abort()
+
+    threads = [threading.Thread(target=body, args=(k,)) for k in range(C)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=300)
+    assert not errors, errors
+    ref_o, ref_l, _ = o8.attn_fp8_rows(m8.q, m8.k8_pages, m8.v8_pages, m8.k_scale, m8.v_scale, m8.page_table, P, w.Hkv, w.scale,
+                                       np.arange(R))
+    L = P + R
+    for k in range(C):
+        lay = RankLayout(R, P, C, k)
+        out_e, lse_e, out_l, lse_l, k_pages, v_pages, page_table = result[k]
+        for j, o, l in ((lay.early, out_e, lse_e), (lay.late, out_l, lse_l)):
+            b, e = lay.chunk(j)
+            if e > b:
+                assert np.abs(o - ref_o[b:e]).max() < 1e-12 and np.abs(l - ref_l[:, b:e]).max() < 1e-12
+        for got, ref in ((k_pages, m8.k8_pages), (v_pages, m8.v8_pages)):
+            a = o8.e4m3_decode(orc.kv_gather(got, page_table, 0, L))
+            assert np.array_equal(a, o8.e4m3_decode(orc.kv_gather(ref, m8.page_table, 0, L)))

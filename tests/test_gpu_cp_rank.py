@@ -250,3 +250,59 @@ def test_large_schedule_refuses_capture():
     ctx.poll_status()
     assert not bool(torch.isnan(out.float()).any())
     ctx.close()
+
+
+@pytest.mark.parametrize("R,P,C", [(1500, 640, 4), (333, 192, 3), (5, 0, 4)])
+def test_ranks_as_threads_on_one_gpu_fp8_cache(R, P, C):
+    # the rank worker on FP8 caches with the library's kernels: quantising append of the own rows, raw byte gathers,
+    # raw segment appends, FP8 chunk attention; results within the FP8 variant's bound of the oracle on the stored
+    # bytes, and every rank's cache holds the whole request's bytes afterwards
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from cp_rank_util import ThreadFabric, rank_inputs8
+    from oracle import fp8 as o8
+    from paper_2609_04774_b200 import binding
+    from paper_2609_04774_b200.cp_rank import CpRankWorker, LibraryOps8, RankLayout
+    from tests.test_gpu_fp8 import compare8
+    w = wl.Workload("cp_rank_gpu8", 66, 8, 2, [wl.Request(R, P, C)])
+    m8, mat = wl.materialize_fp8(w), wl.materialize(w)
+    ro, rl, ra = o8.attn_fp8_rows(m8.q, m8.k8_pages, m8.v8_pages, m8.k_scale, m8.v_scale, m8.page_table, P, w.Hkv, w.scale,
+                                  np.arange(R))
+    fabric = ThreadFabric(C)
+    result, errors = {}, []
+
+    def body(k):
+        try:
+            torch.cuda.set_device(0)
+            lay = RankLayout(R, P, C, k)
+            k_pages, v_pages, page_table, rows = rank_inputs8(m8, mat, lay, 66)
+            ops = LibraryOps8(binding.Context(0), torch.from_numpy(k_pages).cuda(), torch.from_numpy(v_pages).cuda(),
+                              torch.from_numpy(m8.k_scale).cuda(), torch.from_numpy(m8.v_scale).cuda(),
+                              torch.from_numpy(page_table).cuda(), w.Hq, w.scale)
+            t = {n: _dev(x) for n, x in rows.items()}
+            out = CpRankWorker(lay, fabric.comm(k), ops).prefill(t["q_early"], t["q_late"], t["k_early"], t["v_early"],
+                                                                   t["k_late"], t["v_late"])
+            torch.cuda.synchronize()
+            ops.ctx.poll_status()
+            result[k] = tuple(x.clone() for x in out) + (ops.k_pages.cpu().numpy(), ops.v_pages.cpu().numpy(), page_table)
+        except Exception as e:
+            errors.append(e)
+            fabric.barrier.abort()
+
+    threads = [threading.Thread(target=body, args=(k,)) for k in range(C)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=600)
+    assert not errors, errors
+    L = P + R
+    for k in range(C):
+        lay = RankLayout(R, P, C, k)
+        out_e, lse_e, out_l, lse_l, k_pages, v_pages, page_table = result[k]
+        for j, o, l in ((lay.early, out_e, lse_e), (lay.late, out_l, lse_l)):
+            b, e = lay.chunk(j)
+            assert o.shape[0] == e - b
+            if e > b:
+                compare8(_f64(o), _f64(l), ro[b:e], rl[:, b:e], ra[b:e], "fp8 rank %d chunk %d" % (k, j))
+        for got, ref in ((k_pages, m8.k8_pages), (v_pages, m8.v8_pages)):
+            assert np.array_equal(o8.e4m3_decode(orc.kv_gather(got, page_table, 0, L)),
+                                  o8.e4m3_decode(orc.kv_gather(ref, m8.page_table, 0, L)))
