@@ -278,6 +278,21 @@ def _library_extras():
                                        self.scale, part, lse, self._ws)
         return part, lse
 
+    def attn_kvranges(self, lay, q_full, ranges):
+        """All R queries against each of the key ranges: partials written straight into one stacked, persistent
+        buffer (parts [n, R, Hq, D] fp32, lses [n, Hq, R]), ready for cp_merge."""
+        torch = self.torch
+        R, n = lay.R, len(ranges)
+        parts = self.buffer("kvr_parts", (n, R, self.Hq, self.D), torch.float32)
+        lses = self.buffer("kvr_lses", (n, self.Hq, R), torch.float32)
+        if self._ws is None:
+            nbytes = self.b.cp_workspace_bytes([lay.R], [lay.C], self.Hq)
+            self._ws = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        for i, (lo, hi) in enumerate(ranges):
+            self.b.cp_prefill_attn_kvrange(self.ctx, q_full, self.cache, self.page_table, lay.P, R, lo, hi, self.Hq,
+                                           self.scale, parts[i], lses[i], self._ws)
+        return parts, lses
+
     def merge(self, parts, lses, final):
         """parts [N, T, Hq, D] fp32, lses [N, Hq, T] -> (out [T, Hq, D] bf16 if final else fp32, lse [Hq, T])."""
         torch = self.torch
@@ -292,6 +307,7 @@ def _library_extras():
         return self.torch.zeros(tuple(shape), dtype=self.torch.float32, device=self.device)
 
     LibraryOps.attn_kvrange, LibraryOps.merge, LibraryOps.empty_f32 = attn_kvrange, merge, empty_f32
+    LibraryOps.attn_kvranges = attn_kvranges
 
 
 _library_extras()
@@ -379,6 +395,15 @@ class CpRankWorker:
         out_l, lse_l = ops.attn_chunk(lay, lay.late, q_late)
         return out_e, lse_e, out_l, lse_l
 
+    def _return_index(self, like):
+        """The send-buffer row index as a tensor on the device of `like` (built once per worker)."""
+        import torch
+        if getattr(self, "_ret_idx", None) is None:
+            idx, pad = _return_index_of(self.lay)
+            self._ret_idx = torch.tensor(idx, dtype=torch.long, device=like.device)
+            self._ret_pad = torch.tensor(pad, dtype=torch.bool, device=like.device) if any(pad) else None
+        return self._ret_idx, self._ret_pad
+
     def prefill_pass_q(self, q_early, q_late, k_early, v_early, k_late, v_late):
         """Same inputs and outputs as prefill(), but the K/V never leaves its rank: the rank's cache must hold
         its prefix block; its own chunks' K/V are appended here, nothing else is ever read from the cache."""
@@ -394,33 +419,36 @@ class CpRankWorker:
         ops.kv_append(lay.P + lb, le - lb, k_late, v_late)
         he.wait()
         hl.wait()
+        # rank order is token order for the early chunks; the late chunks arrive in reverse (rank r sent chunk 2C-1-r)
         q_full = ops.empty_rows(lay.R, Hq)
         n_first = min(lay.R, lay.C * lay.cl)
         q_full[:n_first] = ge.reshape((-1,) + tuple(ge.shape[2:]))[:n_first]
-        for r in range(lay.C):
-            b, e = lay.chunk(lay.late_chunk_of(r))
-            q_full[b:e] = gl[r][:e - b]
+        if lay.R > n_first:
+            late = gl.flip(0).reshape((-1,) + tuple(gl.shape[2:]))      # chunks C, C+1, ... in order, cl rows each
+            q_full[n_first:] = late[:lay.R - n_first]
 
         # 3. partial attention of all queries over each of the rank's key ranges, merged locally
         pb, pe = lay.prefix_block(lay.rank)
         ranges = [(lo, hi) for lo, hi in ((pb, pe), (lay.P + eb, lay.P + ee), (lay.P + lb, lay.P + le)) if hi > lo]
-        parts = [ops.attn_kvrange(lay, q_full, lo, hi) for lo, hi in ranges]
-        if len(parts) == 1:
-            mine_o, mine_l = parts[0]
-        elif parts:
-            mine_o, mine_l = ops.merge(_stack([p for p, _ in parts]), _stack([l for _, l in parts]), final=False)
+        if ranges and hasattr(ops, "attn_kvranges"):
+            po, pl = ops.attn_kvranges(lay, q_full, ranges)             # stacked by the ops, no copies
+            mine_o, mine_l = (po[0], pl[0]) if len(ranges) == 1 else ops.merge(po, pl, final=False)
+        elif ranges:
+            parts = [ops.attn_kvrange(lay, q_full, lo, hi) for lo, hi in ranges]
+            mine_o, mine_l = parts[0] if len(parts) == 1 else \
+                ops.merge(_stack([p for p, _ in parts]), _stack([l for _, l in parts]), final=False)
         else:                                   # the rank holds no key at all (more ranks than blocks and chunks)
             mine_o = ops.empty_f32((lay.R, Hq, ops.D))
             mine_l = ops.empty_f32((Hq, lay.R)) - float("inf")
 
         # 4. every row's partial goes back to the rank that owns the row: block d = chunk d, then chunk 2C-1-d
-        send_o = ops.empty_f32((lay.C, 2 * lay.cl, Hq, ops.D))
-        send_l = ops.empty_f32((lay.C, Hq, 2 * lay.cl)) - float("inf")
-        for d in range(lay.C):
-            for half, j in enumerate((d, lay.late_chunk_of(d))):
-                b, e = lay.chunk(j)
-                send_o[d, half * lay.cl:half * lay.cl + e - b] = mine_o[b:e]
-                send_l[d, :, half * lay.cl:half * lay.cl + e - b] = mine_l[:, b:e]
+        #    (one gather by row index per tensor; rows of the padding take row 0's values and lse = -inf)
+        idx, pad = self._return_index(mine_l)
+        send_o = mine_o.index_select(0, idx).reshape((lay.C, 2 * lay.cl, Hq, ops.D))
+        send_l = mine_l.index_select(1, idx)
+        if pad is not None:
+            send_l = send_l.masked_fill(pad, float("-inf"))
+        send_l = send_l.reshape((Hq, lay.C, 2 * lay.cl)).transpose(0, 1).contiguous()
         (ro, ho), (rl, hl2) = comm.all_to_all(send_o), comm.all_to_all(send_l)
         ho.wait()
         hl2.wait()
@@ -429,6 +457,18 @@ class CpRankWorker:
         out, lse = ops.merge(ro, rl, final=True)
         n_e, n_l = ee - eb, le - lb
         return out[:n_e], lse[:, :n_e], out[lay.cl:lay.cl + n_l], lse[:, lay.cl:lay.cl + n_l]
+
+
+def _return_index_of(lay):
+    """Row index of the all-to-all's send buffer: block d holds chunk d, then chunk 2C-1-d, cl rows each; rows of the
+    padding point at row 0 and are flagged."""
+    idx, pad = [], []
+    for d in range(lay.C):
+        for j in (d, lay.late_chunk_of(d)):
+            b, e = lay.chunk(j)
+            idx += list(range(b, e)) + [0] * (lay.cl - (e - b))
+            pad += [False] * (e - b) + [True] * (lay.cl - (e - b))
+    return idx, pad
 
 
 def _stack(tensors):
