@@ -34,7 +34,7 @@ def _stale(target: str, deps) -> bool:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every source to an object in ``build/`` and link ``libcpattn.so``.  Returns its path."""
-    headers = [os.path.join(CSRC, "internal.h"), os.path.join(ROOT, "include", "cpattn.h"),
+    headers = [os.path.join(CSRC, "internal.h"), os.path.join(CSRC, "attn_kernel.cuh"), os.path.join(ROOT, "include", "cpattn.h"),
                os.path.join(ROOT, "include", "cpcache.h"), os.path.abspath(__file__)]
     objdir = os.path.join(_HERE, "build")
     os.makedirs(objdir, exist_ok=True)
