@@ -284,6 +284,13 @@ int cp_kv_gather(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_tabl
 int cp_kv_append(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int64_t t_begin,
                  int64_t n, const void* k_rows, const void* v_rows, void* stream);
 
+/* cp_check_page_table -- debug aid (the paper has no counterpart): enqueues a small kernel that compares every one of
+ * the n_entries of a device page table with the pool size.  The table is only read.  After the stream has been
+ * synchronised, cp_ctx_poll_status returns CP_ERR_BOUNDS with detail {code, index of the first bad entry found, block,
+ * its page id} if an entry lies outside [0, num_pages).  The attention calls never fault on such an entry (the page
+ * reads as zeros) and the copies skip it; this call is for finding it.  Errors: INVALID_ARG, CUDA. */
+int cp_check_page_table(cp_ctx* ctx, const int32_t* page_table, int64_t n_entries, int64_t num_pages, void* stream);
+
 /* cp_kv_append_segments -- cp_kv_append for several runs of rows in ONE launch: segment i writes rows
  * [row0, row0 + n) of k_rows / v_rows (device [*, Hkv, D] bf16) to logical tokens [t_begin, t_begin + n).  What a
  * CP rank needs after an all-gather of K and V (Section 2.1): the gathered blocks of the C ranks land at C

@@ -23,7 +23,7 @@ EXPORTS = ["cp_strerror", "cp_last_error", "cp_ctx_create", "cp_ctx_destroy", "c
            "cp_workspace_bytes", "cp_schedule_inspect", "cp_prefill_attn", "cp_prefill_attn_batch", "cp_prefill_attn_shard", "cp_prefill_attn_chunk", "cp_prefill_attn_kvrange", "cp_prefill_attn_static", "cp_merge",
            "cp_kv_gather", "cp_kv_append", "cp_workspace_bytes_fp8", "cp_prefill_attn_fp8", "cp_prefill_attn_fp8_batch",
            "cp_kv_append_fp8", "cp_kv_append_segments", "cp_prefill_attn_fp8_shard", "cp_prefill_attn_fp8_chunk",
-           "cp_prefill_attn_fp8_kvrange", "cp_kv_gather_fp8", "cp_kv_append_segments_fp8"]
+           "cp_prefill_attn_fp8_kvrange", "cp_kv_gather_fp8", "cp_kv_append_segments_fp8", "cp_check_page_table"]
 
 
 class CpError(RuntimeError):
@@ -349,3 +349,9 @@ def cp_kv_append_segments_fp8(ctx, cache, page_table, segments, k_bytes, v_bytes
     seg = np.ascontiguousarray(np.asarray(list(segments), dtype=np.int64).reshape(-1, 3))
     _check(load().cp_kv_append_segments_fp8(ctx._h, ctypes.byref(cache), _ptr(page_table), ctypes.c_int32(seg.shape[0]),
                                             _hp(seg), _ptr(k_bytes), _ptr(v_bytes), _stream(stream)))
+
+
+def cp_check_page_table(ctx, page_table, num_pages, stream=None):
+    """Enqueue the page-table check; a bad entry shows as CP_ERR_BOUNDS at the next poll_status() after a sync."""
+    _check(load().cp_check_page_table(ctx._h, _ptr(page_table), ctypes.c_int64(page_table.numel()),
+                                      ctypes.c_int64(num_pages), _stream(stream)))

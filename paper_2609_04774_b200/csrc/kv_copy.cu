@@ -104,6 +104,20 @@ kv_append_segments_kernel(uint4* __restrict__ paged_k, uint4* __restrict__ paged
     }
 }
 
+// Debug aid: every entry of a device page table against the pool size.  The table is only read, never used as an
+// address; the first entry outside [0, num_pages) lands in the status words {code, index, block, page id}.
+__global__ void __launch_bounds__(256)
+check_page_table_kernel(const int32_t* __restrict__ page_table, int64_t n, int64_t num_pages, int32_t* status) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t page = page_table[i];
+        if ((page < 0 || page >= num_pages) && atomicCAS(status, 0, CP_ERR_BOUNDS) == 0) {
+            status[1] = (int32_t)i;
+            status[2] = (int32_t)blockIdx.x;
+            status[3] = (int32_t)page;
+        }
+    }
+}
+
 // FP8 cache writer: eight bf16 values of a row -> eight E4M3 bytes, each e4m3_rne_satfinite(x / scale[g]) with
 // the quotient rounded to fp32 first.  Page ids outside the pool are skipped and reported like in the copies.
 __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d, float sc) {
@@ -231,6 +245,16 @@ extern "C" int cp_kv_append_segments(cp_ctx* ctx, const cp_kv_cache* cache, cons
 // Raw byte copies of an FP8 cache (no conversion): the same kernels with one-byte elements, i.e. 8 vectors of 16
 // bytes per head row.  What a CP rank exchanges when the cache is FP8: stored bytes travel, and because all ranks
 // share the per-head scales they can be appended as they are.
+extern "C" int cp_check_page_table(cp_ctx* ctx, const int32_t* page_table, int64_t n_entries, int64_t num_pages, void* stream) {
+    if (!ctx || !page_table || n_entries < 0 || num_pages < 1)
+        return set_error(CP_ERR_INVALID_ARG, "cp_check_page_table: null pointer, negative count or empty pool");
+    if (n_entries == 0) return CP_OK;
+    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+    const int blocks = (int)std::min<int64_t>((n_entries + 255) / 256, (int64_t)ctx->num_sms * 8);
+    check_page_table_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(page_table, n_entries, num_pages, ctx->d_status);
+    return check_cuda(cudaGetLastError(), "cp_check_page_table");
+}
+
 extern "C" int cp_kv_gather_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,
                                 int64_t n, void* k_bytes, void* v_bytes, void* stream) {
     const char* who = "cp_kv_gather_fp8";

@@ -150,6 +150,29 @@ def test_kv_append_segments_bit_exact(ctx):
     assert e.value.code == binding.CP_ERR_UNSUPPORTED
 
 
+def test_page_table_check_reports_bad_entries(ctx):
+    # the checker only reads the table: a good table passes, an entry beyond the pool (or negative) is reported with
+    # its index and value, and the context computes on afterwards
+    pt = torch.arange(1000, dtype=torch.int32, device="cuda")
+    binding.cp_check_page_table(ctx, pt, 1000)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    pt[617] = 1000
+    binding.cp_check_page_table(ctx, pt, 1000)
+    torch.cuda.synchronize()
+    with pytest.raises(binding.CpError) as e:
+        ctx.poll_status()
+    assert e.value.code == binding.CP_ERR_BOUNDS and "entry 617 holds page id 1000" in str(e.value)
+    pt[617] = -3
+    binding.cp_check_page_table(ctx, pt, 1000)
+    torch.cuda.synchronize()
+    with pytest.raises(binding.CpError) as e:
+        ctx.poll_status()
+    assert e.value.code == binding.CP_ERR_BOUNDS and "page id -3" in str(e.value)
+    ctx.poll_status()                                    # cleared
+    check_batch(ctx, wl.Workload("after_bounds", 51, 8, 2, [wl.Request(200, 64, 2)]))
+
+
 def test_attention_small_mixed_batch(ctx):
     dev, out, lse, _ = check_batch(ctx, wl.small_mixed())
     # run-to-run bitwise determinism
