@@ -165,10 +165,11 @@ int cp_schedule_inspect(int32_t B, const int64_t* cu_new, const int64_t* prefix_
  * Hq % Hkv == 0 (query head h uses KV head h / (Hq / Hkv)).  With an even group size a work unit is one
  * 128-row query tile for two query heads of a group, which share every K/V tile in shared memory; with an
  * odd one (e.g. Hq == Hkv) a unit is one head and two consecutive query tiles, which share the K/V tiles
- * the same way (measured on config 2's lengths: 1137 TFLOP/s with 16/16 heads against 1211 with 32/8).  One persistent launch computes all tiles; the few units that were split along KV
- * to balance the SMs are combined by a second small launch (an LSE merge of their partials).  Work lists of
- * up to 3 KB travel in the launch parameters; larger ones are first copied into the workspace by a small
- * kernel.  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ * the same way (measured on config 2's lengths: 1137 TFLOP/s with 16/16 heads against 1211 with 32/8).
+ * One persistent launch computes all tiles; the few units that were split along KV to balance the SMs are
+ * combined by a second small launch (an LSE merge of their partials).  Work lists of up to 24 KB travel in
+ * the launch parameters; larger ones are first copied into the workspace by a small kernel.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
  * ------------------------------------------------------------------------------------------- */
 int cp_prefill_attn(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int32_t* page_table,
                     int64_t prefix_len, int64_t new_len, int32_t C, int32_t Hq, float scale,
