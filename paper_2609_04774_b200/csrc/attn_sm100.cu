@@ -186,13 +186,15 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     // With schedule reuse on, a call whose schedule-relevant arguments and workspace equal the previous call's
     // (the next layer of the same batch) launches on the work lists that are already in the workspace.
-    uint64_t key = 0;
+    std::vector<int64_t> key;
     if (ctx->cache_on) {
-        key = 1469598103934665603ull;
-        auto mix = [&key](int64_t v) { key = (key ^ (uint64_t)v) * 1099511628211ull; };
-        mix(B); mix(Hq); mix(cache->Hkv); mix(cache->page_size); mix(only_shard); mix(only_chunk); mix(kv_lo); mix(kv_hi);
-        mix(grid_max); mix(out_f32); mix(want_fill); mix(cache8 != nullptr);
-        for (int32_t b = 0; b < B; ++b) { mix(cu_new[b + 1]); mix(prefix_len[b]); mix(C[b]); mix(cu_pages[b + 1]); }
+        key.reserve(14 + 4 * (size_t)B);
+        const int64_t head[] = {B, Hq, cache->Hkv, cache->page_size, only_shard, only_chunk, kv_lo, kv_hi,
+                                grid_max, out_f32, want_fill, cache8 != nullptr};
+        key.assign(head, head + sizeof head / sizeof head[0]);
+        for (int32_t b = 0; b < B; ++b) {
+            key.push_back(cu_new[b + 1]); key.push_back(prefix_len[b]); key.push_back(C[b]); key.push_back(cu_pages[b + 1]);
+        }
     }
     WorkspaceLayout lay;        // where the partial results (and the lists of a large schedule) sit in the workspace
     WorkspaceLayout ilay;       // offsets of the lists inside the launch-parameter copy of a small schedule
@@ -200,10 +202,11 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
     int32_t fill[2 * kMaxFillRanges] = {0};
     int64_t total_rows;
     bool inl_on = false;
+    bool fill_all = false;      // more uncovered row ranges than the kernel takes: a fill launch precedes the attention launch
     InlineSched inl_local;
     inl_local.bytes[0] = 0;
     const InlineSched* inl = &inl_local;
-    if (ctx->cache_on && ctx->cache_valid && ctx->cache_key == key && ctx->cache_ws == workspace) {
+    if (ctx->cache_on && ctx->cache_valid && ctx->cache_ws == workspace && ctx->cache_args == key) {
         lay = ctx->cache_lay;
         grid = ctx->cache_grid;
         n_items = ctx->cache_items;
@@ -213,6 +216,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         inl = &ctx->cache_inl;
         n_fill = ctx->cache_n_fill;
         memcpy(fill, ctx->cache_fill, sizeof fill);
+        fill_all = ctx->cache_fill_all;
     } else {
         ctx->cache_valid = false;
         Schedule sch;
@@ -231,7 +235,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
             int64_t gaps[2 * kMaxFillRanges];
             const int n = uncovered_rows(sch.items, total_rows, gaps, kMaxFillRanges);
             if (n > kMaxFillRanges) {     // more gaps than the kernel takes: fill everything first, in stream order
-                if (int rc = launch_fill_rows(static_cast<float*>(out), lse, total_rows, 0, total_rows, Hq, s)) return rc;
+                fill_all = true;
             } else {
                 n_fill = n;
                 for (int i = 0; i < 2 * n; ++i) fill[i] = (int32_t)gaps[i];
@@ -291,7 +295,7 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
         n_merges = (int32_t)sch.merges.size();
         if (ctx->cache_on) {
             ctx->cache_valid = true;
-            ctx->cache_key = key;
+            ctx->cache_args = std::move(key);
             ctx->cache_ws = workspace;
             ctx->cache_lay = lay;
             ctx->cache_grid = grid;
@@ -302,9 +306,12 @@ int attn_common(cp_ctx* ctx, const void* q, const cp_kv_cache* cache, const int3
             if (inl_on) memcpy(ctx->cache_inl.bytes, inl_local.bytes, kInlineSchedBytes);
             ctx->cache_n_fill = n_fill;
             memcpy(ctx->cache_fill, fill, sizeof fill);
+            ctx->cache_fill_all = fill_all;
         }
     }
 
+    if (fill_all)
+        if (int rc = launch_fill_rows(static_cast<float*>(out), lse, total_rows, 0, total_rows, Hq, s)) return rc;
     CUtensorMap tmQ, tmK, tmV;
     uint8_t* q8 = ws + base_ws;
     float* q_scale = reinterpret_cast<float*>(q8 + (size_t)total_rows * Hq * kD);

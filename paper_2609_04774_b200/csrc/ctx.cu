@@ -53,8 +53,7 @@ extern "C" int cp_ctx_create(cp_ctx** out, int device) {
     if (prop.major != 10)
         return set_error(CP_ERR_UNSUPPORTED, "cp_ctx_create: device is sm_%d%d, this library is sm_100a only",
                          prop.major, prop.minor);
-    cp_ctx* c = new cp_ctx();
-    memset(c, 0, sizeof *c);
+    cp_ctx* c = new cp_ctx();      // value-initialised: every plain member starts as zero
     c->device = device;
     c->num_sms = prop.multiProcessorCount;
     c->stage_bytes = 2u << 20;

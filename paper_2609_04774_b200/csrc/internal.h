@@ -133,7 +133,7 @@ struct cp_ctx {
     // schedule reuse (cp_ctx_cache_schedule): what the last attention call left in its workspace
     bool cache_on;
     bool cache_valid;
-    uint64_t cache_key;                // hash of every argument the schedule depends on
+    std::vector<int64_t> cache_args;   // every argument the schedule depends on, compared element by element
     const void* cache_ws;              // workspace the cached schedule lives in
     cpattn::WorkspaceLayout cache_lay;
     int32_t cache_grid, cache_items, cache_merges;
@@ -146,5 +146,6 @@ struct cp_ctx {
     bool cache_inline;                 // the remembered work lists travel in the launch parameters
     cpattn::InlineSched cache_inl;
     int32_t cache_n_fill;
+    bool cache_fill_all;
     int32_t cache_fill[2 * cpattn::kMaxFillRanges];
 };
