@@ -888,7 +888,7 @@ def run_cprank(args, out):
     bandwidth are printed beside the measured local time."""
     import torch
     from paper_2609_04774_b200 import binding, build
-    from paper_2609_04774_b200.cp_rank import CpRankWorker, LibraryOps, LibraryOps8, RankLayout
+    from paper_2609_04774_b200.cp_rank import CpRankWorker, LibraryOps, LibraryOps8, RankLayout, landing_pages
     build.build()
     D = 128
     for cfg in args.configs:
@@ -899,15 +899,21 @@ def run_cprank(args, out):
         R, P, C = r.new_len, r.prefix_len, r.C
         n_pages = r.n_pages
         pt = torch.from_numpy(wl.permutation(w.seed, wl.TID_PERM, n_pages)).cuda()
+        # landing mode (the default here when the chunks are whole pages): the gathers write into a run of pages behind
+        # the request's own pages and no append runs; --no-landing times the arena + append path
+        land_pages = landing_pages(RankLayout(R, P, C, 0))
+        a0 = None if args.no_landing else n_pages
+        pool = n_pages + land_pages
         if args.fp8:      # E4M3 pages (finite codes), per-head scales shared by all ranks; stored bytes travel
-            k = (torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda") * 70).to(torch.float8_e4m3fn).view(torch.uint8)
-            v = (torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda") * 70).to(torch.float8_e4m3fn).view(torch.uint8)
+            k = (torch.randn((pool, wl.PAGE, w.Hkv, D), device="cuda") * 70).to(torch.float8_e4m3fn).view(torch.uint8)
+            v = (torch.randn((pool, wl.PAGE, w.Hkv, D), device="cuda") * 70).to(torch.float8_e4m3fn).view(torch.uint8)
             sc = torch.full((w.Hkv,), 6.0 / 448.0, dtype=torch.float32, device="cuda")
-            ops = LibraryOps8(binding.Context(0), k, v, sc, sc.clone(), pt, w.Hq, w.scale)
+            ops = LibraryOps8(binding.Context(0), k, v, sc, sc.clone(), pt, w.Hq, w.scale, arena_page0=a0)
         else:
-            k = torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
-            v = torch.randn((n_pages, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
-            ops = LibraryOps(binding.Context(0), k, v, pt, w.Hq, w.scale)
+            k = torch.randn((pool, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
+            v = torch.randn((pool, wl.PAGE, w.Hkv, D), device="cuda").to(torch.bfloat16)
+            ops = LibraryOps(binding.Context(0), k, v, pt, w.Hq, w.scale, arena_page0=a0)
+        landed = ops.landing(RankLayout(R, P, C, 0)) is not None
         per_rank, per_rank_graph = [], []
         for rank in range(C):
             lay = RankLayout(R, P, C, rank)
@@ -964,7 +970,8 @@ def run_cprank(args, out):
             recv = (C - 1) * 2 * lay0.cl * w.Hq * (D * 2 + D * 4 + 4)
         else:             # K and V of the other ranks' prefix blocks and chunks
             recv = (C - 1) * 2 * (1 if args.fp8 else 2) * w.Hkv * D * (lay0.block_pages * wl.PAGE + 2 * lay0.cl)
-        out.write(json.dumps({"mode": "cprank", "exchange": "pass-q" if args.pass_q else ("all-gather-kv, fp8 bytes" if args.fp8 else "all-gather-kv"), "config": cfg, "workload": w.name, "R": R, "P": P, "C": C,
+        out.write(json.dumps({"mode": "cprank", "exchange": "pass-q" if args.pass_q else ("all-gather-kv, fp8 bytes" if args.fp8 else "all-gather-kv"),
+                              "landing": bool(landed and not args.pass_q), "config": cfg, "workload": w.name, "R": R, "P": P, "C": C,
                               "rank_local_ms": per_rank, "slowest_rank_ms": max(per_rank),
                               "rank_local_ms_graph_replay": per_rank_graph,
                               "tflops_per_gpu_slowest_rank": flops_of(w) / C / (max(per_rank) * 1e-3) / 1e12,
@@ -1044,6 +1051,8 @@ def main():
     ap.add_argument("--page", type=int, default=None, help="configs mode: tokens per cache page (16, 32, 64, 128)")
     ap.add_argument("--rank-reps", type=int, default=5)
     ap.add_argument("--pass-q", action="store_true", help="cprank mode: K/V stays sharded, queries travel")
+    ap.add_argument("--no-landing", action="store_true",
+                    help="cprank mode: gather into separate arenas and append into the cache instead of landing in pool pages")
     ap.add_argument("--cache-requests", type=int, default=20000)
     ap.add_argument("--merge-T", type=int, nargs="*", default=[4096, 16384, 65536, 262144])
     ap.add_argument("--merge-reps", type=int, default=20)

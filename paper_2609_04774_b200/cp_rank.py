@@ -15,6 +15,12 @@ step is five library launches (own prefix block read out, two appends, two atten
 KV-split units where the schedule cuts any.  Remote data is always copied into local HBM before a kernel reads
 it.  The module holds no arithmetic of the method: it moves rows and calls the library.
 
+Landing mode (LibraryOps(..., arena_page0=n)): when the chunks are whole pages (cl a multiple of the page size) and
+the caller sets aside a run of pages of the cache pool, the arenas ARE those pages: every gather writes into the
+pool, a page table built once per layout maps each logical token to the page its row landed in (prefix block r and
+early chunk r at rank r's slot, late chunk 2C-1-r at rank r's slot, i.e. in reverse token order), and the two append
+launches disappear: a rank step is the read-out of the own prefix block plus the two attention calls.
+
 A second mode, prefill_pass_q, keeps the K/V sharded (a rank holds its prefix block and the K/V of its own
 two chunks) and lets the queries travel: all-gather of Q, cp_prefill_attn_kvrange over each of the rank's key
 ranges, a local cp_merge of those partials, an all-to-all that returns every row's partials to the rank that
@@ -94,6 +100,39 @@ class RankLayout:
         return b, e
 
 
+def landing_rows(lay: RankLayout):
+    """Arena row of every logical token of the request when the gathers land in the layout
+    prefix blocks (C x n_blk rows) | early chunks (C x cl) | late chunks (C x cl), rank r's contribution at slot r:
+    a list of (token_begin, n_tokens, arena_row) runs covering [0, P + R), in token order."""
+    C, cl, n_blk = lay.C, lay.cl, lay.block_pages * lay.page
+    runs = []
+    if lay.P:
+        runs.append((0, lay.P, 0))                    # block r starts at token r * n_blk and at arena row r * n_blk
+    for j in range(2 * C):
+        b, e = lay.chunk(j)
+        if e > b:
+            slot = j if j < C else 2 * C - 1 - j      # early chunk j came from rank j, late chunk j from rank 2C-1-j
+            runs.append((lay.P + b, e - b, C * n_blk + (0 if j < C else C * cl) + slot * cl))
+    return runs
+
+
+def landing_table(lay: RankLayout, arena_page0: int):
+    """Page ids (one per page of [0, P + R)) that read the landed rows back in token order, or None when a chunk
+    does not start on a page boundary (cl not a multiple of the page size)."""
+    if lay.cl % lay.page:
+        return None
+    table = []
+    for t0, n, a0 in landing_rows(lay):
+        assert t0 % lay.page == 0 and a0 % lay.page == 0 and len(table) == t0 // lay.page
+        table += [arena_page0 + a0 // lay.page + i for i in range(-(-n // lay.page))]
+    return table
+
+
+def landing_pages(lay: RankLayout) -> int:
+    """Pages the landing arena takes in the pool."""
+    return lay.C * lay.block_pages + 2 * lay.C * (-(-lay.cl // lay.page))
+
+
 class TorchComm:
     """All-gather of equally sized row blocks over a torch.distributed group (NCCL on GPUs, gloo on CPU)."""
 
@@ -146,10 +185,11 @@ class TorchComm:
 class LibraryOps:
     """The three device steps of a rank, on this rank's paged cache, through the C-ABI library."""
 
-    def __init__(self, ctx, k_pages, v_pages, page_table, Hq, scale):
+    def __init__(self, ctx, k_pages, v_pages, page_table, Hq, scale, arena_page0=None):
         import torch
         from . import binding
         self.b, self.ctx, self.torch = binding, ctx, torch
+        self.arena_page0, self._landing = arena_page0, {}
         self.cache = binding.make_cache(k_pages, v_pages)
         self.k_pages, self.v_pages, self.page_table = k_pages, v_pages, page_table
         self.Hq, self.scale = Hq, scale
@@ -176,7 +216,26 @@ class LibraryOps:
         """Element type of K/V rows as they travel between ranks and sit in the arenas."""
         return self.torch.bfloat16
 
-    def to_wire(self, name, t_begin, k_rows, v_rows):
+    def landing(self, lay: RankLayout):
+        """Landing mode for this layout: (k_rows, v_rows, page_table) -- the arena as row views
+        [C * (n_blk + 2 cl), Hkv, D] of the pools' pages from arena_page0 on, and the device page table that reads
+        the landed rows in token order -- or None (no pages set aside, chunks not whole pages, pool not contiguous
+        or too small)."""
+        key = (lay.R, lay.P, lay.C, lay.rank, lay.page)
+        if key not in self._landing:
+            land = None
+            table = landing_table(lay, self.arena_page0) if self.arena_page0 is not None else None
+            n_pg = landing_pages(lay)
+            if (table is not None and lay.page == self.k_pages.shape[1] and self.k_pages.is_contiguous()
+                    and self.v_pages.is_contiguous() and self.arena_page0 + n_pg <= self.k_pages.shape[0]):
+                rows = n_pg * lay.page
+                kr = self.k_pages[self.arena_page0:self.arena_page0 + n_pg].view(rows, self.Hkv, self.D)
+                vr = self.v_pages[self.arena_page0:self.arena_page0 + n_pg].view(rows, self.Hkv, self.D)
+                land = (kr, vr, self.torch.tensor(table, dtype=self.torch.int32, device=self.device))
+            self._landing[key] = land
+        return self._landing[key]
+
+    def to_wire(self, name, t_begin, k_rows, v_rows, page_table=None):
         """This rank's new K/V rows (bf16, logical tokens t_begin..) in the form they travel in: as they are."""
         return k_rows, v_rows
 
@@ -193,7 +252,7 @@ class LibraryOps:
         if n > 0:
             self.b.cp_kv_append(self.ctx, self.cache, self.page_table, t_begin, n, k_rows, v_rows)
 
-    def attn_chunk(self, lay: RankLayout, chunk, q_chunk):
+    def attn_chunk(self, lay: RankLayout, chunk, q_chunk, page_table=None):
         n = q_chunk.shape[0]
         out = self.buffer("out_%d" % chunk, (n, self.Hq, self.D), self.torch.bfloat16)
         lse = self.buffer("lse_%d" % chunk, (self.Hq, n), self.torch.float32)
@@ -202,18 +261,19 @@ class LibraryOps:
         if self._ws is None:
             nbytes = self.b.cp_workspace_bytes([lay.R], [lay.C], self.Hq)
             self._ws = self.torch.empty(nbytes, dtype=self.torch.uint8, device=self.device)
-        self.b.cp_prefill_attn_chunk(self.ctx, q_chunk, self.cache, self.page_table, lay.P, lay.R, lay.C, chunk,
-                                     self.Hq, self.scale, out, lse, self._ws)
+        self.b.cp_prefill_attn_chunk(self.ctx, q_chunk, self.cache, self.page_table if page_table is None else page_table,
+                                     lay.P, lay.R, lay.C, chunk, self.Hq, self.scale, out, lse, self._ws)
         return out, lse
 
 
 class LibraryOps8(LibraryOps):
     """The device steps of a rank on an FP8 K/V cache (E4M3 pages, one fp32 scale per KV head shared by all ranks)."""
 
-    def __init__(self, ctx, k8_pages, v8_pages, k_scale, v_scale, page_table, Hq, scale):
+    def __init__(self, ctx, k8_pages, v8_pages, k_scale, v_scale, page_table, Hq, scale, arena_page0=None):
         import torch
         from . import binding
         self.b, self.ctx, self.torch = binding, ctx, torch
+        self.arena_page0, self._landing = arena_page0, {}
         self.cache = binding.make_cache_fp8(k8_pages, v8_pages, k_scale, v_scale)
         self.k_pages, self.v_pages, self.page_table = k8_pages, v8_pages, page_table
         self.k_scale, self.v_scale = k_scale, v_scale
@@ -230,14 +290,15 @@ class LibraryOps8(LibraryOps):
     def empty_rows(self, n, heads):
         return self.torch.zeros((n, heads, self.D), dtype=self.torch.uint8, device=self.device)
 
-    def to_wire(self, name, t_begin, k_rows, v_rows):
+    def to_wire(self, name, t_begin, k_rows, v_rows, page_table=None):
         """Quantise the rank's own new rows into its cache (they belong there anyway) and read the stored bytes
         back: what the other ranks receive is exactly what this rank attends to."""
         n = k_rows.shape[0]
+        pt = self.page_table if page_table is None else page_table
         kb, vb = self.buffer("wire_k_" + name, (n, self.Hkv, self.D)), self.buffer("wire_v_" + name, (n, self.Hkv, self.D))
         if n > 0:
-            self.b.cp_kv_append_fp8(self.ctx, self.cache, self.page_table, t_begin, n, k_rows, v_rows)
-            self.b.cp_kv_gather_fp8(self.ctx, self.cache, self.page_table, t_begin, n, kb, vb)
+            self.b.cp_kv_append_fp8(self.ctx, self.cache, pt, t_begin, n, k_rows, v_rows)
+            self.b.cp_kv_gather_fp8(self.ctx, self.cache, pt, t_begin, n, kb, vb)
         return kb, vb
 
     def kv_gather(self, t_begin, n, k_rows, v_rows):
@@ -249,7 +310,7 @@ class LibraryOps8(LibraryOps):
         if segments:
             self.b.cp_kv_append_segments_fp8(self.ctx, self.cache, self.page_table, segments, k_rows, v_rows)
 
-    def attn_chunk(self, lay: RankLayout, chunk, q_chunk):
+    def attn_chunk(self, lay: RankLayout, chunk, q_chunk, page_table=None):
         n = q_chunk.shape[0]
         out = self.buffer("out_%d" % chunk, (n, self.Hq, self.D), self.torch.bfloat16)
         lse = self.buffer("lse_%d" % chunk, (self.Hq, n), self.torch.float32)
@@ -258,8 +319,8 @@ class LibraryOps8(LibraryOps):
         if self._ws is None:
             nbytes = self.b.cp_workspace_bytes_fp8([lay.R], [lay.C], self.Hq)
             self._ws = self.torch.empty(nbytes, dtype=self.torch.uint8, device=self.device)
-        self.b.cp_prefill_attn_fp8_chunk(self.ctx, q_chunk, self.cache, self.page_table, lay.P, lay.R, lay.C, chunk,
-                                         self.Hq, self.scale, out, lse, self._ws)
+        self.b.cp_prefill_attn_fp8_chunk(self.ctx, q_chunk, self.cache, self.page_table if page_table is None else page_table,
+                                         lay.P, lay.R, lay.C, chunk, self.Hq, self.scale, out, lse, self._ws)
         return out, lse
 
 
@@ -345,10 +406,17 @@ class CpRankWorker:
 
         C, cl = lay.C, lay.cl
         n_blk = lay.block_pages * lay.page
-        # one arena per tensor: gathered prefix blocks | gathered early chunks | gathered late chunks (rows)
+        # one arena per tensor: gathered prefix blocks | gathered early chunks | gathered late chunks (rows).
+        # Landing mode: the arena is a run of pages of the cache pool itself and `table` reads it in token order.
         off_e, off_l = C * n_blk, C * (n_blk + cl)
-        ak = ops.buffer("arena_k", (C * (n_blk + 2 * cl), ops.Hkv, ops.D))
-        av = ops.buffer("arena_v", (C * (n_blk + 2 * cl), ops.Hkv, ops.D))
+        land = ops.landing(lay) if hasattr(ops, "landing") else None
+        if land is not None:
+            ak, av, table = land
+            kw = {"page_table": table}
+        else:
+            ak = ops.buffer("arena_k", (C * (n_blk + 2 * cl), ops.Hkv, ops.D))
+            av = ops.buffer("arena_v", (C * (n_blk + 2 * cl), ops.Hkv, ops.D))
+            kw = {}
 
         # 1. contributions: own prefix block read out of the cache, own chunks (padded to cl rows when short);
         #    every gather lands in its part of the arena
@@ -359,8 +427,8 @@ class CpRankWorker:
             ops.kv_gather(pb, pe - pb, sk, sv)
             hp = (comm.all_gather_into(ak[:off_e], sk), comm.all_gather_into(av[:off_e], sv))
         if hasattr(ops, "to_wire"):       # an FP8 cache sends stored bytes; a bf16 cache the rows as they are
-            k_early, v_early = ops.to_wire("early", lay.P + eb, k_early, v_early)
-            k_late, v_late = ops.to_wire("late", lay.P + lb, k_late, v_late)
+            k_early, v_early = ops.to_wire("early", lay.P + eb, k_early, v_early, **kw)
+            k_late, v_late = ops.to_wire("late", lay.P + lb, k_late, v_late, **kw)
         he = (comm.all_gather_into(ak[off_e:off_l], _padded(ops, k_early, cl, "send_early_k")),
               comm.all_gather_into(av[off_e:off_l], _padded(ops, v_early, cl, "send_early_v")))
         hl = (comm.all_gather_into(ak[off_l:], _padded(ops, k_late, cl, "send_late_k")),
@@ -379,10 +447,11 @@ class CpRankWorker:
         for r in range(C):
             b, e = lay.chunk(r)
             segs.append((lay.P + b, e - b, off_e + r * cl))
-        ops.kv_append_segments(segs, ak, av)
+        if land is None:
+            ops.kv_append_segments(segs, ak, av)
 
         # 3. early chunk: its keys are all here; the late all-gather is still in flight
-        out_e, lse_e = ops.attn_chunk(lay, lay.early, q_early)
+        out_e, lse_e = ops.attn_chunk(lay, lay.early, q_early, **kw)
 
         # 4. late chunks (rank r sent chunk 2C-1-r), one launch, then the late chunk's attention
         hl[0].wait()
@@ -391,8 +460,9 @@ class CpRankWorker:
         for r in range(C):
             b, e = lay.chunk(lay.late_chunk_of(r))
             segs.append((lay.P + b, e - b, off_l + r * cl))
-        ops.kv_append_segments(segs, ak, av)
-        out_l, lse_l = ops.attn_chunk(lay, lay.late, q_late)
+        if land is None:
+            ops.kv_append_segments(segs, ak, av)
+        out_l, lse_l = ops.attn_chunk(lay, lay.late, q_late, **kw)
         return out_e, lse_e, out_l, lse_l
 
     def _return_index(self, like):

@@ -56,10 +56,24 @@ class ThreadComm:
 class OracleOps:
     """kv_gather / kv_append / attn_chunk of one rank on numpy page pools, through the oracle."""
 
-    def __init__(self, k_pages, v_pages, page_table, Hq, scale):
+    def __init__(self, k_pages, v_pages, page_table, Hq, scale, arena_page0=None):
         self.k_pages, self.v_pages, self.page_table = k_pages, v_pages, np.asarray(page_table)
         self.Hq, self.scale = Hq, scale
         self.Hkv, self.D = k_pages.shape[2], k_pages.shape[3]
+        self.arena_page0 = arena_page0
+
+    def landing(self, lay):
+        """Landing mode on the numpy pools: torch views of the arena pages (shared memory) and the page table."""
+        from paper_2609_04774_b200 import cp_rank
+        table = cp_rank.landing_table(lay, self.arena_page0) if self.arena_page0 is not None else None
+        if table is None:
+            return None
+        n_pg, a0 = cp_rank.landing_pages(lay), self.arena_page0
+        assert a0 + n_pg <= self.k_pages.shape[0]
+        dt = np.int16 if self.k_pages.dtype == np.uint16 else self.k_pages.dtype
+        kr = torch.from_numpy(self.k_pages.view(dt))[a0:a0 + n_pg].view(n_pg * lay.page, self.Hkv, self.D)
+        vr = torch.from_numpy(self.v_pages.view(dt))[a0:a0 + n_pg].view(n_pg * lay.page, self.Hkv, self.D)
+        return kr, vr, np.asarray(table)
 
     def empty_rows(self, n, heads):
         return torch.zeros((n, heads, self.D), dtype=torch.int16)
@@ -89,13 +103,14 @@ class OracleOps:
             orc.kv_append(self.k_pages, self.page_table, t_begin, self._bits(k_rows)[:n])
             orc.kv_append(self.v_pages, self.page_table, t_begin, self._bits(v_rows)[:n])
 
-    def attn_chunk(self, lay, chunk, q_chunk):
+    def attn_chunk(self, lay, chunk, q_chunk, page_table=None):
         b, e = lay.chunk(chunk)
         q = np.zeros((lay.R, self.Hq, self.D), dtype=np.uint16)
         q[b:e] = self._bits(q_chunk)
         if e == b:
             return np.zeros((0, self.Hq, self.D)), np.zeros((self.Hq, 0))
-        return orc.attn_rows(q, self.k_pages, self.v_pages, self.page_table, lay.P, self.Hkv, self.scale, np.arange(b, e))
+        pt = self.page_table if page_table is None else page_table
+        return orc.attn_rows(q, self.k_pages, self.v_pages, pt, lay.P, self.Hkv, self.scale, np.arange(b, e))
 
 
     # ---- pass-Q mode: partial attention over a key range, LSE merge (fp64 torch tensors) ----
@@ -119,8 +134,8 @@ class OracleOps:
 class OracleOps8(OracleOps):
     """The same steps on E4M3 byte pools with per-head scales, through the FP8 oracle."""
 
-    def __init__(self, k8_pages, v8_pages, k_scale, v_scale, page_table, Hq, scale):
-        super().__init__(k8_pages, v8_pages, page_table, Hq, scale)
+    def __init__(self, k8_pages, v8_pages, k_scale, v_scale, page_table, Hq, scale, arena_page0=None):
+        super().__init__(k8_pages, v8_pages, page_table, Hq, scale, arena_page0)
         self.k_scale, self.v_scale = k_scale, v_scale
 
     def empty_rows(self, n, heads):
@@ -137,13 +152,14 @@ class OracleOps8(OracleOps):
     def _bits(t):
         return t.contiguous().numpy()
 
-    def to_wire(self, name, t_begin, k_rows, v_rows):
+    def to_wire(self, name, t_begin, k_rows, v_rows, page_table=None):
         from oracle import fp8 as o8
+        pt = self.page_table if page_table is None else page_table
         kc = o8.quantize_kv(k_rows.contiguous().numpy().view(np.uint16), self.k_scale)
         vc = o8.quantize_kv(v_rows.contiguous().numpy().view(np.uint16), self.v_scale)
         if kc.shape[0]:
-            orc.kv_append(self.k_pages, self.page_table, t_begin, kc)
-            orc.kv_append(self.v_pages, self.page_table, t_begin, vc)
+            orc.kv_append(self.k_pages, pt, t_begin, kc)
+            orc.kv_append(self.v_pages, pt, t_begin, vc)
         return torch.from_numpy(kc), torch.from_numpy(vc)
 
     def kv_gather(self, t_begin, n, k_rows, v_rows):
@@ -151,14 +167,15 @@ class OracleOps8(OracleOps):
             k_rows[:n] = torch.from_numpy(orc.kv_gather(self.k_pages, self.page_table, t_begin, t_begin + n))
             v_rows[:n] = torch.from_numpy(orc.kv_gather(self.v_pages, self.page_table, t_begin, t_begin + n))
 
-    def attn_chunk(self, lay, chunk, q_chunk):
+    def attn_chunk(self, lay, chunk, q_chunk, page_table=None):
         from oracle import fp8 as o8
         b, e = lay.chunk(chunk)
         q = np.zeros((lay.R, self.Hq, self.D), dtype=np.uint16)
         q[b:e] = q_chunk.contiguous().numpy().view(np.uint16)
         if e == b:
             return np.zeros((0, self.Hq, self.D)), np.zeros((self.Hq, 0))
-        o, l, _ = o8.attn_fp8_rows(q, self.k_pages, self.v_pages, self.k_scale, self.v_scale, self.page_table, lay.P, self.Hkv,
+        o, l, _ = o8.attn_fp8_rows(q, self.k_pages, self.v_pages, self.k_scale, self.v_scale,
+                                   self.page_table if page_table is None else page_table, lay.P, self.Hkv,
                                    self.scale, np.arange(b, e))
         return o, l
 

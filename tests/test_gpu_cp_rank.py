@@ -306,3 +306,82 @@ def test_ranks_as_threads_on_one_gpu_fp8_cache(R, P, C):
         for got, ref in ((k_pages, m8.k8_pages), (v_pages, m8.v8_pages)):
             assert np.array_equal(o8.e4m3_decode(orc.kv_gather(got, page_table, 0, L)),
                                   o8.e4m3_decode(orc.kv_gather(ref, m8.page_table, 0, L)))
+
+
+@pytest.mark.parametrize("fp8", [False, True])
+@pytest.mark.parametrize("R,P,C", [(2048, 1024, 4), (509, 192, 4), (1533, 0, 3)])
+def test_ranks_on_one_gpu_landing_mode(R, P, C, fp8):
+    # landing mode: the gathers write into pages of the rank's own pool, a page table reads them in token order, no
+    # append runs (the method is taken away); results against the oracle, and the pool read through the landing table
+    # holds the whole request bit for bit.  The step is run twice on the same worker (layer after layer).
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from cp_rank_util import ThreadFabric, rank_inputs, rank_inputs8
+    from oracle import fp8 as o8
+    from paper_2609_04774_b200 import binding
+    from paper_2609_04774_b200.cp_rank import CpRankWorker, LibraryOps, LibraryOps8, RankLayout, landing_pages
+    from tests.test_gpu_fp8 import compare8
+    w = wl.Workload("cp_rank_land_gpu", 68, 8, 2, [wl.Request(R, P, C)])
+    mat = wl.materialize(w)
+    L = P + R
+    if fp8:
+        m8 = wl.materialize_fp8(w)
+        ro, rl, ra = o8.attn_fp8_rows(m8.q, m8.k8_pages, m8.v8_pages, m8.k_scale, m8.v_scale, m8.page_table, P, w.Hkv, w.scale,
+                                      np.arange(R))
+        ref_k, ref_v = orc.kv_gather(m8.k8_pages, m8.page_table, 0, L), orc.kv_gather(m8.v8_pages, m8.page_table, 0, L)
+    else:
+        ro, rl = orc.attn_full(mat.q, mat.k_pages, mat.v_pages, mat.page_table, P, w.Hkv, w.scale)
+        ref_k, ref_v = orc.kv_gather(mat.k_pages, mat.page_table, 0, L), orc.kv_gather(mat.v_pages, mat.page_table, 0, L)
+    fabric = ThreadFabric(C)
+    result, errors = {}, []
+
+    def body(k):
+        try:
+            torch.cuda.set_device(0)
+            lay = RankLayout(R, P, C, k)
+            assert lay.cl % lay.page == 0
+            k_pages, v_pages, page_table, rows = rank_inputs8(m8, mat, lay, 68) if fp8 else rank_inputs(mat, lay, 68)
+            a0 = k_pages.shape[0]
+            extra = np.zeros((landing_pages(lay),) + k_pages.shape[1:], dtype=k_pages.dtype)
+            k_pages, v_pages = np.concatenate([k_pages, extra]), np.concatenate([v_pages, extra])
+            pt = torch.from_numpy(page_table).cuda()
+            if fp8:
+                ops = LibraryOps8(binding.Context(0), torch.from_numpy(k_pages).cuda(), torch.from_numpy(v_pages).cuda(),
+                                  torch.from_numpy(m8.k_scale).cuda(), torch.from_numpy(m8.v_scale).cuda(), pt, w.Hq, w.scale,
+                                  arena_page0=a0)
+            else:
+                ops = LibraryOps(binding.Context(0), _dev(k_pages), _dev(v_pages), pt, w.Hq, w.scale, arena_page0=a0)
+            assert ops.landing(lay) is not None
+            ops.kv_append_segments = None
+            t = {n: _dev(x) for n, x in rows.items()}
+            worker = CpRankWorker(lay, fabric.comm(k), ops)
+            for _ in range(2):
+                out = worker.prefill(t["q_early"], t["q_late"], t["k_early"], t["v_early"], t["k_late"], t["v_late"])
+            torch.cuda.synchronize()
+            ops.ctx.poll_status()
+            pool = lambda p: p.cpu().numpy() if fp8 else p.view(torch.int16).cpu().numpy().view(np.uint16)
+            result[k] = tuple(x.clone() for x in out) + (pool(ops.k_pages), pool(ops.v_pages), ops.landing(lay)[2].cpu().numpy())
+        except Exception as e:
+            errors.append(e)
+            fabric.barrier.abort()
+
+    threads = [threading.Thread(target=body, args=(k,)) for k in range(C)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=600)
+    assert not errors, errors
+    for k in range(C):
+        lay = RankLayout(R, P, C, k)
+        out_e, lse_e, out_l, lse_l, k_pages, v_pages, table = result[k]
+        for j, o, l in ((lay.early, out_e, lse_e), (lay.late, out_l, lse_l)):
+            b, e = lay.chunk(j)
+            assert o.shape[0] == e - b and e > b
+            if fp8:
+                compare8(_f64(o), _f64(l), ro[b:e], rl[:, b:e], ra[b:e], "landing fp8 rank %d chunk %d" % (k, j))
+            else:
+                _compare(o, l, ro[b:e], rl[:, b:e], "landing rank %d chunk %d" % (k, j))
+        got_k, got_v = orc.kv_gather(k_pages, table, 0, L), orc.kv_gather(v_pages, table, 0, L)
+        if fp8:
+            assert np.array_equal(o8.e4m3_decode(got_k), o8.e4m3_decode(ref_k)) and np.array_equal(o8.e4m3_decode(got_v), o8.e4m3_decode(ref_v))
+        else:
+            assert np.array_equal(got_k, ref_k) and np.array_equal(got_v, ref_v)

@@ -497,7 +497,7 @@ def _random_workload(seed):
     return wl.Workload("random_%d" % seed, seed, heads[0], heads[1], reqs)
 
 
-@pytest.mark.parametrize("seed", range(1000, 1000 + int(os.environ.get("CPATTN_FUZZ_CASES", "16"))))
+@pytest.mark.parametrize("seed", range(1000, 1000 + int(os.environ.get("CPATTN_FUZZ_CASES", "48"))))
 def test_attention_random_batches(ctx, seed):
     # seeded random batches: head shapes with even, odd and unit group sizes, ragged lengths from one token
     # up, prefixes that are absent, page-aligned or not, every supported kind of C
