@@ -572,8 +572,8 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, const InlineSche
 }
 
 // P*V issuer: O_h += P_h V_j in the order (tile, head), each in the two pieces P is handed over in.  In a
-// single-head unit the tiles alternate between the two P / O column sets (two independent online-softmax
-// streams over the even and the odd tiles of the piece, combined in the epilogue).
+// single-head unit (a pair of consecutive query tiles of one head) the second P / O column set belongs to the
+// unit's second query tile instead of a second head; the loop is the same.
 template <bool kFp8>
 __device__ __forceinline__ void mma_pv_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
                                             volatile uint32_t* abort_flag) {
