@@ -10,41 +10,81 @@ using namespace cpattn;
 
 namespace {
 
-// kToPaged = false: paged -> rows (gather); true: rows -> paged (append).
+// One token's row of vec_per_tok 16-byte vectors, copied by one warp: four vectors per lane and tensor are in flight
+// before the first store.  `paged` is the address of the token's slot (head 0, vector 0); head g starts
+// stride_head8 vectors further.  vph_shift = log2(vectors per head row): 4 (bf16) or 3 (one-byte elements).
+template <bool kToPaged>
+__device__ __forceinline__ void copy_token(uint4* __restrict__ paged_k, uint4* __restrict__ paged_v, uint4* __restrict__ rows_k,
+                                           uint4* __restrict__ rows_v, int64_t paged_off, int64_t rows_off, int vec_per_tok,
+                                           int vph_shift, int64_t stride_head8, int lane) {
+    for (int v0 = 0; v0 < vec_per_tok; v0 += 128) {
+        int64_t po[4];
+        uint4 a[4], b[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int v = v0 + u * 32 + lane;
+            const int g = v >> vph_shift;
+            po[u] = paged_off + (int64_t)g * stride_head8 + (v - (g << vph_shift));
+            if (v < vec_per_tok) {
+                if (rows_k) a[u] = kToPaged ? rows_k[rows_off + v] : paged_k[po[u]];
+                if (rows_v) b[u] = kToPaged ? rows_v[rows_off + v] : paged_v[po[u]];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int v = v0 + u * 32 + lane;
+            if (v < vec_per_tok) {
+                if (kToPaged) {
+                    if (rows_k) paged_k[po[u]] = a[u];
+                    if (rows_v) paged_v[po[u]] = b[u];
+                } else {
+                    if (rows_k) rows_k[rows_off + v] = a[u];
+                    if (rows_v) rows_v[rows_off + v] = b[u];
+                }
+            }
+        }
+    }
+}
+
+// Records the first page id outside the pool in the status words {code, table index, block, page id}.
+__device__ __forceinline__ void report_bad_page(int32_t* status, int64_t table_index, int64_t page) {
+    if (atomicCAS(status, 0, CP_ERR_BOUNDS) == 0) {
+        status[1] = (int32_t)table_index;
+        status[2] = (int32_t)blockIdx.x;
+        status[3] = (int32_t)page;
+    }
+}
+
+// kToPaged = false: paged -> rows (gather); true: rows -> paged (append).  One warp per token (the page id is looked up
+// once per token); page_shift = log2(page_size).
 template <bool kToPaged>
 __global__ void __launch_bounds__(256)
 kv_copy_kernel(uint4* __restrict__ paged_k, uint4* __restrict__ paged_v, uint4* __restrict__ rows_k,
                uint4* __restrict__ rows_v, const int32_t* __restrict__ page_table, int64_t t_begin, int64_t n,
-               int page_size, int Hkv, int vec_per_head, int64_t stride_page8, int64_t stride_tok8,
+               int page_shift, int Hkv, int vph_shift, int64_t stride_page8, int64_t stride_tok8,
                int64_t stride_head8, int64_t num_pages, int32_t* status) {
-    const int vec_per_tok = Hkv * vec_per_head;
-    const int64_t total = n * vec_per_tok;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t tok = i / vec_per_tok;
-        const int rem = (int)(i - tok * vec_per_tok);
-        const int g = rem / vec_per_head;
-        const int c = rem - g * vec_per_head;
+    const int vec_per_tok = Hkv << vph_shift;
+    const int lane = threadIdx.x & 31;
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t tok = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; tok < n; tok += n_warps) {
         const int64_t t = t_begin + tok;
-        const int64_t page = page_table[t / page_size];
+        const int64_t page = page_table[t >> page_shift];
         if (page < 0 || page >= num_pages) {
-            // a page id outside the pool: the element is skipped (nothing is read or written through it) and the
-            // first such entry is recorded in the status words {code, table index, block, page id}
-            if (atomicCAS(status, 0, CP_ERR_BOUNDS) == 0) {
-                status[1] = (int32_t)(t / page_size);
-                status[2] = (int32_t)blockIdx.x;
-                status[3] = (int32_t)page;
-            }
+            // a page id outside the pool: the token is skipped (nothing is read or written through it)
+            if (lane == 0) report_bad_page(status, t >> page_shift, page);
             continue;
         }
-        const int64_t off = page * stride_page8 + (t % page_size) * stride_tok8 + (int64_t)g * stride_head8 + c;
-        if (kToPaged) {
-            if (rows_k) paged_k[off] = rows_k[i];
-            if (rows_v) paged_v[off] = rows_v[i];
-        } else {
-            if (rows_k) rows_k[i] = paged_k[off];
-            if (rows_v) rows_v[i] = paged_v[off];
-        }
+        copy_token<kToPaged>(paged_k, paged_v, rows_k, rows_v,
+                             page * stride_page8 + (t & ((1ll << page_shift) - 1)) * stride_tok8, tok * vec_per_tok, vec_per_tok,
+                             vph_shift, stride_head8, lane);
     }
+}
+
+// page sizes are powers of two (validate_cache): log2
+inline int log2_of(int v) {
+    int s = 0;
+    while ((1 << s) < v) ++s;
+    return s;
 }
 
 int validate_cache(const cp_kv_cache* c, const char* who) {
@@ -74,33 +114,26 @@ struct SegmentTable {
 __global__ void __launch_bounds__(256)
 kv_append_segments_kernel(uint4* __restrict__ paged_k, uint4* __restrict__ paged_v, const uint4* __restrict__ rows_k,
                           const uint4* __restrict__ rows_v, const int32_t* __restrict__ page_table,
-                          const __grid_constant__ SegmentTable seg, int page_size, int Hkv, int vec_per_head,
+                          const __grid_constant__ SegmentTable seg, int page_shift, int Hkv, int vph_shift,
                           int64_t stride_page8, int64_t stride_tok8, int64_t stride_head8, int64_t num_pages,
                           int32_t* status) {
-    const int vec_per_tok = Hkv * vec_per_head;
-    const int64_t total = seg.cum[seg.n_segments] * vec_per_tok;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t tok = i / vec_per_tok;
-        const int rem = (int)(i - tok * vec_per_tok);
-        int sg = 0;
-        while (tok >= seg.cum[sg + 1]) ++sg;                       // few segments: a linear walk
+    const int vec_per_tok = Hkv << vph_shift;
+    const int lane = threadIdx.x & 31;
+    const int64_t n = seg.cum[seg.n_segments];
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    int sg = 0;
+    for (int64_t tok = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; tok < n; tok += n_warps) {
+        while (tok >= seg.cum[sg + 1]) ++sg;                       // tokens ascend: the walk never goes back
         const int64_t k = tok - seg.cum[sg];
         const int64_t t = seg.t_begin[sg] + k;
-        const int64_t src = (seg.row0[sg] + k) * vec_per_tok + rem;
-        const int g = rem / vec_per_head;
-        const int c = rem - g * vec_per_head;
-        const int64_t page = page_table[t / page_size];
+        const int64_t page = page_table[t >> page_shift];
         if (page < 0 || page >= num_pages) {
-            if (atomicCAS(status, 0, CP_ERR_BOUNDS) == 0) {
-                status[1] = (int32_t)(t / page_size);
-                status[2] = (int32_t)blockIdx.x;
-                status[3] = (int32_t)page;
-            }
+            if (lane == 0) report_bad_page(status, t >> page_shift, page);
             continue;
         }
-        const int64_t off = page * stride_page8 + (t % page_size) * stride_tok8 + (int64_t)g * stride_head8 + c;
-        if (rows_k) paged_k[off] = rows_k[src];
-        if (rows_v) paged_v[off] = rows_v[src];
+        copy_token<true>(paged_k, paged_v, const_cast<uint4*>(rows_k), const_cast<uint4*>(rows_v),
+                         page * stride_page8 + (t & ((1ll << page_shift) - 1)) * stride_tok8, (seg.row0[sg] + k) * vec_per_tok,
+                         vec_per_tok, vph_shift, stride_head8, lane);
     }
 }
 
@@ -189,12 +222,10 @@ int kv_copy(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, in
         return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
     if (n == 0) return CP_OK;
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    const int vec_per_head = cache->D / 8;
-    const int64_t total = n * cache->Hkv * vec_per_head;
-    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
+    const int blocks = (int)std::min<int64_t>((n + 7) / 8, (int64_t)ctx->num_sms * 16);      // one warp per token
     kv_copy_kernel<kToPaged><<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        (uint4*)cache->k, (uint4*)cache->v, (uint4*)k_rows, (uint4*)v_rows, page_table, t_begin, n, cache->page_size,
-        cache->Hkv, vec_per_head, cache->stride_page / 8, cache->stride_tok / 8, cache->stride_head / 8, cache->num_pages,
+        (uint4*)cache->k, (uint4*)cache->v, (uint4*)k_rows, (uint4*)v_rows, page_table, t_begin, n, log2_of(cache->page_size),
+        cache->Hkv, 4, cache->stride_page / 8, cache->stride_tok / 8, cache->stride_head / 8, cache->num_pages,
         ctx->d_status);
     return check_cuda(cudaGetLastError(), who);
 }
@@ -232,19 +263,14 @@ extern "C" int cp_kv_append_segments(cp_ctx* ctx, const cp_kv_cache* cache, cons
     }
     if (tab.n_segments == 0) return CP_OK;
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    const int vec_per_head = cache->D / 8;
-    const int64_t total = tab.cum[tab.n_segments] * cache->Hkv * vec_per_head;
-    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
+    const int blocks = (int)std::min<int64_t>((tab.cum[tab.n_segments] + 7) / 8, (int64_t)ctx->num_sms * 16);
     kv_append_segments_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        (uint4*)cache->k, (uint4*)cache->v, (const uint4*)k_rows, (const uint4*)v_rows, page_table, tab, cache->page_size,
-        cache->Hkv, vec_per_head, cache->stride_page / 8, cache->stride_tok / 8, cache->stride_head / 8, cache->num_pages,
+        (uint4*)cache->k, (uint4*)cache->v, (const uint4*)k_rows, (const uint4*)v_rows, page_table, tab, log2_of(cache->page_size),
+        cache->Hkv, 4, cache->stride_page / 8, cache->stride_tok / 8, cache->stride_head / 8, cache->num_pages,
         ctx->d_status);
     return check_cuda(cudaGetLastError(), who);
 }
 
-// Raw byte copies of an FP8 cache (no conversion): the same kernels with one-byte elements, i.e. 8 vectors of 16
-// bytes per head row.  What a CP rank exchanges when the cache is FP8: stored bytes travel, and because all ranks
-// share the per-head scales they can be appended as they are.
 extern "C" int cp_check_page_table(cp_ctx* ctx, const int32_t* page_table, int64_t n_entries, int64_t num_pages, void* stream) {
     if (!ctx || !page_table || n_entries < 0 || num_pages < 1)
         return set_error(CP_ERR_INVALID_ARG, "cp_check_page_table: null pointer, negative count or empty pool");
@@ -255,6 +281,9 @@ extern "C" int cp_check_page_table(cp_ctx* ctx, const int32_t* page_table, int64
     return check_cuda(cudaGetLastError(), "cp_check_page_table");
 }
 
+// Raw byte copies of an FP8 cache (no conversion): the same kernels with one-byte elements, i.e. 8 vectors of 16
+// bytes per head row.  What a CP rank exchanges when the cache is FP8: stored bytes travel, and because all ranks
+// share the per-head scales they can be appended as they are.
 extern "C" int cp_kv_gather_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,
                                 int64_t n, void* k_bytes, void* v_bytes, void* stream) {
     const char* who = "cp_kv_gather_fp8";
@@ -266,12 +295,10 @@ extern "C" int cp_kv_gather_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const
         return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
     if (n == 0) return CP_OK;
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    const int vec_per_head = cache->D / 16;
-    const int64_t total = n * cache->Hkv * vec_per_head;
-    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
+    const int blocks = (int)std::min<int64_t>((n + 7) / 8, (int64_t)ctx->num_sms * 16);
     kv_copy_kernel<false><<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        (uint4*)cache->k, (uint4*)cache->v, (uint4*)k_bytes, (uint4*)v_bytes, page_table, t_begin, n, cache->page_size,
-        cache->Hkv, vec_per_head, cache->stride_page / 16, cache->stride_tok / 16, cache->stride_head / 16, cache->num_pages,
+        (uint4*)cache->k, (uint4*)cache->v, (uint4*)k_bytes, (uint4*)v_bytes, page_table, t_begin, n, log2_of(cache->page_size),
+        cache->Hkv, 3, cache->stride_page / 16, cache->stride_tok / 16, cache->stride_head / 16, cache->num_pages,
         ctx->d_status);
     return check_cuda(cudaGetLastError(), who);
 }
@@ -303,12 +330,10 @@ extern "C" int cp_kv_append_segments_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cac
     }
     if (tab.n_segments == 0) return CP_OK;
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    const int vec_per_head = cache->D / 16;
-    const int64_t total = tab.cum[tab.n_segments] * cache->Hkv * vec_per_head;
-    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
+    const int blocks = (int)std::min<int64_t>((tab.cum[tab.n_segments] + 7) / 8, (int64_t)ctx->num_sms * 16);
     kv_append_segments_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        (uint4*)cache->k, (uint4*)cache->v, (const uint4*)k_bytes, (const uint4*)v_bytes, page_table, tab, cache->page_size,
-        cache->Hkv, vec_per_head, cache->stride_page / 16, cache->stride_tok / 16, cache->stride_head / 16, cache->num_pages,
+        (uint4*)cache->k, (uint4*)cache->v, (const uint4*)k_bytes, (const uint4*)v_bytes, page_table, tab, log2_of(cache->page_size),
+        cache->Hkv, 3, cache->stride_page / 16, cache->stride_tok / 16, cache->stride_head / 16, cache->num_pages,
         ctx->d_status);
     return check_cuda(cudaGetLastError(), who);
 }
