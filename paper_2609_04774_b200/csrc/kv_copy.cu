@@ -163,36 +163,34 @@ __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d, f
 __global__ void __launch_bounds__(256)
 kv_append_fp8_kernel(uint8_t* __restrict__ paged_k, uint8_t* __restrict__ paged_v, const uint4* __restrict__ rows_k,
                      const uint4* __restrict__ rows_v, const float* __restrict__ k_scale, const float* __restrict__ v_scale,
-                     const int32_t* __restrict__ page_table, int64_t t_begin, int64_t n, int page_size, int Hkv,
+                     const int32_t* __restrict__ page_table, int64_t t_begin, int64_t n, int page_shift, int Hkv,
                      int64_t stride_page, int64_t stride_tok, int64_t stride_head, int64_t num_pages, int32_t* status) {
-    const int vec_per_tok = Hkv * 16;                 // 8 elements per thread
-    const int64_t total = n * vec_per_tok;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t tok = i / vec_per_tok;
-        const int rem = (int)(i - tok * vec_per_tok);
-        const int g = rem >> 4, c = rem & 15;
+    const int vec_per_tok = Hkv * 16;                 // one warp per token, 8 elements (16 bytes in, 8 bytes out) per lane and step
+    const int lane = threadIdx.x & 31;
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t tok = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; tok < n; tok += n_warps) {
         const int64_t t = t_begin + tok;
-        const int64_t page = page_table[t / page_size];
+        const int64_t page = page_table[t >> page_shift];
         if (page < 0 || page >= num_pages) {
-            if (atomicCAS(status, 0, CP_ERR_BOUNDS) == 0) {
-                status[1] = (int32_t)(t / page_size);
-                status[2] = (int32_t)blockIdx.x;
-                status[3] = (int32_t)page;
-            }
+            if (lane == 0) report_bad_page(status, t >> page_shift, page);
             continue;
         }
-        const int64_t off = page * stride_page + (t % page_size) * stride_tok + (int64_t)g * stride_head + c * 8;
+        const int64_t tok_off = page * stride_page + (t & ((1ll << page_shift) - 1)) * stride_tok;
+        for (int v = lane; v < vec_per_tok; v += 32) {
+            const int g = v >> 4, c = v & 15;
+            const int64_t off = tok_off + (int64_t)g * stride_head + c * 8;
 #pragma unroll
-        for (int kv = 0; kv < 2; ++kv) {
-            const uint4* rows = kv ? rows_v : rows_k;
-            if (!rows) continue;
-            const uint4 raw = rows[i];
-            const float sc = kv ? v_scale[g] : k_scale[g];
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
-            uint2 o;
-            o.x = quant4(__low2float(h[0]), __high2float(h[0]), __low2float(h[1]), __high2float(h[1]), sc);
-            o.y = quant4(__low2float(h[2]), __high2float(h[2]), __low2float(h[3]), __high2float(h[3]), sc);
-            *reinterpret_cast<uint2*>((kv ? paged_v : paged_k) + off) = o;
+            for (int kv = 0; kv < 2; ++kv) {
+                const uint4* rows = kv ? rows_v : rows_k;
+                if (!rows) continue;
+                const uint4 raw = rows[tok * vec_per_tok + v];
+                const float sc = kv ? v_scale[g] : k_scale[g];
+                const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+                uint2 o;
+                o.x = quant4(__low2float(h[0]), __high2float(h[0]), __low2float(h[1]), __high2float(h[1]), sc);
+                o.y = quant4(__low2float(h[2]), __high2float(h[2]), __low2float(h[3]), __high2float(h[3]), sc);
+                *reinterpret_cast<uint2*>((kv ? paged_v : paged_k) + off) = o;
+            }
         }
     }
 }
@@ -349,11 +347,10 @@ extern "C" int cp_kv_append_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const
         return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
     if (n == 0) return CP_OK;
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    const int64_t total = n * cache->Hkv * 16;
-    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)ctx->num_sms * 16);
+    const int blocks = (int)std::min<int64_t>((n + 7) / 8, (int64_t)ctx->num_sms * 16);       // one warp per token
     kv_append_fp8_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         (uint8_t*)cache->k, (uint8_t*)cache->v, (const uint4*)k_rows, (const uint4*)v_rows, cache->k_scale, cache->v_scale,
-        page_table, t_begin, n, cache->page_size, cache->Hkv, cache->stride_page, cache->stride_tok, cache->stride_head,
+        page_table, t_begin, n, log2_of(cache->page_size), cache->Hkv, cache->stride_page, cache->stride_tok, cache->stride_head,
         cache->num_pages, ctx->d_status);
     return check_cuda(cudaGetLastError(), who);
 }
