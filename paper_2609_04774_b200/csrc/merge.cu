@@ -117,7 +117,6 @@ extern "C" int cp_merge(cp_ctx* ctx, const float* partials, const float* lses, i
     if (((uintptr_t)partials | (uintptr_t)out) & 15)
         return set_error(CP_ERR_INVALID_ARG, "cp_merge: partials and out must be 16-byte aligned");
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // heads per warp: measured.  Two partials: 2 heads per warp (4 row loads in flight per warp, many warps)
     // reach 6.2-6.6 TB/s where 4 heads gave 5.9-6.1 and 8 heads 4.4; one head per warp loses 10 %.  The output
