@@ -71,3 +71,37 @@ def test_gpu_calls_fail_cleanly_without_a_device(lib):
     with pytest.raises(binding.CpError) as e:
         binding.Context(0)
     assert e.value.code in (binding.CP_ERR_CUDA, binding.CP_ERR_INVALID_ARG)
+
+
+def test_headers_compile_as_c99_and_link_from_c(lib, tmp_path):
+    # the boundary is a C ABI: both public headers must be valid C (not only C++), and a plain C program linked
+    # against the library must get the planner's numbers (compared with the oracle's plan)
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no gcc on this machine")
+    src = tmp_path / "use_cpattn.c"
+    src.write_text(
+        '#include "cpattn.h"\n#include "cpcache.h"\n#include <stdio.h>\n'
+        "int main(void) {\n"
+        "    cp_shard_plan plan[4];\n"
+        "    int rc = cp_plan(4096, 12288, 4, plan);\n"
+        "    for (int k = 0; k < 4 && rc == 0; ++k)\n"
+        '        printf("%lld %lld %lld %lld %lld %lld %llu\\n", (long long)plan[k].q_begin[0], (long long)plan[k].q_end[0],\n'
+        "               (long long)plan[k].q_begin[1], (long long)plan[k].q_end[1], (long long)plan[k].kv_end[0],\n"
+        "               (long long)plan[k].kv_end[1], (unsigned long long)plan[k].pairs);\n"
+        '    printf("%s\\n", cp_strerror(rc));\n'
+        "    return rc;\n}\n")
+    exe = tmp_path / "use_cpattn"
+    libdir = os.path.dirname(build.LIB_PATH)
+    subprocess.check_call([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(build.ROOT, "include"),
+                           str(src), "-o", str(exe), "-L", libdir, "-l:" + os.path.basename(build.LIB_PATH),
+                           "-Wl,-rpath," + libdir])
+    out = subprocess.check_output([str(exe)], text=True).split("\n")
+    ref = orc.plan(4096, 12288, 4)
+    for k in range(4):
+        got = [int(x) for x in out[k].split()]
+        assert got == [ref[k]["q_begin"][0], ref[k]["q_end"][0], ref[k]["q_begin"][1], ref[k]["q_end"][1],
+                       ref[k]["kv_end"][0], ref[k]["kv_end"][1], ref[k]["pairs"]]
+    assert out[4] == "CP_OK"
