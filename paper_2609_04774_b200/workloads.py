@@ -180,7 +180,9 @@ class Workload:
 
     @property
     def scale(self) -> float:
-        return 1.0 / math.sqrt(self.D)
+        """Softmax scale passed to the calls: 1/sqrt(D) unless ``meta["scale"]`` overrides it (tests use large scales to
+        make the row maxima jump between key tiles)."""
+        return float(self.meta.get("scale", 1.0 / math.sqrt(self.D)))
 
     @property
     def total_new(self) -> int:

@@ -271,3 +271,11 @@ def test_fp8_attention_config2_shape_sampled(ctx):
 
 def test_fp8_attention_config5_shape_sampled(ctx):
     check_batch8(ctx, wl.config5(), rows_per_request=24)
+
+
+@pytest.mark.parametrize("scale", [0.5, 2.0])
+def test_fp8_attention_peaked_scores_exercise_the_rescale_path(ctx, scale):
+    # a large softmax scale makes new row maxima arrive in later key tiles, so the rescale of O and of the running sum
+    # (threshold 2^4 in this variant, weights scaled by 16 and saturating at 448) really runs
+    w = wl.Workload("fp8_peaked_%g" % scale, 79, 8, 2, [wl.Request(600, 1280, 2), wl.Request(260, 0, 1)], meta={"scale": scale})
+    check_batch8(ctx, w)
