@@ -246,6 +246,22 @@ def test_attention_kv_split_units(ctx):
     assert torch.equal(o1.view(torch.int16), dev.out.view(torch.int16)) and torch.equal(l1, dev.lse)
 
 
+def test_attention_one_unit_cut_over_all_sms(ctx):
+    # a single work unit (one query tile, one pair of heads) behind a quarter of a million cached tokens: the planner
+    # cuts it into one piece per SM, so the fix-up merges far more than 32 partials per row (it walks them in groups
+    # of 32)
+    w = wl.Workload("one_unit", 45, 2, 1, [wl.Request(100, 250000, 1)])
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    info, _, _ = binding.cp_schedule_inspect(w.cu_new, [250000], [1], w.Hq, w.Hkv, sms, want_lists=False)
+    assert info["split_units"] == 1 and info["slots"] > 64, info
+    check_batch(ctx, w, pair_budget=1e10)
+    # the same with an odd group (a tile-pair unit of one head): 200 rows, two tiles
+    w1 = wl.Workload("one_unit_mha", 46, 1, 1, [wl.Request(200, 180000, 1)])
+    info, _, _ = binding.cp_schedule_inspect(w1.cu_new, [180000], [1], w1.Hq, w1.Hkv, sms, want_lists=False)
+    assert info["split_units"] == 1 and info["slots"] > 64, info
+    check_batch(ctx, w1, pair_budget=1e10)
+
+
 def test_attention_strided_cache_view(ctx):
     # the cache is a view into a wider allocation (one unused head slot per token, an unused token row
     # per page): only the three strides say where things are
