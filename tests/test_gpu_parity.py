@@ -150,6 +150,88 @@ def test_kv_append_segments_bit_exact(ctx):
     assert e.value.code == binding.CP_ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("Hkv,page", [(1, 16), (3, 128), (16, 32), (8, 64)])
+def test_kv_copies_other_head_counts_and_page_sizes(ctx, Hkv, page):
+    # one warp copies one token: rows of 16 vectors (one KV head) up to 256 (sixteen heads, two passes of the warp),
+    # a count that is no multiple of 32, every page size; the cache is a strided view; gather, append and the
+    # segment form against the oracle, bit for bit
+    w = wl.Workload("copies", 52, Hkv, Hkv, [wl.Request(333, 5 * page, 1)], page=page)
+    mat = wl.materialize(w, need_q=False)
+    npg = mat.k_pages.shape[0]
+    big_k = torch.zeros((npg, page + 1, Hkv + 1, w.D), dtype=torch.bfloat16, device="cuda")
+    big_v = torch.zeros_like(big_k)
+    k, v = big_k[:, :page, :Hkv], big_v[:, :page, :Hkv]
+    k.copy_(bits_to_bf16(mat.k_pages))
+    v.copy_(bits_to_bf16(mat.v_pages))
+    cache = binding.make_cache(k, v)
+    pt = torch.from_numpy(mat.page_table).cuda()
+    L = w.requests[0].total_len
+    t0, n = 7, L - 7
+    kr = torch.zeros((n, Hkv, w.D), dtype=torch.bfloat16, device="cuda")
+    vr = torch.zeros_like(kr)
+    binding.cp_kv_gather(ctx, cache, pt, t0, n, kr, vr)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    bits = lambda t: t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(bits(kr), orc.kv_gather(mat.k_pages, mat.page_table, t0, t0 + n))
+    assert np.array_equal(bits(vr), orc.kv_gather(mat.v_pages, mat.page_table, t0, t0 + n))
+    newk, newv = wl.normal_bf16(53, wl.TID_K, (n, Hkv, w.D)), wl.normal_bf16(53, wl.TID_V, (n, Hkv, w.D))
+    kp, vp = mat.k_pages.copy(), mat.v_pages.copy()
+    binding.cp_kv_append(ctx, cache, pt, t0, 100, bits_to_bf16(newk), bits_to_bf16(newv))
+    orc.kv_append(kp, mat.page_table, t0, newk[:100])
+    orc.kv_append(vp, mat.page_table, t0, newv[:100])
+    segs = [(200, 57, 120), (130, 33, 300), (L - 9, 9, 0)]
+    binding.cp_kv_append_segments(ctx, cache, pt, segs, bits_to_bf16(newk), bits_to_bf16(newv))
+    for s0, sn, r0 in segs:
+        orc.kv_append(kp, mat.page_table, s0, newk[r0:r0 + sn])
+        orc.kv_append(vp, mat.page_table, s0, newv[r0:r0 + sn])
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    assert np.array_equal(bits(k), kp) and np.array_equal(bits(v), vp)
+    assert not bool(big_k[:, page].any()) and not bool(big_k[:, :, Hkv].any())      # nothing outside the view was touched
+
+
+def test_kv_copies_skip_page_ids_outside_the_pool(ctx):
+    # the copies compare every page id with the pool size before they use it: tokens behind a bad entry are left alone
+    # (rows keep their fill on a gather, the pool is untouched on an append) and the first bad entry is reported
+    w = wl.Workload("bad_pages", 54, 4, 2, [wl.Request(200, 256, 1)])
+    mat = wl.materialize(w, need_q=False)
+    k, v = bits_to_bf16(mat.k_pages), bits_to_bf16(mat.v_pages)
+    cache = binding.make_cache(k, v)
+    pt_host = mat.page_table.copy()
+    pt_host[2], pt_host[5] = k.shape[0], -1                    # one beyond the pool, one negative
+    pt = torch.from_numpy(pt_host).cuda()
+    L = w.requests[0].total_len
+    bad = np.zeros(L, dtype=bool)
+    bad[2 * wl.PAGE:3 * wl.PAGE] = bad[5 * wl.PAGE:6 * wl.PAGE] = True
+    kr = torch.full((L, w.Hkv, w.D), 7.0, dtype=torch.bfloat16, device="cuda")
+    vr = torch.full_like(kr, 7.0)
+    binding.cp_kv_gather(ctx, cache, pt, 0, L, kr, vr)
+    torch.cuda.synchronize()
+    with pytest.raises(binding.CpError) as e:
+        ctx.poll_status()
+    assert e.value.code == binding.CP_ERR_BOUNDS
+    bits = lambda t: t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+    ref = orc.kv_gather(mat.k_pages, mat.page_table, 0, L)
+    assert np.array_equal(bits(kr)[~bad], ref[~bad]) and bool((kr[torch.from_numpy(bad).cuda()] == 7.0).all())
+    before_k, before_v = k.clone(), v.clone()
+    rows = bits_to_bf16(wl.normal_bf16(55, wl.TID_K, (L, w.Hkv, w.D)))
+    binding.cp_kv_append(ctx, cache, pt, 0, L, rows, rows)
+    binding.cp_kv_append_segments(ctx, cache, pt, [(2 * wl.PAGE, wl.PAGE, 0)], rows, rows)      # entirely behind the bad entry
+    torch.cuda.synchronize()
+    with pytest.raises(binding.CpError) as e:
+        ctx.poll_status()
+    assert e.value.code == binding.CP_ERR_BOUNDS
+    good = torch.from_numpy(mat.page_table[[i for i in range(len(pt_host)) if i not in (2, 5)]].astype(np.int64)).cuda()
+    touched = torch.zeros(k.shape[0], dtype=torch.bool, device="cuda")
+    touched[good] = True
+    assert torch.equal(k[~touched], before_k[~touched]) and torch.equal(v[~touched], before_v[~touched])
+    got = orc.kv_gather(bits(k), mat.page_table, 0, L)
+    assert np.array_equal(got[~bad], bits(rows)[~bad])
+    ctx.poll_status()                                          # cleared; the context is usable
+    check_batch(ctx, wl.Workload("after_bad_pages", 56, 8, 2, [wl.Request(150, 64, 2)]))
+
+
 def test_page_table_check_reports_bad_entries(ctx):
     # the checker only reads the table: a good table passes, an entry beyond the pool (or negative) is reported with
     # its index and value, and the context computes on afterwards
