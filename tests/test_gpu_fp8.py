@@ -99,8 +99,9 @@ def check_batch8(ctx, w, rows_per_request=None, seed=7):
     return dev, stats
 
 
-def test_fp8_append_matches_oracle_bit_for_bit(ctx):
-    w = wl.Workload("fp8_append", 51, 8, 2, [wl.Request(300, 192, 1)])
+@pytest.mark.parametrize("Hkv,page", [(2, 64), (1, 16), (3, 128), (16, 32)])
+def test_fp8_append_matches_oracle_bit_for_bit(ctx, Hkv, page):
+    w = wl.Workload("fp8_append", 51, 4 * Hkv, Hkv, [wl.Request(300, 3 * page, 1)], page=page)
     m8 = wl.materialize_fp8(w)
     dev = Device8(m8)
     r = w.requests[0]
@@ -114,12 +115,29 @@ def test_fp8_append_matches_oracle_bit_for_bit(ctx):
     kc, vc = o8.quantize_kv(newk, m8.k_scale), o8.quantize_kv(newv, m8.v_scale)
     kp, vp = m8.k8_pages.copy(), m8.v8_pages.copy()
     t = np.arange(t0, t0 + n)
-    kp[m8.page_table[t // wl.PAGE], t % wl.PAGE] = kc
-    vp[m8.page_table[t // wl.PAGE], t % wl.PAGE] = vc
+    kp[m8.page_table[t // page], t % page] = kc
+    vp[m8.page_table[t // page], t % page] = vc
     got_k, got_v = dev.k8.cpu().numpy(), dev.v8.cpu().numpy()
     assert np.array_equal(o8.e4m3_decode(got_k), o8.e4m3_decode(kp))          # (+0 and -0 codes both stand for zero)
     assert np.array_equal(o8.e4m3_decode(got_v), o8.e4m3_decode(vp))
     assert np.array_equal(got_k & 0x7F, kp & 0x7F) and np.array_equal(got_v & 0x7F, vp & 0x7F)
+    # the raw byte copies: read the stored bytes out, write them back at other tokens in two runs
+    kb = torch.zeros((n, Hkv, w.D), dtype=torch.uint8, device="cuda")
+    vb = torch.zeros_like(kb)
+    binding.cp_kv_gather_fp8(ctx, dev.cache, dev.page_table, t0, n, kb, vb)
+    torch.cuda.synchronize()
+    assert np.array_equal(kb.cpu().numpy(), got_k[m8.page_table[t // page], t % page])
+    assert np.array_equal(vb.cpu().numpy(), got_v[m8.page_table[t // page], t % page])
+    segs = [(0, 30, 100), (t0 + 50, 41, 7)]
+    binding.cp_kv_append_segments_fp8(ctx, dev.cache, dev.page_table, segs, kb, vb)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    exp_k, exp_v = got_k.copy(), got_v.copy()
+    for s0, sn, r0 in segs:
+        ts = np.arange(s0, s0 + sn)
+        exp_k[m8.page_table[ts // page], ts % page] = kb.cpu().numpy()[r0:r0 + sn]
+        exp_v[m8.page_table[ts // page], ts % page] = vb.cpu().numpy()[r0:r0 + sn]
+    assert np.array_equal(dev.k8.cpu().numpy(), exp_k) and np.array_equal(dev.v8.cpu().numpy(), exp_v)
 
 
 def test_fp8_attention_small_mixed_batch(ctx):
