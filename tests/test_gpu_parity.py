@@ -344,6 +344,30 @@ def test_attention_one_unit_cut_over_all_sms(ctx):
     check_batch(ctx, w1, pair_budget=1e10)
 
 
+def test_attention_reads_zeros_behind_page_ids_outside_the_pool(ctx):
+    # a page id outside [0, num_pages) is a tensor-map coordinate outside the tensor: the copy engine fills zeros, the
+    # same mechanism that serves the unused tail of every request's last key tile.  Reference: the oracle with those
+    # table entries pointed at a page of zeros.
+    w = wl.Workload("oob_pages", 58, 8, 2, [wl.Request(300, 640, 2)])
+    mat = wl.materialize(w)
+    dev = DeviceWorkload(mat)
+    used = set(int(x) for x in mat.page_table)
+    spare = [i for i in range(mat.k_pages.shape[0]) if i not in used][0]
+    k_ref, v_ref = mat.k_pages.copy(), mat.v_pages.copy()
+    k_ref[spare] = 0
+    v_ref[spare] = 0
+    pt_ref = mat.page_table.copy()
+    pt_dev = mat.page_table.copy()
+    for idx, bad in ((3, mat.k_pages.shape[0] + 7), (9, -2), (12, 2 ** 31 - 1)):
+        pt_ref[idx] = spare
+        pt_dev[idx] = bad
+    dev.page_table = torch.from_numpy(pt_dev).cuda()
+    out, lse = dev.run_batch(ctx)
+    r = w.requests[0]
+    ref_o, ref_l = orc.attn_full(mat.q, k_ref, v_ref, pt_ref, r.prefix_len, w.Hkv, w.scale)
+    compare(out, lse, ref_o, ref_l, "oob pages")
+
+
 def test_attention_strided_cache_view(ctx):
     # the cache is a view into a wider allocation (one unused head slot per token, an unused token row
     # per page): only the three strides say where things are
