@@ -785,7 +785,7 @@ def run_kvcopy(args, out):
     import torch
     from paper_2609_04774_b200 import build
     build.build()
-    for m in kvcopy_points(torch, load_peaks(), (16384, 131072, 1048576)):
+    for m in kvcopy_points(torch, load_peaks(), tuple(args.kv_tokens)):
         out.write(json.dumps(dict(mode="kvcopy", **m)) + "\n")
     out.flush()
 
@@ -1051,6 +1051,7 @@ def main():
     ap.add_argument("--page", type=int, default=None, help="configs mode: tokens per cache page (16, 32, 64, 128)")
     ap.add_argument("--rank-reps", type=int, default=5)
     ap.add_argument("--pass-q", action="store_true", help="cprank mode: K/V stays sharded, queries travel")
+    ap.add_argument("--kv-tokens", type=int, nargs="*", default=[16384, 131072, 1048576], help="kvcopy mode: tokens per point")
     ap.add_argument("--no-landing", action="store_true",
                     help="cprank mode: gather into separate arenas and append into the cache instead of landing in pool pages")
     ap.add_argument("--cache-requests", type=int, default=20000)
