@@ -228,21 +228,12 @@ int kv_copy(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, in
     return check_cuda(cudaGetLastError(), who);
 }
 
-}  // namespace
-
-namespace cpattn {
-int validate_kv_cache(const cp_kv_cache* c, const char* who) { return validate_cache(c, who); }
-int validate_kv_cache_fp8(const cp_kv_cache_fp8* c, const char* who) { return validate_cache_fp8(c, who); }
-}
-
-extern "C" int cp_kv_append_segments(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int32_t n_segments,
-                                     const cp_kv_segment* segments, const void* k_rows, const void* v_rows, void* stream) {
-    const char* who = "cp_kv_append_segments";
-    if (!ctx || !page_table || !segments || n_segments < 0)
-        return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or negative segment count", who);
-    if (n_segments > kMaxSegments)
-        return set_error(CP_ERR_UNSUPPORTED, "%s: %d segments, at most %d per call", who, n_segments, kMaxSegments);
-    if (int rc = validate_cache(cache, who)) return rc;
+// The segment form for both cache kinds: `elem_shift` = log2(bytes per element) turns the caller's strides into
+// 16-byte vectors (bf16: strides in elements, 8 per vector; one-byte elements: strides in bytes, 16 per vector).
+int append_segments(cp_ctx* ctx, void* cache_k, void* cache_v, int32_t page_size, int32_t Hkv, int64_t stride_page,
+                    int64_t stride_tok, int64_t stride_head, int64_t num_pages, bool one_byte, const int32_t* page_table,
+                    int32_t n_segments, const cp_kv_segment* segments, const void* k_rows, const void* v_rows, void* stream,
+                    const char* who) {
     if (!k_rows && !v_rows) return set_error(CP_ERR_INVALID_ARG, "%s: both row pointers are NULL", who);
     if (((uintptr_t)k_rows | (uintptr_t)v_rows) & 15)
         return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
@@ -261,12 +252,31 @@ extern "C" int cp_kv_append_segments(cp_ctx* ctx, const cp_kv_cache* cache, cons
     }
     if (tab.n_segments == 0) return CP_OK;
     if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    const int blocks = (int)std::min<int64_t>((tab.cum[tab.n_segments] + 7) / 8, (int64_t)ctx->num_sms * 16);
+    const int per_vec = one_byte ? 16 : 8;          // stride units per 16-byte vector
+    const int blocks = (int)std::min<int64_t>((tab.cum[tab.n_segments] + 7) / 8, (int64_t)ctx->num_sms * 16);   // one warp per token
     kv_append_segments_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        (uint4*)cache->k, (uint4*)cache->v, (const uint4*)k_rows, (const uint4*)v_rows, page_table, tab, log2_of(cache->page_size),
-        cache->Hkv, 4, cache->stride_page / 8, cache->stride_tok / 8, cache->stride_head / 8, cache->num_pages,
-        ctx->d_status);
+        (uint4*)cache_k, (uint4*)cache_v, (const uint4*)k_rows, (const uint4*)v_rows, page_table, tab, log2_of(page_size), Hkv,
+        one_byte ? 3 : 4, stride_page / per_vec, stride_tok / per_vec, stride_head / per_vec, num_pages, ctx->d_status);
     return check_cuda(cudaGetLastError(), who);
+}
+
+}  // namespace
+
+namespace cpattn {
+int validate_kv_cache(const cp_kv_cache* c, const char* who) { return validate_cache(c, who); }
+int validate_kv_cache_fp8(const cp_kv_cache_fp8* c, const char* who) { return validate_cache_fp8(c, who); }
+}
+
+extern "C" int cp_kv_append_segments(cp_ctx* ctx, const cp_kv_cache* cache, const int32_t* page_table, int32_t n_segments,
+                                     const cp_kv_segment* segments, const void* k_rows, const void* v_rows, void* stream) {
+    const char* who = "cp_kv_append_segments";
+    if (!ctx || !page_table || !segments || n_segments < 0)
+        return set_error(CP_ERR_INVALID_ARG, "%s: null pointer or negative segment count", who);
+    if (n_segments > kMaxSegments)
+        return set_error(CP_ERR_UNSUPPORTED, "%s: %d segments, at most %d per call", who, n_segments, kMaxSegments);
+    if (int rc = validate_cache(cache, who)) return rc;
+    return append_segments(ctx, const_cast<void*>(cache->k), const_cast<void*>(cache->v), cache->page_size, cache->Hkv, cache->stride_page, cache->stride_tok,
+                           cache->stride_head, cache->num_pages, false, page_table, n_segments, segments, k_rows, v_rows, stream, who);
 }
 
 extern "C" int cp_check_page_table(cp_ctx* ctx, const int32_t* page_table, int64_t n_entries, int64_t num_pages, void* stream) {
@@ -310,30 +320,9 @@ extern "C" int cp_kv_append_segments_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cac
     if (n_segments > kMaxSegments)
         return set_error(CP_ERR_UNSUPPORTED, "%s: %d segments, at most %d per call", who, n_segments, kMaxSegments);
     if (int rc = validate_cache_fp8(cache, who)) return rc;
-    if (!k_bytes && !v_bytes) return set_error(CP_ERR_INVALID_ARG, "%s: both row pointers are NULL", who);
-    if (((uintptr_t)k_bytes | (uintptr_t)v_bytes) & 15)
-        return set_error(CP_ERR_INVALID_ARG, "%s: row buffers must be 16-byte aligned", who);
-    SegmentTable tab;
-    tab.n_segments = 0;
-    tab.cum[0] = 0;
-    for (int32_t i = 0; i < n_segments; ++i) {
-        const cp_kv_segment& sg = segments[i];
-        if (sg.t_begin < 0 || sg.n < 0 || sg.row0 < 0)
-            return set_error(CP_ERR_INVALID_ARG, "%s: segment %d has a negative field", who, i);
-        if (sg.n == 0) continue;
-        const int k = tab.n_segments++;
-        tab.t_begin[k] = sg.t_begin;
-        tab.row0[k] = sg.row0;
-        tab.cum[k + 1] = tab.cum[k] + sg.n;
-    }
-    if (tab.n_segments == 0) return CP_OK;
-    if (int rc = check_cuda(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
-    const int blocks = (int)std::min<int64_t>((tab.cum[tab.n_segments] + 7) / 8, (int64_t)ctx->num_sms * 16);
-    kv_append_segments_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        (uint4*)cache->k, (uint4*)cache->v, (const uint4*)k_bytes, (const uint4*)v_bytes, page_table, tab, log2_of(cache->page_size),
-        cache->Hkv, 3, cache->stride_page / 16, cache->stride_tok / 16, cache->stride_head / 16, cache->num_pages,
-        ctx->d_status);
-    return check_cuda(cudaGetLastError(), who);
+    return append_segments(ctx, const_cast<void*>(cache->k), const_cast<void*>(cache->v), cache->page_size, cache->Hkv,
+                           cache->stride_page, cache->stride_tok, cache->stride_head, cache->num_pages, true, page_table,
+                           n_segments, segments, k_bytes, v_bytes, stream, who);
 }
 
 extern "C" int cp_kv_append_fp8(cp_ctx* ctx, const cp_kv_cache_fp8* cache, const int32_t* page_table, int64_t t_begin,
