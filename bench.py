@@ -10,7 +10,8 @@ whose KV range was split across CTAs.  `value` is measured with inputs resident 
 the same C-ABI calls from pinned HOST buffers (q, the new tokens' K/V rows appended into the paged cache,
 page table up; out and lse down).  At one GPU the same line also carries: `sustained` (the headline
 workload repeated for at least two seconds of GPU time, clocks sampled), `configs` (configurations 1-5,
-each with its own clocks), `merge` (cp_merge bandwidth points), `kvcopy` (paged copy bandwidth) and the
+each with its own clocks), `merge` (cp_merge bandwidth points), `kvcopy` (paged copy bandwidth), `cp_rank` (local
+time of the slowest rank of a degree-4 worker on configuration 2, call by call and from a CUDA graph) and the
 `cpu_baseline` legs (the fp64 oracle on the host cores).
 
 Other modes (`--mode merge|table|configs|kvcopy|cprank|cachemgr|cpu`) write the cp_merge sweep, the measured
@@ -741,10 +742,12 @@ def run_ours(args):
         line["merge"] = merge_points(torch, peaks, [(T, N, bf) for T in (4096, 16384, 65536) for N in (2, 4, 8)] +
                                      [(16384, N, f32) for N in (2, 4, 8)])
         line["kvcopy"] = kvcopy_points(torch, peaks)
+        line["cp_rank"] = cp_rank_leg(args)
         targets = {c["workload"]: c["ms"] for c in line["configs"]}
         line["targets"] = {
             "cfg2_ms_le_0.855": targets.get("cfg2_R4096_P12288_C4"), "cfg3_ms_le_125.1": targets.get("cfg3_R131072_P0_C8"),
-            "merge_points_below_5600_GBps": [(m["T"], m["N"], m["out"], round(m["GBps"])) for m in line["merge"] if m["GBps"] < 5600.0]}
+            "merge_points_below_5600_GBps": [(m["T"], m["N"], m["out"], round(m["GBps"])) for m in line["merge"] if m["GBps"] < 5600.0],
+            "cp_rank_graph_ms_le_0.30": line["cp_rank"]["slowest_rank_ms_graph_replay"]}
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline_legs(w, mat_headline, args)
     elif not args.no_cpu_baseline and world == 1:
@@ -879,6 +882,24 @@ class _LoopbackComm:
 
     def all_to_all(self, blocks):
         return blocks.clone(), self._Done()
+
+
+def cp_rank_leg(args):
+    """The rank worker's local time on the headline configuration for the default line: slowest rank, issued call by
+    call and replayed from a CUDA graph (bf16 cache, all-gather-KV exchange, landing mode)."""
+    import copy
+    import io
+    a = copy.copy(args)
+    a.configs, a.fp8, a.pass_q, a.no_landing = [2], False, False, False
+    buf = io.StringIO()
+    run_cprank(a, buf)
+    d = json.loads(buf.getvalue().strip().splitlines()[-1])
+    g = [x for x in d["rank_local_ms_graph_replay"] if x]
+    return {"workload": d["workload"], "C": d["C"], "exchange": d["exchange"], "landing": d["landing"],
+            "slowest_rank_ms": d["slowest_rank_ms"], "slowest_rank_ms_graph_replay": max(g) if g else None,
+            "nvlink_bytes_received_per_rank": d["nvlink_bytes_received_per_rank"],
+            "nvlink_ms_modelled_at_770GBps": d["nvlink_ms_modelled_at_770GBps"],
+            "note": "one GPU: local work of each rank measured with loopback gathers; the link time is modelled, not measured"}
 
 
 def run_cprank(args, out):
