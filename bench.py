@@ -12,7 +12,8 @@ page table up; out and lse down).  At one GPU the same line also carries: `susta
 workload repeated for at least two seconds of GPU time, clocks sampled), `configs` (configurations 1-5,
 each with its own clocks), `merge` (cp_merge bandwidth points), `kvcopy` (paged copy bandwidth), `cp_rank` (local
 time of the slowest rank of a degree-4 worker on configuration 2, call by call and from a CUDA graph) and the
-`cpu_baseline` legs (the fp64 oracle on the host cores).
+`cpu_baseline` legs (the fp64 oracle on the host cores), plus `prefill_time_table`, a corner of the measured
+t(new_len, prefix_len, C) table (the whole table: `--mode table`).
 
 Other modes (`--mode merge|table|configs|kvcopy|cprank|cachemgr|cpu`) write the cp_merge sweep, the measured
 prefill-time table over (new_len, prefix_len, C), the per-config numbers, the paged KV copy bandwidth, one CP rank's
@@ -743,6 +744,7 @@ def run_ours(args):
                                      [(16384, N, f32) for N in (2, 4, 8)])
         line["kvcopy"] = kvcopy_points(torch, peaks)
         line["cp_rank"] = cp_rank_leg(args)
+        line["prefill_time_table"] = table_leg(torch)
         targets = {c["workload"]: c["ms"] for c in line["configs"]}
         line["targets"] = {
             "cfg2_ms_le_0.855": targets.get("cfg2_R4096_P12288_C4"), "cfg3_ms_le_125.1": targets.get("cfg3_R131072_P0_C8"),
@@ -793,6 +795,66 @@ def run_kvcopy(args, out):
     out.flush()
 
 
+def _time_call(torch, fn):
+    """Best of three batch means of one call; a batch runs for about 10 ms (2 to 50 launches)."""
+    for _ in range(2):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    fn()
+    e1.record()
+    torch.cuda.synchronize()
+    reps = int(max(2, min(50, 10.0 / max(e0.elapsed_time(e1), 1e-3))))
+    best = float("inf")
+    for _ in range(3):
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1) / reps)
+    return best
+
+
+def table_leg(torch):
+    """A corner of the prefill-time table for the default line: (new_len, prefix_len) in {4096, 16384} x hit ratio
+    {0, 0.75}, C in {1, 2, 4, 8}: time of all shards in one launch and of the slowest / fastest single shard (what one
+    CP rank computes), with W(R, P) of Eq. 1.  Random K/V made on the device (the values do not matter for the time)."""
+    from paper_2609_04774_b200 import binding
+    ctx = binding.Context(torch.cuda.current_device())
+    Hq, Hkv, D = 32, 8, 128
+    scale = D ** -0.5
+    rows = []
+    for R in (4096, 16384):
+        for hit in (0.0, 0.75):
+            P = (int(round(R / (1 - hit))) - R) // wl.PAGE * wl.PAGE
+            pages = (P + R + wl.PAGE - 1) // wl.PAGE
+            q = torch.randn((R, Hq, D), device="cuda").to(torch.bfloat16)
+            k = torch.randn((pages, wl.PAGE, Hkv, D), device="cuda").to(torch.bfloat16)
+            v = torch.randn((pages, wl.PAGE, Hkv, D), device="cuda").to(torch.bfloat16)
+            pt = torch.from_numpy(wl.permutation(11, wl.TID_PERM, pages)).cuda()
+            cache = binding.make_cache(k, v)
+            o = torch.empty((R, Hq, D), dtype=torch.bfloat16, device="cuda")
+            lse = torch.empty((Hq, R), dtype=torch.float32, device="cuda")
+            po = torch.empty((R, Hq, D), dtype=torch.float32, device="cuda")
+            ws = torch.zeros(binding.cp_workspace_bytes([R], [8], Hq), dtype=torch.uint8, device="cuda")
+            W = R * P + R * (R + 1) // 2
+            for C in (1, 2, 4, 8):
+                t_all = _time_call(torch, lambda: binding.cp_prefill_attn(ctx, q, cache, pt, P, R, C, Hq, scale, o, lse, ws))
+                ts = [_time_call(torch, lambda: binding.cp_prefill_attn_shard(ctx, q, cache, pt, P, R, C, s, Hq, scale, po, lse, ws))
+                      for s in range(C)]
+                rows.append({"R": R, "P": P, "C": C, "W": W, "t_all_ms": t_all, "t_shard_max_ms": max(ts), "t_shard_min_ms": min(ts)})
+            ctx.poll_status()
+            del q, k, v, o, po, lse, ws
+            torch.cuda.empty_cache()
+    ctx.close()
+    base = {(r["R"], r["P"]): r["t_shard_max_ms"] for r in rows if r["C"] == 1}
+    for r in rows:
+        r["speedup_vs_C1"] = base[(r["R"], r["P"])] / r["t_shard_max_ms"]
+    return rows
+
+
 def run_table(args, out):
     """Measured prefill-time table over (new_len, prefix_len, C): all-shard time and the slowest /
     fastest single shard (what one CP rank would compute), with W(R,P) of Eq. (1) -- the inputs of the
@@ -819,26 +881,7 @@ def run_table(args, out):
             po = torch.empty((R, Hq, D), dtype=torch.float32, device="cuda")
             ws = torch.zeros(binding.cp_workspace_bytes([R], [8], Hq), dtype=torch.uint8, device="cuda")
 
-            def timeit(fn):
-                """Best of three batch means; a batch runs for about 10 ms (2 to 50 launches)."""
-                for _ in range(2):
-                    fn()
-                torch.cuda.synchronize()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                fn()
-                e1.record()
-                torch.cuda.synchronize()
-                reps = int(max(2, min(50, 10.0 / max(e0.elapsed_time(e1), 1e-3))))
-                best = float("inf")
-                for _ in range(3):
-                    e0.record()
-                    for _ in range(reps):
-                        fn()
-                    e1.record()
-                    torch.cuda.synchronize()
-                    best = min(best, e0.elapsed_time(e1) / reps)
-                return best
+            timeit = lambda fn: _time_call(torch, fn)
 
             W = R * P + R * (R + 1) // 2
             for C in (1, 2, 4, 8):

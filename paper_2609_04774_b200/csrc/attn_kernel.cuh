@@ -834,6 +834,28 @@ __device__ __forceinline__ void softmax_tile(float (&c0)[32], float (&c1)[32], f
     l += st.x + st.y;
 }
 
+// 4 x 4 transpose of 16-byte items inside every group of four lanes: on return v[s] holds what lane (quad * 4 + s)
+// had in v[t], t = this lane's position in its quad.  Two exchange stages (lane ^ 1, lane ^ 2), 16 shuffles.
+__device__ __forceinline__ uint4 shfl_xor16(uint4 a, int mask) {
+    a.x = __shfl_xor_sync(0xffffffffu, a.x, mask);
+    a.y = __shfl_xor_sync(0xffffffffu, a.y, mask);
+    a.z = __shfl_xor_sync(0xffffffffu, a.z, mask);
+    a.w = __shfl_xor_sync(0xffffffffu, a.w, mask);
+    return a;
+}
+__device__ __forceinline__ void quad_transpose(uint4 (&v)[4], int t) {
+    {
+        const bool hi = t & 1;
+        const uint4 r0 = shfl_xor16(hi ? v[0] : v[1], 1), r1 = shfl_xor16(hi ? v[2] : v[3], 1);
+        if (hi) { v[0] = r0; v[2] = r1; } else { v[1] = r0; v[3] = r1; }
+    }
+    {
+        const bool hi = t & 2;
+        const uint4 r0 = shfl_xor16(hi ? v[0] : v[2], 2), r1 = shfl_xor16(hi ? v[1] : v[3], 2);
+        if (hi) { v[0] = r0; v[1] = r1; } else { v[2] = r0; v[3] = r1; }
+    }
+}
+
 template <bool kFp8>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSched& inl, uint32_t smem_base, uint32_t tmem_base,
                                              volatile uint32_t* abort_flag, int wg) {
@@ -904,33 +926,53 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
         const bool partial = u.slot >= 0;
         const bool valid = row < u.it.n_rows;
         const int64_t grow_idx = (int64_t)u.it.q_row0 + row;
-        float* part_row = p.partial_o + (((int64_t)max(u.slot, 0) * 2 + wg) * kBlockM + (row - row_base)) * kD;
+        // A thread holds 32 consecutive columns of its own row; written as they are, every store instruction of a warp
+        // would touch 32 rows with 16 bytes each.  The four lanes of a quad swap their 16-byte pieces first, so that
+        // a store instruction writes 64 contiguous bytes of each of 8 rows (a quarter of the memory transactions).
+        const int qt = lane & 3;
+        const int row_q0 = row - qt;                                        // first row of this lane's quad
+        const bool f32 = partial || p.out_f32;
+        // element (not byte) offset of row row_q0, column 0, in the destination this call writes
+        const int64_t base_q0 = partial ? (((int64_t)u.slot * 2 + wg) * kBlockM + (row_q0 - row_base)) * kD
+                                        : (((int64_t)u.it.q_row0 + row_q0) * p.Hq + head) * kD;
+        const int64_t row_pitch = partial ? kD : (int64_t)p.Hq * kD;        // elements between consecutive rows
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
             float o[32];
             TMEM_LD32(o_tmem + cc * 32, o, 0);
             tc_wait_ld();
-            if (valid) {
-                if (partial || p.out_f32) {
-                    float4* dst = partial ? reinterpret_cast<float4*>(part_row + cc * 32)
-                                          : reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) +
-                                                                      (grow_idx * p.Hq + head) * kD + cc * 32);
+            if (f32) {
+                float* dstf = partial ? p.partial_o : reinterpret_cast<float*>(p.out);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        dst[i] = make_float4(o[4 * i] * inv_l, o[4 * i + 1] * inv_l, o[4 * i + 2] * inv_l, o[4 * i + 3] * inv_l);
-                } else {
-                    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) +
-                                                          (grow_idx * p.Hq + head) * kD + cc * 32);
+                for (int hlf = 0; hlf < 2; ++hlf) {
+                    uint4 v[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        uint4 v;
-                        v.x = pack_bf16(o[8 * i + 0] * inv_l, o[8 * i + 1] * inv_l);
-                        v.y = pack_bf16(o[8 * i + 2] * inv_l, o[8 * i + 3] * inv_l);
-                        v.z = pack_bf16(o[8 * i + 4] * inv_l, o[8 * i + 5] * inv_l);
-                        v.w = pack_bf16(o[8 * i + 6] * inv_l, o[8 * i + 7] * inv_l);
-                        dst[i] = v;
+                        const int c0 = hlf * 16 + 4 * i;
+                        v[i] = make_uint4(__float_as_uint(o[c0] * inv_l), __float_as_uint(o[c0 + 1] * inv_l),
+                                          __float_as_uint(o[c0 + 2] * inv_l), __float_as_uint(o[c0 + 3] * inv_l));
                     }
+                    quad_transpose(v, qt);
+#pragma unroll
+                    for (int sdx = 0; sdx < 4; ++sdx)
+                        if (row_q0 + sdx < u.it.n_rows)
+                            *reinterpret_cast<uint4*>(dstf + base_q0 + sdx * row_pitch + cc * 32 + hlf * 16 + qt * 4) = v[sdx];
                 }
+            } else {
+                uint4 v[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    v[i].x = pack_bf16(o[8 * i + 0] * inv_l, o[8 * i + 1] * inv_l);
+                    v[i].y = pack_bf16(o[8 * i + 2] * inv_l, o[8 * i + 3] * inv_l);
+                    v[i].z = pack_bf16(o[8 * i + 4] * inv_l, o[8 * i + 5] * inv_l);
+                    v[i].w = pack_bf16(o[8 * i + 6] * inv_l, o[8 * i + 7] * inv_l);
+                }
+                quad_transpose(v, qt);
+                __nv_bfloat16* dsth = reinterpret_cast<__nv_bfloat16*>(p.out);
+#pragma unroll
+                for (int sdx = 0; sdx < 4; ++sdx)
+                    if (row_q0 + sdx < u.it.n_rows)
+                        *reinterpret_cast<uint4*>(dsth + base_q0 + sdx * row_pitch + cc * 32 + qt * 8) = v[sdx];
             }
         }
         if (valid) {
