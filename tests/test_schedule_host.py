@@ -84,6 +84,19 @@ def test_schedule_balances_short_no_prefix_requests():
             assert info["max_load"] <= max(1.25 * share, share + 8), (R, C, info)
 
 
+def test_schedule_counts_a_fixed_cost_per_piece_for_small_kv():
+    # small K/V (one group): the slowest CTA's estimated cost -- its KV tile steps plus two per piece of work -- stays
+    # within 6 % (+2) of the mean cost for mid-size requests without a prefix; coverage is checked as everywhere
+    for R, bound in ((3072, 42), (4096, 68), (6144, 144)):
+        w = wl.Workload("mid", 1, 32, 8, [wl.Request(R, 0, 1)])
+        info, loads = check(w)
+        _, pieces, _ = binding.cp_schedule_inspect(w.cu_new, [0], [1], w.Hq, w.Hkv, 148)
+        cnt = np.bincount(pieces[:, 0], minlength=info["grid"])
+        cost = loads + 2 * cnt
+        assert cost.max() <= bound, (R, cost.max())
+        assert cost.max() <= 1.06 * cost.mean() + 2, (R, cost.max(), cost.mean())
+
+
 def test_schedule_small_and_odd_shapes():
     for w in (wl.small_mixed(), wl.Workload("one_row", 1, 4, 2, [wl.Request(1, 0, 1)]),
               wl.Workload("long_prefix", 2, 8, 2, [wl.Request(7, 100000, 2)]),
