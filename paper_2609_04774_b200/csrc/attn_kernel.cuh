@@ -525,9 +525,12 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, const InlineSche
     uint32_t s_par = 1;                // parity of "previous score tile was read"; 1: no tile yet (passes)
     const uint64_t q_desc0 = make_desc(smem_base + kSmemQ, 16, 1024);
     const uint64_t k_desc0 = make_desc(smem_base + kSmemKV, 16, 1024);           // K-major view of a ring slot
-    for (int round = 0;; ++round) {
-        UnitInfo u;
-        if (!fetch_unit(p, inl, round, u)) break;
+    // the next unit's description is fetched while the current one runs (three dependent loads otherwise sit between
+    // the last score tile of a unit and the first of the next)
+    UnitInfo u, nu;
+    bool have = fetch_unit(p, inl, 0, u);
+    for (int round = 0; have; ++round) {
+        const bool have_next = fetch_unit(p, inl, round + 1, nu);
         const int j0 = u.t_begin, n = u.t_end;
         mbar_wait(bars, kBarQFull, round & 1, abort_flag, p.status, round);
         RingPos kpos = unit_pos;
@@ -568,6 +571,8 @@ __device__ __forceinline__ void mma_s_role(const AttnParams& p, const InlineSche
         const uint32_t q5 = adv / kKvStages, r5 = adv - q5 * kKvStages;
         unit_pos = unit_pos.plus(r5);
         unit_pos.par ^= (q5 & 1u);
+        u = nu;
+        have = have_next;
     }
 }
 
@@ -582,9 +587,10 @@ __device__ __forceinline__ void mma_pv_role(const AttnParams& p, const InlineSch
     RingPos unit_pos = {0, 0};
     uint32_t p_par0 = 0, p_par1 = 0;   // phase parity of p_ready per softmax warpgroup
     const uint64_t v_desc0 = make_desc(smem_base + kSmemKV, kHalfBytes, 1024);   // MN-major view of a ring slot
-    for (int round = 0;; ++round) {
-        UnitInfo u;
-        if (!fetch_unit(p, inl, round, u)) break;
+    UnitInfo u, nu;
+    bool have = fetch_unit(p, inl, 0, u);
+    for (int round = 0; have; ++round) {
+        const bool have_next = fetch_unit(p, inl, round + 1, nu);      // fetched ahead, as in the score issuer
         const int j0 = u.t_begin, n = u.t_end;
         RingPos vpos = unit_pos.plus(n - j0 == 1 ? 1 : 2);   // V(j0)
 #pragma unroll 1
@@ -635,6 +641,8 @@ __device__ __forceinline__ void mma_pv_role(const AttnParams& p, const InlineSch
         const uint32_t q5 = adv / kKvStages, r5 = adv - q5 * kKvStages;
         unit_pos = unit_pos.plus(r5);
         unit_pos.par ^= (q5 & 1u);
+        u = nu;
+        have = have_next;
     }
 }
 
@@ -881,9 +889,9 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
     __syncwarp();
     uint32_t s_par = 0;        // phase parity of s_ready for this head
 
-    for (int round = 0;; ++round) {
-        UnitInfo u;
-        if (!fetch_unit(p, inl, round, u)) break;
+    UnitInfo u, nu;
+    bool have = fetch_unit(p, inl, 0, u);
+    for (int round = 0; have; ++round) {
         const int n = u.t_end;
         const int head = u.head0 + head_sel;
         const int j_first = u.t_begin;
@@ -917,6 +925,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
                                    j == j_first, m, l, sy);
             ++tile_cnt;
         }
+        // the next unit's description is fetched under the epilogue
+        const bool have_next = fetch_unit(p, inl, round + 1, nu);
         // epilogue: O / l -> global at the row's original position; LSE in natural log
         SM_WAIT(kBarPvDone + wg, (tile_cnt - 1) & 1, n);
         tc_fence_after();
@@ -983,6 +993,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, const InlineSc
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + (kBarOFree + wg) * 8);
+        u = nu;
+        have = have_next;
     }
 #undef SM_WAIT
 }
