@@ -51,7 +51,7 @@ NOMINAL_HBM_GBS = 8000.0
 MUFU_ROOFLINE_TFLOPS = 148 * 16 * 512 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum of one cp_attn_kernel launch, from the ncu captures
 # summarised in profiles/ (per workload name; a workload without a capture reports null)
-ATTN_TRAFFIC_BYTES = {"cfg2_R4096_P12288_C4": 117_532_416, "cfg3_R131072_P0_C8": 7_200_575_488}
+ATTN_TRAFFIC_BYTES = {"cfg2_R4096_P12288_C4": 121_965_056, "cfg3_R131072_P0_C8": 7_200_575_488}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
