@@ -122,7 +122,8 @@ WorkspaceLayout workspace_layout(size_t n_items, size_t n_pieces, size_t n_merge
     return w;
 }
 
-// Estimated time of a schedule's slowest CTA in KV tile steps: its tiles plus kPieceCostTiles per piece of work.
+// Estimated time of a schedule in KV tile steps: the slowest CTA's tiles plus kPieceCostTiles per piece of work,
+// plus the merge launch when any unit is cut.
 static int64_t schedule_cost(const Schedule& s) {
     int64_t worst = 0;
     for (int32_t g = 0; g < s.grid; ++g) {
@@ -130,7 +131,8 @@ static int64_t schedule_cost(const Schedule& s) {
         for (int32_t k = s.cta_off[g]; k < s.cta_off[g + 1]; ++k) cost += s.pieces[k].t_end - s.pieces[k].t_begin + kPieceCostTiles;
         worst = std::max(worst, cost);
     }
-    return worst;
+    // a schedule with cut units is followed by the merge launch (about ten microseconds: six tile steps)
+    return worst + (s.merges.empty() ? 0 : kMergeLaunchCostTiles);
 }
 
 // Schedule for batches whose K/V is small enough that the order of the units does not matter for L2 (one group).
@@ -138,8 +140,10 @@ static int64_t schedule_cost(const Schedule& s) {
 // tile steps, measured), so a CTA with many short pieces gets fewer tiles.  Whole units go, longest first, to the CTA
 // with the smallest cost so far while they fit under the share; the rest are cut into KV ranges that fill the
 // least-loaded CTAs up to the share (raised one step at a time when nothing fits any more).
+// With cuts = false nothing is cut (plain longest-first dealing to the least-loaded CTA): no partial results and no
+// merge launch, which wins for small batches of many short units.
 // Returns false when the cuts need more partial slots than there are (the caller then uses the dealing scheme).
-static bool build_schedule_lpt(int32_t HP, int32_t grid_max, int64_t W, int32_t longest, Schedule& s) {
+static bool build_schedule_lpt(int32_t HP, int32_t grid_max, int64_t W, int32_t longest, bool cuts, Schedule& s) {
     const int64_t n_items = (int64_t)s.items.size();
     const int64_t n_units = n_items * HP;
     const int64_t c = kPieceCostTiles;
@@ -160,7 +164,7 @@ static bool build_schedule_lpt(int32_t HP, int32_t grid_max, int64_t W, int32_t 
         const int32_t n = s.items[i].n_kv_tiles;
         for (int32_t pr = 0; pr < HP; ++pr) {
             const Slot top = heap.top();
-            if (top.first + n + c <= T) {
+            if (!cuts || top.first + n + c <= T) {      // without cuts: every unit whole, to the least-loaded CTA
                 heap.pop();
                 ps.push_back({(int32_t)i, pr, 0, n, -1, top.second});
                 heap.push({top.first + n + c, top.second});
@@ -238,11 +242,13 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t pairs_per_kv, int
     // small K/V (one group): the least-loaded-first scheme is built as well and kept when its slowest CTA's
     // estimated cost is lower by at least 3 % (measured: 9-10 % less time for 3072 and 4096 new tokens without a
     // prefix at 32/8 heads; no difference below the margin)
-    Schedule alt;
-    bool have_alt = false;
+    Schedule alt, whole;
+    bool have_alt = false, have_whole = false;
     if (!one_each && allow_split && PK == HP) {
         alt.items = s.items;
-        have_alt = build_schedule_lpt(HP, grid_max, W, longest, alt);
+        have_alt = build_schedule_lpt(HP, grid_max, W, longest, true, alt);
+        whole.items = s.items;
+        have_whole = build_schedule_lpt(HP, grid_max, W, longest, false, whole);
     }
     const int32_t G = one_each ? (int32_t)n_units
                                : (int32_t)std::max<int64_t>(1, std::min<int64_t>(grid_max, (W + T - 1) / T));
@@ -343,14 +349,16 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t pairs_per_kv, int
     }
     for (const Cut& k : cuts)
         s.pieces[(size_t)fill[k.cta]++] = {tail[k.unit].item, (int16_t)tail[k.unit].pair, (int16_t)k.slot, k.t_begin, k.t_end};
-    if (have_alt && schedule_cost(alt) * 100 < schedule_cost(s) * 97) {     // by a margin: the estimate is coarse
-        s.pieces.swap(alt.pieces);
-        s.cta_off.swap(alt.cta_off);
-        s.merges.swap(alt.merges);
-        s.merge_slots.swap(alt.merge_slots);
-        s.grid = alt.grid;
-        s.n_slots = alt.n_slots;
-    }
+    auto take = [&s](Schedule& o) {
+        s.pieces.swap(o.pieces);
+        s.cta_off.swap(o.cta_off);
+        s.merges.swap(o.merges);
+        s.merge_slots.swap(o.merge_slots);
+        s.grid = o.grid;
+        s.n_slots = o.n_slots;
+    };
+    if (have_alt && schedule_cost(alt) * 100 < schedule_cost(s) * 97) take(alt);     // by a margin: the estimate is coarse
+    if (have_whole && schedule_cost(whole) * 100 < schedule_cost(s) * 97) take(whole);
     return CP_OK;
 }
 

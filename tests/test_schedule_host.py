@@ -87,14 +87,16 @@ def test_schedule_balances_short_no_prefix_requests():
 def test_schedule_counts_a_fixed_cost_per_piece_for_small_kv():
     # small K/V (one group): the slowest CTA's estimated cost -- its KV tile steps plus two per piece of work -- stays
     # within 6 % (+2) of the mean cost for mid-size requests without a prefix; coverage is checked as everywhere
-    for R, bound in ((3072, 42), (4096, 68), (6144, 144)):
+    for R, bound in ((1536, 14), (2048, 20), (3072, 42), (4096, 66), (6144, 140)):
         w = wl.Workload("mid", 1, 32, 8, [wl.Request(R, 0, 1)])
         info, loads = check(w)
         _, pieces, _ = binding.cp_schedule_inspect(w.cu_new, [0], [1], w.Hq, w.Hkv, 148)
         cnt = np.bincount(pieces[:, 0], minlength=info["grid"])
         cost = loads + 2 * cnt
         assert cost.max() <= bound, (R, cost.max())
-        assert cost.max() <= 1.06 * cost.mean() + 2, (R, cost.max(), cost.mean())
+        assert cost.max() <= 1.06 * cost.mean() + 4, (R, cost.max(), cost.mean())
+        # these batches of many short units are dealt whole: nothing is cut, so the call is one launch
+        assert info["split_units"] == 0 and info["launches"] == 1, info
 
 
 def test_schedule_small_and_odd_shapes():
