@@ -143,7 +143,7 @@ static int64_t schedule_cost(const Schedule& s) {
 // With cuts = false nothing is cut (plain longest-first dealing to the least-loaded CTA): no partial results and no
 // merge launch, which wins for small batches of many short units.
 // Returns false when the cuts need more partial slots than there are (the caller then uses the dealing scheme).
-static bool build_schedule_lpt(int32_t HP, int32_t grid_max, int64_t W, int32_t longest, bool cuts, Schedule& s) {
+static bool build_schedule_lpt(int32_t HP, int32_t PK, int32_t grid_max, int64_t W, int32_t longest, bool cuts, Schedule& s) {
     const int64_t n_items = (int64_t)s.items.size();
     const int64_t n_units = n_items * HP;
     const int64_t c = kPieceCostTiles;
@@ -160,9 +160,11 @@ static bool build_schedule_lpt(int32_t HP, int32_t grid_max, int64_t W, int32_t 
     // items are sorted longest first (build_tiles), so walking them in order is longest first
     struct TailUnit { int32_t item; int32_t pair; int32_t n; };
     std::vector<TailUnit> tail;
+    // PK < HP: KV head by KV head (all CTAs then read one head's K/V at a time), longest first within a head
+    for (int32_t g0 = 0; g0 < HP; g0 += PK)
     for (int64_t i = 0; i < n_items; ++i) {
         const int32_t n = s.items[i].n_kv_tiles;
-        for (int32_t pr = 0; pr < HP; ++pr) {
+        for (int32_t pr = g0; pr < g0 + PK; ++pr) {
             const Slot top = heap.top();
             if (!cuts || top.first + n + c <= T) {      // without cuts: every unit whole, to the least-loaded CTA
                 heap.pop();
@@ -239,16 +241,17 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t pairs_per_kv, int
     // When there are no more units than CTAs and none is longer than the share, every unit gets a CTA of its own:
     // the same critical path as packing them, and nothing is cut, so no partial results and no merge launch.
     const bool one_each = n_units <= grid_max && longest <= T;
-    // small K/V (one group): the least-loaded-first scheme is built as well and kept when its slowest CTA's
-    // estimated cost is lower by at least 3 % (measured: 9-10 % less time for 3072 and 4096 new tokens without a
-    // prefix at 32/8 heads; no difference below the margin)
+    // Small shares (a CTA gets at most kLptMaxShareTiles KV tile steps, so the fixed cost of a piece of work is
+    // felt): two more schedules are built, least-loaded-first with and without cuts, and the cheapest of the three
+    // by estimate is kept (the others must lose by at least 3 %).  Larger batches are balanced within a per cent
+    // by the dealing scheme below, and three schedules would only cost host time.
     Schedule alt, whole;
     bool have_alt = false, have_whole = false;
-    if (!one_each && allow_split && PK == HP) {
+    if (!one_each && allow_split && T <= kLptMaxShareTiles) {
         alt.items = s.items;
-        have_alt = build_schedule_lpt(HP, grid_max, W, longest, true, alt);
+        have_alt = build_schedule_lpt(HP, PK, grid_max, W, longest, true, alt);
         whole.items = s.items;
-        have_whole = build_schedule_lpt(HP, grid_max, W, longest, false, whole);
+        have_whole = build_schedule_lpt(HP, PK, grid_max, W, longest, false, whole);
     }
     const int32_t G = one_each ? (int32_t)n_units
                                : (int32_t)std::max<int64_t>(1, std::min<int64_t>(grid_max, (W + T - 1) / T));
