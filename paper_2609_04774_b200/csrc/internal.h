@@ -70,6 +70,7 @@ constexpr int kMinShareTiles = 8;                      // smallest per-CTA share
 constexpr int kMinPieceTiles = 4;                      // never cut a unit into pieces shorter than this
 constexpr int kMergeLaunchCostTiles = 6;                // the merge launch behind a schedule with cut units, in KV tile steps
 constexpr int kLptMaxShareTiles = 256;                 // per-CTA share up to which the least-loaded-first schedules are tried
+constexpr int kLptMaxUnitsPerCta = 16;                 // ... and units per CTA (more than that balance by their number)
 constexpr int kPieceCostTiles = 2;                     // fixed cost of a piece of work (prologue, epilogue, ramp) in KV tile steps
 constexpr size_t kPartialRowFloats = 128;              // fp32 values of one partial row
 constexpr size_t kPartialSlotRows = 2 * 128;           // two heads x 128 query rows per slot

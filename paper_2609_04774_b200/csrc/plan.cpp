@@ -153,9 +153,16 @@ static bool build_schedule_lpt(int32_t HP, int32_t PK, int32_t grid_max, int64_t
     struct Piece { int32_t item; int32_t pair; int32_t t_begin; int32_t t_end; int32_t slot; int32_t cta; };
     std::vector<Piece> ps;
     ps.reserve((size_t)n_units + 2 * (size_t)G);
-    // least-loaded CTA first; equal costs: lowest CTA index (the schedule is a pure function of its inputs)
-    typedef std::pair<int64_t, int32_t> Slot;
-    std::priority_queue<Slot, std::vector<Slot>, std::greater<Slot>> heap;
+    // least-loaded CTA first; equal costs: lowest CTA index (the schedule is a pure function of its inputs).
+    // Heap keys are cost * 256 + CTA index in one integer (kMaxGrid < 256): one comparison per step.
+    struct Slot { int64_t first; int32_t second; };
+    struct Heap {
+        std::priority_queue<int64_t, std::vector<int64_t>, std::greater<int64_t>> q;
+        void push(Slot v) { q.push(v.first * 256 + v.second); }
+        Slot top() const { return {q.top() >> 8, (int32_t)(q.top() & 255)}; }
+        void pop() { q.pop(); }
+    } heap;
+    static_assert(kMaxGrid <= 256, "CTA index must fit the key's low byte");
     for (int32_t g = 0; g < G; ++g) heap.push({0, g});
     // items are sorted longest first (build_tiles), so walking them in order is longest first
     struct TailUnit { int32_t item; int32_t pair; int32_t n; };
@@ -242,12 +249,12 @@ static int build_schedule_impl(int32_t pairs_per_tile, int32_t pairs_per_kv, int
     // the same critical path as packing them, and nothing is cut, so no partial results and no merge launch.
     const bool one_each = n_units <= grid_max && longest <= T;
     // Small shares (a CTA gets at most kLptMaxShareTiles KV tile steps, so the fixed cost of a piece of work is
-    // felt): two more schedules are built, least-loaded-first with and without cuts, and the cheapest of the three
+    // felt) and few units per CTA (many short units balance by their number alone): two more schedules are built, least-loaded-first with and without cuts, and the cheapest of the three
     // by estimate is kept (the others must lose by at least 3 %).  Larger batches are balanced within a per cent
     // by the dealing scheme below, and three schedules would only cost host time.
     Schedule alt, whole;
     bool have_alt = false, have_whole = false;
-    if (!one_each && allow_split && T <= kLptMaxShareTiles) {
+    if (!one_each && allow_split && T <= kLptMaxShareTiles && n_units <= (int64_t)kLptMaxUnitsPerCta * grid_max) {
         alt.items = s.items;
         have_alt = build_schedule_lpt(HP, PK, grid_max, W, longest, true, alt);
         whole.items = s.items;
