@@ -99,6 +99,17 @@ def test_schedule_counts_a_fixed_cost_per_piece_for_small_kv():
         assert info["split_units"] == 0 and info["launches"] == 1, info
 
 
+def test_schedule_is_a_pure_function_of_its_inputs():
+    # the same arguments give the same lists, whichever of the three schemes wins (ties in the least-loaded-first
+    # dealing go to the lowest CTA index): a remembered schedule can stand in for a rebuilt one
+    for w in (wl.Workload("p1", 1, 32, 8, [wl.Request(4096, 0, 1)]), wl.Workload("p2", 1, 32, 8, [wl.Request(2048, 4096, 2)]),
+              wl.small_mixed(), wl.config2()):
+        a = (w.cu_new, [r.prefix_len for r in w.requests], [r.C for r in w.requests], w.Hq, w.Hkv, 148)
+        i1, p1, t1 = binding.cp_schedule_inspect(*a)
+        i2, p2, t2 = binding.cp_schedule_inspect(*a)
+        assert i1 == i2 and np.array_equal(p1, p2) and np.array_equal(t1, t2)
+
+
 def test_schedule_small_and_odd_shapes():
     for w in (wl.small_mixed(), wl.Workload("one_row", 1, 4, 2, [wl.Request(1, 0, 1)]),
               wl.Workload("long_prefix", 2, 8, 2, [wl.Request(7, 100000, 2)]),
